@@ -1,0 +1,162 @@
+/*
+ * libblockdialect: BlockDialect W4A4 quantized linear layer for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Every tensor pointer is a DEVICE pointer owned by the caller unless a
+ * parameter says "host".  `stream` is a cudaStream_t passed as void* (NULL = the
+ * legacy default stream).  Calls enqueue work on the stream and return; argument
+ * errors are reported synchronously through the return value and nothing is
+ * enqueued.  Device-side conditions (non-finite input, an expired bounded wait)
+ * are recorded in a device status word that bd_poll_status reads.  The library
+ * never allocates or frees device memory on these paths: scratch is passed in as
+ * `workspace` (sizes from the *_workspace_size calls).  There is no CPU fallback.
+ *
+ * The method (arXiv 2501.01144, "BlockDialect"):
+ *   - operands are cut into blocks of 32 consecutive elements along the
+ *     multiplication dimension K (Sec. 3.1; Appendix "Quantization Dimension");
+ *   - each block stores a shared power-of-two exponent e = floor(log2 max|x|) - 2
+ *     (Sec. 3.1), a 4-bit dialect id into the 16-entry DialectFP4 formatbook
+ *     (Sec. 3.1, Fig. 4) and, per element, a sign bit and a 3-bit index into the
+ *     dialect's eight magnitudes 0.5 * {0..15} (Sec. 3.1, Sec. 3.3);
+ *   - a product of two operands sums 4-bit integer products exactly inside a
+ *     block and rescales once per block by 2^(eA + eB - 2) (Sec. 3.3, Fig. 6).
+ */
+#ifndef BD_H
+#define BD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BD_OK = 0,
+    BD_ERR_INVALID_ARG = 1, /* null pointer, negative size, bad enum                      */
+    BD_ERR_SHAPE = 2,       /* K not a multiple of 32, operand shapes disagree, ld < K    */
+    BD_ERR_ALIGN = 3,       /* pointer or leading dimension not 16-byte aligned           */
+    BD_ERR_UNSUPPORTED = 4, /* combination not implemented                                */
+    BD_ERR_CUDA = 5,        /* a CUDA call failed; bd_last_cuda_error gives the code      */
+    BD_ERR_NONFINITE = 6,   /* Inf/NaN met by a quantizer (from bd_poll_status)           */
+    BD_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired (from bd_poll_status)   */
+    BD_ERR_WORKSPACE = 8    /* workspace missing or too small                             */
+} bd_status;
+
+typedef enum { BD_F32 = 0, BD_BF16 = 1, BD_F16 = 2 } bd_dtype;
+
+/* Dialect selection rule.
+ * BD_SELECT_TWO_STAGE: the online rule of Sec. 3.2 (Fig. 5): stage 1 picks the
+ *   dialect pair whose maximum equals the block maximum rounded to the 0.5 grid,
+ *   stage 2 the member of the pair with more block elements inside its beneficial
+ *   range (equal counts: the even-numbered dialect).
+ * BD_SELECT_MSE: the offline rule for weights (Sec. 3.2 first paragraph, Sec. 4.3):
+ *   the dialect with the smallest exact squared error over all 16, lowest id on
+ *   equal error; errors are summed in fp64 in element order.                        */
+typedef enum { BD_SELECT_TWO_STAGE = 0, BD_SELECT_MSE = 1 } bd_select;
+
+/* Which axis of the source the blocks run along.
+ * BD_AXIS_CONTIG:  source is [rows, K] with K contiguous (activations per token,
+ *                  weights per output channel, Q and K per head dimension).
+ * BD_AXIS_STRIDED: source is [K, rows] with `rows` contiguous and blocks made of 32
+ *                  consecutive source rows (the value matrix V, quantised along the
+ *                  token axis; Appendix "Quantization Dimension").  The result is the
+ *                  quantised TRANSPOSE: a [rows, K] operand.                         */
+typedef enum { BD_AXIS_CONTIG = 0, BD_AXIS_STRIDED = 1 } bd_axis;
+
+/* GEMM implementation choice (bd_set_gemm_impl). */
+typedef enum {
+    BD_GEMM_AUTO = 0,   /* by shape                                                    */
+    BD_GEMM_SIMT = 1,   /* CUDA-core kernel: exact integer in-block sums, any shape     */
+    BD_GEMM_TCGEN05 = 2 /* tensor-core kernel (block-scaled E4M3 MMA, TMEM accumulators) */
+} bd_gemm_impl;
+
+/* A quantised [rows, K] operand in the library's physical layout.  All three
+ * buffers are caller-allocated device memory of the sizes bd_qtensor_sizes
+ * returns; the library never frees them.  The layout is opaque (it is arranged
+ * for bulk copies into shared memory and for the tensor-core scale-factor
+ * format); bd_export_canonical converts it to the documented canonical layout. */
+typedef struct {
+    void *codes;   /* 4 bits per element                                  */
+    void *ids;     /* 4 bits per block                                    */
+    void *scales;  /* 8 bits per block: e + 127                           */
+    int64_t rows;
+    int64_t K;
+} bd_qtensor;
+
+/* Buffer sizes in bytes for a [rows, K] operand.  K must be a multiple of 32. */
+bd_status bd_qtensor_sizes(int64_t rows, int64_t K, size_t *codes_bytes, size_t *ids_bytes,
+                           size_t *scales_bytes);
+
+/* Offline weight quantisation (Sec. 3.3 "the optimal dialect for each block is
+ * precomputed").  W: [N, K] of `dtype`, row stride ldw elements, blocks along K.
+ * out->rows must be N and out->K must be K. */
+bd_status bd_quantize_weights(const void *W, bd_dtype dtype, int64_t N, int64_t K, int64_t ldw,
+                              bd_select select, bd_qtensor *out, void *stream);
+
+/* Online activation quantisation with the two-stage rule (Sec. 3.2, Sec. 3.3):
+ * per block absmax -> shared exponent, 5-bit truncated magnitudes, pair by rounded
+ * block maximum, dialect by beneficial-range counts, round-to-nearest (ties to the
+ * larger magnitude) onto the dialect's grid, 4-bit codes.
+ * BD_AXIS_CONTIG:  X is [M, K], row stride ldx.  out is [M, K].
+ * BD_AXIS_STRIDED: X is [K, M], row stride ldx.  out is [M, K] (the transpose).
+ * X and ldx*sizeof(element) must be 16-byte aligned. */
+bd_status bd_quantize_act(const void *X, bd_dtype dtype, int64_t M, int64_t K, int64_t ldx,
+                          bd_axis axis, bd_qtensor *out, void *stream);
+
+/* Y[M,N] = dq(A)[M,K] * dq(B)[N,K]^T (Sec. 3.3, Fig. 6).  ydtype is BD_F32 or BD_BF16
+ * (bf16 = round-to-nearest-even of the fp32 accumulator); ldy = row stride of Y in
+ * elements.  workspace: bd_gemm_workspace_size bytes, 256-byte aligned, or NULL when
+ * that size is 0. */
+bd_status bd_gemm_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes);
+bd_status bd_gemm(const bd_qtensor *A, const bd_qtensor *B, void *Y, bd_dtype ydtype, int64_t ldy,
+                  void *workspace, size_t workspace_bytes, void *stream);
+
+/* Batched product for attention (Appendix "Quantization Dimension"): `batch`
+ * independent products; operand b of A uses operand b / b_group of B (grouped-query
+ * attention shares one K/V head among b_group query heads).  A points to `batch`
+ * descriptors, B to batch / b_group descriptors (host arrays); Y + b * stride_y
+ * elements is product b. */
+bd_status bd_gemm_batched(const bd_qtensor *A, const bd_qtensor *B, int64_t batch, int64_t b_group,
+                          void *Y, bd_dtype ydtype, int64_t ldy, int64_t stride_y, void *workspace,
+                          size_t workspace_bytes, void *stream);
+
+/* The quantised linear layer: quantise X [M,K] online (two-stage rule), then
+ * Y = dq(X) * dq(Wq)^T.  The quantised activation lives only in `workspace`. */
+bd_status bd_linear_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes);
+bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx,
+                    const bd_qtensor *Wq, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace,
+                    size_t workspace_bytes, void *stream);
+
+/* Canonical layout (what is compared bit for bit with a reference):
+ *   codes  [rows][K/2]   byte j of a row: element 2j in bits 3:0, element 2j+1 in
+ *                        bits 7:4; nibble = sign << 3 | index (index ascending in
+ *                        magnitude, Sec. 3.3: the example value 10 has index 110b)
+ *   ids    [rows][K/32]  one byte per block, 0..15
+ *   scales [rows][K/32]  one byte per block, e + 127                               */
+bd_status bd_export_canonical(const bd_qtensor *q, uint8_t *codes, uint8_t *ids, uint8_t *scales,
+                              void *stream);
+bd_status bd_import_canonical(const uint8_t *codes, const uint8_t *ids, const uint8_t *scales,
+                              bd_qtensor *q, void *stream);
+
+/* out[rows][ld] (fp32) = sign * 0.5 * value[id][index] * 2^e (Sec. 3.3, Fig. 6). */
+bd_status bd_dequantize(const bd_qtensor *q, float *out, int64_t ld, void *stream);
+
+/* The DialectFP4 formatbook (Sec. 3.1, Fig. 4) as a HOST table: magnitudes in units
+ * of 0.5, ascending. */
+bd_status bd_get_formatbook(uint8_t out[16][8]);
+
+/* Synchronises `stream`, then returns and clears the device status word:
+ * BD_OK, BD_ERR_NONFINITE or BD_ERR_TIMEOUT (or BD_ERR_CUDA). */
+bd_status bd_poll_status(void *stream);
+
+bd_status bd_set_gemm_impl(bd_gemm_impl impl);
+/* Number of kernels this library has launched in this process (host counter). */
+uint64_t bd_launch_count(void);
+int bd_last_cuda_error(void);
+const char *bd_status_string(bd_status s);
+int bd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BD_H */

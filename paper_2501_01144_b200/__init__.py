@@ -1,0 +1,12 @@
+"""BlockDialect W4A4 quantized linear layer for B200: Python binding of libblockdialect.
+
+The binding marshals arguments only; every step runs in the CUDA library.
+Importing the package does not load the library; the first call does, and it
+raises if the shared object has not been built (there is no fallback path).
+"""
+from .binding import (  # noqa: F401
+    AXIS_CONTIG, AXIS_STRIDED, BF16, F16, F32, GEMM_AUTO, GEMM_SIMT, GEMM_TCGEN05, SELECT_MSE,
+    SELECT_TWO_STAGE, BdError, QTensor, build, dequantize, export_canonical, gemm, gemm_batched,
+    gemm_workspace_size, get_formatbook, import_canonical, launch_count, library_path, linear, linear_workspace_size,
+    load, poll_status, quantize_act, quantize_weights, set_gemm_impl, version,
+)

@@ -1,0 +1,257 @@
+"""ctypes binding of the C ABI in include/bd.h (same names without the bd_ prefix)."""
+import ctypes
+import os
+import subprocess
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libblockdialect.so")
+_SRC = os.path.join(_HERE, "csrc", "bd_lib.cu")
+
+F32, BF16, F16 = 0, 1, 2
+SELECT_TWO_STAGE, SELECT_MSE = 0, 1
+AXIS_CONTIG, AXIS_STRIDED = 0, 1
+GEMM_AUTO, GEMM_SIMT, GEMM_TCGEN05 = 0, 1, 2
+
+_TORCH_DTYPE = {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}
+
+_lib = None
+
+
+class BdError(RuntimeError):
+    def __init__(self, status, text):
+        super().__init__(f"libblockdialect: status {status}: {text}")
+        self.status = status
+
+
+class _CQTensor(ctypes.Structure):
+    _fields_ = [("codes", ctypes.c_void_p), ("ids", ctypes.c_void_p), ("scales", ctypes.c_void_p),
+                ("rows", ctypes.c_int64), ("K", ctypes.c_int64)]
+
+
+def library_path():
+    return _LIB_PATH
+
+
+def build(verbose=False):
+    """Compile the CUDA library in-tree for sm_100a."""
+    srcs = [os.path.join(_HERE, "csrc", f) for f in os.listdir(os.path.join(_HERE, "csrc"))]
+    if os.path.exists(_LIB_PATH) and all(os.path.getmtime(_LIB_PATH) >= os.path.getmtime(s) for s in srcs):
+        return _LIB_PATH
+    cmd = ["nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "-shared", "-Xcompiler", "-fPIC", "-o", _LIB_PATH, _SRC]
+    if verbose:
+        cmd.insert(1, "-Xptxas=-v")
+    subprocess.run(cmd, check=True)
+    return _LIB_PATH
+
+
+def load():
+    """Load the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise BdError(-1, f"{_LIB_PATH} is missing: run __graft_entry__.build() (nvcc, sm_100a) first")
+    lib = ctypes.CDLL(_LIB_PATH)
+    i64, vp, ci, sz = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    qp = ctypes.POINTER(_CQTensor)
+    szp = ctypes.POINTER(sz)
+    lib.bd_qtensor_sizes.argtypes = [i64, i64, szp, szp, szp]
+    lib.bd_quantize_weights.argtypes = [vp, ci, i64, i64, i64, ci, qp, vp]
+    lib.bd_quantize_act.argtypes = [vp, ci, i64, i64, i64, ci, qp, vp]
+    lib.bd_gemm_workspace_size.argtypes = [i64, i64, i64, szp]
+    lib.bd_gemm.argtypes = [qp, qp, vp, ci, i64, vp, sz, vp]
+    lib.bd_gemm_batched.argtypes = [qp, qp, i64, i64, vp, ci, i64, i64, vp, sz, vp]
+    lib.bd_linear_workspace_size.argtypes = [i64, i64, i64, szp]
+    lib.bd_linear.argtypes = [vp, ci, i64, i64, i64, qp, vp, ci, i64, vp, sz, vp]
+    lib.bd_export_canonical.argtypes = [qp, vp, vp, vp, vp]
+    lib.bd_import_canonical.argtypes = [vp, vp, vp, qp, vp]
+    lib.bd_dequantize.argtypes = [qp, vp, i64, vp]
+    lib.bd_get_formatbook.argtypes = [vp]
+    lib.bd_poll_status.argtypes = [vp]
+    lib.bd_set_gemm_impl.argtypes = [ci]
+    lib.bd_launch_count.restype = ctypes.c_uint64
+    lib.bd_status_string.argtypes = [ci]
+    lib.bd_status_string.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def _check(status):
+    if status:
+        lib = load()
+        text = lib.bd_status_string(status).decode()
+        if status == 5:
+            text += f" (cuda error {lib.bd_last_cuda_error()})"
+        raise BdError(status, text)
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def version():
+    return load().bd_version()
+
+
+def launch_count():
+    """Kernels launched by the library so far in this process."""
+    return int(load().bd_launch_count())
+
+
+def set_gemm_impl(impl):
+    _check(load().bd_set_gemm_impl(impl))
+
+
+def get_formatbook():
+    """The DialectFP4 table, 16 x 8, magnitudes in units of 0.5 (Sec. 3.1, Fig. 4)."""
+    buf = (ctypes.c_uint8 * 128)()
+    _check(load().bd_get_formatbook(buf))
+    return torch.tensor(list(buf), dtype=torch.uint8).reshape(16, 8)
+
+
+def poll_status(stream=None):
+    """Synchronise the stream and raise if a kernel recorded a device-side condition."""
+    _check(load().bd_poll_status(_stream(stream)))
+
+
+class QTensor:
+    """A quantised [rows, K] operand: three device byte buffers in the library's layout."""
+
+    def __init__(self, rows, K, device="cuda"):
+        c, i, s = (ctypes.c_size_t() for _ in range(3))
+        _check(load().bd_qtensor_sizes(rows, K, ctypes.byref(c), ctypes.byref(i), ctypes.byref(s)))
+        self.rows, self.K = rows, K
+        self.codes = torch.empty(c.value, dtype=torch.uint8, device=device)
+        self.ids = torch.empty(i.value, dtype=torch.uint8, device=device)
+        self.scales = torch.empty(s.value, dtype=torch.uint8, device=device)
+
+    def c_struct(self):
+        return _CQTensor(self.codes.data_ptr(), self.ids.data_ptr(), self.scales.data_ptr(), self.rows, self.K)
+
+    def nbytes(self):
+        return self.codes.numel() + self.ids.numel() + self.scales.numel()
+
+
+def _src(x):
+    if x.dtype not in _TORCH_DTYPE or x.dim() != 2 or x.stride(1) != 1 or not x.is_cuda:
+        raise ValueError("source must be a 2-D CUDA tensor of fp32/bf16/fp16 with a contiguous last axis")
+    return ctypes.c_void_p(x.data_ptr()), _TORCH_DTYPE[x.dtype], x.stride(0)
+
+
+def quantize_weights(W, select=SELECT_MSE, out=None, stream=None):
+    """Offline weight quantisation of W [N, K] along K (Sec. 3.3)."""
+    ptr, dt, ld = _src(W)
+    N, K = W.shape
+    out = out or QTensor(N, K, W.device)
+    cq = out.c_struct()
+    _check(load().bd_quantize_weights(ptr, dt, N, K, ld, select, ctypes.byref(cq), _stream(stream)))
+    return out
+
+
+def quantize_act(X, axis=AXIS_CONTIG, out=None, stream=None):
+    """Online two-stage quantisation (Sec. 3.2).  AXIS_CONTIG: X [M, K]; AXIS_STRIDED: X [K, M]."""
+    ptr, dt, ld = _src(X)
+    M, K = X.shape if axis == AXIS_CONTIG else (X.shape[1], X.shape[0])
+    out = out or QTensor(M, K, X.device)
+    cq = out.c_struct()
+    _check(load().bd_quantize_act(ptr, dt, M, K, ld, axis, ctypes.byref(cq), _stream(stream)))
+    return out
+
+
+def gemm_workspace_size(M, N, K):
+    b = ctypes.c_size_t()
+    _check(load().bd_gemm_workspace_size(M, N, K, ctypes.byref(b)))
+    return b.value
+
+
+def linear_workspace_size(M, N, K):
+    b = ctypes.c_size_t()
+    _check(load().bd_linear_workspace_size(M, N, K, ctypes.byref(b)))
+    return b.value
+
+
+def _ydtype(dtype):
+    if dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("output dtype must be float32 or bfloat16")
+    return _TORCH_DTYPE[dtype]
+
+
+def _ws(workspace, need, device):
+    if workspace is None and need:
+        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    ptr = ctypes.c_void_p(workspace.data_ptr() if workspace is not None else 0)
+    return workspace, ptr, (workspace.numel() if workspace is not None else 0)
+
+
+def gemm(A, B, out=None, dtype=torch.float32, workspace=None, stream=None):
+    """Y [M, N] = dq(A) dq(B)^T (Sec. 3.3, Fig. 6)."""
+    if out is None:
+        out = torch.empty(A.rows, B.rows, dtype=dtype, device=A.codes.device)
+    workspace, wptr, wbytes = _ws(workspace, gemm_workspace_size(A.rows, B.rows, A.K), A.codes.device)
+    ca, cb = A.c_struct(), B.c_struct()
+    _check(load().bd_gemm(ctypes.byref(ca), ctypes.byref(cb), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
+                          out.stride(0), wptr, wbytes, _stream(stream)))
+    return out
+
+
+def gemm_batched(As, Bs, b_group=1, out=None, dtype=torch.float32, workspace=None, stream=None):
+    """Batched product; A[b] pairs with B[b // b_group] (grouped-query attention)."""
+    batch = len(As)
+    M, N, K = As[0].rows, Bs[0].rows, As[0].K
+    if out is None:
+        out = torch.empty(batch, M, N, dtype=dtype, device=As[0].codes.device)
+    workspace, wptr, wbytes = _ws(workspace, gemm_workspace_size(M, N, K), As[0].codes.device)
+    ca = (_CQTensor * batch)(*[a.c_struct() for a in As])
+    cb = (_CQTensor * len(Bs))(*[b.c_struct() for b in Bs])
+    _check(load().bd_gemm_batched(ca, cb, batch, b_group, ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
+                                  out.stride(1), out.stride(0), wptr, wbytes, _stream(stream)))
+    return out
+
+
+def linear(X, Wq, out=None, dtype=torch.bfloat16, workspace=None, stream=None):
+    """The quantised linear layer: two-stage quantisation of X [M, K], then the product with Wq [N, K]."""
+    ptr, dt, ld = _src(X)
+    M, K = X.shape
+    if out is None:
+        out = torch.empty(M, Wq.rows, dtype=dtype, device=X.device)
+    workspace, wptr, wbytes = _ws(workspace, linear_workspace_size(M, Wq.rows, K), X.device)
+    cw = Wq.c_struct()
+    _check(load().bd_linear(ptr, dt, M, K, ld, ctypes.byref(cw), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
+                            out.stride(0), wptr, wbytes, _stream(stream)))
+    return out
+
+
+def export_canonical(q, stream=None):
+    """(codes [rows, K/2], ids [rows, K/32], scales [rows, K/32]) as uint8 CUDA tensors."""
+    dev = q.codes.device
+    codes = torch.empty(q.rows, q.K // 2, dtype=torch.uint8, device=dev)
+    ids = torch.empty(q.rows, q.K // 32, dtype=torch.uint8, device=dev)
+    scales = torch.empty(q.rows, q.K // 32, dtype=torch.uint8, device=dev)
+    cq = q.c_struct()
+    _check(load().bd_export_canonical(ctypes.byref(cq), ctypes.c_void_p(codes.data_ptr()),
+                                      ctypes.c_void_p(ids.data_ptr()), ctypes.c_void_p(scales.data_ptr()),
+                                      _stream(stream)))
+    return codes, ids, scales
+
+
+def import_canonical(codes, ids, scales, stream=None):
+    """Build a QTensor from canonical uint8 CUDA tensors."""
+    rows, K = codes.shape[0], codes.shape[1] * 2
+    q = QTensor(rows, K, codes.device)
+    cq = q.c_struct()
+    codes, ids, scales = codes.contiguous(), ids.contiguous(), scales.contiguous()
+    _check(load().bd_import_canonical(ctypes.c_void_p(codes.data_ptr()), ctypes.c_void_p(ids.data_ptr()),
+                                      ctypes.c_void_p(scales.data_ptr()), ctypes.byref(cq), _stream(stream)))
+    return q
+
+
+def dequantize(q, stream=None):
+    """fp32 [rows, K] values of a quantised operand (Sec. 3.3, Fig. 6)."""
+    out = torch.empty(q.rows, q.K, dtype=torch.float32, device=q.codes.device)
+    cq = q.c_struct()
+    _check(load().bd_dequantize(ctypes.byref(cq), ctypes.c_void_p(out.data_ptr()), out.stride(0), _stream(stream)))
+    return out

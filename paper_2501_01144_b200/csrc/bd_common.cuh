@@ -1,0 +1,176 @@
+// Shared definitions of the CUDA library: the DialectFP4 formatbook and the
+// tables derived from it, the physical storage layout, and the status word.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/bd.h"
+
+namespace bd {
+
+constexpr int kBlock = 32;          // elements per block along K (Sec. 3.1; Sec. 4.1 "Block size is 32")
+constexpr int kRowTile = 128;       // rows per scale/id atom
+constexpr int kBlocksPerAtom = 4;   // k-blocks per scale/id atom (128 elements of K)
+constexpr int kScaleAtomBytes = 512;
+constexpr int kIdAtomBytes = 256;
+
+// ---------------------------------------------------------------------------
+// DialectFP4 formatbook (Sec. 3.1, Fig. 4): 16 dialects x 8 magnitudes in units
+// of 0.5, ascending.  Eight pairs, one per possible rounded block maximum
+// 7.5 ... 4.0; the two members share the maximum (index 7) and differ in the
+// value at index 6, the even member holding the larger.  Dialect 4 is the one
+// the paper prints (0.5 * {0,1,2,3,4,6,10,13}); dialect 7 is FP4 E2M1.
+// Everything below (thresholds, ranges, decode tables) is computed from this
+// one table at compile time.
+// ---------------------------------------------------------------------------
+struct Formatbook {
+    uint8_t v[16][8];
+};
+constexpr Formatbook kBook = {{
+    {0, 1, 2, 3, 4, 6, 12, 15}, {0, 1, 2, 3, 4, 6, 10, 15},
+    {0, 1, 2, 3, 4, 6, 11, 14}, {0, 1, 2, 3, 4, 6, 9, 14},
+    {0, 1, 2, 3, 4, 6, 10, 13}, {0, 1, 2, 3, 4, 6, 8, 13},
+    {0, 1, 2, 3, 4, 6, 9, 12},  {0, 1, 2, 3, 4, 6, 8, 12},
+    {0, 1, 2, 3, 4, 6, 9, 11},  {0, 1, 2, 3, 4, 6, 8, 11},
+    {0, 1, 2, 3, 4, 6, 8, 10},  {0, 1, 2, 3, 4, 6, 7, 10},
+    {0, 1, 2, 3, 4, 6, 8, 9},   {0, 1, 2, 3, 4, 6, 7, 9},
+    {0, 1, 2, 3, 4, 5, 7, 8},   {0, 1, 2, 3, 4, 5, 6, 8},
+}};
+
+// Rounding thresholds on the 5-bit code q5 (units of 0.25): a code rounds to
+// index j or above exactly when q5 >= v[j-1] + v[j] (midpoint of two multiples
+// of 0.5, ties to the larger magnitude; Sec. 3.3).  Stored as a bit mask with
+// bit t set for each threshold t, so that index = popcount(mask & ((2 << q5) - 1)).
+constexpr uint32_t round_mask(int d) {
+    uint32_t m = 0;
+    for (int j = 1; j < 8; j++) m |= 1u << (kBook.v[d][j - 1] + kBook.v[d][j]);
+    return m;
+}
+
+// Beneficial ranges (Sec. 3.2, Fig. 5c) as bit masks over q5.
+//   even member: [ (dE + dO)/2 , (dE + max)/2 )   -> q5 in [dE + dO, dE + max)
+//   odd member:  [ (dO + next lower)/2 , (dE + dO)/2 ) -> q5 in [dO + v5, dE + dO)
+constexpr uint32_t range_bits(int lo, int hi) {
+    uint32_t m = 0;
+    for (int q = lo; q < hi && q < 32; q++) m |= 1u << q;
+    return m;
+}
+constexpr uint32_t even_range_mask(int p) {
+    return range_bits(kBook.v[2 * p][6] + kBook.v[2 * p + 1][6], kBook.v[2 * p][6] + kBook.v[2 * p][7]);
+}
+constexpr uint32_t odd_range_mask(int p) {
+    return range_bits(kBook.v[2 * p + 1][6] + kBook.v[2 * p + 1][5], kBook.v[2 * p][6] + kBook.v[2 * p + 1][6]);
+}
+
+// E4M3 encoding of the magnitude 0.5 * h, h in 0..15 (exact: four significant bits).
+constexpr uint8_t e4m3_of_half_units(int h) {
+    if (h == 0) return 0;
+    int msb = 0;
+    for (int b = 3; b >= 0; b--)
+        if (h >> b & 1) { msb = b; break; }
+    int exp_field = msb - 1 + 7;                           // value = 2^(msb-1) * 1.mmm
+    int mant = ((h << 3) >> msb) & 7;                      // three bits below the leading one
+    return (uint8_t)(exp_field << 3 | mant);
+}
+// Eight-byte decode tables of a dialect: byte i = operand byte of index i.
+constexpr uint64_t e4m3_lut(int d) {
+    uint64_t t = 0;
+    for (int i = 0; i < 8; i++) t |= (uint64_t)e4m3_of_half_units(kBook.v[d][i]) << (8 * i);
+    return t;
+}
+constexpr uint64_t int_lut(int d) {
+    uint64_t t = 0;
+    for (int i = 0; i < 8; i++) t |= (uint64_t)kBook.v[d][i] << (8 * i);
+    return t;
+}
+
+struct DeviceTables {
+    uint32_t round_mask[16];
+    uint32_t even_mask[8];
+    uint32_t odd_mask[8];
+    uint32_t e4m3_lo[16], e4m3_hi[16];
+    uint32_t int_lo[16], int_hi[16];
+};
+constexpr DeviceTables make_tables() {
+    DeviceTables t{};
+    for (int d = 0; d < 16; d++) {
+        t.round_mask[d] = round_mask(d);
+        t.e4m3_lo[d] = (uint32_t)e4m3_lut(d);
+        t.e4m3_hi[d] = (uint32_t)(e4m3_lut(d) >> 32);
+        t.int_lo[d] = (uint32_t)int_lut(d);
+        t.int_hi[d] = (uint32_t)(int_lut(d) >> 32);
+    }
+    for (int p = 0; p < 8; p++) {
+        t.even_mask[p] = even_range_mask(p);
+        t.odd_mask[p] = odd_range_mask(p);
+    }
+    return t;
+}
+constexpr DeviceTables kTables = make_tables();
+
+// ---------------------------------------------------------------------------
+// Physical layout of a quantised [rows, K] operand.
+//
+// codes: [rows][K/2] bytes, row-major.  Each aligned group of 8 elements is one
+//   little-endian 32-bit word w: the 3-bit index of element j sits in bits
+//   4j+2 .. 4j; the sign of element j sits in bit 8j+7 for j < 4 and in bit
+//   8(j-4)+3 for j >= 4.  With this order a word decodes to eight operand bytes
+//   with two byte-permute lookups (the masked word is the selector) and two
+//   and-or operations that move the signs into bit 7 of each byte.
+//
+// scales: atoms of 512 bytes covering 128 rows x 4 k-blocks, atom index
+//   kg * row_tiles + rt; inside an atom the byte of (row r, block b) is at
+//   (r % 32) * 16 + (r % 128 / 32) * 4 + b % 4: the order tcgen05.cp expects for
+//   block-scaled MMA scale factors (32 lanes x 16 bytes, four row groups side by
+//   side).  Padding entries hold 0.
+//
+// ids: atoms of 256 bytes in the same atom order; (row r, block b) is nibble
+//   b % 2 of byte (r % 128) * 2 + (b % 4) / 2.
+// ---------------------------------------------------------------------------
+__host__ __device__ inline int64_t row_tiles(int64_t rows) { return (rows + kRowTile - 1) / kRowTile; }
+__host__ __device__ inline int64_t k_groups(int64_t K) { return (K / kBlock + kBlocksPerAtom - 1) / kBlocksPerAtom; }
+
+__host__ __device__ inline int64_t scale_offset(int64_t rows, int64_t r, int64_t b) {
+    int64_t atom = (b / kBlocksPerAtom) * row_tiles(rows) + r / kRowTile;
+    int rr = (int)(r % kRowTile);
+    return atom * kScaleAtomBytes + (rr % 32) * 16 + (rr / 32) * 4 + (int)(b % kBlocksPerAtom);
+}
+__host__ __device__ inline int64_t id_byte_offset(int64_t rows, int64_t r, int64_t b) {
+    int64_t atom = (b / kBlocksPerAtom) * row_tiles(rows) + r / kRowTile;
+    return atom * kIdAtomBytes + (r % kRowTile) * 2 + (b % kBlocksPerAtom) / 2;
+}
+
+// Decode one code word into eight operand bytes (lo = elements 0..3, hi = 4..7)
+// through the dialect's eight-byte table.
+__device__ __forceinline__ void decode_word(uint32_t w, uint32_t lut_lo, uint32_t lut_hi, uint32_t &lo,
+                                            uint32_t &hi) {
+    uint32_t sel = w & 0x77777777u;
+    lo = (w & 0x80808080u) | __byte_perm(lut_lo, lut_hi, sel);
+    hi = ((w << 4) & 0x80808080u) | __byte_perm(lut_lo, lut_hi, sel >> 16);
+}
+
+// Index and sign of element j (0..7) of a code word.
+__host__ __device__ inline uint32_t word_index(uint32_t w, int j) { return (w >> (4 * j)) & 7u; }
+__host__ __device__ inline uint32_t word_sign(uint32_t w, int j) {
+    return (w >> (j < 4 ? 8 * j + 7 : 8 * (j - 4) + 3)) & 1u;
+}
+__host__ __device__ inline uint32_t word_insert(uint32_t idx, uint32_t sign, int j) {
+    return idx << (4 * j) | sign << (j < 4 ? 8 * j + 7 : 8 * (j - 4) + 3);
+}
+
+// Bits of the device status word (defined in quantize.cuh; the library is one
+// translation unit).  bd_poll_status reads and clears it.
+enum : uint32_t { kStatusNonfinite = 1u, kStatusTimeout = 2u };
+
+// Launch helpers shared by the translation units.
+struct QView {                 // a qtensor as kernels see it
+    uint8_t *codes;
+    uint8_t *ids;
+    uint8_t *scales;
+    int64_t rows, K;
+};
+inline QView view_of(const bd_qtensor *q) {
+    return QView{(uint8_t *)q->codes, (uint8_t *)q->ids, (uint8_t *)q->scales, q->rows, q->K};
+}
+
+}  // namespace bd

@@ -1,0 +1,309 @@
+// libblockdialect: the extern "C" entry points declared in include/bd.h.
+// Host-side validation and kernel dispatch only; all arithmetic is in the kernels.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "bd_common.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include "quantize.cuh"
+
+using namespace bd;
+
+namespace {
+
+int g_last_cuda_error = 0;
+uint64_t g_launches = 0;
+bd_gemm_impl g_gemm_impl = BD_GEMM_AUTO;
+
+bd_status cuda_result(cudaError_t e) {
+    if (e == cudaSuccess) return BD_OK;
+    g_last_cuda_error = (int)e;
+    return BD_ERR_CUDA;
+}
+bd_status launch_result(int kernels = 1) {
+    g_launches += (uint64_t)kernels;
+    return cuda_result(cudaGetLastError());
+}
+
+bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+
+bd_status check_qtensor(const bd_qtensor *q) {
+    if (!q || !q->codes || !q->ids || !q->scales) return BD_ERR_INVALID_ARG;
+    if (q->rows <= 0 || q->K <= 0) return BD_ERR_INVALID_ARG;
+    if (q->K % kBlock) return BD_ERR_SHAPE;
+    if (!aligned16(q->codes) || !aligned16(q->ids) || !aligned16(q->scales)) return BD_ERR_ALIGN;
+    return BD_OK;
+}
+
+int elem_bytes(bd_dtype dt) { return dt == BD_F32 ? 4 : 2; }
+
+unsigned grid_for(int64_t threads, int block) { return (unsigned)((threads + block - 1) / block); }
+
+template <int SELECT, bool WC, bool WE>
+bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out, uint8_t *e4m3, cudaStream_t st) {
+    const int nb = (int)(out.K / kBlock), nb_pad = (int)k_groups(out.K) * kBlocksPerAtom;
+    const int64_t rows_pad = row_tiles(out.rows) * kRowTile;
+    const unsigned grid = grid_for(rows_pad * nb_pad, 256);
+    switch (dt) {
+        case BD_F32: quantize_contig_kernel<BD_F32, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad); break;
+        case BD_BF16: quantize_contig_kernel<BD_BF16, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad); break;
+        case BD_F16: quantize_contig_kernel<BD_F16, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad); break;
+        default: return BD_ERR_INVALID_ARG;
+    }
+    return launch_result();
+}
+
+bd_status check_source(const void *X, bd_dtype dt, int64_t rows, int64_t K, int64_t ld, int64_t min_ld) {
+    if (!X || rows <= 0 || K <= 0) return BD_ERR_INVALID_ARG;
+    if (dt != BD_F32 && dt != BD_BF16 && dt != BD_F16) return BD_ERR_INVALID_ARG;
+    if (K % kBlock || ld < min_ld) return BD_ERR_SHAPE;
+    if (!aligned16(X) || (ld * elem_bytes(dt)) % 16) return BD_ERR_ALIGN;
+    return BD_OK;
+}
+
+template <typename OutT>
+bd_status launch_simt(const QView &A, const QView &B, void *Y, int64_t ldy, cudaStream_t st) {
+    dim3 grid((unsigned)((B.rows + kSimtTile - 1) / kSimtTile), (unsigned)((A.rows + kSimtTile - 1) / kSimtTile));
+    gemm_simt_kernel<OutT><<<grid, 256, 0, st>>>(A, B, (OutT *)Y, ldy);
+    return launch_result();
+}
+
+bool use_tc(int64_t M, int64_t N, int64_t K) {
+    if (g_gemm_impl == BD_GEMM_SIMT) return false;
+    if (g_gemm_impl == BD_GEMM_TCGEN05) return true;
+    return tc_supported(M, N, K) && M >= 64;
+}
+
+bd_status check_gemm(const bd_qtensor *A, const bd_qtensor *B, const void *Y, bd_dtype ydt, int64_t ldy) {
+    bd_status s = check_qtensor(A);
+    if (s) return s;
+    s = check_qtensor(B);
+    if (s) return s;
+    if (!Y || (ydt != BD_F32 && ydt != BD_BF16)) return BD_ERR_INVALID_ARG;
+    if (A->K != B->K || ldy < B->rows) return BD_ERR_SHAPE;
+    return BD_OK;
+}
+
+bd_status gemm_dispatch(const QView &A, const QView &B, void *Y, bd_dtype ydt, int64_t ldy, void *ws, size_t ws_bytes,
+                        cudaStream_t st) {
+    if (use_tc(A.rows, B.rows, A.K)) {
+        if (!tc_supported(A.rows, B.rows, A.K)) return BD_ERR_UNSUPPORTED;
+        size_t need = tc_gemm_workspace(A.rows, B.rows, A.K);
+        if (need && (!ws || ws_bytes < need)) return BD_ERR_WORKSPACE;
+        if (need && ((uintptr_t)ws & 255u)) return BD_ERR_ALIGN;
+        // decode both operands to plain operand-byte matrices, then the block-scaled MMA kernel
+        uint8_t *a8 = (uint8_t *)ws;
+        uint8_t *b8 = a8 + tc_operand_bytes(A.rows, A.K);
+        const int nb = (int)(A.K / kBlock);
+        decode_e4m3_kernel<<<grid_for(A.rows * nb, 256), 256, 0, st>>>(A, a8, nb);
+        decode_e4m3_kernel<<<grid_for(B.rows * nb, 256), 256, 0, st>>>(B, b8, nb);
+        bd_status s = launch_result(2);
+        if (s) return s;
+        g_launches += 1;
+        return cuda_result(tc_gemm(a8, A.scales, A.rows, b8, B.scales, B.rows, A.K, Y, ydt == BD_BF16, ldy, st));
+    }
+    if (ydt == BD_F32) return launch_simt<float>(A, B, Y, ldy, st);
+    return launch_simt<__nv_bfloat16>(A, B, Y, ldy, st);
+}
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+}  // namespace
+
+extern "C" {
+
+bd_status bd_qtensor_sizes(int64_t rows, int64_t K, size_t *codes_bytes, size_t *ids_bytes, size_t *scales_bytes) {
+    if (rows <= 0 || K <= 0) return BD_ERR_INVALID_ARG;
+    if (K % kBlock) return BD_ERR_SHAPE;
+    const size_t atoms = (size_t)(row_tiles(rows) * k_groups(K));
+    if (codes_bytes) *codes_bytes = (size_t)rows * (size_t)(K / 2);
+    if (ids_bytes) *ids_bytes = atoms * kIdAtomBytes;
+    if (scales_bytes) *scales_bytes = atoms * kScaleAtomBytes;
+    return BD_OK;
+}
+
+bd_status bd_quantize_weights(const void *W, bd_dtype dtype, int64_t N, int64_t K, int64_t ldw, bd_select select,
+                              bd_qtensor *out, void *stream) {
+    bd_status s = check_source(W, dtype, N, K, ldw, K);
+    if (s) return s;
+    s = check_qtensor(out);
+    if (s) return s;
+    if (out->rows != N || out->K != K) return BD_ERR_SHAPE;
+    QView v = view_of(out);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (select == BD_SELECT_MSE) return launch_contig<BD_SELECT_MSE, true, false>(W, dtype, ldw, v, nullptr, st);
+    if (select == BD_SELECT_TWO_STAGE) return launch_contig<BD_SELECT_TWO_STAGE, true, false>(W, dtype, ldw, v, nullptr, st);
+    return BD_ERR_INVALID_ARG;
+}
+
+bd_status bd_quantize_act(const void *X, bd_dtype dtype, int64_t M, int64_t K, int64_t ldx, bd_axis axis,
+                          bd_qtensor *out, void *stream) {
+    if (axis != BD_AXIS_CONTIG && axis != BD_AXIS_STRIDED) return BD_ERR_INVALID_ARG;
+    bd_status s = check_source(X, dtype, M, K, ldx, axis == BD_AXIS_CONTIG ? K : M);
+    if (s) return s;
+    s = check_qtensor(out);
+    if (s) return s;
+    if (out->rows != M || out->K != K) return BD_ERR_SHAPE;
+    QView v = view_of(out);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (axis == BD_AXIS_CONTIG) return launch_contig<BD_SELECT_TWO_STAGE, true, false>(X, dtype, ldx, v, nullptr, st);
+    const int nb = (int)(K / kBlock), nb_pad = (int)k_groups(K) * kBlocksPerAtom;
+    const int64_t rows_pad = row_tiles(M) * kRowTile;
+    const unsigned grid = grid_for(rows_pad * (nb_pad / 2), 256);
+    switch (dtype) {
+        case BD_F32: quantize_strided_kernel<BD_F32><<<grid, 256, 0, st>>>(X, ldx, v, rows_pad, nb, nb_pad); break;
+        case BD_BF16: quantize_strided_kernel<BD_BF16><<<grid, 256, 0, st>>>(X, ldx, v, rows_pad, nb, nb_pad); break;
+        default: quantize_strided_kernel<BD_F16><<<grid, 256, 0, st>>>(X, ldx, v, rows_pad, nb, nb_pad); break;
+    }
+    return launch_result();
+}
+
+bd_status bd_gemm_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes) {
+    if (!bytes || M <= 0 || N <= 0 || K <= 0) return BD_ERR_INVALID_ARG;
+    if (K % kBlock) return BD_ERR_SHAPE;
+    *bytes = tc_supported(M, N, K) ? tc_gemm_workspace(M, N, K) : 0;
+    return BD_OK;
+}
+
+bd_status bd_gemm(const bd_qtensor *A, const bd_qtensor *B, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace,
+                  size_t workspace_bytes, void *stream) {
+    bd_status s = check_gemm(A, B, Y, ydtype, ldy);
+    if (s) return s;
+    return gemm_dispatch(view_of(A), view_of(B), Y, ydtype, ldy, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+bd_status bd_gemm_batched(const bd_qtensor *A, const bd_qtensor *B, int64_t batch, int64_t b_group, void *Y,
+                          bd_dtype ydtype, int64_t ldy, int64_t stride_y, void *workspace, size_t workspace_bytes,
+                          void *stream) {
+    if (!A || !B || batch <= 0 || b_group <= 0 || batch % b_group) return BD_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < batch; i++) {
+        bd_status s = check_gemm(&A[i], &B[i / b_group], Y, ydtype, ldy);
+        if (s) return s;
+    }
+    const int ysz = ydtype == BD_F32 ? 4 : 2;
+    for (int64_t i = 0; i < batch; i++) {
+        bd_status s = gemm_dispatch(view_of(&A[i]), view_of(&B[i / b_group]), (char *)Y + i * stride_y * ysz, ydtype,
+                                    ldy, workspace, workspace_bytes, (cudaStream_t)stream);
+        if (s) return s;
+    }
+    return BD_OK;
+}
+
+bd_status bd_linear_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes) {
+    if (!bytes || M <= 0 || N <= 0 || K <= 0) return BD_ERR_INVALID_ARG;
+    if (K % kBlock) return BD_ERR_SHAPE;
+    size_t c, i, s;
+    bd_qtensor_sizes(M, K, &c, &i, &s);
+    size_t gemm_ws = tc_supported(M, N, K) ? tc_gemm_workspace(M, N, K) : 0;
+    *bytes = align256(c) + align256(i) + align256(s) + align256(gemm_ws);
+    return BD_OK;
+}
+
+bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, const bd_qtensor *Wq, void *Y,
+                    bd_dtype ydtype, int64_t ldy, void *workspace, size_t workspace_bytes, void *stream) {
+    bd_status s = check_source(X, xdtype, M, K, ldx, K);
+    if (s) return s;
+    s = check_qtensor(Wq);
+    if (s) return s;
+    if (Wq->K != K || ldy < Wq->rows) return BD_ERR_SHAPE;
+    if (!Y || (ydtype != BD_F32 && ydtype != BD_BF16)) return BD_ERR_INVALID_ARG;
+    size_t need;
+    bd_linear_workspace_size(M, Wq->rows, K, &need);
+    if (!workspace || workspace_bytes < need) return BD_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 255u) return BD_ERR_ALIGN;
+    size_t c, i, sc;
+    bd_qtensor_sizes(M, K, &c, &i, &sc);
+    char *p = (char *)workspace;
+    bd_qtensor xq{p, p + align256(c), p + align256(c) + align256(i), M, K};
+    char *gemm_ws = p + align256(c) + align256(i) + align256(sc);
+    cudaStream_t st = (cudaStream_t)stream;
+    s = launch_contig<BD_SELECT_TWO_STAGE, true, false>(X, xdtype, ldx, view_of(&xq), nullptr, st);
+    if (s) return s;
+    return gemm_dispatch(view_of(&xq), view_of(Wq), Y, ydtype, ldy, gemm_ws, need - (size_t)(gemm_ws - p), st);
+}
+
+bd_status bd_export_canonical(const bd_qtensor *q, uint8_t *codes, uint8_t *ids, uint8_t *scales, void *stream) {
+    bd_status s = check_qtensor(q);
+    if (s) return s;
+    if (!codes || !ids || !scales) return BD_ERR_INVALID_ARG;
+    if (!aligned16(codes)) return BD_ERR_ALIGN;
+    const int nb = (int)(q->K / kBlock);
+    export_canonical_kernel<<<grid_for(q->rows * nb, 256), 256, 0, (cudaStream_t)stream>>>(view_of(q), codes, ids,
+                                                                                          scales, nb);
+    return launch_result();
+}
+
+bd_status bd_import_canonical(const uint8_t *codes, const uint8_t *ids, const uint8_t *scales, bd_qtensor *q,
+                              void *stream) {
+    bd_status s = check_qtensor(q);
+    if (s) return s;
+    if (!codes || !ids || !scales) return BD_ERR_INVALID_ARG;
+    if (!aligned16(codes)) return BD_ERR_ALIGN;
+    const int nb = (int)(q->K / kBlock), nb_pad = (int)k_groups(q->K) * kBlocksPerAtom;
+    const int64_t rows_pad = row_tiles(q->rows) * kRowTile;
+    import_canonical_kernel<<<grid_for(rows_pad * nb_pad, 256), 256, 0, (cudaStream_t)stream>>>(
+        codes, ids, scales, view_of(q), rows_pad, nb, nb_pad);
+    return launch_result();
+}
+
+bd_status bd_dequantize(const bd_qtensor *q, float *out, int64_t ld, void *stream) {
+    bd_status s = check_qtensor(q);
+    if (s) return s;
+    if (!out) return BD_ERR_INVALID_ARG;
+    if (ld < q->K) return BD_ERR_SHAPE;
+    const int nb = (int)(q->K / kBlock);
+    dequantize_kernel<<<grid_for(q->rows * nb, 256), 256, 0, (cudaStream_t)stream>>>(view_of(q), out, ld, nb);
+    return launch_result();
+}
+
+bd_status bd_get_formatbook(uint8_t out[16][8]) {
+    if (!out) return BD_ERR_INVALID_ARG;
+    for (int d = 0; d < 16; d++)
+        for (int i = 0; i < 8; i++) out[d][i] = kBook.v[d][i];
+    return BD_OK;
+}
+
+bd_status bd_poll_status(void *stream) {
+    bd_status s = cuda_result(cudaStreamSynchronize((cudaStream_t)stream));
+    if (s) return s;
+    uint32_t word = 0, zero = 0;
+    s = cuda_result(cudaMemcpyFromSymbol(&word, g_status_word, sizeof(word)));
+    if (s) return s;
+    if (word) {
+        s = cuda_result(cudaMemcpyToSymbol(g_status_word, &zero, sizeof(zero)));
+        if (s) return s;
+    }
+    if (word & kStatusTimeout) return BD_ERR_TIMEOUT;
+    if (word & kStatusNonfinite) return BD_ERR_NONFINITE;
+    return BD_OK;
+}
+
+bd_status bd_set_gemm_impl(bd_gemm_impl impl) {
+    if (impl != BD_GEMM_AUTO && impl != BD_GEMM_SIMT && impl != BD_GEMM_TCGEN05) return BD_ERR_INVALID_ARG;
+    g_gemm_impl = impl;
+    return BD_OK;
+}
+
+uint64_t bd_launch_count(void) { return g_launches; }
+
+int bd_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char *bd_status_string(bd_status s) {
+    switch (s) {
+        case BD_OK: return "ok";
+        case BD_ERR_INVALID_ARG: return "invalid argument";
+        case BD_ERR_SHAPE: return "shape error (K must be a multiple of 32; operand shapes must agree)";
+        case BD_ERR_ALIGN: return "pointer or leading dimension not 16-byte aligned";
+        case BD_ERR_UNSUPPORTED: return "unsupported combination";
+        case BD_ERR_CUDA: return "CUDA error (see bd_last_cuda_error)";
+        case BD_ERR_NONFINITE: return "non-finite input met by a quantizer";
+        case BD_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        case BD_ERR_WORKSPACE: return "workspace missing or too small";
+    }
+    return "unknown status";
+}
+
+int bd_version(void) { return 100; }
+
+}  // extern "C"

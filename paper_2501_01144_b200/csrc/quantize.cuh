@@ -1,0 +1,396 @@
+// BlockDialect quantizer kernels: one thread owns one block of 32 elements.
+//
+// Per block (Sec. 3.2 preprocessing, two-stage selection; Sec. 3.3 rounding):
+//   amax  -> shared exponent e = floor(log2 amax) - 2 (kept >= -127)
+//   q5[k] = floor(4 * |x_k| * 2^-e)            (3 integer + 2 fraction bits, truncated)
+//   pair  = the dialect pair whose maximum equals (max q5 + 1) >> 1 (saturated at 15)
+//   id    = even member unless more elements fall in the odd member's beneficial range
+//   idx_k = number of rounding thresholds of dialect id that are <= q5[k]
+// All decisions are integer; the only floating-point step is an exact
+// power-of-two scaling followed by truncation (fma with round-toward-zero onto 2^23).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "bd_common.cuh"
+
+namespace bd {
+
+__device__ uint32_t g_status_word = 0;
+
+__constant__ DeviceTables c_tables = kTables;
+
+// Tables in shared memory: 32-bit words, at most 32 per table group, so that any
+// mix of per-thread indices is free of bank conflicts (one word per bank).
+struct SmemTables {
+    uint32_t round_mask[16];
+    uint32_t even_mask[8];
+    uint32_t odd_mask[8];
+    uint32_t e4m3_lo[16], e4m3_hi[16];
+};
+__device__ __forceinline__ void load_tables(SmemTables &s) {
+    for (int i = threadIdx.x; i < 16; i += blockDim.x) {
+        s.round_mask[i] = c_tables.round_mask[i];
+        s.e4m3_lo[i] = c_tables.e4m3_lo[i];
+        s.e4m3_hi[i] = c_tables.e4m3_hi[i];
+        if (i < 8) {
+            s.even_mask[i] = c_tables.even_mask[i];
+            s.odd_mask[i] = c_tables.odd_mask[i];
+        }
+    }
+    __syncthreads();
+}
+
+// ---- loading 32 elements of a block as fp32 bit patterns -------------------
+template <int DT>
+struct Loader;
+template <>
+struct Loader<BD_F32> {
+    static constexpr int kElemBytes = 4;
+    __device__ static void contiguous(const void *p, uint32_t (&bits)[32]) {
+        const uint4 *q = (const uint4 *)p;
+#pragma unroll
+        for (int i = 0; i < 8; i++) {
+            uint4 u = __ldg(q + i);
+            bits[4 * i] = u.x; bits[4 * i + 1] = u.y; bits[4 * i + 2] = u.z; bits[4 * i + 3] = u.w;
+        }
+    }
+    __device__ static uint32_t one(const void *p) { return __ldg((const uint32_t *)p); }
+};
+template <>
+struct Loader<BD_BF16> {
+    static constexpr int kElemBytes = 2;
+    __device__ static void contiguous(const void *p, uint32_t (&bits)[32]) {
+        const uint4 *q = (const uint4 *)p;
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            uint4 u = __ldg(q + i);
+            uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                bits[8 * i + 2 * j] = w[j] << 16;
+                bits[8 * i + 2 * j + 1] = w[j] & 0xffff0000u;
+            }
+        }
+    }
+    __device__ static uint32_t one(const void *p) { return (uint32_t)__ldg((const uint16_t *)p) << 16; }
+};
+template <>
+struct Loader<BD_F16> {
+    static constexpr int kElemBytes = 2;
+    __device__ static uint32_t cvt(uint16_t h) { return __float_as_uint(__half2float(__ushort_as_half(h))); }
+    __device__ static void contiguous(const void *p, uint32_t (&bits)[32]) {
+        const uint4 *q = (const uint4 *)p;
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            uint4 u = __ldg(q + i);
+            uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int j = 0; j < 4; j++) {
+                bits[8 * i + 2 * j] = cvt((uint16_t)(w[j] & 0xffffu));
+                bits[8 * i + 2 * j + 1] = cvt((uint16_t)(w[j] >> 16));
+            }
+        }
+    }
+    __device__ static uint32_t one(const void *p) { return cvt(__ldg((const uint16_t *)p)); }
+};
+
+// floor(|x| * 2^(2-e)) for |x| given as fp32 bits (sign cleared).  eadj = max(biased
+// exponent of the block maximum, 2), so that e = eadj - 129.
+struct Scaler {
+    float s1, s2;
+    bool two_step;
+    __device__ explicit Scaler(uint32_t eadj) {
+        two_step = eadj < 4;                                     // 2^(131-eadj) would overflow fp32
+        s1 = two_step ? 18446744073709551616.0f /* 2^64 */ : __uint_as_float((258u - eadj) << 23);
+        s2 = __uint_as_float((two_step ? 194u - eadj : 127u) << 23);   // 2^(67-eadj) or 1
+    }
+    __device__ __forceinline__ uint32_t q5(uint32_t abits) const {
+        float a = __uint_as_float(abits);
+        float t = two_step ? __fmaf_rz(a * s1, s2, 8388608.0f) : __fmaf_rz(a, s1, 8388608.0f);
+        return __float_as_uint(t) & 63u;
+    }
+};
+
+struct BlockResult {
+    uint32_t words[4];
+    uint32_t id;
+    uint32_t scale;   // e + 127
+};
+
+// Element rounding and packing for a chosen dialect.
+__device__ __forceinline__ void encode_block(const uint32_t (&bits)[32], const Scaler &sc, uint32_t mask,
+                                             uint32_t (&words)[4]) {
+#pragma unroll
+    for (int w = 0; w < 4; w++) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            uint32_t b = bits[8 * w + j];
+            uint32_t q = sc.q5(b & 0x7fffffffu);
+            uint32_t idx = __popc(mask & ((2u << q) - 1u));
+            word |= word_insert(idx, b >> 31, j);
+        }
+        words[w] = word;
+    }
+}
+
+// Two-stage rule (Sec. 3.2).
+__device__ __forceinline__ BlockResult quantize_two_stage(const uint32_t (&bits)[32], const SmemTables &tab,
+                                                          bool &nonfinite) {
+    uint32_t amax = 0;
+#pragma unroll
+    for (int k = 0; k < 32; k++) amax = max(amax, bits[k] & 0x7fffffffu);
+    nonfinite = amax >= 0x7f800000u;
+    uint32_t eadj = max(amax >> 23, 2u);
+    Scaler sc(eadj);
+    uint32_t m5 = sc.q5(amax);
+    uint32_t max_hu = min(15u, (m5 + 1u) >> 1);
+    uint32_t pair = min(7u, 15u - max_hu);                       // pair maxima are 15 - pair
+    uint32_t em = tab.even_mask[pair], om = tab.odd_mask[pair];
+    int balance = 0;
+#pragma unroll
+    for (int k = 0; k < 32; k++) {
+        uint32_t q = sc.q5(bits[k] & 0x7fffffffu);
+        balance += (int)((em >> q) & 1u) - (int)((om >> q) & 1u);
+    }
+    BlockResult r;
+    r.id = 2u * pair + (balance < 0 ? 1u : 0u);
+    r.scale = eadj - 2u;                                         // (eadj - 129) + 127
+    encode_block(bits, sc, tab.round_mask[r.id], r.words);
+    return r;
+}
+
+// Exact-MSE rule (Sec. 3.2 first paragraph; Sec. 4.3): all 16 dialects, squared
+// error against the untruncated scaled magnitude, fp64, element order, no
+// contraction; the lowest id wins equal sums.
+__device__ __forceinline__ BlockResult quantize_mse(const uint32_t (&bits)[32], const SmemTables &tab,
+                                                    bool &nonfinite) {
+    uint32_t amax = 0;
+#pragma unroll
+    for (int k = 0; k < 32; k++) amax = max(amax, bits[k] & 0x7fffffffu);
+    nonfinite = amax >= 0x7f800000u;
+    uint32_t eadj = max(amax >> 23, 2u);
+    Scaler sc(eadj);
+    // 2^-e as a double: e = eadj - 129  ->  biased double exponent 1023 - e
+    double inv = __longlong_as_double((long long)(1023 + 129 - (int)eadj) << 52);
+    uint32_t best = 0;
+    double best_err = __longlong_as_double(0x7ff0000000000000LL);
+    for (uint32_t d = 0; d < 16; d++) {
+        uint32_t mask = tab.round_mask[d];
+        uint64_t lut = (uint64_t)c_tables.int_hi[d] << 32 | c_tables.int_lo[d];
+        double err = 0.0;
+#pragma unroll
+        for (int k = 0; k < 32; k++) {
+            uint32_t a = bits[k] & 0x7fffffffu;
+            uint32_t idx = __popc(mask & ((2u << sc.q5(a)) - 1u));
+            double h = (double)((lut >> (8 * idx)) & 0xff);
+            double t = __dsub_rn(__dmul_rn((double)__uint_as_float(a), inv), __dmul_rn(0.5, h));
+            err = __dadd_rn(err, __dmul_rn(t, t));
+        }
+        if (err < best_err) {
+            best_err = err;
+            best = d;
+        }
+    }
+    BlockResult r;
+    r.id = best;
+    r.scale = eadj - 2u;
+    encode_block(bits, sc, tab.round_mask[best], r.words);
+    return r;
+}
+
+// ---------------------------------------------------------------------------
+// Contiguous-axis quantizer.  Thread t of the grid owns block (r, b) with
+// t = r * nb_pad + b, nb_pad = 4 * k_groups: four neighbouring lanes share one
+// row and one scale/id atom, so they merge their scale bytes into one 32-bit
+// store and their id nibbles into one 16-bit store.  Threads past the real rows
+// or blocks write the zero padding of the atoms.
+// Optional second output: the decoded operand bytes (E4M3 of 0.5 * value, sign in
+// bit 7) as a plain [rows][K] byte matrix, the form the tensor-core GEMM loads.
+// ---------------------------------------------------------------------------
+template <int DT, int SELECT, bool WRITE_CODES, bool WRITE_E4M3>
+__global__ void __launch_bounds__(256) quantize_contig_kernel(const void *__restrict__ X, int64_t ld, QView out,
+                                                              uint8_t *__restrict__ e4m3, int64_t rows_pad,
+                                                              int nb, int nb_pad) {
+    __shared__ SmemTables tab;
+    load_tables(tab);
+    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= rows_pad * nb_pad) return;                          // whole groups of 4 lanes leave together
+    int64_t r = t / nb_pad;
+    int b = (int)(t - r * nb_pad);
+    bool valid = r < out.rows && b < nb;
+    BlockResult res;
+    res.id = 0; res.scale = 0;
+    res.words[0] = res.words[1] = res.words[2] = res.words[3] = 0;
+    if (valid) {
+        uint32_t bits[32];
+        Loader<DT>::contiguous((const char *)X + (r * ld + (int64_t)b * 32) * Loader<DT>::kElemBytes, bits);
+        bool nonfinite;
+        if (SELECT == BD_SELECT_MSE) res = quantize_mse(bits, tab, nonfinite);
+        else res = quantize_two_stage(bits, tab, nonfinite);
+        if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
+        if (WRITE_CODES)
+            *(uint4 *)(out.codes + r * (out.K / 2) + (int64_t)b * 16) =
+                make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
+        if (WRITE_E4M3) {
+            uint32_t lo = tab.e4m3_lo[res.id], hi = tab.e4m3_hi[res.id];
+            uint32_t o[8];
+#pragma unroll
+            for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, o[2 * w], o[2 * w + 1]);
+            uint4 *dst = (uint4 *)(e4m3 + r * out.K + (int64_t)b * 32);
+            dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+            dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+        }
+    }
+    // merge the four lanes of a k-group (lane & 3 = b % 4)
+    uint32_t sc = res.scale << (8 * (b & 3));
+    uint32_t idn = res.id << (4 * (b & 3));
+    sc |= __shfl_xor_sync(0xffffffffu, sc, 1);
+    idn |= __shfl_xor_sync(0xffffffffu, idn, 1);
+    sc |= __shfl_xor_sync(0xffffffffu, sc, 2);
+    idn |= __shfl_xor_sync(0xffffffffu, idn, 2);
+    if ((b & 3) == 0) {
+        *(uint32_t *)(out.scales + scale_offset(out.rows, r, b)) = sc;
+        if (WRITE_CODES) *(uint16_t *)(out.ids + id_byte_offset(out.rows, r, b)) = (uint16_t)idn;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Strided-axis quantizer (the value matrix V, blocks along the token axis).
+// Source X is [K, rows] with `rows` contiguous; thread t owns output row
+// r = t % rows_pad and the pair of blocks (2*bp, 2*bp+1), bp = t / rows_pad, so
+// that consecutive lanes read consecutive addresses and each id byte has one
+// writer.
+// ---------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(256) quantize_strided_kernel(const void *__restrict__ X, int64_t ld, QView out,
+                                                               int64_t rows_pad, int nb, int nb_pad) {
+    __shared__ SmemTables tab;
+    load_tables(tab);
+    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= rows_pad * (nb_pad / 2)) return;
+    int64_t bp = t / rows_pad;
+    int64_t r = t - bp * rows_pad;
+    uint32_t idbyte = 0;
+    for (int h = 0; h < 2; h++) {
+        int b = (int)(2 * bp + h);
+        BlockResult res;
+        res.id = 0; res.scale = 0;
+        if (r < out.rows && b < nb) {
+            uint32_t bits[32];
+#pragma unroll
+            for (int k = 0; k < 32; k++)
+                bits[k] = Loader<DT>::one((const char *)X + (((int64_t)b * 32 + k) * ld + r) * Loader<DT>::kElemBytes);
+            bool nonfinite;
+            res = quantize_two_stage(bits, tab, nonfinite);
+            if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
+            *(uint4 *)(out.codes + r * (out.K / 2) + (int64_t)b * 16) =
+                make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
+        }
+        out.scales[scale_offset(out.rows, r, b)] = (uint8_t)res.scale;
+        idbyte |= res.id << (4 * h);
+    }
+    out.ids[id_byte_offset(out.rows, r, 2 * bp)] = (uint8_t)idbyte;
+}
+
+// ---------------------------------------------------------------------------
+// Layout conversion and dequantisation: one thread per block.
+// ---------------------------------------------------------------------------
+__global__ void export_canonical_kernel(QView q, uint8_t *__restrict__ codes, uint8_t *__restrict__ ids,
+                                        uint8_t *__restrict__ scales, int nb) {
+    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= q.rows * nb) return;
+    int64_t r = t / nb;
+    int b = (int)(t - r * nb);
+    uint4 u = *(const uint4 *)(q.codes + r * (q.K / 2) + (int64_t)b * 16);
+    uint32_t w[4] = {u.x, u.y, u.z, u.w}, o[4];
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        uint32_t c = 0;
+#pragma unroll
+        for (int j = 0; j < 8; j++) c |= (word_sign(w[i], j) << 3 | word_index(w[i], j)) << (4 * j);
+        o[i] = c;
+    }
+    *(uint4 *)(codes + r * (q.K / 2) + (int64_t)b * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+    ids[r * nb + b] = (q.ids[id_byte_offset(q.rows, r, b)] >> (4 * (b & 1))) & 15;
+    scales[r * nb + b] = q.scales[scale_offset(q.rows, r, b)];
+}
+
+// Thread t owns (r, b) over the padded grid, as in the contiguous quantizer.
+__global__ void import_canonical_kernel(const uint8_t *__restrict__ codes, const uint8_t *__restrict__ ids,
+                                        const uint8_t *__restrict__ scales, QView q, int64_t rows_pad, int nb,
+                                        int nb_pad) {
+    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= rows_pad * nb_pad) return;
+    int64_t r = t / nb_pad;
+    int b = (int)(t - r * nb_pad);
+    bool valid = r < q.rows && b < nb;
+    uint32_t id = 0, sc = 0;
+    if (valid) {
+        uint4 u = *(const uint4 *)(codes + r * (q.K / 2) + (int64_t)b * 16);
+        uint32_t c[4] = {u.x, u.y, u.z, u.w}, o[4];
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int j = 0; j < 8; j++) {
+                uint32_t nib = (c[i] >> (4 * j)) & 15u;
+                w |= word_insert(nib & 7u, nib >> 3, j);
+            }
+            o[i] = w;
+        }
+        *(uint4 *)(q.codes + r * (q.K / 2) + (int64_t)b * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+        id = ids[r * nb + b] & 15u;
+        sc = scales[r * nb + b];
+    }
+    uint32_t scw = sc << (8 * (b & 3)), idn = id << (4 * (b & 3));
+    scw |= __shfl_xor_sync(0xffffffffu, scw, 1);
+    idn |= __shfl_xor_sync(0xffffffffu, idn, 1);
+    scw |= __shfl_xor_sync(0xffffffffu, scw, 2);
+    idn |= __shfl_xor_sync(0xffffffffu, idn, 2);
+    if ((b & 3) == 0) {
+        *(uint32_t *)(q.scales + scale_offset(q.rows, r, b)) = scw;
+        *(uint16_t *)(q.ids + id_byte_offset(q.rows, r, b)) = (uint16_t)idn;
+    }
+}
+
+__global__ void dequantize_kernel(QView q, float *__restrict__ out, int64_t ld, int nb) {
+    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= q.rows * nb) return;
+    int64_t r = t / nb;
+    int b = (int)(t - r * nb);
+    uint4 u = *(const uint4 *)(q.codes + r * (q.K / 2) + (int64_t)b * 16);
+    uint32_t w[4] = {u.x, u.y, u.z, u.w};
+    uint32_t id = (q.ids[id_byte_offset(q.rows, r, b)] >> (4 * (b & 1))) & 15;
+    int e = (int)q.scales[scale_offset(q.rows, r, b)] - 127;
+    uint64_t lut = (uint64_t)c_tables.int_hi[id] << 32 | c_tables.int_lo[id];
+    float *dst = out + r * ld + (int64_t)b * 32;
+#pragma unroll
+    for (int i = 0; i < 4; i++)
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            float h = (float)((lut >> (8 * word_index(w[i], j))) & 0xff);
+            float v = scalbnf(h, e - 1);                          // 0.5 * h * 2^e, exact
+            dst[8 * i + j] = word_sign(w[i], j) ? -v : v;
+        }
+}
+
+// Decode a packed operand into the plain [rows][K] operand-byte matrix (E4M3).
+__global__ void decode_e4m3_kernel(QView q, uint8_t *__restrict__ out, int nb) {
+    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= q.rows * nb) return;
+    int64_t r = t / nb;
+    int b = (int)(t - r * nb);
+    uint4 u = *(const uint4 *)(q.codes + r * (q.K / 2) + (int64_t)b * 16);
+    uint32_t w[4] = {u.x, u.y, u.z, u.w}, o[8];
+    uint32_t id = (q.ids[id_byte_offset(q.rows, r, b)] >> (4 * (b & 1))) & 15;
+    uint32_t lo = c_tables.e4m3_lo[id], hi = c_tables.e4m3_hi[id];
+#pragma unroll
+    for (int i = 0; i < 4; i++) decode_word(w[i], lo, hi, o[2 * i], o[2 * i + 1]);
+    uint4 *dst = (uint4 *)(out + r * q.K + (int64_t)b * 32);
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
+}  // namespace bd

@@ -1,0 +1,75 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every declared symbol,
+and its host-only entry points behave.  No kernel is launched here."""
+import ctypes
+import os
+import re
+
+import numpy as np
+
+import oracle
+import paper_2501_01144_b200 as bd
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "bd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(bd_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = bd.load()
+    names = _declared_symbols()
+    assert len(names) >= 15
+    for name in names:
+        assert hasattr(lib, name), f"{name} declared in include/bd.h but not exported"
+
+
+def test_version_and_status_strings():
+    lib = bd.load()
+    assert bd.version() >= 100
+    for code in range(9):
+        assert lib.bd_status_string(code)
+    assert lib.bd_status_string(0) == b"ok"
+
+
+def test_formatbook_matches_independent_oracle_table():
+    # the CUDA library and the oracle each carry their own copy of the table
+    assert (bd.get_formatbook().numpy() == oracle.formatbook()).all()
+
+
+def test_qtensor_sizes_and_argument_errors():
+    lib = bd.load()
+    c, i, s = (ctypes.c_size_t() for _ in range(3))
+    assert lib.bd_qtensor_sizes(8192, 4096, ctypes.byref(c), ctypes.byref(i), ctypes.byref(s)) == 0
+    assert c.value == 8192 * 4096 // 2
+    assert i.value == 8192 * 4096 // 32 // 2          # 4 bits per block
+    assert s.value == 8192 * 4096 // 32               # 8 bits per block
+    # ragged shapes are padded to whole 128-row x 4-block atoms
+    assert lib.bd_qtensor_sizes(130, 96, ctypes.byref(c), ctypes.byref(i), ctypes.byref(s)) == 0
+    assert c.value == 130 * 48 and s.value == 2 * 1 * 512 and i.value == 2 * 1 * 256
+    assert lib.bd_qtensor_sizes(16, 100, None, None, None) == 2      # K % 32
+    assert lib.bd_qtensor_sizes(0, 64, None, None, None) == 1
+    b = ctypes.c_size_t()
+    assert lib.bd_linear_workspace_size(16, 128, 100, ctypes.byref(b)) == 2
+    assert lib.bd_gemm_workspace_size(16, 128, 256, None) == 1
+    assert lib.bd_set_gemm_impl(7) == 1 and lib.bd_set_gemm_impl(0) == 0
+
+
+def test_null_and_misaligned_arguments_rejected_before_any_launch():
+    lib = bd.load()
+    q = bd.binding._CQTensor(0, 0, 0, 16, 64)
+    assert lib.bd_quantize_act(None, bd.BF16, 16, 64, 64, 0, ctypes.byref(q), None) == 1
+    buf = np.zeros(4096, np.uint8)
+    base = buf.ctypes.data + (-buf.ctypes.data % 16)          # host memory: only the checks run
+    q = bd.binding._CQTensor(base, base + 1024, base + 2048, 16, 64)
+    assert lib.bd_quantize_act(ctypes.c_void_p(base + 4), bd.BF16, 16, 64, 64, 0, ctypes.byref(q), None) == 3
+    assert lib.bd_quantize_act(ctypes.c_void_p(base), bd.BF16, 16, 64, 60, 0, ctypes.byref(q), None) == 2
+    assert lib.bd_quantize_act(ctypes.c_void_p(base), 9, 16, 64, 64, 0, ctypes.byref(q), None) == 1
+    q2 = bd.binding._CQTensor(base, base + 1024, base + 2048, 8, 64)
+    assert lib.bd_quantize_act(ctypes.c_void_p(base), bd.BF16, 16, 64, 64, 0, ctypes.byref(q2), None) == 2
+    qa = bd.binding._CQTensor(base, base + 1024, base + 2048, 16, 64)
+    qb = bd.binding._CQTensor(base, base + 1024, base + 2048, 16, 96)
+    assert lib.bd_gemm(ctypes.byref(qa), ctypes.byref(qb), ctypes.c_void_p(base), bd.F32, 16, None, 0, None) == 2
+    assert lib.bd_gemm(ctypes.byref(qa), ctypes.byref(qa), ctypes.c_void_p(base), bd.F16, 16, None, 0, None) == 1

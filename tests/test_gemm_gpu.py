@@ -1,0 +1,111 @@
+"""GPU parity of the block-scaled product against the fp64 oracle:
+|Y - Yref| <= 1e-6 * sum_k |a_k||w_k| per output element (fp32 output)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2501_01144_b200 as bd
+from paper_2501_01144_b200 import inputs
+from util import gemm_tolerance_ok, oracle_quantize, to_device
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = [bd.GEMM_SIMT, bd.GEMM_TCGEN05]
+
+
+@pytest.fixture(autouse=True)
+def _reset_impl():
+    yield
+    bd.set_gemm_impl(bd.GEMM_AUTO)
+
+
+def _ref(qa, qb):
+    return oracle.gemm(oracle.dequantize(*qa), oracle.dequantize(*qb))
+
+
+def _run(impl, qa_ref, qb_ref, dtype=torch.float32):
+    bd.set_gemm_impl(impl)
+    A = bd.import_canonical(*(torch.from_numpy(t).cuda() for t in qa_ref))
+    B = bd.import_canonical(*(torch.from_numpy(t).cuda() for t in qb_ref))
+    try:
+        return bd.gemm(A, B, dtype=dtype)
+    except bd.BdError as e:
+        if e.status == 4:
+            pytest.skip("implementation does not take this shape")
+        raise
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_tiny_case(impl):
+    X, W = inputs.tiny_case()
+    qa, qb = oracle.quantize(X), oracle.quantize(W, oracle.SELECT_MSE)
+    Yref, T = _ref(qa, qb)
+    Y = _run(impl, qa, qb).cpu().numpy()
+    ok, ratio = gemm_tolerance_ok(Y, Yref, T)
+    assert ok, f"max err / bound = {ratio}"
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("M,N,K", [(1, 8, 32), (5, 130, 96), (128, 128, 128), (130, 257, 352), (200, 384, 1024)])
+def test_ragged_shapes(impl, M, N, K):
+    rng = np.random.default_rng(M + 31 * N + 977 * K)
+    a = rng.standard_t(4, (M, K)).astype(np.float32)
+    a[:, rng.integers(0, K)] *= 50
+    b = (0.02 * rng.standard_normal((N, K))).astype(np.float32)
+    qa, qb = oracle.quantize(a), oracle.quantize(b)
+    Yref, T = _ref(qa, qb)
+    Y = _run(impl, qa, qb).cpu().numpy()
+    ok, ratio = gemm_tolerance_ok(Y, Yref, T)
+    assert ok, f"max err / bound = {ratio}"
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_in_block_sums_are_exact(impl):
+    # one huge block contribution plus many tiny ones of opposite sign: only exact in-block
+    # integer sums and a full-precision cross-block accumulation meet the bound
+    K = 1024
+    a = np.full((128, K), 0.5, np.float32)
+    b = np.full((128, K), 0.5, np.float32)
+    a[:, :32] = 6.0 * 2.0 ** 8
+    b[:, :32] = 6.0 * 2.0 ** 8
+    b[:, 32:] *= -1
+    a[1::2] *= -1
+    qa, qb = oracle.quantize(a), oracle.quantize(b)
+    Yref, T = _ref(qa, qb)
+    Y = _run(impl, qa, qb).cpu().numpy()
+    ok, ratio = gemm_tolerance_ok(Y, Yref, T)
+    assert ok, f"max err / bound = {ratio}"
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_bf16_output_is_rounded_fp32_result(impl):
+    X, W = inputs.tiny_case()
+    qa, qb = oracle.quantize(X), oracle.quantize(W, oracle.SELECT_MSE)
+    y32 = _run(impl, qa, qb, torch.float32)
+    y16 = _run(impl, qa, qb, torch.bfloat16)
+    assert torch.equal(y16, y32.to(torch.bfloat16))
+
+
+def test_linear_tiny_case_end_to_end():
+    X, W = inputs.tiny_case()
+    Wq = bd.quantize_weights(to_device(W, torch.float32), bd.SELECT_MSE)
+    Y = bd.linear(to_device(X, torch.float32), Wq, dtype=torch.float32).cpu().numpy()
+    Yref, T = _ref(oracle.quantize(X), oracle.quantize(W, oracle.SELECT_MSE))
+    ok, ratio = gemm_tolerance_ok(Y, Yref, T)
+    assert ok, f"max err / bound = {ratio}"
+    bd.poll_status()
+
+
+def test_batched_grouped_query_product():
+    rng = np.random.default_rng(21)
+    heads, kv, S, d = 4, 2, 96, 128
+    q = inputs.to_bf16_bits(rng.standard_normal((heads, S, d)).astype(np.float32))
+    k = inputs.to_bf16_bits(rng.standard_normal((kv, S, d)).astype(np.float32))
+    As = [bd.quantize_act(to_device(q[h], torch.bfloat16)) for h in range(heads)]
+    Bs = [bd.quantize_act(to_device(k[g], torch.bfloat16)) for g in range(kv)]
+    Y = bd.gemm_batched(As, Bs, b_group=heads // kv).cpu().numpy()
+    for h in range(heads):
+        Yref, T = _ref(oracle_quantize(q[h], torch.bfloat16), oracle_quantize(k[h // 2], torch.bfloat16))
+        ok, ratio = gemm_tolerance_ok(Y[h], Yref, T)
+        assert ok, f"head {h}: max err / bound = {ratio}"

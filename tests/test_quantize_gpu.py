@@ -1,0 +1,122 @@
+"""GPU parity of the quantizers against the CPU oracle: codes, dialect ids and
+shared exponents must match bit for bit (through the canonical export)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2501_01144_b200 as bd
+from paper_2501_01144_b200 import inputs
+from util import assert_bit_exact, oracle_quantize, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def test_tiny_case_activations_two_stage_and_weights_mse():
+    X, W = inputs.tiny_case()
+    qx = bd.quantize_act(to_device(X, torch.float32))
+    assert_bit_exact(qx, oracle.quantize(X), "X two-stage")
+    qw = bd.quantize_weights(to_device(W, torch.float32), bd.SELECT_MSE)
+    assert_bit_exact(qw, oracle.quantize(W, oracle.SELECT_MSE), "W mse")
+    qw2 = bd.quantize_weights(to_device(W, torch.float32), bd.SELECT_TWO_STAGE)
+    assert_bit_exact(qw2, oracle.quantize(W), "W two-stage")
+    bd.poll_status()
+
+
+def test_activation_bandwidth_workload_full_size():
+    # the benchmarked configuration: bf16 [8192, 4096] with 1 % outlier channels
+    xb = inputs.act_normal_outliers(8192, 4096, seed=1)
+    q = bd.quantize_act(to_device(xb, torch.bfloat16))
+    assert_bit_exact(q, oracle_quantize(xb, torch.bfloat16), "config 2")
+    bd.poll_status()
+
+
+@pytest.mark.parametrize("rows,K", [(1, 32), (3, 96), (127, 160), (129, 4096), (300, 352), (16, 11008)])
+@pytest.mark.parametrize("kind", [torch.float32, torch.bfloat16, torch.float16])
+def test_ragged_shapes_and_dtypes(rows, K, kind):
+    rng = np.random.default_rng(rows * 7919 + K)
+    x = rng.standard_normal((rows, K)).astype(np.float32) * np.exp2(rng.integers(-6, 6, (rows, 1))).astype(np.float32)
+    x[:, rng.integers(0, K)] *= 30
+    if kind == torch.float32:
+        host = x
+    elif kind == torch.bfloat16:
+        host = inputs.to_bf16_bits(x)
+    else:
+        host = inputs.to_f16_bits(x)
+    q = bd.quantize_act(to_device(host, kind))
+    assert_bit_exact(q, oracle_quantize(host, kind), f"{rows}x{K} {kind}")
+    qm = bd.quantize_weights(to_device(host, kind), bd.SELECT_MSE)
+    assert_bit_exact(qm, oracle_quantize(host, kind, oracle.SELECT_MSE), f"mse {rows}x{K} {kind}")
+
+
+def test_degenerate_blocks():
+    x = np.zeros((8, 64), np.float32)
+    x[0, 3] = -0.0                                   # all-zero block with a negative zero
+    x[1, :32] = 1e-44; x[1, 5] = -3e-45              # fp32 subnormals: exponent clamp
+    x[2, :32] = 2.0 ** -125                          # exponent exactly at the clamp
+    x[2, 32:] = 2.0 ** -124 * 1.7
+    x[3, :32] = 3.0e38; x[3, 7] = -1.0               # near the top of the fp32 range
+    x[4, :] = np.linspace(-7.75, 7.75, 64)           # every quarter step: ties on every boundary
+    x[5, :32] = 7.99; x[5, 32:] = 7.75               # block maximum rounding up to 8.0 saturates at 7.5
+    x[6, :32] = np.float32(6.74999); x[6, 32:] = 6.75
+    x[7, ::2] = 5.0; x[7, 1::2] = -4.0; x[7, 0] = 6.5   # equal beneficial-range counts
+    q = bd.quantize_act(to_device(x, torch.float32))
+    assert_bit_exact(q, oracle.quantize(x), "degenerate")
+    h = (x * 1e-3).astype(np.float16)
+    h[0, :8] = np.float16(6e-8) * np.arange(8)       # fp16 subnormals
+    hb = h.view(np.uint16)
+    q = bd.quantize_act(to_device(hb, torch.float16))
+    assert_bit_exact(q, oracle_quantize(hb, torch.float16), "fp16 subnormal")
+
+
+def test_leading_dimension_and_output_guard_bands():
+    rng = np.random.default_rng(5)
+    big = rng.standard_normal((40, 512)).astype(np.float32)
+    xd = to_device(inputs.to_bf16_bits(big), torch.bfloat16)
+    view = xd[:, 128:128 + 256]                      # ld = 512 > K = 256, 16-byte aligned start
+    q = bd.QTensor(40, 256)
+    guard = 4096
+    bufs = {}
+    for name in ("codes", "ids", "scales"):          # place each buffer between pattern-filled guards
+        n = getattr(q, name).numel()
+        raw = torch.full((n + 2 * guard,), 0xA5, dtype=torch.uint8, device="cuda")
+        bufs[name] = raw
+        setattr(q, name, raw[guard:guard + n])
+    bd.quantize_act(view, out=q)
+    ref = oracle_quantize(inputs.to_bf16_bits(big[:, 128:384]), torch.bfloat16)
+    assert_bit_exact(q, ref, "strided rows")
+    for name, raw in bufs.items():
+        n = raw.numel() - 2 * guard
+        assert (raw[:guard] == 0xA5).all() and (raw[guard + n:] == 0xA5).all(), f"{name}: write outside the buffer"
+
+
+@pytest.mark.parametrize("kind", [torch.bfloat16, torch.float32])
+def test_strided_axis_quantizes_the_transpose(kind):
+    # V [tokens, head_dim] quantised along tokens: result equals quantising V^T along its rows
+    rng = np.random.default_rng(9)
+    v = rng.standard_normal((320, 128)).astype(np.float32)
+    host = v if kind == torch.float32 else inputs.to_bf16_bits(v)
+    q = bd.quantize_act(to_device(host, kind), axis=bd.AXIS_STRIDED)
+    assert (q.rows, q.K) == (128, 320)
+    ref = oracle_quantize(np.ascontiguousarray(host.T), kind)
+    assert_bit_exact(q, ref, "strided axis")
+
+
+def test_nonfinite_input_sets_status():
+    x = torch.ones(4, 64, device="cuda")
+    x[2, 40] = float("inf")
+    bd.quantize_act(x)
+    with pytest.raises(bd.BdError) as e:
+        bd.poll_status()
+    assert e.value.status == 6
+    bd.poll_status()                                 # the word is cleared by the read
+
+
+def test_import_export_roundtrip_and_dequantize():
+    X, _ = inputs.tiny_case()
+    ref = oracle.quantize(X)
+    q = bd.import_canonical(*(torch.from_numpy(t).cuda() for t in ref))
+    assert_bit_exact(q, ref, "import")
+    dq = bd.dequantize(q).cpu().numpy().astype(np.float64)
+    assert (dq == oracle.dequantize(*ref)).all()
+    assert (np.signbit(dq) == np.signbit(oracle.dequantize(*ref))).all()
