@@ -11,6 +11,14 @@ namespace bd {
 
 constexpr int kSimtTile = 64;
 
+// Each byte of the result is 0xff if bit 7 of the same byte of x is set, else 0
+// (prmt in its default mode replicates the byte's top bit when the selector's bit 3 is set).
+__device__ __forceinline__ uint32_t sign_bytes(uint32_t x) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %1, 0xba98;" : "=r"(r) : "r"(x));
+    return r;
+}
+
 __device__ __forceinline__ void simt_decode_block(const QView &q, int64_t row, int b, uint32_t (&dst)[8],
                                                   int &scale) {
     if (row >= q.rows) {
@@ -28,8 +36,8 @@ __device__ __forceinline__ void simt_decode_block(const QView &q, int64_t row, i
         uint32_t m0, m1;
         decode_word(w[i] & 0x77777777u, lo, hi, m0, m1);          // magnitudes only
         // two's-complement negate the bytes whose sign bit is set
-        uint32_t s0 = __byte_perm(w[i], 0, 0xba98);               // 0xff where elements 0..3 are negative
-        uint32_t s1 = __byte_perm(w[i] << 4, 0, 0xba98);          // elements 4..7
+        uint32_t s0 = sign_bytes(w[i]);                           // 0xff where elements 0..3 are negative
+        uint32_t s1 = sign_bytes(w[i] << 4);                      // elements 4..7
         dst[2 * i] = __vsub4(m0 ^ s0, s0);
         dst[2 * i + 1] = __vsub4(m1 ^ s1, s1);
     }

@@ -62,7 +62,9 @@ def test_degenerate_blocks():
     x[7, ::2] = 5.0; x[7, 1::2] = -4.0; x[7, 0] = 6.5   # equal beneficial-range counts
     q = bd.quantize_act(to_device(x, torch.float32))
     assert_bit_exact(q, oracle.quantize(x), "degenerate")
+    x[3] = np.linspace(-60000, 60000, 64)            # keep the fp16 copy finite
     h = (x * 1e-3).astype(np.float16)
+    h[3] = x[3].astype(np.float16)                   # top of the fp16 range
     h[0, :8] = np.float16(6e-8) * np.arange(8)       # fp16 subnormals
     hb = h.view(np.uint16)
     q = bd.quantize_act(to_device(hb, torch.float16))
