@@ -1,15 +1,339 @@
-// Tensor-core GEMM (tcgen05, block-scaled E4M3 MMA with TMEM accumulators): interface.
+// Tensor-core GEMM for sm_100a: Y[M,N] = A[M,K] * B[N,K]^T with one power-of-two
+// scale per 32 elements of K on each operand (Sec. 3.3: products inside a block
+// share the exponent sum eA + eB; here the block-scaled MMA applies it in hardware).
+//
+// Operands arrive as plain [rows][K] byte matrices holding the E4M3 encoding of
+// 0.5 * value (exact: every DialectFP4 magnitude has at most four significant bits)
+// and as scale atoms (bd_common.cuh) holding e + 127 as UE8M0.  TMA loads 128-byte
+// swizzled K-major tiles and the scale atoms into a ring of shared-memory stages;
+// one thread issues tcgen05.cp (scales -> TMEM) and tcgen05.mma.kind::mxf8f6f4
+// .block_scale (K = 32 per instruction = one block) into a TMEM accumulator; four
+// epilogue warps read the accumulator with tcgen05.ld and store fp32 or bf16.
+//
+// Every wait on an mbarrier is bounded: when the limit is reached the kernel
+// records kStatusTimeout, stops waiting everywhere, frees its TMEM and returns.
 #pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+
 #include "bd_common.cuh"
+#include "quantize.cuh"
 
 namespace bd {
+namespace tc {
 
-inline bool tc_supported(int64_t, int64_t, int64_t) { return false; }
+constexpr int BM = 128;            // rows of A per tile = MMA M = TMEM lanes
+constexpr int BK = 128;            // bytes of K per stage = one 128-byte swizzle row = 4 blocks
+constexpr int kThreads = 192;      // warp 0: TMA, warp 1: MMA + TMEM, warps 2..5: epilogue
+constexpr uint32_t kSpinLimit = 1u << 26;
+
+template <int BN>
+struct Config {
+    static constexpr int kStages = BN == 256 ? 4 : 6;
+    static constexpr int kATile = BM * BK;                       // 16 KiB
+    static constexpr int kBTile = BN * BK;
+    static constexpr int kSfA = kScaleAtomBytes;
+    static constexpr int kSfB = (BN / 128) * kScaleAtomBytes;
+    static constexpr int kStageBytes = kATile + kBTile + kSfA + kSfB;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment slack */ + 256 /* barriers */;
+    static constexpr int kAccCols = BN;
+    static constexpr int kSfaCol = BN;
+    static constexpr int kSfbCol = BN + 4;
+    static constexpr int kTmemCols = BN == 256 ? 512 : 256;      // power of two >= BN + 4 + 4 * BN / 128
+};
+
+// ---- PTX wrappers ----------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  `abort_flag` (shared memory) is raised by the first wait that runs out;
+// later waits return at once so that the CTA drains quickly.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag) {
+    for (uint32_t spin = 0; spin < kSpinLimit; spin++) {
+        if (mbar_try_wait(bar, parity)) return;
+        if ((spin & 1023u) == 1023u && *abort_flag) return;
+    }
+    *abort_flag = 1;
+    atomicOr(&g_status_word, kStatusTimeout);
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tcgen05_cp_32x128b_warpx4(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tcgen05_mma_mxf8(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t sfa, uint32_t sfb, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+        ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb) : "memory");
+}
+__device__ __forceinline__ void tcgen05_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tcgen05_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (64 bit): start address, leading and stride byte
+// offsets in 16-byte units, descriptor version 1, swizzle mode in bits 61..63.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+    return (uint64_t)((addr >> 4) & 0x3fffu) | (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16 |
+           (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32 | (uint64_t)1 << 46 | (uint64_t)layout << 61;
+}
+constexpr uint32_t kLayoutSwizzle128 = 2, kLayoutNone = 0;
+
+// Instruction descriptor of the block-scaled MMA: E4M3 x E4M3 (format 0), both K-major,
+// UE8M0 scales, N >> 3 at bit 17, M >> 4 at bit 24, scale byte selectors at bits 4 (B) and 29 (A).
+template <int BN>
+__device__ __forceinline__ uint32_t instr_desc(uint32_t sf_id) {
+    return (uint32_t)(BN >> 3) << 17 | 1u << 23 | (uint32_t)(BM >> 4) << 24 | sf_id << 4 | sf_id << 29;
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+               const uint8_t *__restrict__ sfA, const uint8_t *__restrict__ sfB, int M, int N, int K,
+               int row_tiles_a, int row_tiles_b, void *__restrict__ Y, int64_t ldy, int out_bf16) {
+    using C = Config<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *const base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    // all A tiles, then all B tiles (both 1024-byte aligned for the 128-byte swizzle), then the scale atoms
+    auto a_tile = [&](int s) { return base + (uint32_t)s * C::kATile; };
+    auto b_tile = [&](int s) { return base + (uint32_t)C::kStages * C::kATile + (uint32_t)s * C::kBTile; };
+    auto sfa_tile = [&](int s) { return base + (uint32_t)C::kStages * (C::kATile + C::kBTile) + (uint32_t)s * C::kSfA; };
+    auto sfb_tile = [&](int s) {
+        return base + (uint32_t)C::kStages * (C::kATile + C::kBTile + C::kSfA) + (uint32_t)s * C::kSfB;
+    };
+    const uint32_t bars = base + C::kStages * C::kStageBytes;              // full[S], empty[S], tmem_full
+    volatile uint32_t *const shared_words = (volatile uint32_t *)(base_ptr + C::kStages * C::kStageBytes + 128);
+    volatile uint32_t *const tmem_slot = shared_words;                     // TMEM base address
+    volatile uint32_t *const abort_flag = shared_words + 1;
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int k_tiles = (K + BK - 1) / BK;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (C::kStages + s); };
+    const uint32_t tmem_full_bar = bars + 8u * (2 * C::kStages);
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < C::kStages; s++) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        mbar_init(tmem_full_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32((const void *)tmem_slot)), "r"((uint32_t)C::kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer ----
+            const int atoms_b = min(BN / 128, row_tiles_b - blockIdx.x * (BN / 128));
+            const uint32_t tx = C::kATile + C::kBTile + C::kSfA + (uint32_t)atoms_b * kScaleAtomBytes;
+            int issued = 0;
+            for (int kt = 0; kt < k_tiles; kt++) {
+                const int s = kt % C::kStages;
+                mbar_wait(empty_bar(s), ((kt / C::kStages) & 1) ^ 1, abort_flag);
+                if (*abort_flag) break;
+                mbar_expect_tx(full_bar(s), tx);
+                tma_load_2d(a_tile(s), &mapA, kt * BK, m0, full_bar(s));
+                tma_load_2d(b_tile(s), &mapB, kt * BK, n0, full_bar(s));
+                bulk_load(sfa_tile(s), sfA + ((int64_t)kt * row_tiles_a + blockIdx.y) * kScaleAtomBytes,
+                          kScaleAtomBytes, full_bar(s));
+                bulk_load(sfb_tile(s), sfB + ((int64_t)kt * row_tiles_b + blockIdx.x * (BN / 128)) * kScaleAtomBytes,
+                          (uint32_t)atoms_b * kScaleAtomBytes, full_bar(s));
+                issued = kt + 1;
+            }
+            if (*abort_flag) {
+                // bounded wait for this thread's own copies still in flight before the CTA may exit
+                for (int kt = max(0, issued - C::kStages); kt < issued; kt++)
+                    for (uint32_t spin = 0; spin < (1u << 20); spin++)
+                        if (mbar_try_wait(full_bar(kt % C::kStages), (kt / C::kStages) & 1)) break;
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issuer ----
+            for (int kt = 0; kt < k_tiles; kt++) {
+                const int s = kt % C::kStages;
+                mbar_wait(full_bar(s), (kt / C::kStages) & 1, abort_flag);
+                if (*abort_flag) break;
+                tcgen05_fence_after();
+                const uint32_t sfa_s = sfa_tile(s), sfb_s = sfb_tile(s);
+                tcgen05_cp_32x128b_warpx4(tmem + C::kSfaCol, smem_desc(sfa_s, 0, 128, kLayoutNone));
+#pragma unroll
+                for (int j = 0; j < BN / 128; j++)
+                    tcgen05_cp_32x128b_warpx4(tmem + C::kSfbCol + 4 * j,
+                                              smem_desc(sfb_s + j * kScaleAtomBytes, 0, 128, kLayoutNone));
+#pragma unroll
+                for (int k = 0; k < BK / 32; k++) {
+                    const uint64_t da = smem_desc(a_tile(s) + 32 * k, 16, 1024, kLayoutSwizzle128);
+                    const uint64_t db = smem_desc(b_tile(s) + 32 * k, 16, 1024, kLayoutSwizzle128);
+                    tcgen05_mma_mxf8(tmem, da, db, instr_desc<BN>(k), tmem + C::kSfaCol, tmem + C::kSfbCol,
+                                     (kt | k) != 0);
+                }
+                tcgen05_commit(empty_bar(s));                      // stage free once these MMAs have read it
+            }
+            tcgen05_commit(tmem_full_bar);                         // accumulator complete
+        }
+    } else {
+        // ---- epilogue: warp w reads TMEM lanes 32 * (w % 4) .. + 31 ----
+        mbar_wait(tmem_full_bar, 0, abort_flag);
+        tcgen05_fence_after();
+        const int quad = warp % 4;
+        const int row = m0 + quad * 32 + lane;
+        const bool vec_ok = (ldy % 8 == 0) && (((uintptr_t)Y & 15u) == 0);
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; c++) {
+            uint32_t r[32];
+            tcgen05_ld_32x32b_x32(tmem + ((uint32_t)(quad * 32) << 16) + c * 32, r);
+            tcgen05_wait_ld();
+            const int col = n0 + c * 32;
+            if (row >= M || col >= N || *abort_flag) continue;
+            if (out_bf16) {
+                __nv_bfloat16 *dst = (__nv_bfloat16 *)Y + (int64_t)row * ldy + col;
+                if (vec_ok && col + 32 <= N) {
+#pragma unroll
+                    for (int i = 0; i < 4; i++) {
+                        uint32_t p[4];
+#pragma unroll
+                        for (int j = 0; j < 4; j++) {
+                            __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * i + 2 * j]),
+                                                                     __uint_as_float(r[8 * i + 2 * j + 1]));
+                            p[j] = *(uint32_t *)&h;
+                        }
+                        ((uint4 *)dst)[i] = make_uint4(p[0], p[1], p[2], p[3]);
+                    }
+                } else {
+                    for (int i = 0; i < 32 && col + i < N; i++) dst[i] = __float2bfloat16_rn(__uint_as_float(r[i]));
+                }
+            } else {
+                float *dst = (float *)Y + (int64_t)row * ldy + col;
+                if (vec_ok && col + 32 <= N) {
+#pragma unroll
+                    for (int i = 0; i < 8; i++)
+                        ((uint4 *)dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+                } else {
+                    for (int i = 0; i < 32 && col + i < N; i++) dst[i] = __uint_as_float(r[i]);
+                }
+            }
+        }
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)C::kTmemCols)
+                     : "memory");
+    }
+}
+
+// ---- host side --------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// Tensor map of a [rows][K] byte matrix, box = 128 bytes of K x box_rows rows, 128-byte swizzle, zero fill.
+inline bool make_operand_map(CUtensorMap *map, const uint8_t *ptr, int64_t rows, int64_t K, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)K};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void *)ptr, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+           CUDA_SUCCESS;
+}
+
+template <int BN>
+inline cudaError_t launch(const uint8_t *a8, const uint8_t *sfa, int64_t M, const uint8_t *b8, const uint8_t *sfb,
+                          int64_t N, int64_t K, void *Y, bool out_bf16, int64_t ldy, cudaStream_t st) {
+    using C = Config<BN>;
+    CUtensorMap mapA, mapB;
+    if (!make_operand_map(&mapA, a8, M, K, BM) || !make_operand_map(&mapB, b8, N, K, BN)) return cudaErrorInvalidValue;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
+    gemm_tc_kernel<BN><<<grid, kThreads, C::kSmemBytes, st>>>(mapA, mapB, sfa, sfb, (int)M, (int)N, (int)K,
+                                                             (int)row_tiles(M), (int)row_tiles(N), Y, ldy, out_bf16 ? 1 : 0);
+    return cudaGetLastError();
+}
+
+}  // namespace tc
+
+inline bool tc_supported(int64_t M, int64_t N, int64_t K) {
+    return K % kBlock == 0 && M >= 1 && N >= 1 && M < (1ll << 31) && N < (1ll << 31) && K < (1ll << 31);
+}
 inline size_t tc_operand_bytes(int64_t rows, int64_t K) { return ((size_t)rows * (size_t)K + 255) & ~(size_t)255; }
 inline size_t tc_gemm_workspace(int64_t M, int64_t N, int64_t K) { return tc_operand_bytes(M, K) + tc_operand_bytes(N, K); }
-inline cudaError_t tc_gemm(const uint8_t *, const uint8_t *, int64_t, const uint8_t *, const uint8_t *, int64_t, int64_t,
-                           void *, bool, int64_t, cudaStream_t) {
-    return cudaErrorNotSupported;
+
+inline cudaError_t tc_gemm(const uint8_t *a8, const uint8_t *sfa, int64_t M, const uint8_t *b8, const uint8_t *sfb,
+                           int64_t N, int64_t K, void *Y, bool out_bf16, int64_t ldy, cudaStream_t st) {
+    if (N > 128) return tc::launch<256>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
+    return tc::launch<128>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
 }
 
 }  // namespace bd
