@@ -39,7 +39,9 @@ typedef enum {
     BD_ERR_CUDA = 5,        /* a CUDA call failed; bd_last_cuda_error gives the code      */
     BD_ERR_NONFINITE = 6,   /* Inf/NaN met by a quantizer (from bd_poll_status)           */
     BD_ERR_TIMEOUT = 7,     /* a bounded device-side wait expired (from bd_poll_status)   */
-    BD_ERR_WORKSPACE = 8    /* workspace missing or too small                             */
+    BD_ERR_WORKSPACE = 8,   /* workspace missing or too small                             */
+    BD_ERR_SCRATCH_LIMIT = 9 /* bd_linear_noalloc: the problem needs more scratch than the
+                                library's built-in buffer holds                             */
 } bd_status;
 
 typedef enum { BD_F32 = 0, BD_BF16 = 1, BD_F16 = 2 } bd_dtype;
@@ -126,6 +128,31 @@ bd_status bd_linear_workspace_size(int64_t M, int64_t N, int64_t K, size_t *byte
 bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx,
                     const bd_qtensor *Wq, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace,
                     size_t workspace_bytes, void *stream);
+
+/* bd_linear for callers that can neither allocate device memory nor hand in a
+ * workspace (the paper has no counterpart; this is a convenience of the library).
+ * Think of code that runs where cudaMalloc is off limits: inside a region whose
+ * memory plan is already frozen, in a plugin that was given only its input and
+ * output tensors, or under a memory pool that forbids side allocations.  The
+ * scratch that bd_linear takes as `workspace` lives here in a fixed device array
+ * of BD_NOALLOC_SCRATCH_BYTES that is part of the library image: every GPU whose
+ * context loads the library carries those bytes until the process exits.
+ *
+ * Same arguments, results and errors as bd_linear, minus the workspace pair.
+ * Problems with bd_linear_workspace_size(M, N, K) > BD_NOALLOC_SCRATCH_BYTES are
+ * refused with BD_ERR_SCRATCH_LIMIT and nothing is enqueued.  The call performs no
+ * cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ * The first call on each device looks up the array's device address (a symbol
+ * query, with that device current) and caches it; make that first call outside
+ * any stream capture.  All calls on a device share the one array: it keeps
+ * whatever the previous call left there, which is harmless because every byte a
+ * call reads it has written earlier in the same call, so nothing needs clearing.
+ * Two calls that overlap on the GPU (different streams, or one stream per thread)
+ * race on the array; serialise them. */
+#define BD_NOALLOC_SCRATCH_BYTES (32u << 20)
+bd_status bd_linear_noalloc(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx,
+                            const bd_qtensor *Wq, void *Y, bd_dtype ydtype, int64_t ldy, void *stream);
 
 /* Canonical layout (what is compared bit for bit with a reference):
  *   codes  [rows][K/2]   byte j of a row: element 2j in bits 3:0, element 2j+1 in

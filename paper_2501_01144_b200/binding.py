@@ -66,6 +66,7 @@ def load():
     lib.bd_gemm_batched.argtypes = [qp, qp, i64, i64, vp, ci, i64, i64, vp, sz, vp]
     lib.bd_linear_workspace_size.argtypes = [i64, i64, i64, szp]
     lib.bd_linear.argtypes = [vp, ci, i64, i64, i64, qp, vp, ci, i64, vp, sz, vp]
+    lib.bd_linear_noalloc.argtypes = [vp, ci, i64, i64, i64, qp, vp, ci, i64, vp]
     lib.bd_export_canonical.argtypes = [qp, vp, vp, vp, vp]
     lib.bd_import_canonical.argtypes = [vp, vp, vp, qp, vp]
     lib.bd_dequantize.argtypes = [qp, vp, i64, vp]
@@ -222,6 +223,22 @@ def linear(X, Wq, out=None, dtype=torch.bfloat16, workspace=None, stream=None):
     cw = Wq.c_struct()
     _check(load().bd_linear(ptr, dt, M, K, ld, ctypes.byref(cw), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
                             out.stride(0), wptr, wbytes, _stream(stream)))
+    return out
+
+
+NOALLOC_SCRATCH_BYTES = 32 << 20
+
+
+def linear_noalloc(X, Wq, out, stream=None):
+    """bd_linear without a workspace argument and without any allocation: for callers that may not
+    allocate device memory (frozen memory plans, plugins handed only inputs and outputs).  `out`
+    must be preallocated; problems whose scratch need exceeds NOALLOC_SCRATCH_BYTES raise status 9.
+    Calls share one built-in device buffer, so calls that overlap on the GPU must be serialised."""
+    ptr, dt, ld = _src(X)
+    M, K = X.shape
+    cw = Wq.c_struct()
+    _check(load().bd_linear_noalloc(ptr, dt, M, K, ld, ctypes.byref(cw), ctypes.c_void_p(out.data_ptr()),
+                                    _ydtype(out.dtype), out.stride(0), _stream(stream)))
     return out
 
 

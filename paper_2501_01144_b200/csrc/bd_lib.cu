@@ -111,6 +111,16 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 }  // namespace
 
+// Built-in scratch of bd_linear_noalloc.  In host code this name is only a handle
+// for symbol queries, never a device address: the entry point asks the runtime for
+// the address once per device and passes that pointer on.
+static __device__ __align__(256) uint8_t g_noalloc_scratch[BD_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_noalloc_ptr[kMaxDevices] = {};
+}  // namespace
+
 extern "C" {
 
 bd_status bd_qtensor_sizes(int64_t rows, int64_t K, size_t *codes_bytes, size_t *ids_bytes, size_t *scales_bytes) {
@@ -223,6 +233,26 @@ bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_
     return gemm_dispatch(view_of(&xq), view_of(Wq), Y, ydtype, ldy, gemm_ws, need - (size_t)(gemm_ws - p), st);
 }
 
+bd_status bd_linear_noalloc(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, const bd_qtensor *Wq,
+                            void *Y, bd_dtype ydtype, int64_t ldy, void *stream) {
+    if (!Wq || M <= 0 || K <= 0 || Wq->rows <= 0) return BD_ERR_INVALID_ARG;
+    size_t need = 0;
+    bd_status s = bd_linear_workspace_size(M, Wq->rows, K, &need);
+    if (s) return s;
+    if (need > (size_t)BD_NOALLOC_SCRATCH_BYTES) return BD_ERR_SCRATCH_LIMIT;
+    int dev = -1;
+    s = cuda_result(cudaGetDevice(&dev));
+    if (s) return s;
+    if (dev < 0 || dev >= kMaxDevices) return BD_ERR_UNSUPPORTED;
+    if (!g_noalloc_ptr[dev]) {                       // first call on this device: resolve the symbol
+        void *p = nullptr;
+        s = cuda_result(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        if (s) return s;
+        g_noalloc_ptr[dev] = p;
+    }
+    return bd_linear(X, xdtype, M, K, ldx, Wq, Y, ydtype, ldy, g_noalloc_ptr[dev], BD_NOALLOC_SCRATCH_BYTES, stream);
+}
+
 bd_status bd_export_canonical(const bd_qtensor *q, uint8_t *codes, uint8_t *ids, uint8_t *scales, void *stream) {
     bd_status s = check_qtensor(q);
     if (s) return s;
@@ -300,6 +330,7 @@ const char *bd_status_string(bd_status s) {
         case BD_ERR_NONFINITE: return "non-finite input met by a quantizer";
         case BD_ERR_TIMEOUT: return "a bounded device-side wait expired";
         case BD_ERR_WORKSPACE: return "workspace missing or too small";
+        case BD_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the built-in no-allocation buffer holds";
     }
     return "unknown status";
 }

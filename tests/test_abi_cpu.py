@@ -29,7 +29,7 @@ def test_library_exports_every_declared_symbol():
 def test_version_and_status_strings():
     lib = bd.load()
     assert bd.version() >= 100
-    for code in range(9):
+    for code in range(10):
         assert lib.bd_status_string(code)
     assert lib.bd_status_string(0) == b"ok"
 
