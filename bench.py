@@ -328,18 +328,73 @@ def run_gpu(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def run_case(args):
+    """A few launches of one kernel family on a small, fixed case (for ncu captures).
+    quantizer: bd_quantize_act on bf16 [8192, 4096] (168 MiB of buffers in rotation).
+    linear_<layer>: bd_linear of one LLaMA3-8B layer at M = 2048 (layer in qo_proj, kv_proj, gate_up, down)."""
+    import torch
+
+    import paper_2501_01144_b200 as bd
+    from paper_2501_01144_b200 import inputs
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+
+    def dev_bf16(bits):
+        return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    reps = args.steps
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if args.case == "quantizer":
+        qm, qk = QUANT_SHAPE
+        xs = [dev_bf16(inputs.act_normal_outliers(qm, qk, seed=1 + s)) for s in range(2)]
+        qs = [bd.QTensor(qm, qk, dev) for _ in range(2)]
+        for i in range(args.warmup):
+            bd.quantize_act(xs[i % 2], out=qs[i % 2])
+        e0.record()
+        for i in range(reps):
+            bd.quantize_act(xs[i % 2], out=qs[i % 2])
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        print(json.dumps({"case": args.case, "us_per_launch": us,
+                          "GB/s": qm * qk * BYTES_PER_ELEM_QUANT / us / 1e3}))
+        return
+    name = args.case[len("linear_"):]
+    K, N = {n: (k, nn) for n, k, nn in LAYERS}[name]
+    x = dev_bf16(inputs.act_student_t(M_TOKENS, K, seed=2))
+    wq = bd.quantize_weights(dev_bf16(inputs.weights_normal(N, K, seed=2)), bd.SELECT_TWO_STAGE)
+    y = torch.empty(M_TOKENS, N, dtype=torch.bfloat16, device=dev)
+    ws = torch.empty(bd.linear_workspace_size(M_TOKENS, N, K), dtype=torch.uint8, device=dev)
+    for _ in range(args.warmup):
+        bd.linear(x, wq, out=y, workspace=ws)
+    e0.record()
+    for _ in range(reps):
+        bd.linear(x, wq, out=y, workspace=ws)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / reps * 1e3
+    print(json.dumps({"case": args.case, "us_per_call": us, "TFLOP/s": 2.0 * M_TOKENS * N * K / us / 1e6}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--case", default=None,
+                    choices=["quantizer"] + ["linear_" + n for n, _, _ in LAYERS],
+                    help="run a few launches of one small case (for profiler captures) instead of the benchmark")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.case:
+        run_case(args)
         return
     run_gpu(args, rank, world, local_rank)
 

@@ -14,6 +14,7 @@
 // records kStatusTimeout, stops waiting everywhere, frees its TMEM and returns.
 #pragma once
 #include <cuda.h>
+#include <stdlib.h>
 #include <cuda_bf16.h>
 
 #include "bd_common.cuh"
@@ -123,7 +124,7 @@ __device__ __forceinline__ uint32_t instr_desc(uint32_t sf_id) {
     return (uint32_t)(BN >> 3) << 17 | 1u << 23 | (uint32_t)(BM >> 4) << 24 | sf_id << 4 | sf_id << 29;
 }
 
-template <int BN>
+template <int BN, int MODE = 0>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                const uint8_t *__restrict__ sfA, const uint8_t *__restrict__ sfB, int M, int N, int K,
@@ -178,8 +179,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
             int issued = 0;
             for (int kt = 0; kt < k_tiles; kt++) {
                 const int s = kt % C::kStages;
+                if ((MODE & 8) && kt >= C::kStages) break;
                 mbar_wait(empty_bar(s), ((kt / C::kStages) & 1) ^ 1, abort_flag);
                 if (*abort_flag) break;
+                if ((MODE & 1) && kt >= C::kStages) {               // experiment: no loads after the ring is filled
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(full_bar(s)) : "memory");
+                    issued = kt + 1;
+                    continue;
+                }
                 mbar_expect_tx(full_bar(s), tx);
                 tma_load_2d(a_tile(s), &mapA, kt * BK, m0, full_bar(s));
                 tma_load_2d(b_tile(s), &mapB, kt * BK, n0, full_bar(s));
@@ -201,19 +208,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
             // ---- MMA issuer ----
             for (int kt = 0; kt < k_tiles; kt++) {
                 const int s = kt % C::kStages;
-                mbar_wait(full_bar(s), (kt / C::kStages) & 1, abort_flag);
+                if (!(MODE & 8) || kt < C::kStages) mbar_wait(full_bar(s), (kt / C::kStages) & 1, abort_flag);
                 if (*abort_flag) break;
                 tcgen05_fence_after();
                 const uint32_t sfa_s = sfa_tile(s), sfb_s = sfb_tile(s);
+                if (!(MODE & 4) || kt == 0)
                 tcgen05_cp_32x128b_warpx4(tmem + C::kSfaCol, smem_desc(sfa_s, 0, 128, kLayoutNone));
+                if (!(MODE & 4) || kt == 0)
 #pragma unroll
                 for (int j = 0; j < BN / 128; j++)
                     tcgen05_cp_32x128b_warpx4(tmem + C::kSfbCol + 4 * j,
                                               smem_desc(sfb_s + j * kScaleAtomBytes, 0, 128, kLayoutNone));
 #pragma unroll
-                for (int k = 0; k < BK / 32; k++) {
+                for (int k = 0; k < ((MODE & 2) ? 0 : BK / 32); k++) {
                     const uint64_t da = smem_desc(a_tile(s) + 32 * k, 16, 1024, kLayoutSwizzle128);
                     const uint64_t db = smem_desc(b_tile(s) + 32 * k, 16, 1024, kLayoutSwizzle128);
+                    if (MODE & 16) {                               // experiment: plain (unscaled) FP8 kind, timing only
+                        const uint32_t idesc = 1u << 4 | (uint32_t)(BN >> 3) << 17 | (uint32_t)(BM >> 4) << 24;
+                        asm volatile(
+                            "{\n\t.reg .pred p;\n\t"
+                            "setp.ne.b32 p, %4, 0;\n\t"
+                            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+                            ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"((uint32_t)((kt | k) != 0)) : "memory");
+                    } else
                     tcgen05_mma_mxf8(tmem, da, db, instr_desc<BN>(k), tmem + C::kSfaCol, tmem + C::kSfbCol,
                                      (kt | k) != 0);
                 }
@@ -274,6 +291,207 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
     }
 }
 
+// ---------------------------------------------------------------------------
+// Two-CTA variant: a cluster of two CTAs on neighbouring SMs computes a 256 x 256 tile
+// with tcgen05.mma.cta_group::2.  CTA r of the pair loads rows [128 r, 128 r + 128) of
+// the A tile and of the B tile, so each SM reads half as much B from shared memory per
+// MMA as the one-CTA kernel; the leader (rank 0) issues the scale copies and the MMAs
+// for both; each CTA owns the accumulator rows of its own A half and stores them.
+// All loads complete on the leader's "full" barrier; the leader's commit frees the
+// stage in both CTAs.
+// ---------------------------------------------------------------------------
+constexpr int kStages2 = 6;
+constexpr int kHalfTile = 128 * BK;                               // 16 KiB: A half or B half
+constexpr int kStage2Bytes = 2 * kHalfTile + kScaleAtomBytes + 2 * kScaleAtomBytes;
+constexpr int kSmem2Bytes = kStages2 * kStage2Bytes + 1024 + 256;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tcgen05_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tcgen05_cp_pair(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tcgen05_mma_mxf8_pair(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                      uint32_t sfa, uint32_t sfb, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+        ::"r"(d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb) : "memory");
+}
+
+// Store one 32-column chunk of an accumulator row (fp32 registers) as fp32 or bf16.
+__device__ __forceinline__ void store_chunk(const uint32_t (&r)[32], void *Y, int64_t ldy, int row, int col, int N,
+                                            int out_bf16, bool vec_ok) {
+    if (out_bf16) {
+        __nv_bfloat16 *dst = (__nv_bfloat16 *)Y + (int64_t)row * ldy + col;
+        if (vec_ok && col + 32 <= N) {
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+                uint32_t p[4];
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * i + 2 * j]),
+                                                             __uint_as_float(r[8 * i + 2 * j + 1]));
+                    p[j] = *(uint32_t *)&h;
+                }
+                ((uint4 *)dst)[i] = make_uint4(p[0], p[1], p[2], p[3]);
+            }
+        } else {
+            for (int i = 0; i < 32 && col + i < N; i++) dst[i] = __float2bfloat16_rn(__uint_as_float(r[i]));
+        }
+    } else {
+        float *dst = (float *)Y + (int64_t)row * ldy + col;
+        if (vec_ok && col + 32 <= N) {
+#pragma unroll
+            for (int i = 0; i < 8; i++) ((uint4 *)dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+        } else {
+            for (int i = 0; i < 32 && col + i < N; i++) dst[i] = __uint_as_float(r[i]);
+        }
+    }
+}
+
+template <int MODE = 0>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                const __grid_constant__ CUtensorMap mapSfA, const __grid_constant__ CUtensorMap mapSfB, int M, int N,
+                int K, int row_tiles_a, int row_tiles_b, void *__restrict__ Y, int64_t ldy, int out_bf16) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *const base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    auto a_tile = [&](int s) { return base + (uint32_t)s * kHalfTile; };
+    auto b_tile = [&](int s) { return base + (uint32_t)(kStages2 + s) * kHalfTile; };
+    auto sfa_tile = [&](int s) { return base + (uint32_t)(2 * kStages2) * kHalfTile + (uint32_t)s * kScaleAtomBytes; };
+    auto sfb_tile = [&](int s) {
+        return base + (uint32_t)(2 * kStages2) * kHalfTile + (uint32_t)(kStages2 + 2 * s) * kScaleAtomBytes;
+    };
+    const uint32_t bars = base + kStages2 * kStage2Bytes;
+    volatile uint32_t *const shared_words = (volatile uint32_t *)(base_ptr + kStages2 * kStage2Bytes + 128);
+    volatile uint32_t *const tmem_slot = shared_words;
+    volatile uint32_t *const abort_flag = shared_words + 1;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (kStages2 + s); };
+    const uint32_t tmem_full_bar = bars + 8u * (2 * kStages2);
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const uint32_t rank = cluster_ctarank();                      // 0 = leader
+    const int pair = blockIdx.x / 2;
+    const int m0 = pair * 256 + (int)rank * 128;                  // this CTA's accumulator rows
+    const int n0 = blockIdx.y * 256;
+    const int k_tiles = (K + BK - 1) / BK;
+    constexpr int kAccCols = 256, kSfaCol = 256, kSfbCol = 260, kTmemCols = 512;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < kStages2; s++) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        mbar_init(tmem_full_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32((const void *)tmem_slot)), "r"((uint32_t)kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                           // both CTAs: barriers initialised, TMEM allocated
+    tcgen05_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer (both CTAs); every copy completes on the leader's full barrier ----
+            constexpr uint32_t tx_pair = 2u * (2u * kHalfTile + 3u * kScaleAtomBytes);
+            int issued = 0;
+            for (int kt = 0; kt < k_tiles; kt++) {
+                const int s = kt % kStages2;
+                if ((MODE & 8) && kt >= kStages2) break;
+                mbar_wait(empty_bar(s), ((kt / kStages2) & 1) ^ 1, abort_flag);
+                if (*abort_flag) break;
+                const uint32_t fb = map_to_cta(full_bar(s), 0);
+                if (rank == 0) mbar_expect_tx(full_bar(s), tx_pair);
+                tma_load_2d_pair(a_tile(s), &mapA, kt * BK, m0, fb);
+                tma_load_2d_pair(b_tile(s), &mapB, kt * BK, n0 + (int)rank * 128, fb);
+                tma_load_2d_pair(sfa_tile(s), &mapSfA, 0, kt * row_tiles_a + pair * 2 + (int)rank, fb);
+                tma_load_2d_pair(sfb_tile(s), &mapSfB, 0, kt * row_tiles_b + blockIdx.y * 2, fb);
+                issued = kt + 1;
+            }
+            (void)issued;
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            // ---- MMA issuer (leader only) ----
+            for (int kt = 0; kt < k_tiles; kt++) {
+                const int s = kt % kStages2;
+                if (!(MODE & 8) || kt < kStages2) mbar_wait(full_bar(s), (kt / kStages2) & 1, abort_flag);
+                if (*abort_flag) break;
+                tcgen05_fence_after();
+                if (!(MODE & 4) || kt == 0) {
+                tcgen05_cp_pair(tmem + kSfaCol, smem_desc(sfa_tile(s), 0, 128, kLayoutNone));
+                tcgen05_cp_pair(tmem + kSfbCol, smem_desc(sfb_tile(s), 0, 128, kLayoutNone));
+                tcgen05_cp_pair(tmem + kSfbCol + 4, smem_desc(sfb_tile(s) + kScaleAtomBytes, 0, 128, kLayoutNone));
+                }
+#pragma unroll
+                for (int k = 0; k < BK / 32; k++) {
+                    const uint64_t da = smem_desc(a_tile(s) + 32 * k, 16, 1024, kLayoutSwizzle128);
+                    const uint64_t db = smem_desc(b_tile(s) + 32 * k, 16, 1024, kLayoutSwizzle128);
+                    const uint32_t idesc = (uint32_t)(256 >> 3) << 17 | 1u << 23 | (uint32_t)(256 >> 4) << 24 |
+                                           (uint32_t)k << 4 | (uint32_t)k << 29;
+                    tcgen05_mma_mxf8_pair(tmem, da, db, idesc, tmem + kSfaCol, tmem + kSfbCol, (kt | k) != 0);
+                }
+                tcgen05_commit_pair(empty_bar(s));
+            }
+            tcgen05_commit_pair(tmem_full_bar);
+        }
+    } else {
+        mbar_wait(tmem_full_bar, 0, abort_flag);
+        tcgen05_fence_after();
+        const int quad = warp % 4;
+        const int row = m0 + quad * 32 + lane;
+        const bool vec_ok = (ldy % 8 == 0) && (((uintptr_t)Y & 15u) == 0);
+#pragma unroll 1
+        for (int c = 0; c < kAccCols / 32; c++) {
+            uint32_t r[32];
+            tcgen05_ld_32x32b_x32(tmem + ((uint32_t)(quad * 32) << 16) + c * 32, r);
+            tcgen05_wait_ld();
+            const int col = n0 + c * 32;
+            if (row >= M || col >= N || *abort_flag) continue;
+            store_chunk(r, Y, ldy, row, col, N, out_bf16, vec_ok);
+        }
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                           // the peer may still signal our barriers until here
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols)
+                     : "memory");
+    }
+}
+
 // ---- host side --------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -304,7 +522,40 @@ inline bool make_operand_map(CUtensorMap *map, const uint8_t *ptr, int64_t rows,
            CUDA_SUCCESS;
 }
 
-template <int BN>
+// Tensor map over the scale atoms: [atoms][128 x uint32], box = `atoms_per_box` whole atoms, zero fill.
+inline bool make_scale_map(CUtensorMap *map, const uint8_t *ptr, int64_t atoms, int atoms_per_box) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {128, (cuuint64_t)atoms};
+    cuuint64_t strides[1] = {(cuuint64_t)kScaleAtomBytes};
+    cuuint32_t box[2] = {128, (cuuint32_t)atoms_per_box};
+    cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, (void *)ptr, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+           CUDA_SUCCESS;
+}
+
+template <int MODE = 0>
+inline cudaError_t launch_pair(const uint8_t *a8, const uint8_t *sfa, int64_t M, const uint8_t *b8, const uint8_t *sfb,
+                               int64_t N, int64_t K, void *Y, bool out_bf16, int64_t ldy, cudaStream_t st) {
+    CUtensorMap mapA, mapB, mapSfA, mapSfB;
+    const int64_t rta = row_tiles(M), rtb = row_tiles(N), kg = k_groups(K);
+    if (!make_operand_map(&mapA, a8, M, K, 128) || !make_operand_map(&mapB, b8, N, K, 128) ||
+        !make_scale_map(&mapSfA, sfa, rta * kg, 1) || !make_scale_map(&mapSfB, sfb, rtb * kg, 2))
+        return cudaErrorInvalidValue;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc2_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem2Bytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    dim3 grid((unsigned)(2 * ((M + 255) / 256)), (unsigned)((N + 255) / 256));
+    gemm_tc2_kernel<MODE><<<grid, kThreads, kSmem2Bytes, st>>>(mapA, mapB, mapSfA, mapSfB, (int)M, (int)N, (int)K, (int)rta,
+                                                        (int)rtb, Y, ldy, out_bf16 ? 1 : 0);
+    return cudaGetLastError();
+}
+
+template <int BN, int MODE = 0>
 inline cudaError_t launch(const uint8_t *a8, const uint8_t *sfa, int64_t M, const uint8_t *b8, const uint8_t *sfb,
                           int64_t N, int64_t K, void *Y, bool out_bf16, int64_t ldy, cudaStream_t st) {
     using C = Config<BN>;
@@ -312,12 +563,12 @@ inline cudaError_t launch(const uint8_t *a8, const uint8_t *sfa, int64_t M, cons
     if (!make_operand_map(&mapA, a8, M, K, BM) || !make_operand_map(&mapB, b8, N, K, BN)) return cudaErrorInvalidValue;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<BN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
     dim3 grid((unsigned)((N + BN - 1) / BN), (unsigned)((M + BM - 1) / BM));
-    gemm_tc_kernel<BN><<<grid, kThreads, C::kSmemBytes, st>>>(mapA, mapB, sfa, sfb, (int)M, (int)N, (int)K,
+    gemm_tc_kernel<BN, MODE><<<grid, kThreads, C::kSmemBytes, st>>>(mapA, mapB, sfa, sfb, (int)M, (int)N, (int)K,
                                                              (int)row_tiles(M), (int)row_tiles(N), Y, ldy, out_bf16 ? 1 : 0);
     return cudaGetLastError();
 }
@@ -332,6 +583,20 @@ inline size_t tc_gemm_workspace(int64_t M, int64_t N, int64_t K) { return tc_ope
 
 inline cudaError_t tc_gemm(const uint8_t *a8, const uint8_t *sfa, int64_t M, const uint8_t *b8, const uint8_t *sfb,
                            int64_t N, int64_t K, void *Y, bool out_bf16, int64_t ldy, cudaStream_t st) {
+    static int variant = -1;
+    if (variant < 0) { const char *v = getenv("BD_TC_VARIANT"); variant = v ? atoi(v) : 0; }
+    if (variant == 1) return tc::launch<128>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
+    if (variant == 3) return tc::launch<256, 1>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
+    if (variant == 4) return tc::launch<256, 2>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
+    if (variant == 28) return tc::launch_pair<12>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
+    if (variant == 20) return tc::launch_pair<0>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
+    if (variant == 11) return tc::launch<256, 29>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
+    if (variant == 10) return cudaSuccess;                        // experiment: decode kernels only
+    if (variant == 7) return tc::launch<256, 5>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
+    if (variant == 8) return tc::launch<256, 13>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
+    if (variant == 9) return tc::launch<256, 9>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
+    if (variant == 5) return tc::launch<128, 1>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
+    if (variant == 6) return tc::launch<128, 2>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
     if (N > 128) return tc::launch<256>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
     return tc::launch<128>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
 }

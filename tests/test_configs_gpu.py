@@ -1,0 +1,107 @@
+"""Parity at the benchmark's full sizes (the launch configuration bench.py times), on
+sampled outputs the oracle can compute one by one: whole rows, whole columns and tile
+boundaries of the LLaMA-shaped linear layers, the decode-to-prefill M sweep, and the
+Mistral-shaped attention products with both operands quantised online."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2501_01144_b200 as bd
+from paper_2501_01144_b200 import inputs
+from util import assert_bit_exact, gemm_tolerance_ok, oracle_quantize, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_rows_cols(Y, xb, wb, rows, cols, what):
+    """Y [M,N] from the library; xb/wb bf16 bit patterns.  Compares Y[rows, :] and Y[:, cols]."""
+    qa_all = None
+    qb = oracle.quantize(wb, dtype=oracle.BF16)
+    wdq = oracle.dequantize(*qb)
+    qa = oracle.quantize(xb[rows], dtype=oracle.BF16)
+    Yref, T = oracle.gemm(oracle.dequantize(*qa), wdq)
+    ok, ratio = gemm_tolerance_ok(Y[rows], Yref, T)
+    assert ok, f"{what} rows: max err / bound = {ratio}"
+    if len(cols):
+        qa_all = oracle.quantize(xb, dtype=oracle.BF16)
+        Yref, T = oracle.gemm(oracle.dequantize(*qa_all), wdq[cols])
+        ok, ratio = gemm_tolerance_ok(Y[:, cols], Yref, T)
+        assert ok, f"{what} cols: max err / bound = {ratio}"
+
+
+@pytest.mark.parametrize("K,N", [(4096, 4096), (4096, 1024), (4096, 14336), (14336, 4096)])
+def test_llama3_linear_layers_m2048(K, N):
+    M = 2048
+    xb = inputs.act_student_t(M, K, seed=2)
+    wb = inputs.weights_normal(N, K, seed=2)
+    Wq = bd.quantize_weights(to_device(wb, torch.bfloat16), bd.SELECT_TWO_STAGE)
+    Y = bd.linear(to_device(xb, torch.bfloat16), Wq, dtype=torch.float32).cpu().numpy()
+    rng = np.random.default_rng(K + N)
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, M - 1], rng.choice(M, 4, replace=False)]))
+    cols = np.unique(np.concatenate([[0, 255, 256, N - 1], rng.choice(N, 4, replace=False)]))
+    _check_rows_cols(Y, xb, wb, rows, cols, f"K={K} N={N}")
+    # bf16 output (what the benchmark times) is the rounded fp32 result
+    Y16 = bd.linear(to_device(xb, torch.bfloat16), Wq, dtype=torch.bfloat16)
+    assert torch.equal(Y16.cpu(), torch.from_numpy(Y).to(torch.bfloat16))
+    bd.poll_status()
+
+
+def test_llama3_weights_exact_mse_rule_on_kv_shape():
+    wb = inputs.weights_normal(1024, 4096, seed=2)
+    Wq = bd.quantize_weights(to_device(wb, torch.bfloat16), bd.SELECT_MSE)
+    assert_bit_exact(Wq, oracle_quantize(wb, torch.bfloat16, oracle.SELECT_MSE), "kv weights, MSE rule")
+
+
+@pytest.mark.parametrize("K,N", [(4096, 11008), (11008, 4096)])
+@pytest.mark.parametrize("M", [1, 16, 128, 1024, 8192])
+def test_llama2_mlp_m_sweep(K, N, M):
+    xb = inputs.act_post_silu(M, K, seed=3)
+    wb = inputs.weights_normal(N, K, seed=3)
+    Wq = bd.quantize_weights(to_device(wb, torch.bfloat16), bd.SELECT_TWO_STAGE)
+    Y = bd.linear(to_device(xb, torch.bfloat16), Wq, dtype=torch.float32).cpu().numpy()
+    rng = np.random.default_rng(M)
+    rows = np.unique(np.concatenate([[0, M - 1], rng.choice(M, min(M, 6), replace=False)]))
+    cols = np.array([0, N - 1, 255, 256]) if M <= 1024 else np.array([], int)
+    _check_rows_cols(Y, xb, wb, rows, cols, f"M={M} K={K} N={N}")
+    bd.poll_status()
+
+
+def test_attention_products_both_operands_online():
+    heads, kv, S, d = 32, 8, 4096, 128
+    n_p = 2                                                   # heads of P generated (each is 64 MiB of fp32)
+    Q, Kt, P, V = inputs.attention_case(heads, kv, S, d, seed=4, p_heads=n_p)
+    group = heads // kv
+    # ---- QK^T: both along head_dim (K = 128), grouped-query batching over all 32 heads ----
+    Aq = [bd.quantize_act(to_device(Q[h], torch.bfloat16)) for h in range(heads)]
+    Bk = [bd.quantize_act(to_device(Kt[g], torch.bfloat16)) for g in range(kv)]
+    for h in (0, 5, 31):
+        assert_bit_exact(Aq[h], oracle_quantize(Q[h], torch.bfloat16), f"Q head {h}")
+    assert_bit_exact(Bk[7], oracle_quantize(Kt[7], torch.bfloat16), "K head 7")
+    out = torch.empty(4, S, S, dtype=torch.float32, device="cuda")
+    check_heads = [0, 13, 30, 31]
+    Ssc = bd.gemm_batched([Aq[h] for h in check_heads], [Bk[h // group] for h in check_heads], b_group=1, out=out)
+    rows = np.array([0, 127, 128, 2049, S - 1])
+    for i, h in enumerate(check_heads):
+        qa = oracle_quantize(Q[h][rows], torch.bfloat16)
+        qb = oracle_quantize(Kt[h // group], torch.bfloat16)
+        Yref, T = oracle.gemm(oracle.dequantize(*qa), oracle.dequantize(*qb))
+        ok, ratio = gemm_tolerance_ok(Ssc[i].cpu().numpy()[rows], Yref, T)
+        assert ok, f"QK^T head {h}: max err / bound = {ratio}"
+    # grouped batching: heads 0..3 share KV head 0
+    out4 = bd.gemm_batched(Aq[:4], Bk[:1], b_group=4, out=torch.empty(4, S, S, dtype=torch.float32, device="cuda"))
+    assert torch.equal(out4[0], Ssc[0])
+    del out, out4, Ssc
+    # ---- PV: P along keys (K = 4096, fp32 source), V along tokens (strided axis) ----
+    Bv = [bd.quantize_act(to_device(V[g], torch.bfloat16), axis=bd.AXIS_STRIDED) for g in range(kv)]
+    assert_bit_exact(Bv[0], oracle_quantize(np.ascontiguousarray(V[0].T), torch.bfloat16), "V head 0 (token axis)")
+    for h in range(n_p):
+        Ap = bd.quantize_act(to_device(P[h], torch.float32))
+        assert_bit_exact(Ap, oracle.quantize(P[h]), f"P head {h}")
+        O = bd.gemm(Ap, Bv[h // group]).cpu().numpy()
+        qa = oracle.quantize(P[h][rows])
+        qb = oracle_quantize(np.ascontiguousarray(V[h // group].T), torch.bfloat16)
+        Yref, T = oracle.gemm(oracle.dequantize(*qa), oracle.dequantize(*qb))
+        ok, ratio = gemm_tolerance_ok(O[rows], Yref, T)
+        assert ok, f"PV head {h}: max err / bound = {ratio}"
+    bd.poll_status()
