@@ -84,29 +84,7 @@ constexpr uint64_t int_lut(int d) {
     return t;
 }
 
-struct DeviceTables {
-    uint32_t round_mask[16];
-    uint32_t even_mask[8];
-    uint32_t odd_mask[8];
-    uint32_t e4m3_lo[16], e4m3_hi[16];
-    uint32_t int_lo[16], int_hi[16];
-};
-constexpr DeviceTables make_tables() {
-    DeviceTables t{};
-    for (int d = 0; d < 16; d++) {
-        t.round_mask[d] = round_mask(d);
-        t.e4m3_lo[d] = (uint32_t)e4m3_lut(d);
-        t.e4m3_hi[d] = (uint32_t)(e4m3_lut(d) >> 32);
-        t.int_lo[d] = (uint32_t)int_lut(d);
-        t.int_hi[d] = (uint32_t)(int_lut(d) >> 32);
-    }
-    for (int p = 0; p < 8; p++) {
-        t.even_mask[p] = even_range_mask(p);
-        t.odd_mask[p] = odd_range_mask(p);
-    }
-    return t;
-}
-constexpr DeviceTables kTables = make_tables();
+
 
 // ---------------------------------------------------------------------------
 // Physical layout of a quantised [rows, K] operand.
@@ -149,14 +127,94 @@ __device__ __forceinline__ void decode_word(uint32_t w, uint32_t lut_lo, uint32_
     hi = ((w << 4) & 0x80808080u) | __byte_perm(lut_lo, lut_hi, sel >> 16);
 }
 
-// Index and sign of element j (0..7) of a code word.
-__host__ __device__ inline uint32_t word_index(uint32_t w, int j) { return (w >> (4 * j)) & 7u; }
-__host__ __device__ inline uint32_t word_sign(uint32_t w, int j) {
-    return (w >> (j < 4 ? 8 * j + 7 : 8 * (j - 4) + 3)) & 1u;
+// Where logical element e (0..7) of an 8-element group sits in its code word.  The order
+// inside a group is a fixed permutation chosen so that the signs of four bf16 pairs can be
+// gathered with shifts by 0, 4, 8 and 12 bits (see the bf16 quantizer); every producer and
+// consumer of code words goes through these helpers or through decode_word, and a block of
+// 32 shares one scale, so the permutation never shows outside the library.
+//   slot s: index in bits 4s..4s+2; sign in bit 8s+7 (s < 4) or 8(s-4)+3 (s >= 4);
+//   decode_word emits slot s as operand byte s (lo = slots 0..3, hi = slots 4..7).
+__host__ __device__ constexpr int slot_of(int e) { return e < 4 ? 2 * e + 1 : 2 * (e - 4); }
+__host__ __device__ constexpr int sign_bit_of_slot(int s) { return s < 4 ? 8 * s + 7 : 8 * (s - 4) + 3; }
+__host__ __device__ inline uint32_t word_index(uint32_t w, int e) { return (w >> (4 * slot_of(e))) & 7u; }
+__host__ __device__ inline uint32_t word_sign(uint32_t w, int e) { return (w >> sign_bit_of_slot(slot_of(e))) & 1u; }
+__host__ __device__ inline uint32_t word_insert(uint32_t idx, uint32_t sign, int e) {
+    return idx << (4 * slot_of(e)) | sign << sign_bit_of_slot(slot_of(e));
 }
-__host__ __device__ inline uint32_t word_insert(uint32_t idx, uint32_t sign, int j) {
-    return idx << (4 * j) | sign << (j < 4 ? 8 * j + 7 : 8 * (j - 4) + 3);
+
+// ---------------------------------------------------------------------------
+// Merged thresholds of a dialect pair, for the one-pass quantizer.  With v5 the common
+// value below the differing slot, dE > dO the two differing values and mx the shared
+// maximum, the ten thresholds on q5
+//   t0..t4 (common), v5+dO, v5+dE, dE+dO, dO+mx, dE+mx
+// are strictly increasing.  u = #{thresholds <= q5} then decides everything:
+//   u in {6,7}: inside the odd member's beneficial range [v5+dO, dE+dO);
+//   u in {8,9}: inside the even member's range [dE+dO, dE+mx);
+//   index under the even member = u - [u>=6] - [u>=8] - [u>=9];
+//   index under the odd member  = u - [u>=7] - [u>=8] - [u>=10].
+// pair_tables_ok() checks all of this against the plain definitions for every code.
+// ---------------------------------------------------------------------------
+constexpr uint32_t merged_mask(int p) {
+    const uint8_t *ev = kBook.v[2 * p], *od = kBook.v[2 * p + 1];
+    uint32_t m = 0;
+    for (int j = 1; j <= 5; j++) m |= 1u << (ev[j - 1] + ev[j]);
+    m |= 1u << (od[5] + od[6]);
+    m |= 1u << (ev[5] + ev[6]);
+    m |= 1u << (ev[6] + od[6]);
+    m |= 1u << (od[6] + od[7]);
+    m |= 1u << (ev[6] + ev[7]);
+    return m;
 }
+constexpr int popcount32(uint32_t x) {
+    int c = 0;
+    for (; x; x &= x - 1) c++;
+    return c;
+}
+constexpr bool pair_tables_ok() {
+    for (int p = 0; p < 8; p++) {
+        const uint32_t mm = merged_mask(p);
+        if (popcount32(mm) != 10) return false;
+        for (int j = 0; j < 6; j++)
+            if (kBook.v[2 * p][j] != kBook.v[2 * p + 1][j]) return false;
+        for (int q = 0; q < 32; q++) {
+            const int u = popcount32(mm & ((2u << q) - 1u));
+            const int idx_e = u - (u >= 6) - (u >= 8) - (u >= 9);
+            const int idx_o = u - (u >= 7) - (u >= 8) - (u >= 10);
+            if (idx_e != popcount32(round_mask(2 * p) & ((2u << q) - 1u))) return false;
+            if (idx_o != popcount32(round_mask(2 * p + 1) & ((2u << q) - 1u))) return false;
+            if (((even_range_mask(p) >> q) & 1u) != (uint32_t)(u == 8 || u == 9)) return false;
+            if (((odd_range_mask(p) >> q) & 1u) != (uint32_t)(u == 6 || u == 7)) return false;
+        }
+    }
+    return true;
+}
+static_assert(pair_tables_ok(), "merged-threshold shortcut does not match the formatbook");
+
+struct DeviceTables {
+    uint32_t round_mask[16];
+    uint32_t even_mask[8];
+    uint32_t odd_mask[8];
+    uint32_t e4m3_lo[16], e4m3_hi[16];
+    uint32_t int_lo[16], int_hi[16];
+    uint32_t merged_above[8];     // merged_mask(p) >> 1: popcount(x >> q5) = thresholds above q5
+};
+constexpr DeviceTables make_tables() {
+    DeviceTables t{};
+    for (int d = 0; d < 16; d++) {
+        t.round_mask[d] = round_mask(d);
+        t.e4m3_lo[d] = (uint32_t)e4m3_lut(d);
+        t.e4m3_hi[d] = (uint32_t)(e4m3_lut(d) >> 32);
+        t.int_lo[d] = (uint32_t)int_lut(d);
+        t.int_hi[d] = (uint32_t)(int_lut(d) >> 32);
+    }
+    for (int p = 0; p < 8; p++) {
+        t.even_mask[p] = even_range_mask(p);
+        t.odd_mask[p] = odd_range_mask(p);
+        t.merged_above[p] = merged_mask(p) >> 1;
+    }
+    return t;
+}
+constexpr DeviceTables kTables = make_tables();
 
 // Bits of the device status word (defined in quantize.cuh; the library is one
 // translation unit).  bd_poll_status reads and clears it.

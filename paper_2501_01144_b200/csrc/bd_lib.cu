@@ -47,7 +47,12 @@ bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out
     const unsigned grid = grid_for(rows_pad * nb_pad, 256);
     switch (dt) {
         case BD_F32: quantize_contig_kernel<BD_F32, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad); break;
-        case BD_BF16: quantize_contig_kernel<BD_BF16, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad); break;
+        case BD_BF16:
+            if (SELECT == BD_SELECT_TWO_STAGE)
+                quantize_bf16_kernel<WC, WE><<<grid, 256, 0, st>>>((const uint16_t *)X, ld, out, e4m3, rows_pad, nb, nb_pad);
+            else
+                quantize_contig_kernel<BD_BF16, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad);
+            break;
         case BD_F16: quantize_contig_kernel<BD_F16, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad); break;
         default: return BD_ERR_INVALID_ARG;
     }
@@ -225,9 +230,27 @@ bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_
     size_t c, i, sc;
     bd_qtensor_sizes(M, K, &c, &i, &sc);
     char *p = (char *)workspace;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t N = Wq->rows;
+    if (use_tc(M, N, K)) {
+        if (!tc_supported(M, N, K)) return BD_ERR_UNSUPPORTED;
+        // tensor-core path: the quantizer writes the operand bytes and the scale atoms directly
+        // (no codes, no ids); the weights are decoded to operand bytes; then the block-scaled MMA
+        uint8_t *sfa = (uint8_t *)p;
+        uint8_t *a8 = sfa + align256(sc);
+        uint8_t *b8 = a8 + tc_operand_bytes(M, K);
+        bd_qtensor xq{nullptr, nullptr, sfa, M, K};
+        s = launch_contig<BD_SELECT_TWO_STAGE, false, true>(X, xdtype, ldx, view_of(&xq), a8, st);
+        if (s) return s;
+        QView W = view_of(Wq);
+        decode_e4m3_kernel<<<grid_for(N * (K / kBlock), 256), 256, 0, st>>>(W, b8, (int)(K / kBlock));
+        s = launch_result();
+        if (s) return s;
+        g_launches += 1;
+        return cuda_result(tc_gemm(a8, sfa, M, b8, W.scales, N, K, Y, ydtype == BD_BF16, ldy, st));
+    }
     bd_qtensor xq{p, p + align256(c), p + align256(c) + align256(i), M, K};
     char *gemm_ws = p + align256(c) + align256(i) + align256(sc);
-    cudaStream_t st = (cudaStream_t)stream;
     s = launch_contig<BD_SELECT_TWO_STAGE, true, false>(X, xdtype, ldx, view_of(&xq), nullptr, st);
     if (s) return s;
     return gemm_dispatch(view_of(&xq), view_of(Wq), Y, ydtype, ldy, gemm_ws, need - (size_t)(gemm_ws - p), st);

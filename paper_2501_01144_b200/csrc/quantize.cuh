@@ -27,6 +27,7 @@ struct SmemTables {
     uint32_t even_mask[8];
     uint32_t odd_mask[8];
     uint32_t e4m3_lo[16], e4m3_hi[16];
+    uint32_t merged_above[8];
 };
 __device__ __forceinline__ void load_tables(SmemTables &s) {
     for (int i = threadIdx.x; i < 16; i += blockDim.x) {
@@ -36,6 +37,7 @@ __device__ __forceinline__ void load_tables(SmemTables &s) {
         if (i < 8) {
             s.even_mask[i] = c_tables.even_mask[i];
             s.odd_mask[i] = c_tables.odd_mask[i];
+            s.merged_above[i] = c_tables.merged_above[i];
         }
     }
     __syncthreads();
@@ -135,7 +137,48 @@ __device__ __forceinline__ void encode_block(const uint32_t (&bits)[32], const S
     }
 }
 
-// Two-stage rule (Sec. 3.2).
+__device__ __forceinline__ uint32_t prmt_b32(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
+__device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ uint32_t byte_sum(uint32_t x) { return (x * 0x01010101u) >> 24; }
+
+// Second half of the two-stage rule, on packed nibbles.  v[w] holds, for the eight
+// elements of group w (nibble = slot), the number of merged thresholds of the pair
+// ABOVE the element's 5-bit code (0..10).  u = 10 - v is the number at or below it
+// (see merged_mask).  Counts the two beneficial ranges with one byte-permute table
+// lookup per four elements, picks the dialect, and turns u into the 3-bit index with
+// nibble-parallel arithmetic.  signs[w] already holds the sign bits in place.
+__device__ __forceinline__ void finish_two_stage(const uint32_t (&v)[4], const uint32_t (&signs)[4], uint32_t pair,
+                                                 uint32_t &id, uint32_t (&words)[4]) {
+    // table byte of v: 0x01 for v in {1,2} (u in {9,8}: even range), 0x10 for v in {3,4} (odd range);
+    // v >= 8 selects "replicate the top bit" of bytes 0..2, which is 0.
+    uint32_t acc = 0;
+#pragma unroll
+    for (int w = 0; w < 4; w++)
+        acc += prmt_b32(0x10010100u, 0x00000010u, v[w]) + prmt_b32(0x10010100u, 0x00000010u, v[w] >> 16);
+    const uint32_t cnt_even = byte_sum(acc & 0x0f0f0f0fu), cnt_odd = byte_sum((acc >> 4) & 0x0f0f0f0fu);
+    const uint32_t odd = cnt_odd > cnt_even ? 1u : 0u;             // equal counts: the even member
+    id = 2u * pair + odd;
+    const uint32_t first_step = odd ? 0x11111111u : 0x22222222u;   // [u >= 7] or [u >= 6] via a carry into bit 3
+    const uint32_t odd_mask = 0u - odd;
+#pragma unroll
+    for (int w = 0; w < 4; w++) {
+        const uint32_t u = 0xaaaaaaaau - v[w];                      // nibble-wise 10 - v, no borrows
+        const uint32_t b3 = (u >> 3) & 0x11111111u, b1 = (u >> 1) & 0x11111111u, b0 = u & 0x11111111u;
+        const uint32_t f = ((u + first_step) >> 3) & 0x11111111u;
+        const uint32_t top = b3 & (b1 | (b0 & ~odd_mask));          // [u >= 9] (even) or [u >= 10] (odd)
+        words[w] = (u - f - b3 - top) | signs[w];
+    }
+}
+
+// Two-stage rule (Sec. 3.2) for a block given as fp32 bit patterns.
 __device__ __forceinline__ BlockResult quantize_two_stage(const uint32_t (&bits)[32], const SmemTables &tab,
                                                           bool &nonfinite) {
     uint32_t amax = 0;
@@ -147,17 +190,17 @@ __device__ __forceinline__ BlockResult quantize_two_stage(const uint32_t (&bits)
     uint32_t m5 = sc.q5(amax);
     uint32_t max_hu = min(15u, (m5 + 1u) >> 1);
     uint32_t pair = min(7u, 15u - max_hu);                       // pair maxima are 15 - pair
-    uint32_t em = tab.even_mask[pair], om = tab.odd_mask[pair];
-    int balance = 0;
+    const uint32_t above = tab.merged_above[pair];
+    uint32_t v[4] = {0, 0, 0, 0}, signs[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int k = 0; k < 32; k++) {
-        uint32_t q = sc.q5(bits[k] & 0x7fffffffu);
-        balance += (int)((em >> q) & 1u) - (int)((om >> q) & 1u);
+        const uint32_t q = sc.q5(bits[k] & 0x7fffffffu);
+        v[k / 8] += (uint32_t)__popc(above >> q) << (4 * slot_of(k % 8));
+        signs[k / 8] |= (bits[k] >> 31) << sign_bit_of_slot(slot_of(k % 8));
     }
     BlockResult r;
-    r.id = 2u * pair + (balance < 0 ? 1u : 0u);
     r.scale = eadj - 2u;                                         // (eadj - 129) + 127
-    encode_block(bits, sc, tab.round_mask[r.id], r.words);
+    finish_two_stage(v, signs, pair, r.id, r.words);
     return r;
 }
 
@@ -198,6 +241,107 @@ __device__ __forceinline__ BlockResult quantize_mse(const uint32_t (&bits)[32], 
     r.scale = eadj - 2u;
     encode_block(bits, sc, tab.round_mask[best], r.words);
     return r;
+}
+
+// ---------------------------------------------------------------------------
+// bf16 fast path of the contiguous-axis quantizer (same thread-to-block map and outputs
+// as quantize_contig_kernel).  The 32 elements stay packed two per register:
+//   absmax      and + max.u16x2 on the packed magnitudes;
+//   q5          one fma.rz per element; the upper element of a pair is used in place (the
+//               lower half then only adds less than one bf16 ulp, which cannot reach the
+//               next integer of the scaled value), the lower one after a 16-bit shift;
+//   selection   popcount of the pair's merged threshold mask shifted by q5, accumulated as
+//               nibbles, then finish_two_stage;
+//   signs       the four pair registers of a group land on the eight sign bits of the code
+//               word with shifts by 0, 4, 8 and 12.
+// Blocks whose exponent is clamped (maximum below 2^-123) take the generic routine.
+// ---------------------------------------------------------------------------
+__device__ __noinline__ void quantize_bf16_clamped_block(const uint32_t (&R)[16], const SmemTables &tab,
+                                                         BlockResult &res) {
+    uint32_t bits[32];
+#pragma unroll
+    for (int i = 0; i < 16; i++) {
+        bits[2 * i] = R[i] << 16;
+        bits[2 * i + 1] = R[i] & 0xffff0000u;
+    }
+    bool nonfinite;
+    res = quantize_two_stage(bits, tab, nonfinite);
+}
+
+template <bool WRITE_CODES, bool WRITE_E4M3>
+__global__ void __launch_bounds__(256) quantize_bf16_kernel(const uint16_t *__restrict__ X, int64_t ld, QView out,
+                                                            uint8_t *__restrict__ e4m3, int64_t rows_pad, int nb,
+                                                            int nb_pad) {
+    __shared__ SmemTables tab;
+    load_tables(tab);
+    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= rows_pad * nb_pad) return;
+    int64_t r = t / nb_pad;
+    int b = (int)(t - r * nb_pad);
+    BlockResult res;
+    res.id = 0; res.scale = 0;
+    res.words[0] = res.words[1] = res.words[2] = res.words[3] = 0;
+    if (r < out.rows && b < nb) {
+        const uint4 *src = (const uint4 *)(X + r * ld + (int64_t)b * 32);
+        const uint4 l0 = __ldg(src), l1 = __ldg(src + 1), l2 = __ldg(src + 2), l3 = __ldg(src + 3);
+        const uint32_t R[16] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w,
+                                l2.x, l2.y, l2.z, l2.w, l3.x, l3.y, l3.z, l3.w};
+        uint32_t a[16];
+#pragma unroll
+        for (int i = 0; i < 16; i++) a[i] = R[i] & 0x7fff7fffu;
+        uint32_t m = a[0];
+#pragma unroll
+        for (int i = 1; i < 16; i++) m = max_u16x2(m, a[i]);
+        const uint32_t amax = max(m & 0xffffu, m >> 16);          // bf16 magnitude bits of the block maximum
+        if (amax >= 0x7f80u) atomicOr(&g_status_word, kStatusNonfinite);
+        const uint32_t eadj = max(amax >> 7, 2u);
+        if (eadj >= 4u) {
+            const float scale = __uint_as_float((258u - eadj) << 23);     // 2^(2 - e), e = eadj - 129
+            const uint32_t m5 = __float_as_uint(__fmaf_rz(__uint_as_float(amax << 16), scale, 8388608.0f)) & 63u;
+            const uint32_t pair = min(7u, 15u - min(15u, (m5 + 1u) >> 1));
+            const uint32_t above = tab.merged_above[pair];
+            uint32_t v[4] = {0, 0, 0, 0}, signs[4];
+#pragma unroll
+            for (int i = 0; i < 16; i++) {
+                const uint32_t t_lo = __float_as_uint(__fmaf_rz(__uint_as_float(a[i] << 16), scale, 8388608.0f));
+                const uint32_t t_hi = __float_as_uint(__fmaf_rz(__uint_as_float(a[i]), scale, 8388608.0f));
+                // funnel shift in wrap mode uses only the low five bits of the count, i.e. q5
+                const uint32_t v_lo = __popc(__funnelshift_r(above, 0u, t_lo));
+                const uint32_t v_hi = __popc(__funnelshift_r(above, 0u, t_hi));
+                v[i / 4] += (v_lo << (4 * slot_of(2 * (i % 4)))) + (v_hi << (4 * slot_of(2 * (i % 4) + 1)));
+            }
+#pragma unroll
+            for (int w = 0; w < 4; w++)
+                signs[w] = (R[4 * w] & 0x80008000u) | ((R[4 * w + 1] & 0x80008000u) >> 4) |
+                           ((R[4 * w + 2] & 0x80008000u) >> 8) | ((R[4 * w + 3] & 0x80008000u) >> 12);
+            res.scale = eadj - 2u;
+            finish_two_stage(v, signs, pair, res.id, res.words);
+        } else {
+            quantize_bf16_clamped_block(R, tab, res);
+        }
+        if (WRITE_CODES)
+            *(uint4 *)(out.codes + r * (out.K / 2) + (int64_t)b * 16) =
+                make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
+        if (WRITE_E4M3) {
+            uint32_t lo = tab.e4m3_lo[res.id], hi = tab.e4m3_hi[res.id];
+            uint32_t o[8];
+#pragma unroll
+            for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, o[2 * w], o[2 * w + 1]);
+            uint4 *dst = (uint4 *)(e4m3 + r * out.K + (int64_t)b * 32);
+            dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+            dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+        }
+    }
+    uint32_t sc = res.scale << (8 * (b & 3));
+    uint32_t idn = res.id << (4 * (b & 3));
+    sc |= __shfl_xor_sync(0xffffffffu, sc, 1);
+    idn |= __shfl_xor_sync(0xffffffffu, idn, 1);
+    sc |= __shfl_xor_sync(0xffffffffu, sc, 2);
+    idn |= __shfl_xor_sync(0xffffffffu, idn, 2);
+    if ((b & 3) == 0) {
+        *(uint32_t *)(out.scales + scale_offset(out.rows, r, b)) = sc;
+        if (WRITE_CODES) *(uint16_t *)(out.ids + id_byte_offset(out.rows, r, b)) = (uint16_t)idn;
+    }
 }
 
 // ---------------------------------------------------------------------------
