@@ -13,10 +13,13 @@
 #include <cuda_fp16.h>
 
 #include "bd_common.cuh"
+#include "ptx_sm100.cuh"
+
+#ifndef BD_QUANT_MIN_BLOCKS
+#define BD_QUANT_MIN_BLOCKS 5
+#endif
 
 namespace bd {
-
-__device__ uint32_t g_status_word = 0;
 
 __constant__ DeviceTables c_tables = kTables;
 
@@ -269,7 +272,7 @@ __device__ __noinline__ void quantize_bf16_clamped_block(const uint32_t (&R)[16]
 }
 
 template <bool WRITE_CODES, bool WRITE_E4M3>
-__global__ void __launch_bounds__(256) quantize_bf16_kernel(const uint16_t *__restrict__ X, int64_t ld, QView out,
+__global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel(const uint16_t *__restrict__ X, int64_t ld, QView out,
                                                             uint8_t *__restrict__ e4m3, int64_t rows_pad, int nb,
                                                             int nb_pad) {
     __shared__ SmemTables tab;
@@ -286,7 +289,11 @@ __global__ void __launch_bounds__(256) quantize_bf16_kernel(const uint16_t *__re
         const uint4 l0 = __ldg(src), l1 = __ldg(src + 1), l2 = __ldg(src + 2), l3 = __ldg(src + 3);
         const uint32_t R[16] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w,
                                 l2.x, l2.y, l2.z, l2.w, l3.x, l3.y, l3.z, l3.w};
-        uint32_t a[16];
+        uint32_t a[16], signs[4];
+#pragma unroll
+        for (int w = 0; w < 4; w++)
+            signs[w] = (R[4 * w] & 0x80008000u) | ((R[4 * w + 1] >> 4) & 0x08000800u) |
+                       ((R[4 * w + 2] >> 8) & 0x00800080u) | ((R[4 * w + 3] >> 12) & 0x00080008u);
 #pragma unroll
         for (int i = 0; i < 16; i++) a[i] = R[i] & 0x7fff7fffu;
         uint32_t m = a[0];
@@ -300,7 +307,7 @@ __global__ void __launch_bounds__(256) quantize_bf16_kernel(const uint16_t *__re
             const uint32_t m5 = __float_as_uint(__fmaf_rz(__uint_as_float(amax << 16), scale, 8388608.0f)) & 63u;
             const uint32_t pair = min(7u, 15u - min(15u, (m5 + 1u) >> 1));
             const uint32_t above = tab.merged_above[pair];
-            uint32_t v[4] = {0, 0, 0, 0}, signs[4];
+            uint32_t v[4] = {0, 0, 0, 0};
 #pragma unroll
             for (int i = 0; i < 16; i++) {
                 const uint32_t t_lo = __float_as_uint(__fmaf_rz(__uint_as_float(a[i] << 16), scale, 8388608.0f));
@@ -308,16 +315,16 @@ __global__ void __launch_bounds__(256) quantize_bf16_kernel(const uint16_t *__re
                 // funnel shift in wrap mode uses only the low five bits of the count, i.e. q5
                 const uint32_t v_lo = __popc(__funnelshift_r(above, 0u, t_lo));
                 const uint32_t v_hi = __popc(__funnelshift_r(above, 0u, t_hi));
-                v[i / 4] += (v_lo << (4 * slot_of(2 * (i % 4)))) + (v_hi << (4 * slot_of(2 * (i % 4) + 1)));
+                v[i / 4] = v_lo * (1u << (4 * slot_of(2 * (i % 4)))) + v[i / 4];
+                v[i / 4] = v_hi * (1u << (4 * slot_of(2 * (i % 4) + 1))) + v[i / 4];
             }
-#pragma unroll
-            for (int w = 0; w < 4; w++)
-                signs[w] = (R[4 * w] & 0x80008000u) | ((R[4 * w + 1] & 0x80008000u) >> 4) |
-                           ((R[4 * w + 2] & 0x80008000u) >> 8) | ((R[4 * w + 3] & 0x80008000u) >> 12);
             res.scale = eadj - 2u;
             finish_two_stage(v, signs, pair, res.id, res.words);
         } else {
-            quantize_bf16_clamped_block(R, tab, res);
+            uint32_t copy[16];                                   // only this branch spills the block to local memory
+#pragma unroll
+            for (int i = 0; i < 16; i++) copy[i] = R[i];
+            quantize_bf16_clamped_block(copy, tab, res);
         }
         if (WRITE_CODES)
             *(uint4 *)(out.codes + r * (out.K / 2) + (int64_t)b * 16) =
