@@ -41,6 +41,8 @@ bd_status check_qtensor(const bd_qtensor *q) {
 
 int elem_bytes(bd_dtype dt) { return dt == BD_F32 ? 4 : 2; }
 
+unsigned grid_for(int64_t threads, int block) { return (unsigned)((threads + block - 1) / block); }
+
 template <int SELECT, bool WC, bool WE>
 bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out, uint8_t *e4m3, cudaStream_t st) {
     const int nb = (int)(out.K / kBlock), nb_pad = (int)k_groups(out.K) * kBlocksPerAtom;
