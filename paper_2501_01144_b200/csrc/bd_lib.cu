@@ -105,6 +105,12 @@ bd_status gemm_dispatch(const QView &A, const QView &B, void *Y, bd_dtype ydt, i
         uint8_t *b8 = a8 + tc_operand_bytes(A.rows, A.K);
         const int nb = (int)(A.K / kBlock);
         decode_e4m3_kernel<<<grid_for(A.rows * nb, 256), 256, 0, st>>>(A, a8, nb);
+        if (tc_fused_b()) {
+            bd_status s = launch_result(1);
+            if (s) return s;
+            g_launches += 1;
+            return cuda_result(tc_gemm_fused(a8, A.scales, A.rows, B, A.K, Y, ydt == BD_BF16, ldy, st));
+        }
         decode_e4m3_kernel<<<grid_for(B.rows * nb, 256), 256, 0, st>>>(B, b8, nb);
         bd_status s = launch_result(2);
         if (s) return s;
@@ -246,6 +252,10 @@ bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_
         s = launch_contig<BD_SELECT_TWO_STAGE, false, true>(X, xdtype, ldx, view_of(&xq), a8, st);
         if (s) return s;
         QView W = view_of(Wq);
+        if (tc_fused_b()) {
+            g_launches += 1;
+            return cuda_result(tc_gemm_fused(a8, sfa, M, W, K, Y, ydtype == BD_BF16, ldy, st));
+        }
         decode_e4m3_kernel<<<grid_for(N * (K / kBlock), 256), 256, 0, st>>>(W, b8, (int)(K / kBlock));
         s = launch_result();
         if (s) return s;

@@ -21,6 +21,10 @@
 #include "ptx_sm100.cuh"
 #include "quantize.cuh"
 
+#ifndef BD_FUSED_EXP
+#define BD_FUSED_EXP 0
+#endif
+
 namespace bd {
 namespace tc {
 
@@ -79,6 +83,16 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
            (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32 | (uint64_t)1 << 46 | (uint64_t)layout << 61;
 }
 constexpr uint32_t kLayoutSwizzle128 = 2, kLayoutNone = 0;
+// The same descriptor split in two words, so that the issuing thread only adds to the low one:
+// low = (addr >> 4) | (lbo >> 4) << 16, high = (sbo >> 4) | version 1 << 14 | layout << 29.
+__device__ __forceinline__ uint32_t desc_hi(uint32_t sbo_bytes, uint32_t layout) {
+    return ((sbo_bytes >> 4) & 0x3fffu) | 1u << 14 | layout << 29;
+}
+__device__ __forceinline__ uint64_t desc_join(uint32_t lo, uint32_t hi) {
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
 
 // Instruction descriptor of the block-scaled MMA: E4M3 x E4M3 (format 0), both K-major,
 // UE8M0 scales, N >> 3 at bit 17, M >> 4 at bit 24, scale byte selectors at bits 4 (B) and 29 (A).
@@ -203,7 +217,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__
         }
     } else {
         // ---- epilogue: warp w reads TMEM lanes 32 * (w % 4) .. + 31 ----
-        mbar_wait(tmem_full_bar, 0, abort_flag);
+        mbar_wait(tmem_full_bar, 0, abort_flag, 256);
         tcgen05_fence_after();
         const int quad = warp % 4;
         const int row = m0 + quad * 32 + lane;
@@ -429,7 +443,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             tcgen05_commit_pair(tmem_full_bar);
         }
     } else {
-        mbar_wait(tmem_full_bar, 0, abort_flag);
+        mbar_wait(tmem_full_bar, 0, abort_flag, 256);
         tcgen05_fence_after();
         const int quad = warp % 4;
         const int row = m0 + quad * 32 + lane;
@@ -448,6 +462,234 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     tcgen05_fence_before();
     __syncthreads();
     cluster_sync_all();                                           // the peer may still signal our barriers until here
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols)
+                     : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Two-CTA kernel with the weight decode fused in: the B operand stays in its packed
+// 4-bit form in HBM and in the shared-memory stages (64 bytes of codes per row and
+// k-step, loaded by TMA with the 64-byte swizzle, plus the 256-byte id atom); four
+// decode warps per CTA expand each stage's codes through the dialect byte tables into a
+// small ring of operand buffers in the 128-byte-swizzled K-major layout the MMA reads;
+// a proxy fence and an mbarrier hand each buffer to the MMA issuer of the leader CTA.
+// A arrives as operand bytes (from the quantizer or the decode kernel) exactly as in
+// gemm_tc2_kernel.  Freed resources come back through tcgen05.commit to both CTAs.
+// ---------------------------------------------------------------------------
+constexpr int kStagesF = 6;           // raw stages: A tile + packed B codes + ids + scale atoms
+constexpr int kDecBufs = 4;           // decoded-B operand buffers
+constexpr int kCodeTile = 128 * 64;   // 8 KiB: 128 rows x 64 bytes of codes
+constexpr int kDecodeGroups = 4;
+constexpr int kDecodeWarps = 4 * kDecodeGroups;
+constexpr int kFusedThreads = 32 * (2 + kDecodeWarps + 4);   // warp 0 TMA, warp 1 MMA, the decode warps, 4 epilogue warps
+struct FusedSmem {
+    static constexpr int a = 0;
+    static constexpr int codes = a + kStagesF * kHalfTile;
+    static constexpr int dec = codes + kStagesF * kCodeTile;
+    static constexpr int sfa = dec + kDecBufs * kHalfTile;
+    static constexpr int sfb = sfa + kStagesF * kScaleAtomBytes;
+    static constexpr int ids = sfb + kStagesF * 2 * kScaleAtomBytes;
+    static constexpr int bars = ids + kStagesF * kIdAtomBytes;
+    static constexpr int words = bars + 256;
+    static constexpr int luts = words + 64;
+    static constexpr int total = luts + 128 + 1024 /* alignment slack */;
+};
+
+// One lane of a converged warp (the same lane every time).  Loops that issue TMA / tcgen05
+// instructions run with the whole warp converged and only predicate the instruction on this,
+// so that addresses and descriptors stay in uniform registers instead of being moved per instruction.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFusedThreads, 1)
+gemm_tc2f_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapCodes,
+                 const __grid_constant__ CUtensorMap mapSfA, const __grid_constant__ CUtensorMap mapSfB,
+                 const uint8_t *__restrict__ idsB, int M, int N, int K, int row_tiles_a, int row_tiles_b,
+                 void *__restrict__ Y, int64_t ldy, int out_bf16) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *const base_ptr = smem_raw + (base - smem_u32(smem_raw));
+    auto a_tile = [&](int s) { return base + FusedSmem::a + (uint32_t)s * kHalfTile; };
+    auto code_tile = [&](int s) { return base + FusedSmem::codes + (uint32_t)s * kCodeTile; };
+    auto dec_tile = [&](int d) { return base + FusedSmem::dec + (uint32_t)d * kHalfTile; };
+    auto sfa_tile = [&](int s) { return base + FusedSmem::sfa + (uint32_t)s * kScaleAtomBytes; };
+    auto sfb_tile = [&](int s) { return base + FusedSmem::sfb + (uint32_t)s * 2 * kScaleAtomBytes; };
+    auto id_tile = [&](int s) { return base + FusedSmem::ids + (uint32_t)s * kIdAtomBytes; };
+    const uint32_t bars = base + FusedSmem::bars;
+    auto full_bar = [&](int s) { return bars + 8u * s; };                         // leader: A + scales of both CTAs
+    auto empty_bar = [&](int s) { return bars + 8u * (kStagesF + s); };           // both: stage s consumed
+    auto raw_bar = [&](int s) { return bars + 8u * (2 * kStagesF + s); };         // local: codes + ids landed
+    auto dec_full_bar = [&](int d) { return bars + 8u * (3 * kStagesF + d); };    // leader: buffer d decoded in both CTAs
+    auto dec_empty_bar = [&](int d) { return bars + 8u * (3 * kStagesF + kDecBufs + d); };   // both: buffer d consumed
+    const uint32_t tmem_full_bar = bars + 8u * (3 * kStagesF + 2 * kDecBufs);
+    volatile uint32_t *const shared_words = (volatile uint32_t *)(base_ptr + FusedSmem::words);
+    volatile uint32_t *const tmem_slot = shared_words;
+    volatile uint32_t *const abort_flag = shared_words + 1;
+    uint32_t *const luts = (uint32_t *)(base_ptr + FusedSmem::luts);              // e4m3_lo[16], e4m3_hi[16]
+
+    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    const uint32_t rank = cluster_ctarank();
+    const int pair = blockIdx.x / 2;
+    const int m0 = pair * 256 + (int)rank * 128;
+    const int n0 = blockIdx.y * 256;
+    const int k_tiles = (K + BK - 1) / BK;
+    constexpr int kAccCols = 256, kSfaCol = 256, kSfbCol = 260, kTmemCols = 512;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < kStagesF; s++) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+            mbar_init(raw_bar(s), 1);
+        }
+        for (int d = 0; d < kDecBufs; d++) {
+            mbar_init(dec_full_bar(d), 2);                        // one arrival per CTA of the pair
+            mbar_init(dec_empty_bar(d), 1);
+        }
+        mbar_init(tmem_full_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (threadIdx.x < 32) {
+        luts[threadIdx.x] = threadIdx.x < 16 ? c_tables.e4m3_lo[threadIdx.x] : c_tables.e4m3_hi[threadIdx.x - 16];
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32((const void *)tmem_slot)), "r"((uint32_t)kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tcgen05_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        // ---- TMA producer (whole warp converged, one elected lane issues) ----
+        constexpr uint32_t tx_pair = 2u * (kHalfTile + 3u * kScaleAtomBytes);
+        const int my_row_tile = blockIdx.y * 2 + (int)rank;                       // this CTA's 128 rows of B
+        const bool have_ids = my_row_tile < row_tiles_b;
+        int s = 0;
+        uint32_t ph = 1;
+        for (int kt = 0; kt < k_tiles; kt++) {
+            mbar_wait(empty_bar(s), ph, abort_flag);
+            if (*abort_flag) break;
+            const uint32_t fb = map_to_cta(full_bar(s), 0);
+            if (elect_one()) {
+                mbar_expect_tx(raw_bar(s), kCodeTile + (have_ids ? kIdAtomBytes : 0));
+                tma_load_2d(code_tile(s), &mapCodes, kt * (BK / 2), n0 + (int)rank * 128, raw_bar(s));
+                if (have_ids)
+                    bulk_load(id_tile(s), idsB + ((int64_t)kt * row_tiles_b + my_row_tile) * kIdAtomBytes, kIdAtomBytes,
+                              raw_bar(s));
+                if (rank == 0) mbar_expect_tx(full_bar(s), tx_pair);
+                tma_load_2d_pair(a_tile(s), &mapA, kt * BK, m0, fb);
+                tma_load_2d_pair(sfa_tile(s), &mapSfA, 0, kt * row_tiles_a + pair * 2 + (int)rank, fb);
+                tma_load_2d_pair(sfb_tile(s), &mapSfB, 0, kt * row_tiles_b + blockIdx.y * 2, fb);
+            }
+            __syncwarp();
+            if (++s == kStagesF) { s = 0; ph ^= 1u; }
+        }
+    } else if (warp == 1) {
+        if (rank == 0) {
+            // ---- MMA issuer (leader CTA; whole warp converged, one elected lane issues) ----
+            // Everything that does not depend on the k-step is computed once: descriptor high words,
+            // the four instruction descriptors (one per scale byte), TMEM addresses.
+            const uint32_t hi_op = desc_hi(1024, kLayoutSwizzle128), hi_sf = desc_hi(128, kLayoutNone);
+            const uint32_t lo_a0 = (a_tile(0) >> 4) | 1u << 16, lo_b0 = (dec_tile(0) >> 4) | 1u << 16;
+            const uint32_t lo_sfa0 = sfa_tile(0) >> 4, lo_sfb0 = sfb_tile(0) >> 4;
+            const uint32_t idesc0 = (uint32_t)(256 >> 3) << 17 | 1u << 23 | (uint32_t)(256 >> 4) << 24;
+            const uint32_t t_sfa = tmem + kSfaCol, t_sfb = tmem + kSfbCol;
+            int s = 0, d = 0;
+            uint32_t ph_s = 0, ph_d = 0;
+            for (int kt = 0; kt < k_tiles; kt++) {
+                mbar_wait(full_bar(s), ph_s, abort_flag);
+                mbar_wait(dec_full_bar(d), ph_d, abort_flag);
+                if (*abort_flag) break;
+                tcgen05_fence_after();
+                const uint32_t lo_sfa = lo_sfa0 + (uint32_t)s * (kScaleAtomBytes >> 4);
+                const uint32_t lo_sfb = lo_sfb0 + (uint32_t)s * (2 * kScaleAtomBytes >> 4);
+                const uint32_t lo_a = lo_a0 + (uint32_t)s * (kHalfTile >> 4), lo_b = lo_b0 + (uint32_t)d * (kHalfTile >> 4);
+                if (elect_one()) {
+                    tcgen05_cp_pair(t_sfa, desc_join(lo_sfa, hi_sf));
+                    tcgen05_cp_pair(t_sfb, desc_join(lo_sfb, hi_sf));
+                    tcgen05_cp_pair(t_sfb + 4, desc_join(lo_sfb + (kScaleAtomBytes >> 4), hi_sf));
+#pragma unroll
+                    for (int k = 0; k < BK / 32; k++)
+                        tcgen05_mma_mxf8_pair(tmem, desc_join(lo_a + 2 * k, hi_op), desc_join(lo_b + 2 * k, hi_op),
+                                              idesc0 | (uint32_t)k << 4 | (uint32_t)k << 29, t_sfa, t_sfb, (kt | k) != 0);
+                    tcgen05_commit_pair(empty_bar(s));
+                    tcgen05_commit_pair(dec_empty_bar(d));
+                }
+                __syncwarp();
+                if (++s == kStagesF) { s = 0; ph_s ^= 1u; }
+                if (++d == kDecBufs) { d = 0; ph_d ^= 1u; }
+            }
+            if (elect_one()) tcgen05_commit_pair(tmem_full_bar);
+            __syncwarp();
+        }
+    } else if (warp < 2 + kDecodeWarps) {
+        // ---- decode warps, in kDecodeGroups groups of four: group g takes the k-steps kt = g (mod groups),
+        // so that consecutive k-steps are decoded concurrently; thread j of a group expands row j ----
+        const int group = (warp - 2) / 4;
+        const int j = ((warp - 2) % 4) * 32 + lane;
+        const uint32_t swz64 = (uint32_t)(j >> 1) & 3u, swz128 = (uint32_t)j & 7u;
+        const uint32_t dec_full_leader = map_to_cta(dec_full_bar(0), 0);
+        for (int kt = group; kt < k_tiles; kt += kDecodeGroups) {
+            const int s = kt % kStagesF, d = kt % kDecBufs;
+            mbar_wait(raw_bar(s), (kt / kStagesF) & 1, abort_flag);
+            mbar_wait(dec_empty_bar(d), ((kt / kDecBufs) & 1) ^ 1, abort_flag);
+            if (*abort_flag) break;
+            const uint8_t *codes = base_ptr + FusedSmem::codes + s * kCodeTile + j * 64;
+            const uint32_t ids16 = *(const uint16_t *)(base_ptr + FusedSmem::ids + s * kIdAtomBytes + j * 2);
+            uint8_t *dst = base_ptr + FusedSmem::dec + d * kHalfTile + j * 128;
+            uint4 w[4];
+#pragma unroll
+            for (int c = 0; c < 4; c++) w[c] = *(const uint4 *)(codes + 16 * (c ^ swz64));
+#pragma unroll
+            for (int c = 0; c < 4; c++) {
+                const uint32_t id = (ids16 >> (4 * c)) & 15u;
+                const uint32_t lo = luts[id], hi = luts[16 + id];
+                uint32_t o[8];
+                decode_word(w[c].x, lo, hi, o[0], o[1]);
+                decode_word(w[c].y, lo, hi, o[2], o[3]);
+                decode_word(w[c].z, lo, hi, o[4], o[5]);
+                decode_word(w[c].w, lo, hi, o[6], o[7]);
+                *(uint4 *)(dst + 16 * ((2 * c) ^ swz128)) = make_uint4(o[0], o[1], o[2], o[3]);
+                *(uint4 *)(dst + 16 * ((2 * c + 1) ^ swz128)) = make_uint4(o[4], o[5], o[6], o[7]);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA's reads
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory"); // the four warps of this group are done
+            if (j == 0) mbar_arrive_cluster(dec_full_leader + 8u * d);
+        }
+    } else {
+        // ---- epilogue ----
+        mbar_wait(tmem_full_bar, 0, abort_flag, 256);
+        tcgen05_fence_after();
+        const int quad = warp % 4;
+        const int row = m0 + quad * 32 + lane;
+        const bool vec_ok = (ldy % 8 == 0) && (((uintptr_t)Y & 15u) == 0);
+#pragma unroll 1
+        for (int c = 0; c < kAccCols / 32; c++) {
+            uint32_t r[32];
+            tcgen05_ld_32x32b_x32(tmem + ((uint32_t)(quad * 32) << 16) + c * 32, r);
+            tcgen05_wait_ld();
+            const int col = n0 + c * 32;
+            if (row >= M || col >= N || *abort_flag) continue;
+            store_chunk(r, Y, ldy, row, col, N, out_bf16, vec_ok);
+        }
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();
     if (warp == 1) {
         tcgen05_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols)
@@ -518,6 +760,39 @@ inline cudaError_t launch_pair(const uint8_t *a8, const uint8_t *sfa, int64_t M,
     return cudaGetLastError();
 }
 
+// Tensor map of packed codes [rows][K/2] bytes: box = 64 bytes x 128 rows, 64-byte swizzle, zero fill.
+inline bool make_codes_map(CUtensorMap *map, const uint8_t *ptr, int64_t rows, int64_t K) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
+    cuuint32_t box[2] = {64, 128};
+    cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void *)ptr, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+           CUDA_SUCCESS;
+}
+
+// A as operand bytes + scale atoms, B as a packed operand (codes, ids, scale atoms).
+inline cudaError_t launch_fused(const uint8_t *a8, const uint8_t *sfa, int64_t M, const QView &B, int64_t K, void *Y,
+                                bool out_bf16, int64_t ldy, cudaStream_t st) {
+    CUtensorMap mapA, mapCodes, mapSfA, mapSfB;
+    const int64_t N = B.rows, rta = row_tiles(M), rtb = row_tiles(N), kg = k_groups(K);
+    if (!make_operand_map(&mapA, a8, M, K, 128) || !make_codes_map(&mapCodes, B.codes, N, K) ||
+        !make_scale_map(&mapSfA, sfa, rta * kg, 1) || !make_scale_map(&mapSfB, B.scales, rtb * kg, 2))
+        return cudaErrorInvalidValue;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tc2f_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedSmem::total);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    dim3 grid((unsigned)(2 * ((M + 255) / 256)), (unsigned)((N + 255) / 256));
+    gemm_tc2f_kernel<<<grid, kFusedThreads, FusedSmem::total, st>>>(mapA, mapCodes, mapSfA, mapSfB, B.ids, (int)M, (int)N,
+                                                                   (int)K, (int)rta, (int)rtb, Y, ldy, out_bf16 ? 1 : 0);
+    return cudaGetLastError();
+}
+
 template <int BN, int MODE = 0>
 inline cudaError_t launch(const uint8_t *a8, const uint8_t *sfa, int64_t M, const uint8_t *b8, const uint8_t *sfb,
                           int64_t N, int64_t K, void *Y, bool out_bf16, int64_t ldy, cudaStream_t st) {
@@ -544,10 +819,22 @@ inline bool tc_supported(int64_t M, int64_t N, int64_t K) {
 inline size_t tc_operand_bytes(int64_t rows, int64_t K) { return ((size_t)rows * (size_t)K + 255) & ~(size_t)255; }
 inline size_t tc_gemm_workspace(int64_t M, int64_t N, int64_t K) { return tc_operand_bytes(M, K) + tc_operand_bytes(N, K); }
 
-inline cudaError_t tc_gemm(const uint8_t *a8, const uint8_t *sfa, int64_t M, const uint8_t *b8, const uint8_t *sfb,
-                           int64_t N, int64_t K, void *Y, bool out_bf16, int64_t ldy, cudaStream_t st) {
+inline int tc_variant() {
     static int variant = -1;
     if (variant < 0) { const char *v = getenv("BD_TC_VARIANT"); variant = v ? atoi(v) : 0; }
+    return variant;
+}
+// true: B is consumed in packed form by the fused kernel (no decoded copy of B needed)
+inline bool tc_fused_b() { return tc_variant() == 0; }
+
+inline cudaError_t tc_gemm_fused(const uint8_t *a8, const uint8_t *sfa, int64_t M, const QView &B, int64_t K, void *Y,
+                                 bool out_bf16, int64_t ldy, cudaStream_t st) {
+    return tc::launch_fused(a8, sfa, M, B, K, Y, out_bf16, ldy, st);
+}
+
+inline cudaError_t tc_gemm(const uint8_t *a8, const uint8_t *sfa, int64_t M, const uint8_t *b8, const uint8_t *sfb,
+                           int64_t N, int64_t K, void *Y, bool out_bf16, int64_t ldy, cudaStream_t st) {
+    const int variant = tc_variant();
     if (variant == 1) return tc::launch<128>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
     if (variant == 3) return tc::launch<256, 1>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);
     if (variant == 4) return tc::launch<256, 2>(a8, sfa, M, b8, sfb, N, K, Y, out_bf16, ldy, st);

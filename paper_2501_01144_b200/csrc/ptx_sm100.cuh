@@ -13,7 +13,7 @@ __device__ uint32_t g_status_word = 0;
 
 namespace tc {
 
-constexpr uint32_t kSpinLimit = 1u << 26;
+constexpr uint32_t kSpinLimit = 1u << 24;   // polls; with the sleeps below roughly a second
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -33,10 +33,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  `abort_flag` (shared memory) is raised by the first wait that runs out;
-// later waits return at once so that the CTA drains quickly.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag) {
+// later waits return at once so that the CTA drains quickly.  After a few failed polls the
+// warp sleeps between polls (`sleep_ns`), so that a long wait does not take issue slots
+// from the warps that are working.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          uint32_t sleep_ns = 32) {
     for (uint32_t spin = 0; spin < kSpinLimit; spin++) {
         if (mbar_try_wait(bar, parity)) return;
+        if (spin >= 8) __nanosleep(sleep_ns);
         if ((spin & 1023u) == 1023u && *abort_flag) return;
     }
     *abort_flag = 1;
