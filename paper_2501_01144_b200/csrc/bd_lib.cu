@@ -98,24 +98,16 @@ bd_status gemm_dispatch(const QView &A, const QView &B, void *Y, bd_dtype ydt, i
     if (use_tc(A.rows, B.rows, A.K)) {
         if (!tc_supported(A.rows, B.rows, A.K)) return BD_ERR_UNSUPPORTED;
         size_t need = tc_gemm_workspace(A.rows, B.rows, A.K);
-        if (need && (!ws || ws_bytes < need)) return BD_ERR_WORKSPACE;
-        if (need && ((uintptr_t)ws & 255u)) return BD_ERR_ALIGN;
-        // decode both operands to plain operand-byte matrices, then the block-scaled MMA kernel
+        if (!ws || ws_bytes < need) return BD_ERR_WORKSPACE;
+        if ((uintptr_t)ws & 255u) return BD_ERR_ALIGN;
+        // A is expanded to operand bytes by a kernel; B stays packed and is expanded inside the GEMM
         uint8_t *a8 = (uint8_t *)ws;
-        uint8_t *b8 = a8 + tc_operand_bytes(A.rows, A.K);
         const int nb = (int)(A.K / kBlock);
         decode_e4m3_kernel<<<grid_for(A.rows * nb, 256), 256, 0, st>>>(A, a8, nb);
-        if (tc_fused_b()) {
-            bd_status s = launch_result(1);
-            if (s) return s;
-            g_launches += 1;
-            return cuda_result(tc_gemm_fused(a8, A.scales, A.rows, B, A.K, Y, ydt == BD_BF16, ldy, st));
-        }
-        decode_e4m3_kernel<<<grid_for(B.rows * nb, 256), 256, 0, st>>>(B, b8, nb);
-        bd_status s = launch_result(2);
+        bd_status s = launch_result(1);
         if (s) return s;
         g_launches += 1;
-        return cuda_result(tc_gemm(a8, A.scales, A.rows, b8, B.scales, B.rows, A.K, Y, ydt == BD_BF16, ldy, st));
+        return cuda_result(tc::launch(a8, A.scales, A.rows, B, A.K, Y, ydt == BD_BF16, ldy, st));
     }
     if (ydt == BD_F32) return launch_simt<float>(A, B, Y, ldy, st);
     return launch_simt<__nv_bfloat16>(A, B, Y, ldy, st);
@@ -219,8 +211,10 @@ bd_status bd_linear_workspace_size(int64_t M, int64_t N, int64_t K, size_t *byte
     if (K % kBlock) return BD_ERR_SHAPE;
     size_t c, i, s;
     bd_qtensor_sizes(M, K, &c, &i, &s);
-    size_t gemm_ws = tc_supported(M, N, K) ? tc_gemm_workspace(M, N, K) : 0;
-    *bytes = align256(c) + align256(i) + align256(s) + align256(gemm_ws);
+    // tensor-core path: scale atoms + operand bytes of X; CUDA-core path: a packed X
+    const size_t tc_bytes = tc_supported(M, N, K) ? align256(s) + tc_gemm_workspace(M, N, K) : 0;
+    const size_t simt_bytes = align256(c) + align256(i) + align256(s);
+    *bytes = tc_bytes > simt_bytes ? tc_bytes : simt_bytes;
     return BD_OK;
 }
 
@@ -244,29 +238,19 @@ bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_
     if (use_tc(M, N, K)) {
         if (!tc_supported(M, N, K)) return BD_ERR_UNSUPPORTED;
         // tensor-core path: the quantizer writes the operand bytes and the scale atoms directly
-        // (no codes, no ids); the weights are decoded to operand bytes; then the block-scaled MMA
+        // (no codes, no ids); the weights stay packed and are expanded inside the GEMM
         uint8_t *sfa = (uint8_t *)p;
         uint8_t *a8 = sfa + align256(sc);
-        uint8_t *b8 = a8 + tc_operand_bytes(M, K);
         bd_qtensor xq{nullptr, nullptr, sfa, M, K};
         s = launch_contig<BD_SELECT_TWO_STAGE, false, true>(X, xdtype, ldx, view_of(&xq), a8, st);
         if (s) return s;
-        QView W = view_of(Wq);
-        if (tc_fused_b()) {
-            g_launches += 1;
-            return cuda_result(tc_gemm_fused(a8, sfa, M, W, K, Y, ydtype == BD_BF16, ldy, st));
-        }
-        decode_e4m3_kernel<<<grid_for(N * (K / kBlock), 256), 256, 0, st>>>(W, b8, (int)(K / kBlock));
-        s = launch_result();
-        if (s) return s;
         g_launches += 1;
-        return cuda_result(tc_gemm(a8, sfa, M, b8, W.scales, N, K, Y, ydtype == BD_BF16, ldy, st));
+        return cuda_result(tc::launch(a8, sfa, M, view_of(Wq), K, Y, ydtype == BD_BF16, ldy, st));
     }
     bd_qtensor xq{p, p + align256(c), p + align256(c) + align256(i), M, K};
-    char *gemm_ws = p + align256(c) + align256(i) + align256(sc);
     s = launch_contig<BD_SELECT_TWO_STAGE, true, false>(X, xdtype, ldx, view_of(&xq), nullptr, st);
     if (s) return s;
-    return gemm_dispatch(view_of(&xq), view_of(Wq), Y, ydtype, ldy, gemm_ws, need - (size_t)(gemm_ws - p), st);
+    return gemm_dispatch(view_of(&xq), view_of(Wq), Y, ydtype, ldy, nullptr, 0, st);
 }
 
 bd_status bd_linear_noalloc(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, const bd_qtensor *Wq,

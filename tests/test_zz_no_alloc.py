@@ -45,7 +45,7 @@ def test_noalloc_matches_linear_on_two_calls_in_a_row():
 
 
 def test_noalloc_refuses_problems_beyond_its_scratch():
-    M, N, K = 2048, 14336, 4096
+    M, N, K = 8192, 4096, 14336
     assert bd.linear_workspace_size(M, N, K) > bd.binding.NOALLOC_SCRATCH_BYTES
     x = torch.zeros(M, K, dtype=torch.bfloat16, device="cuda")
     wq = bd.QTensor(N, K)
