@@ -80,7 +80,7 @@ bd_status launch_simt(const QView &A, const QView &B, void *Y, int64_t ldy, cuda
 bool use_tc(int64_t M, int64_t N, int64_t K) {
     if (g_gemm_impl == BD_GEMM_SIMT) return false;
     if (g_gemm_impl == BD_GEMM_TCGEN05) return true;
-    return tc_supported(M, N, K) && M >= 64;
+    return tc_supported(M, N, K) && (M >= 16 || (int64_t)N * K >= (1 << 22));
 }
 
 bd_status check_gemm(const bd_qtensor *A, const bd_qtensor *B, const void *Y, bd_dtype ydt, int64_t ldy) {
