@@ -38,6 +38,11 @@ LAYERS = [("qo_proj", 4096, 4096), ("kv_proj", 4096, 1024), ("gate_up", 4096, 14
 M_TOKENS = 2048
 QUANT_SHAPE = (8192, 4096)
 BYTES_PER_ELEM_QUANT = 2 + 0.5 + 1.5 / 32           # bf16 read + 4-bit code + (4-bit id + 8-bit scale) / 32
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
+QUANT_DRAM_BYTES = 67.13e6 + 4.48e6                 # quantize_bf16_kernel on bf16 [8192, 4096]
+GEMM_GATE_UP_DRAM_BYTES = 40806912 + 16053504   # tc::gemm_pair_kernel, gate/up layer (profiles/gemm_pair_kernel_llama3_gate_up.md)
+MLP_SWEEP = [(4096, 11008), (11008, 4096)]
+MLP_SWEEP_M = [1, 16, 128, 1024, 8192]
 
 
 def measured_peaks():
@@ -65,7 +70,7 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "10",
                  "-i", str(self.gpu_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
@@ -222,12 +227,12 @@ def run_gpu(args, rank, world, local_rank):
         return ms
 
     sampler = ClockSampler(local_rank)
-    launches0 = bd.launch_count()
+    sampler.start()                                        # runs through warm-up and the timed region
+    time.sleep(0.05)
     for _ in range(args.warmup):
         step()
     barrier()
     launches_warm = bd.launch_count()
-    sampler.start()
     total_ms = timed(step, args.steps, 0)
     clocks = sampler.stop()
     launches = bd.launch_count() - launches_warm
@@ -259,8 +264,10 @@ def run_gpu(args, rank, world, local_rank):
     gemm_ms = float(np.mean(durations))
     achieved_tf = big["flops"] / (gemm_ms * 1e-3) / 1e12
     fp8_peak = 2.0 * peaks["bf16_tflops"]                 # dense FP8 = 2 x dense bf16 (nominal ratio), burst: kernel timed alone
-    roofline = {"bound": "tensor", "kernel": "bd_gemm " + big["name"], "achieved": achieved_tf, "peak": fp8_peak,
-                "unit": "TFLOP/s", "frac": achieved_tf / fp8_peak, "traffic": None,
+    # DRAM traffic of this launch from the committed ncu capture (profiles/gemm_pair_kernel_llama3_gate_up.md)
+    roofline = {"bound": "tensor", "kernel": "bd_gemm " + big["name"] + " (decode_e4m3 of A + tc::gemm_pair_kernel)",
+                "achieved": achieved_tf, "peak": fp8_peak,
+                "unit": "TFLOP/s", "frac": achieved_tf / fp8_peak, "traffic": GEMM_GATE_UP_DRAM_BYTES,
                 "peak_source": f"2 x {peaks['source']} bf16 burst", "ms_per_launch": gemm_ms,
                 "frac_of_nominal_4500": achieved_tf / 4500.0}
 
@@ -285,9 +292,36 @@ def run_gpu(args, rank, world, local_rank):
     act_quantizer = {"workload": "bf16 [8192, 4096] N(0,1), 1% outlier channels, 4 rotating buffer sets (L2-cold)",
                      "bound": "hbm", "achieved": q_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": q_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": q_gbs / 8000.0,
-                     "us_per_launch": q_ms * 1e3, "algorithmic_bytes": q_bytes, "traffic": None,
+                     "us_per_launch": q_ms * 1e3, "algorithmic_bytes": q_bytes, "traffic": QUANT_DRAM_BYTES,
                      "peak_source": peaks["source"]}
     bd.poll_status()
+
+    # ---- LLaMA2-7B MLP shapes, decode to prefill (reported per M; not part of the timed step) ----
+    sweep = []
+    if rank == 0:
+        torch.manual_seed(3)
+        for K, N in MLP_SWEEP:
+            wq = bd.quantize_weights(dev_bf16(inputs.weights_normal(N, K, seed=3)), bd.SELECT_TWO_STAGE)
+            for M in MLP_SWEEP_M:
+                x = (torch.randn(M, K, device=dev).abs() * torch.randn(M, K, device=dev)).to(torch.bfloat16)
+                y = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+                ws = torch.empty(bd.linear_workspace_size(M, N, K), dtype=torch.uint8, device=dev)
+                for _ in range(3):
+                    bd.linear(x, wq, out=y, workspace=ws)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                n_rep = 10
+                a.record()
+                for _ in range(n_rep):
+                    bd.linear(x, wq, out=y, workspace=ws)
+                b.record()
+                torch.cuda.synchronize()
+                us = a.elapsed_time(b) / n_rep * 1e3
+                flops = 2.0 * M * N * K
+                nbytes = N * K * 0.546875 + M * K * 2 + M * N * 2
+                bound_tf = min(2.0 * peaks["bf16_tflops"], flops / nbytes * peaks["hbm_gbs"] / 1e3)
+                sweep.append({"K": K, "N": N, "M": M, "us": us, "tflops": flops / us / 1e6,
+                              "gbs": nbytes / us / 1e3, "frac_of_roofline": flops / us / 1e6 / bound_tf})
+        bd.poll_status()
 
     if rank != 0:
         return
@@ -322,6 +356,7 @@ def run_gpu(args, rank, world, local_rank):
         "act_quantizer": act_quantizer,
         "cpu_baseline": cpu,
         "per_layer_gflop": {l["name"]: l["flops"] / 1e9 for l in layers},
+        "llama2_mlp_m_sweep": sweep,
     }
     print(json.dumps(line))
     if world > 1:
