@@ -52,7 +52,20 @@ bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out
         case BD_F32: quantize_contig_kernel<BD_F32, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad); break;
         case BD_BF16:
             if (SELECT == BD_SELECT_TWO_STAGE)
-                quantize_bf16_kernel<WC, WE><<<grid, 256, 0, st>>>((const uint16_t *)X, ld, out, e4m3, rows_pad, nb, nb_pad);
+            {
+                // programmatic dependent launch: the blocks may be scheduled while the previous kernel of the
+                // stream drains; the kernel waits for that kernel's results before it touches global memory
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(grid);
+                cfg.blockDim = dim3(256);
+                cfg.stream = st;
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+                attr[0].val.programmaticStreamSerializationAllowed = 1;
+                cfg.attrs = attr;
+                cfg.numAttrs = 1;
+                cudaLaunchKernelEx(&cfg, quantize_bf16_kernel<WC, WE>, (const uint16_t *)X, ld, out, e4m3, rows_pad, nb, nb_pad);
+            }
             else
                 quantize_contig_kernel<BD_BF16, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad);
             break;

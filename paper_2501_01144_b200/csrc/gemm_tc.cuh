@@ -257,6 +257,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
     cluster_sync_all();                                           // both CTAs: barriers initialised, TMEM allocated
     tcgen05_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // programmatic dependent launch: everything above overlapped the tail of the previous kernel in the
+    // stream; its results (the operand bytes the quantizer wrote) are read only after this point
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ---- TMA producer (whole warp converged, one elected lane issues) ----
@@ -538,10 +542,18 @@ inline cudaError_t launch(const uint8_t *a8, const uint8_t *sfa, int64_t M, cons
     const int tiles = sc.m_pairs * sc.n_tiles;
     const int resident = max_resident_clusters();
     sc.clusters = tiles < resident ? tiles : resident;
-    gemm_pair_kernel<<<dim3(2 * sc.clusters), kThreads, Smem::total, st>>>(
-        mapA, mapCodes, mapSfA, mapSfB, B.ids, sc, (int)M, (int)N, (int)rta, (int)rtb, Y, ldy, out_bf16 ? 1 : 0, mapY,
-        use_tma_store);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * sc.clusters);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = Smem::total;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start while the previous kernel drains
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_pair_kernel, mapA, mapCodes, mapSfA, mapSfB, (const uint8_t *)B.ids, sc, (int)M,
+                              (int)N, (int)rta, (int)rtb, Y, ldy, out_bf16 ? 1 : 0, mapY, use_tma_store);
 }
 
 }  // namespace tc

@@ -277,6 +277,7 @@ __global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel
                                                             int nb_pad) {
     __shared__ SmemTables tab;
     load_tables(tab);
+    asm volatile("griddepcontrol.wait;" ::: "memory");           // the source may be the previous kernel's output
     int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= rows_pad * nb_pad) return;
     int64_t r = t / nb_pad;
