@@ -402,27 +402,34 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                     // the previous pass's tensor store must have finished reading the staging buffer
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     __syncwarp();
+                    if (out_bf16) {
+                        // 64 columns: four loads in flight, one wait
+                        uint32_t r[4][16];
 #pragma unroll
-                    for (int c = 0; c < 4; c++) {
-                        if (!out_bf16 && c >= 2) break;
-                        uint32_t r[16];
-                        tcgen05_ld_32x32b_x16(t_base + pass * cols_per_pass + c * 16, r);
+                        for (int c = 0; c < 4; c++) tcgen05_ld_32x32b_x16(t_base + pass * 64 + c * 16, r[c]);
                         tcgen05_wait_ld();
-                        if (out_bf16) {                               // 16 columns -> 32 bytes = chunks 2c, 2c + 1
+#pragma unroll
+                        for (int c = 0; c < 4; c++) {                 // 16 columns -> 32 bytes = chunks 2c, 2c + 1
                             uint32_t p[8];
 #pragma unroll
                             for (int j = 0; j < 8; j++) {
-                                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+                                __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[c][2 * j]), __uint_as_float(r[c][2 * j + 1]));
                                 p[j] = *(uint32_t *)&h;
                             }
                             *(uint4 *)(stage_ptr + 16 * ((2 * c) ^ lane_swz)) = make_uint4(p[0], p[1], p[2], p[3]);
                             *(uint4 *)(stage_ptr + 16 * ((2 * c + 1) ^ lane_swz)) = make_uint4(p[4], p[5], p[6], p[7]);
-                        } else {                                      // 16 columns -> 64 bytes = chunks 4c .. 4c + 3
+                        }
+                    } else {
+                        uint32_t r[2][16];
+#pragma unroll
+                        for (int c = 0; c < 2; c++) tcgen05_ld_32x32b_x16(t_base + pass * 32 + c * 16, r[c]);
+                        tcgen05_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 2; c++)                   // 16 columns -> 64 bytes = chunks 4c .. 4c + 3
 #pragma unroll
                             for (int q = 0; q < 4; q++)
                                 *(uint4 *)(stage_ptr + 16 * ((4 * c + q) ^ lane_swz)) =
-                                    make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
-                        }
+                                    make_uint4(r[c][4 * q], r[c][4 * q + 1], r[c][4 * q + 2], r[c][4 * q + 3]);
                     }
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
