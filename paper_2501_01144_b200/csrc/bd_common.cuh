@@ -102,8 +102,8 @@ constexpr uint64_t int_lut(int d) {
 //   block-scaled MMA scale factors (32 lanes x 16 bytes, four row groups side by
 //   side).  Padding entries hold 0.
 //
-// ids: atoms of 256 bytes in the same atom order; (row r, block b) is nibble
-//   b % 2 of byte (r % 128) * 2 + (b % 4) / 2.
+// ids: atoms of 256 bytes in the same atom order and the same row order as the scales: (row r,
+//   block b) is nibble b % 2 of byte (r % 32) * 8 + (r % 128 / 32) * 2 + (b % 4) / 2.
 // ---------------------------------------------------------------------------
 __host__ __device__ inline int64_t row_tiles(int64_t rows) { return (rows + kRowTile - 1) / kRowTile; }
 __host__ __device__ inline int64_t k_groups(int64_t K) { return (K / kBlock + kBlocksPerAtom - 1) / kBlocksPerAtom; }
@@ -115,8 +115,25 @@ __host__ __device__ inline int64_t scale_offset(int64_t rows, int64_t r, int64_t
 }
 __host__ __device__ inline int64_t id_byte_offset(int64_t rows, int64_t r, int64_t b) {
     int64_t atom = (b / kBlocksPerAtom) * row_tiles(rows) + r / kRowTile;
-    return atom * kIdAtomBytes + (r % kRowTile) * 2 + (b % kBlocksPerAtom) / 2;
+    int rr = (int)(r % kRowTile);
+    return atom * kIdAtomBytes + (rr % 32) * 8 + (rr / 32) * 2 + (int)(b % kBlocksPerAtom) / 2;
 }
+
+// n / d for n < 2^31 as one widening multiply and a shift.  With s = ceil(log2 d), k = 31 + s and
+// mul = floor(2^k / d) + 1 (which fits 32 bits), mul * d = 2^k + e with 0 < e <= d, so
+// n * mul / 2^k = n / d + n * e / (d * 2^k), and the second term is below 1 / d because n * d < 2^k.
+struct FastDiv {
+    uint32_t mul, shift;
+};
+inline FastDiv make_fast_div(uint32_t d) {
+    uint32_t s = 0;
+    while ((1ull << s) < d) s++;
+    FastDiv f;
+    f.shift = 31 + s;
+    f.mul = (uint32_t)((1ull << f.shift) / d + 1);
+    return f;
+}
+__host__ __device__ inline uint32_t fast_div(uint32_t n, FastDiv f) { return (uint32_t)(((uint64_t)n * f.mul) >> f.shift); }
 
 // Decode one code word into eight operand bytes (lo = elements 0..3, hi = 4..7)
 // through the dialect's eight-byte table.
@@ -127,14 +144,14 @@ __device__ __forceinline__ void decode_word(uint32_t w, uint32_t lut_lo, uint32_
     hi = ((w << 4) & 0x80808080u) | __byte_perm(lut_lo, lut_hi, sel >> 16);
 }
 
-// Where logical element e (0..7) of an 8-element group sits in its code word.  The order
-// inside a group is a fixed permutation chosen so that the signs of four bf16 pairs can be
-// gathered with shifts by 0, 4, 8 and 12 bits (see the bf16 quantizer); every producer and
-// consumer of code words goes through these helpers or through decode_word, and a block of
-// 32 shares one scale, so the permutation never shows outside the library.
+// Where logical element e (0..7) of an 8-element group sits in its code word: slot e.  Every
+// producer and consumer of code words goes through these helpers or through decode_word, so the
+// order inside a group is a library-internal choice (a block of 32 shares one scale).
 //   slot s: index in bits 4s..4s+2; sign in bit 8s+7 (s < 4) or 8(s-4)+3 (s >= 4);
 //   decode_word emits slot s as operand byte s (lo = slots 0..3, hi = slots 4..7).
-__host__ __device__ constexpr int slot_of(int e) { return e < 4 ? 2 * e + 1 : 2 * (e - 4); }
+// The sign positions are the ones the bf16 quantizer reaches with two byte permutes (the high
+// bytes of eight packed elements) and one shift by 4.
+__host__ __device__ constexpr int slot_of(int e) { return e; }
 __host__ __device__ constexpr int sign_bit_of_slot(int s) { return s < 4 ? 8 * s + 7 : 8 * (s - 4) + 3; }
 __host__ __device__ inline uint32_t word_index(uint32_t w, int e) { return (w >> (4 * slot_of(e))) & 7u; }
 __host__ __device__ inline uint32_t word_sign(uint32_t w, int e) { return (w >> sign_bit_of_slot(slot_of(e))) & 1u; }

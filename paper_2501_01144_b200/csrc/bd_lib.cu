@@ -43,6 +43,20 @@ int elem_bytes(bd_dtype dt) { return dt == BD_F32 ? 4 : 2; }
 
 unsigned grid_for(int64_t threads, int block) { return (unsigned)((threads + block - 1) / block); }
 
+// Resident CTAs of the bf16 quantizer on the current device (it loops over its chunks).
+unsigned quant_bf16_grid_limit() {
+    static unsigned limit[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64) return 148u * BD_QUANT_MIN_BLOCKS;
+    if (!limit[dev]) {
+        int sms = 0;
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        limit[dev] = (unsigned)(sms > 0 ? sms : 148) * BD_QUANT_MIN_BLOCKS;
+    }
+    return limit[dev];
+}
+
 template <int SELECT, bool WC, bool WE>
 bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out, uint8_t *e4m3, cudaStream_t st) {
     const int nb = (int)(out.K / kBlock), nb_pad = (int)k_groups(out.K) * kBlocksPerAtom;
@@ -51,12 +65,13 @@ bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out
     switch (dt) {
         case BD_F32: quantize_contig_kernel<BD_F32, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad); break;
         case BD_BF16:
-            if (SELECT == BD_SELECT_TWO_STAGE)
+            if (SELECT == BD_SELECT_TWO_STAGE && rows_pad * nb_pad < (1ll << 31))
             {
                 // programmatic dependent launch: the blocks may be scheduled while the previous kernel of the
                 // stream drains; the kernel waits for that kernel's results before it touches global memory
                 cudaLaunchConfig_t cfg = {};
-                cfg.gridDim = dim3(grid);
+                const unsigned chunks = (unsigned)(rows_pad / 64) * (unsigned)(nb_pad / kBlocksPerAtom);
+                cfg.gridDim = dim3(std::min(chunks, quant_bf16_grid_limit()));
                 cfg.blockDim = dim3(256);
                 cfg.stream = st;
                 cudaLaunchAttribute attr[1];
@@ -64,7 +79,9 @@ bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out
                 attr[0].val.programmaticStreamSerializationAllowed = 1;
                 cfg.attrs = attr;
                 cfg.numAttrs = 1;
-                cudaLaunchKernelEx(&cfg, quantize_bf16_kernel<WC, WE>, (const uint16_t *)X, ld, out, e4m3, rows_pad, nb, nb_pad);
+                cudaLaunchKernelEx(&cfg, quantize_bf16_kernel<WC, WE>, (const uint16_t *)X, ld, out, e4m3, chunks,
+                                   (uint32_t)nb, (uint32_t)(nb_pad / kBlocksPerAtom),
+                                   make_fast_div((uint32_t)(nb_pad / kBlocksPerAtom)));
             }
             else
                 quantize_contig_kernel<BD_BF16, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad);

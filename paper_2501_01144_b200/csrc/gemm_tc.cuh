@@ -357,7 +357,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             mbar_wait(dec_empty_bar(d), ((uint32_t)(g / kDecBufs) & 1u) ^ 1u, abort_flag);
             if (*abort_flag) break;
             const uint8_t *codes = base_ptr + Smem::codes + s * kCodeTile + j * 64;
-            const uint32_t ids16 = *(const uint16_t *)(base_ptr + Smem::ids + s * kIdAtomBytes + j * 2);
+            const uint32_t ids16 = *(const uint16_t *)(base_ptr + Smem::ids + s * kIdAtomBytes + (j % 32) * 8 + (j / 32) * 2);
             uint8_t *dst = base_ptr + Smem::dec + d * kHalfTile + j * 128;
             uint4 w[4];
 #pragma unroll

@@ -16,7 +16,7 @@
 #include "ptx_sm100.cuh"
 
 #ifndef BD_QUANT_MIN_BLOCKS
-#define BD_QUANT_MIN_BLOCKS 5
+#define BD_QUANT_MIN_BLOCKS 3
 #endif
 
 namespace bd {
@@ -145,10 +145,12 @@ __device__ __forceinline__ uint32_t prmt_b32(uint32_t a, uint32_t b, uint32_t se
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
     return r;
 }
-__device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
-    uint32_t r;
-    asm("max.u16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
-    return r;
+// max(|a|, |b|) on both bf16 halves (the result's sign bits are the xor of the inputs'); a NaN input
+// gives NaN, so non-finite inputs still show in the maximum.
+__device__ __forceinline__ uint32_t absmax_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.NaN.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
 }
 __device__ __forceinline__ uint32_t byte_sum(uint32_t x) { return (x * 0x01010101u) >> 24; }
 
@@ -249,14 +251,14 @@ __device__ __forceinline__ BlockResult quantize_mse(const uint32_t (&bits)[32], 
 // ---------------------------------------------------------------------------
 // bf16 fast path of the contiguous-axis quantizer (same thread-to-block map and outputs
 // as quantize_contig_kernel).  The 32 elements stay packed two per register:
-//   absmax      and + max.u16x2 on the packed magnitudes;
+//   absmax      max.NaN.xorsign.abs.bf16x2 on the packed elements (off the integer pipe);
 //   q5          one fma.rz per element; the upper element of a pair is used in place (the
 //               lower half then only adds less than one bf16 ulp, which cannot reach the
 //               next integer of the scaled value), the lower one after a 16-bit shift;
 //   selection   popcount of the pair's merged threshold mask shifted by q5, accumulated as
 //               nibbles, then finish_two_stage;
-//   signs       the four pair registers of a group land on the eight sign bits of the code
-//               word with shifts by 0, 4, 8 and 12.
+//   signs       two byte permutes gather the high bytes of a group's eight elements; one shift by 4
+//               puts elements 4..7 on their sign bits.
 // Blocks whose exponent is clamped (maximum below 2^-123) take the generic routine.
 // ---------------------------------------------------------------------------
 __device__ __noinline__ void quantize_bf16_clamped_block(const uint32_t (&R)[16], const SmemTables &tab,
@@ -271,84 +273,125 @@ __device__ __noinline__ void quantize_bf16_clamped_block(const uint32_t (&R)[16]
     res = quantize_two_stage(bits, tab, nonfinite);
 }
 
+// Two-stage rule on one block held as sixteen packed bf16 pairs.
+__device__ __forceinline__ void quantize_bf16_block(const uint32_t (&R)[16], const SmemTables &tab, BlockResult &res) {
+    uint32_t a[16], signs[4];
+#pragma unroll
+    for (int w = 0; w < 4; w++) {
+        // the high byte of each bf16 carries its sign in bit 7: elements 0..3 of the group keep it there,
+        // elements 4..7 move it to bit 3 of the same bytes
+        const uint32_t s03 = prmt_b32(R[4 * w], R[4 * w + 1], 0x7531u), s47 = prmt_b32(R[4 * w + 2], R[4 * w + 3], 0x7531u);
+        signs[w] = (s03 & 0x80808080u) | ((s47 >> 4) & 0x08080808u);
+    }
+#pragma unroll
+    for (int i = 0; i < 16; i++) {
+        a[i] = R[i] & 0x7fff7fffu;
+    }
+    uint32_t m = R[0];
+#pragma unroll
+    for (int i = 1; i < 16; i++) m = absmax_bf16x2(m, R[i]);      // |.| maximum per half; NaN wins; the sign bits are noise
+    m &= 0x7fff7fffu;
+    const uint32_t amax = max(m & 0xffffu, m >> 16);              // bf16 magnitude bits of the block maximum
+    if (amax >= 0x7f80u) atomicOr(&g_status_word, kStatusNonfinite);
+    const uint32_t eadj = max(amax >> 7, 2u);
+    if (eadj >= 4u) {
+        const float scale = __uint_as_float((258u - eadj) << 23);         // 2^(2 - e), e = eadj - 129
+        const uint32_t m5 = __float_as_uint(__fmaf_rz(__uint_as_float(amax << 16), scale, 8388608.0f)) & 63u;
+        const uint32_t pair = min(7u, 15u - min(15u, (m5 + 1u) >> 1));
+        const uint32_t above = tab.merged_above[pair];
+        uint32_t v[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int i = 0; i < 16; i++) {
+            const uint32_t t_lo = __float_as_uint(__fmaf_rz(__uint_as_float(a[i] << 16), scale, 8388608.0f));
+            const uint32_t t_hi = __float_as_uint(__fmaf_rz(__uint_as_float(a[i]), scale, 8388608.0f));
+            // funnel shift in wrap mode uses only the low five bits of the count, i.e. q5
+            const uint32_t v_lo = __popc(__funnelshift_r(above, 0u, t_lo));
+            const uint32_t v_hi = __popc(__funnelshift_r(above, 0u, t_hi));
+            v[i / 4] = v_lo * (1u << (4 * slot_of(2 * (i % 4)))) + v[i / 4];
+            v[i / 4] = v_hi * (1u << (4 * slot_of(2 * (i % 4) + 1))) + v[i / 4];
+        }
+        res.scale = eadj - 2u;
+        finish_two_stage(v, signs, pair, res.id, res.words);
+    } else {
+        uint32_t copy[16];                                       // only this branch spills the block to local memory
+#pragma unroll
+        for (int i = 0; i < 16; i++) copy[i] = R[i];
+        quantize_bf16_clamped_block(copy, tab, res);
+    }
+}
+
+// Work is cut into chunks of 256 blocks = 64 rows x one k-group (4 blocks) that fill whole sectors
+// of the scale and id atoms: chunk c covers k-group c % k_groups of the rows
+//   tile * 128 + 16 * half + i + 32 * j,  i in 0..15, j in 0..3,  (tile, half) = c / k_groups,
+// i.e. bytes [256 * half, +256) of the scale atom and [128 * half, +128) of the id atom.  Lane l of
+// warp w owns i = 2 w + l / 16, j = (l / 4) % 4, block b = l % 4, so the sixteen lanes of one i
+// assemble one 16-byte scale unit and one 8-byte id unit, and every warp store of scales or ids is
+// one contiguous 32- or 16-byte piece.  The four lanes of a row read 256 contiguous bytes.
+// A CTA takes chunks blockIdx.x, blockIdx.x + gridDim.x, ... (consecutive chunks walk along K) and
+// loads the next chunk's elements before it works on the current ones.
 template <bool WRITE_CODES, bool WRITE_E4M3>
 __global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel(const uint16_t *__restrict__ X, int64_t ld, QView out,
-                                                            uint8_t *__restrict__ e4m3, int64_t rows_pad, int nb,
-                                                            int nb_pad) {
+                                                            uint8_t *__restrict__ e4m3, uint32_t chunks, uint32_t nb,
+                                                            uint32_t kgroups, FastDiv div_kgroups) {
     __shared__ SmemTables tab;
     load_tables(tab);
     asm volatile("griddepcontrol.wait;" ::: "memory");           // the source may be the previous kernel's output
-    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= rows_pad * nb_pad) return;
-    int64_t r = t / nb_pad;
-    int b = (int)(t - r * nb_pad);
-    BlockResult res;
-    res.id = 0; res.scale = 0;
-    res.words[0] = res.words[1] = res.words[2] = res.words[3] = 0;
-    if (r < out.rows && b < nb) {
-        const uint4 *src = (const uint4 *)(X + r * ld + (int64_t)b * 32);
-        const uint4 l0 = __ldg(src), l1 = __ldg(src + 1), l2 = __ldg(src + 2), l3 = __ldg(src + 3);
+    const uint32_t rows = (uint32_t)out.rows, tiles = (rows + kRowTile - 1) / kRowTile, half_k = (uint32_t)(out.K / 2);
+    const uint32_t lane = threadIdx.x % 32u, b4 = lane & 3u, j = (lane >> 2) & 3u;
+    const uint32_t row_in_half = 2u * (threadIdx.x / 32u) + (lane >> 4) + 32u * j;      // + 16 * half
+    uint32_t c = blockIdx.x;
+    uint32_t r = 0, b = 0, kg = 0, th = 0;
+    bool valid = false;
+    uint4 l0 = make_uint4(0, 0, 0, 0), l1 = l0, l2 = l0, l3 = l0;
+    auto locate = [&]() {
+        th = fast_div(c, div_kgroups);
+        kg = c - th * kgroups;
+        r = (th >> 1) * kRowTile + (th & 1u) * 16u + row_in_half;
+        b = kg * kBlocksPerAtom + b4;
+        valid = r < rows && b < nb;
+        if (valid) {
+            const uint4 *src = (const uint4 *)(X + (int64_t)r * ld + b * 32u);
+            l0 = __ldg(src); l1 = __ldg(src + 1); l2 = __ldg(src + 2); l3 = __ldg(src + 3);
+        }
+    };
+    if (c < chunks) locate();
+    while (c < chunks) {                                         // the same trip count for the whole CTA
         const uint32_t R[16] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w,
                                 l2.x, l2.y, l2.z, l2.w, l3.x, l3.y, l3.z, l3.w};
-        uint32_t a[16], signs[4];
+        const uint32_t cr = r, cb = b, ckg = kg, cth = th;
+        const bool cvalid = valid;
+        c += gridDim.x;
+        if (c < chunks) locate();
+        BlockResult res;
+        res.id = 0; res.scale = 0;
+        res.words[0] = res.words[1] = res.words[2] = res.words[3] = 0;
+        if (cvalid) {
+            quantize_bf16_block(R, tab, res);
+            if (WRITE_CODES)
+                *(uint4 *)(out.codes + (uint64_t)cr * half_k + cb * 16u) =
+                    make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
+            if (WRITE_E4M3) {
+                uint32_t lo = tab.e4m3_lo[res.id], hi = tab.e4m3_hi[res.id];
+                uint32_t o[8];
 #pragma unroll
-        for (int w = 0; w < 4; w++)
-            signs[w] = (R[4 * w] & 0x80008000u) | ((R[4 * w + 1] >> 4) & 0x08000800u) |
-                       ((R[4 * w + 2] >> 8) & 0x00800080u) | ((R[4 * w + 3] >> 12) & 0x00080008u);
-#pragma unroll
-        for (int i = 0; i < 16; i++) a[i] = R[i] & 0x7fff7fffu;
-        uint32_t m = a[0];
-#pragma unroll
-        for (int i = 1; i < 16; i++) m = max_u16x2(m, a[i]);
-        const uint32_t amax = max(m & 0xffffu, m >> 16);          // bf16 magnitude bits of the block maximum
-        if (amax >= 0x7f80u) atomicOr(&g_status_word, kStatusNonfinite);
-        const uint32_t eadj = max(amax >> 7, 2u);
-        if (eadj >= 4u) {
-            const float scale = __uint_as_float((258u - eadj) << 23);     // 2^(2 - e), e = eadj - 129
-            const uint32_t m5 = __float_as_uint(__fmaf_rz(__uint_as_float(amax << 16), scale, 8388608.0f)) & 63u;
-            const uint32_t pair = min(7u, 15u - min(15u, (m5 + 1u) >> 1));
-            const uint32_t above = tab.merged_above[pair];
-            uint32_t v[4] = {0, 0, 0, 0};
-#pragma unroll
-            for (int i = 0; i < 16; i++) {
-                const uint32_t t_lo = __float_as_uint(__fmaf_rz(__uint_as_float(a[i] << 16), scale, 8388608.0f));
-                const uint32_t t_hi = __float_as_uint(__fmaf_rz(__uint_as_float(a[i]), scale, 8388608.0f));
-                // funnel shift in wrap mode uses only the low five bits of the count, i.e. q5
-                const uint32_t v_lo = __popc(__funnelshift_r(above, 0u, t_lo));
-                const uint32_t v_hi = __popc(__funnelshift_r(above, 0u, t_hi));
-                v[i / 4] = v_lo * (1u << (4 * slot_of(2 * (i % 4)))) + v[i / 4];
-                v[i / 4] = v_hi * (1u << (4 * slot_of(2 * (i % 4) + 1))) + v[i / 4];
+                for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, o[2 * w], o[2 * w + 1]);
+                uint4 *dst = (uint4 *)(e4m3 + (uint64_t)cr * (2u * half_k) + cb * 32u);
+                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
             }
-            res.scale = eadj - 2u;
-            finish_two_stage(v, signs, pair, res.id, res.words);
-        } else {
-            uint32_t copy[16];                                   // only this branch spills the block to local memory
-#pragma unroll
-            for (int i = 0; i < 16; i++) copy[i] = R[i];
-            quantize_bf16_clamped_block(copy, tab, res);
         }
-        if (WRITE_CODES)
-            *(uint4 *)(out.codes + r * (out.K / 2) + (int64_t)b * 16) =
-                make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
-        if (WRITE_E4M3) {
-            uint32_t lo = tab.e4m3_lo[res.id], hi = tab.e4m3_hi[res.id];
-            uint32_t o[8];
-#pragma unroll
-            for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, o[2 * w], o[2 * w + 1]);
-            uint4 *dst = (uint4 *)(e4m3 + r * out.K + (int64_t)b * 32);
-            dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-            dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+        // the four lanes of a row merge their scale bytes and id nibbles
+        uint32_t sc = res.scale << (8 * b4);
+        uint32_t idn = res.id << (4 * b4);
+        sc |= __shfl_xor_sync(0xffffffffu, sc, 1);
+        idn |= __shfl_xor_sync(0xffffffffu, idn, 1);
+        sc |= __shfl_xor_sync(0xffffffffu, sc, 2);
+        idn |= __shfl_xor_sync(0xffffffffu, idn, 2);
+        if (b4 == 0) {
+            const uint32_t atom = ckg * tiles + (cth >> 1), r32 = cr % 32u;
+            *(uint32_t *)(out.scales + (size_t)atom * kScaleAtomBytes + r32 * 16u + j * 4u) = sc;
+            if (WRITE_CODES) *(uint16_t *)(out.ids + (size_t)atom * kIdAtomBytes + r32 * 8u + j * 2u) = (uint16_t)idn;
         }
-    }
-    uint32_t sc = res.scale << (8 * (b & 3));
-    uint32_t idn = res.id << (4 * (b & 3));
-    sc |= __shfl_xor_sync(0xffffffffu, sc, 1);
-    idn |= __shfl_xor_sync(0xffffffffu, idn, 1);
-    sc |= __shfl_xor_sync(0xffffffffu, sc, 2);
-    idn |= __shfl_xor_sync(0xffffffffu, idn, 2);
-    if ((b & 3) == 0) {
-        *(uint32_t *)(out.scales + scale_offset(out.rows, r, b)) = sc;
-        if (WRITE_CODES) *(uint16_t *)(out.ids + id_byte_offset(out.rows, r, b)) = (uint16_t)idn;
     }
 }
 
