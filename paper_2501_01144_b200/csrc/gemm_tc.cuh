@@ -50,8 +50,11 @@ constexpr int kStages = 5;              // raw stages: A tile + packed B codes +
 constexpr int kDecBufs = 4;             // decoded-B operand buffers
 constexpr int kHalfTile = 128 * BK;     // 16 KiB: 128 rows of operand bytes
 constexpr int kCodeTile = 128 * 64;     // 8 KiB: 128 rows x 64 bytes of codes
-constexpr int kDecodeGroups = 4;
-constexpr int kDecodeWarps = 4 * kDecodeGroups;
+#ifndef BD_TC_DECODE_GROUPS
+#define BD_TC_DECODE_GROUPS 4
+#endif
+constexpr int kDecodeWarps = 16;
+constexpr int kDecodeGroups = BD_TC_DECODE_GROUPS;   // groups take alternate k-steps; 16 / groups warps share one k-step
 constexpr int kEpilogueWarp0 = 2 + kDecodeWarps;
 constexpr int kEpilogueWarps = 8;        // two per TMEM lane quadrant, each taking half of the columns
 constexpr int kThreads = 32 * (kEpilogueWarp0 + kEpilogueWarps);
@@ -66,7 +69,7 @@ struct Smem {
     static constexpr int ids = sfb + kStages * 2 * kScaleAtomBytes;
     static constexpr int bars = ids + kStages * kIdAtomBytes;
     static constexpr int words = bars + 256;
-    static constexpr int luts = words + 64;
+    static constexpr int luts = words + 256;
     static constexpr int out = ((luts + 128 + 1023) / 1024) * 1024;          // epilogue staging, 1 KiB aligned
     static constexpr int total = out + kEpilogueWarps * kStageOutBytes + 1024 /* alignment slack */;
 };
@@ -85,6 +88,19 @@ __device__ __forceinline__ bool get_item(const Schedule &sc, int c, int i, Item 
     it.tile = i * sc.clusters + c;
     return it.tile < sc.m_pairs * sc.n_tiles;
 }
+
+#ifdef BD_TC_PROFILE
+__device__ unsigned long long g_prof[32];
+#define PROF_DECL long long prof_t0 = 0; long long prof_acc[4] = {0, 0, 0, 0}; (void)prof_t0; (void)prof_acc
+#define PROF_T0 prof_t0 = clock64()
+#define PROF_ADD(i) prof_acc[i] += clock64() - prof_t0
+#define PROF_OUT(i, slot) if (cluster == 0 && rank == 0 && lane == 0) atomicAdd(&g_prof[slot], (unsigned long long)prof_acc[i])
+#else
+#define PROF_DECL
+#define PROF_T0
+#define PROF_ADD(i)
+#define PROF_OUT(i, slot)
+#endif
 
 // ---- PTX wrappers (cluster pair) ---------------------------------------------
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -268,16 +284,26 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         int s = 0;
         uint32_t ph = 1;
         Item it;
+        PROF_DECL;
         for (int i = 0; get_item(sc, cluster, i, it); i++) {
             const int m_pair = it.tile % sc.m_pairs, n_tile = it.tile / sc.m_pairs;
             const int m0 = m_pair * 256 + (int)rank * 128, n0 = n_tile * 256 + (int)rank * 128;
             const int my_row_tile = n_tile * 2 + (int)rank;                       // this CTA's 128 rows of B
             const bool have_ids = my_row_tile < row_tiles_b;
             for (int kt = 0; kt < sc.k_tiles; kt++) {
+                PROF_T0;
                 mbar_wait(empty_bar(s), ph, abort_flag);
+                PROF_ADD(0);
+#ifdef BD_TC_PROFILE
+                if (cluster == 0 && rank == 0 && lane == 0 && (i > 0 || kt >= kStages))
+                    atomicAdd(&g_prof[18], (unsigned long long)((uint32_t)clock64() - shared_words[8 + s]));
+#endif
                 if (*abort_flag) break;
                 const uint32_t fb = map_to_cta(full_bar(s), 0);
                 if (elect_one()) {
+#ifdef BD_TC_PROFILE
+                    shared_words[2 + s] = (uint32_t)clock64();
+#endif
                     mbar_expect_tx(raw_bar(s), kCodeTile + (have_ids ? kIdAtomBytes : 0));
                     tma_load_2d(code_tile(s), &mapCodes, kt * (BK / 2), n0, raw_bar(s));
                     if (have_ids)
@@ -293,6 +319,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             }
             if (*abort_flag) break;
         }
+        PROF_OUT(0, 0);
     } else if (warp == 1) {
         if (rank == 0) {
             // ---- MMA issuer (leader CTA; whole warp converged, one elected lane issues) ----
@@ -305,14 +332,32 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             const uint32_t t_sfa = tmem + kSfaCol, t_sfb = tmem + kSfbCol;
             int s = 0, d = 0;
             uint32_t ph_s = 0, ph_d = 0;
+            bool ready = false;
             Item it;
+            PROF_DECL;
+#ifdef BD_TC_PROFILE
+            const long long prof_start = clock64();
+#endif
             for (int i = 0; get_item(sc, cluster, i, it); i++) {
+                PROF_T0;
                 if (i > 0) mbar_wait(tmem_empty_bar, (uint32_t)(i - 1) & 1u, abort_flag);
+                PROF_ADD(2);
                 tcgen05_fence_after();
                 for (int kt = 0; kt < sc.k_tiles; kt++) {
-                    mbar_wait(full_bar(s), ph_s, abort_flag);
-                    mbar_wait(dec_full_bar(d), ph_d, abort_flag);
-                    if (*abort_flag) break;
+                    if (!ready) {
+                        // slow path: the probe at the end of the previous k-step found a barrier open
+                        PROF_T0;
+                        mbar_wait(full_bar(s), ph_s, abort_flag);
+                        PROF_ADD(0);
+                        PROF_T0;
+                        mbar_wait(dec_full_bar(d), ph_d, abort_flag);
+                        PROF_ADD(1);
+                        if (*abort_flag) break;
+                    }
+#ifdef BD_TC_PROFILE
+                    const uint32_t prof_iss0 = (uint32_t)clock64();
+                    if (cluster == 0 && lane == 0) atomicAdd(&g_prof[16], (unsigned long long)(prof_iss0 - shared_words[16 + d]));
+#endif
                     tcgen05_fence_after();
                     const uint32_t lo_sfa = lo_sfa0 + (uint32_t)s * (kScaleAtomBytes >> 4);
                     const uint32_t lo_sfb = lo_sfb0 + (uint32_t)s * (2 * kScaleAtomBytes >> 4);
@@ -329,21 +374,42 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
                                                   k == 0 ? first : 1u);
                         tcgen05_commit_pair(empty_bar(s));
                         tcgen05_commit_pair(dec_empty_bar(d));
+#ifdef BD_TC_PROFILE
+                        shared_words[8 + s] = (uint32_t)clock64();
+                        if (cluster == 0) atomicAdd(&g_prof[17], (unsigned long long)((uint32_t)clock64() - prof_iss0));
+#endif
                     }
                     __syncwarp();
                     if (++s == kStages) { s = 0; ph_s ^= 1u; }
                     if (++d == kDecBufs) { d = 0; ph_d ^= 1u; }
+                    // probe the next k-step's barriers now (the rings run across tiles): their shared-memory
+                    // round trip overlaps the instruction issue above instead of opening the next iteration
+                    const bool full_ok = mbar_test_wait(full_bar(s), ph_s), dec_ok = mbar_test_wait(dec_full_bar(d), ph_d);
+                    ready = full_ok && dec_ok;
+#ifdef BD_TC_PROFILE
+                    if (cluster == 0 && lane == 0 && ready) atomicAdd(&g_prof[19], 1ull);
+#endif
                 }
                 if (elect_one()) tcgen05_commit_pair(tmem_full_bar);
                 __syncwarp();
                 if (*abort_flag) break;
             }
+            PROF_OUT(0, 1);
+            PROF_OUT(1, 2);
+            PROF_OUT(2, 3);
+#ifdef BD_TC_PROFILE
+            prof_acc[3] = clock64() - prof_start;
+#endif
+            PROF_OUT(3, 4);
         }
     } else if (warp < kEpilogueWarp0) {
         // ---- decode warps, in groups of four: group g takes this CTA's k-steps g, g + groups, ...;
         // thread j of a group expands row j of the CTA's 128 B rows ----
-        const int group = (warp - 2) / 4;
-        const int j = ((warp - 2) % 4) * 32 + lane;
+        constexpr int kGroupWarps = kDecodeWarps / kDecodeGroups, kGroupThreads = 32 * kGroupWarps;
+        constexpr int kPerRow = kGroupThreads / 128, kBlocksPerThread = 4 / kPerRow;   // threads per B row, blocks per thread
+        const int group = (warp - 2) / kGroupWarps;
+        const int tg = ((warp - 2) % kGroupWarps) * 32 + lane;
+        const int j = tg / kPerRow, c0 = (tg % kPerRow) * kBlocksPerThread;
         const uint32_t swz64 = (uint32_t)(j >> 1) & 3u, swz128 = (uint32_t)j & 7u;
         const uint32_t dec_full_leader = map_to_cta(dec_full_bar(0), 0);
         int total_k = 0;
@@ -351,32 +417,76 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             Item it;
             for (int i = 0; get_item(sc, cluster, i, it); i++) total_k += sc.k_tiles;
         }
+        PROF_DECL;
+#ifdef BD_TC_PROFILE
+        const long long prof_start = clock64();
+#endif
         for (int g = group; g < total_k; g += kDecodeGroups) {
             const int s = g % kStages, d = g % kDecBufs;
+            PROF_T0;
             mbar_wait(raw_bar(s), (uint32_t)(g / kStages) & 1u, abort_flag);
+            PROF_ADD(0);
+#ifdef BD_TC_PROFILE
+            if (cluster == 0 && rank == 0 && tg == 0) {
+                atomicAdd(&g_prof[14], (unsigned long long)((uint32_t)clock64() - shared_words[2 + s]));
+                atomicAdd(&g_prof[15], 1ull);
+            }
+#endif
+            PROF_T0;
             mbar_wait(dec_empty_bar(d), ((uint32_t)(g / kDecBufs) & 1u) ^ 1u, abort_flag);
+            PROF_ADD(1);
             if (*abort_flag) break;
+#ifdef BD_TC_PROFILE
+            const long long pt0 = clock64();
+#endif
             const uint8_t *codes = base_ptr + Smem::codes + s * kCodeTile + j * 64;
             const uint32_t ids16 = *(const uint16_t *)(base_ptr + Smem::ids + s * kIdAtomBytes + (j % 32) * 8 + (j / 32) * 2);
             uint8_t *dst = base_ptr + Smem::dec + d * kHalfTile + j * 128;
-            uint4 w[4];
+            uint4 w[kBlocksPerThread];
 #pragma unroll
-            for (int c = 0; c < 4; c++) w[c] = *(const uint4 *)(codes + 16 * (c ^ swz64));
+            for (int i = 0; i < kBlocksPerThread; i++) w[i] = *(const uint4 *)(codes + 16 * ((c0 + i) ^ swz64));
 #pragma unroll
-            for (int c = 0; c < 4; c++) {
+            for (int i = 0; i < kBlocksPerThread; i++) {
+                const int c = c0 + i;
                 const uint32_t id = (ids16 >> (4 * c)) & 15u;
                 const uint32_t lo = luts[id], hi = luts[16 + id];
                 uint32_t o[8];
-                decode_word(w[c].x, lo, hi, o[0], o[1]);
-                decode_word(w[c].y, lo, hi, o[2], o[3]);
-                decode_word(w[c].z, lo, hi, o[4], o[5]);
-                decode_word(w[c].w, lo, hi, o[6], o[7]);
+                decode_word(w[i].x, lo, hi, o[0], o[1]);
+                decode_word(w[i].y, lo, hi, o[2], o[3]);
+                decode_word(w[i].z, lo, hi, o[4], o[5]);
+                decode_word(w[i].w, lo, hi, o[6], o[7]);
                 *(uint4 *)(dst + 16 * ((2 * c) ^ swz128)) = make_uint4(o[0], o[1], o[2], o[3]);
                 *(uint4 *)(dst + 16 * ((2 * c + 1) ^ swz128)) = make_uint4(o[4], o[5], o[6], o[7]);
             }
+#ifdef BD_TC_PROFILE
+            const long long pt1 = clock64();
+#endif
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the MMA's reads
-            asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory"); // the four warps of this group are done
-            if (j == 0) mbar_arrive_cluster(dec_full_leader + 8u * d);
+#ifdef BD_TC_PROFILE
+            const long long pt2 = clock64();
+#endif
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "n"(kGroupThreads) : "memory");   // this group's warps are done
+#ifdef BD_TC_PROFILE
+            const long long pt3 = clock64();
+#endif
+            if (tg == 0) mbar_arrive_cluster(dec_full_leader + 8u * d);
+#ifdef BD_TC_PROFILE
+            if (tg == 0) shared_words[16 + d] = (uint32_t)pt3;
+            if (cluster == 0 && rank == 0 && tg == 0) {
+                atomicAdd(&g_prof[10], (unsigned long long)(pt1 - pt0));
+                atomicAdd(&g_prof[11], (unsigned long long)(pt2 - pt1));
+                atomicAdd(&g_prof[12], (unsigned long long)(pt3 - pt2));
+                atomicAdd(&g_prof[13], (unsigned long long)(clock64() - pt3));
+            }
+#endif
+        }
+        if (warp == 2) {
+            PROF_OUT(0, 5);
+            PROF_OUT(1, 6);
+#ifdef BD_TC_PROFILE
+            prof_acc[2] = clock64() - prof_start;
+#endif
+            PROF_OUT(2, 7);
         }
     } else {
         // ---- epilogue: warp w reads TMEM lanes 32 * (w % 4) .. + 31 of this CTA's accumulator half,
@@ -390,11 +500,15 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
         const uint32_t lane_swz = (uint32_t)lane & 7u;
         const int cols_per_pass = out_bf16 ? 64 : 32;                 // 128 bytes per row and pass
         Item it;
+        PROF_DECL;
         for (int i = 0; get_item(sc, cluster, i, it); i++) {
             const int m_pair = it.tile % sc.m_pairs, n_tile = it.tile / sc.m_pairs;
             const int row0 = m_pair * 256 + (int)rank * 128 + quad * 32;
             const int n0 = n_tile * 256 + half * 128;
+            PROF_T0;
             mbar_wait(tmem_full_bar, (uint32_t)i & 1u, abort_flag, 256);
+            PROF_ADD(0);
+            PROF_T0;
             tcgen05_fence_after();
             const uint32_t t_base = tmem + ((uint32_t)(quad * 32) << 16) + half * 128;
             if (use_tma_store) {
@@ -454,6 +568,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
+            PROF_ADD(1);
+        }
+        if (ew == 0) {
+            PROF_OUT(0, 8);
+            PROF_OUT(1, 9);
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");    // staging buffers must outlive the stores
         __syncwarp();
