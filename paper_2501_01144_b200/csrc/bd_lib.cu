@@ -9,7 +9,6 @@
 #include "bd_common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
-#include "gemm_wt.cuh"
 #include "quantize.cuh"
 
 using namespace bd;
@@ -41,18 +40,6 @@ bd_status check_qtensor(const bd_qtensor *q) {
 }
 
 int elem_bytes(bd_dtype dt) { return dt == BD_F32 ? 4 : 2; }
-
-// Tensor-core product of operand bytes + scale atoms with a packed operand.
-cudaError_t tc_launch(const uint8_t *a8, const uint8_t *sfa, int64_t M, const QView &B, int64_t K, void *Y, bool out_bf16,
-                      int64_t ldy, cudaStream_t st) {
-    static int which = -1;
-    if (which < 0) {
-        const char *e = getenv("BD_TC_KERNEL");
-        which = (e && e[0] == 's') ? 0 : 1;                      // "smem": decoded weights in shared memory
-    }
-    if (which == 0) return tc::launch(a8, sfa, M, B, K, Y, out_bf16, ldy, st);
-    return wt::launch(a8, sfa, M, B, K, Y, out_bf16, ldy, st);
-}
 
 unsigned grid_for(int64_t threads, int block) { return (unsigned)((threads + block - 1) / block); }
 
@@ -150,7 +137,7 @@ bd_status gemm_dispatch(const QView &A, const QView &B, void *Y, bd_dtype ydt, i
         bd_status s = launch_result(1);
         if (s) return s;
         g_launches += 1;
-        return cuda_result(tc_launch(a8, A.scales, A.rows, B, A.K, Y, ydt == BD_BF16, ldy, st));
+        return cuda_result(tc::launch(a8, A.scales, A.rows, B, A.K, Y, ydt == BD_BF16, ldy, st));
     }
     if (ydt == BD_F32) return launch_simt<float>(A, B, Y, ldy, st);
     return launch_simt<__nv_bfloat16>(A, B, Y, ldy, st);
@@ -288,7 +275,7 @@ bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_
         s = launch_contig<BD_SELECT_TWO_STAGE, false, true>(X, xdtype, ldx, view_of(&xq), a8, st);
         if (s) return s;
         g_launches += 1;
-        return cuda_result(tc_launch(a8, sfa, M, view_of(Wq), K, Y, ydtype == BD_BF16, ldy, st));
+        return cuda_result(tc::launch(a8, sfa, M, view_of(Wq), K, Y, ydtype == BD_BF16, ldy, st));
     }
     bd_qtensor xq{p, p + align256(c), p + align256(c) + align256(i), M, K};
     s = launch_contig<BD_SELECT_TWO_STAGE, true, false>(X, xdtype, ldx, view_of(&xq), nullptr, st);
@@ -401,13 +388,3 @@ const char *bd_status_string(bd_status s) {
 int bd_version(void) { return 100; }
 
 }  // extern "C"
-
-#ifdef BD_TC_PROFILE
-extern "C" int bd_debug_read_prof(unsigned long long *out16) {
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(out16, bd::tc::g_prof, sizeof(unsigned long long) * 32);
-    unsigned long long z[32] = {};
-    cudaMemcpyToSymbol(bd::tc::g_prof, z, sizeof(z));
-    return 0;
-}
-#endif
