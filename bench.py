@@ -22,6 +22,7 @@ With --gpus N > 1 (under torchrun) every rank runs the same per-GPU workload on
 its own tokens (no collective: token batches are independent); value is the sum.
 """
 import argparse
+import datetime
 import json
 import os
 import subprocess
@@ -39,8 +40,8 @@ M_TOKENS = 2048
 QUANT_SHAPE = (8192, 4096)
 BYTES_PER_ELEM_QUANT = 2 + 0.5 + 1.5 / 32           # bf16 read + 4-bit code + (4-bit id + 8-bit scale) / 32
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
-QUANT_DRAM_BYTES = 67.13e6 + 4.48e6                 # quantize_bf16_kernel on bf16 [8192, 4096]
-GEMM_GATE_UP_DRAM_BYTES = 40806912 + 16053504   # tc::gemm_pair_kernel, gate/up layer (profiles/gemm_pair_kernel_llama3_gate_up.md)
+QUANT_DRAM_BYTES = 67.13e6 + 3.28e6                 # quantize_bf16_kernel on bf16 [8192, 4096]
+GEMM_GATE_UP_DRAM_BYTES = 40.82e6 + 18.31e6         # tc::gemm_wtmem_kernel on the gate/up layer
 MLP_SWEEP = [(4096, 11008), (11008, 4096)]
 MLP_SWEEP_M = [1, 16, 128, 1024, 8192]
 
@@ -56,7 +57,7 @@ def measured_peaks():
 
 class ClockSampler:
     """nvidia-smi clock samples taken while the timed region runs."""
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -75,28 +76,42 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Median SM clock and the throttle reasons seen between the wall-clock times t_begin and t_end
+        (the timed region); with no sample inside, the samples nearest to it are used."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.05)
         self.proc.terminate()
         self.proc.wait()
-        sm, smax, reasons = [], None, set()
+        rows, smax = [], None
         for line in open(self.path):
             f = [x.strip() for x in line.split(",")]
             if len(f) < 9:
                 continue
             try:
-                sm.append(float(f[1]))
+                stamp = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                mhz = float(f[1])
                 smax = float(f[2])
+                watts = float(f[3])
             except ValueError:
                 continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
+            active = [name for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                                 "sw_power_cap"), f[5:9]) if val.lower().startswith("active")]
+            rows.append((stamp, mhz, watts, active))
         os.unlink(self.path)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
-                "samples": len(sm)}
+        inside = [r for r in rows if t_begin is not None and t_begin <= r[0] <= t_end]
+        where = "timed region"
+        if not inside and rows and t_begin is not None:
+            mid = 0.5 * (t_begin + t_end)
+            inside = sorted(rows, key=lambda r: abs(r[0] - mid))[:3]
+            where = "nearest samples (region shorter than the sampling period)"
+        elif not inside:
+            inside, where = rows, "whole run"
+        reasons = sorted({a for r in inside for a in r[3]})
+        return {"sm_mhz": float(np.median([r[1] for r in inside])) if inside else None, "sm_max_mhz": smax,
+                "power_w": float(np.median([r[2] for r in inside])) if inside else None, "reasons": reasons,
+                "samples": len(inside), "window": where}
 
 
 # ---------------------------------------------------------------------------
@@ -233,8 +248,10 @@ def run_gpu(args, rank, world, local_rank):
         step()
     barrier()
     launches_warm = bd.launch_count()
+    t_begin = time.time()
     total_ms = timed(step, args.steps, 0)
-    clocks = sampler.stop()
+    t_end = time.time()
+    clocks = sampler.stop(t_begin, t_end)
     launches = bd.launch_count() - launches_warm
     ms_per_step = total_ms / args.steps
     value = world * step_flops / (ms_per_step * 1e-3) / 1e12
@@ -264,8 +281,8 @@ def run_gpu(args, rank, world, local_rank):
     gemm_ms = float(np.mean(durations))
     achieved_tf = big["flops"] / (gemm_ms * 1e-3) / 1e12
     fp8_peak = 2.0 * peaks["bf16_tflops"]                 # dense FP8 = 2 x dense bf16 (nominal ratio), burst: kernel timed alone
-    # DRAM traffic of this launch from the committed ncu capture (profiles/gemm_pair_kernel_llama3_gate_up.md)
-    roofline = {"bound": "tensor", "kernel": "bd_gemm " + big["name"] + " (decode_e4m3 of A + tc::gemm_pair_kernel)",
+    # DRAM traffic of this launch from the committed ncu capture (profiles/gemm_wtmem_kernel_llama3_gate_up.md)
+    roofline = {"bound": "tensor", "kernel": "bd_gemm " + big["name"] + " (decode_e4m3 of the activations + tc::gemm_wtmem_kernel)",
                 "achieved": achieved_tf, "peak": fp8_peak,
                 "unit": "TFLOP/s", "frac": achieved_tf / fp8_peak, "traffic": GEMM_GATE_UP_DRAM_BYTES,
                 "peak_source": f"2 x {peaks['source']} bf16 burst", "ms_per_launch": gemm_ms,
@@ -397,6 +414,23 @@ def run_case(args):
         print(json.dumps({"case": args.case, "us_per_launch": us,
                           "GB/s": qm * qk * BYTES_PER_ELEM_QUANT / us / 1e3}))
         return
+    if args.case == "step":
+        # the benchmark step alone: the four layers through bd_linear, nothing else on the GPU
+        ls = []
+        for i, (_, K, N) in enumerate(LAYERS):
+            ls.append((dev_bf16(inputs.act_student_t(M_TOKENS, K, seed=2 + i)),
+                       bd.quantize_weights(dev_bf16(inputs.weights_normal(N, K, seed=2 + i)), bd.SELECT_TWO_STAGE),
+                       torch.empty(M_TOKENS, N, dtype=torch.bfloat16, device=dev),
+                       torch.empty(bd.linear_workspace_size(M_TOKENS, N, K), dtype=torch.uint8, device=dev)))
+        for it in range(args.warmup + reps):
+            if it == args.warmup:
+                e0.record()
+            for x, wq, y, ws in ls:
+                bd.linear(x, wq, out=y, workspace=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        print(json.dumps({"case": args.case, "us_per_step": e0.elapsed_time(e1) / reps * 1e3}))
+        return
     name = args.case[len("linear_"):]
     K, N = {n: (k, nn) for n, k, nn in LAYERS}[name]
     x = dev_bf16(inputs.act_student_t(M_TOKENS, K, seed=2))
@@ -417,11 +451,11 @@ def run_case(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--case", default=None,
-                    choices=["quantizer"] + ["linear_" + n for n, _, _ in LAYERS],
+                    choices=["quantizer", "step"] + ["linear_" + n for n, _, _ in LAYERS],
                     help="run a few launches of one small case (for profiler captures) instead of the benchmark")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
