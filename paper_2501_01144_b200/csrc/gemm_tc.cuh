@@ -175,16 +175,31 @@ struct Smem {
 static_assert((2 * kXStages + 2 * kCodeStages + 2 * kABufs + 2) * 8 <= 512, "barrier area too small");
 static_assert(Smem::total <= 227 * 1024, "shared memory budget");
 
-// tile = i * clusters + c;  token tile = tile % t_tiles, weight-row pair = tile / t_tiles, so the clusters
-// that run at the same time share the same weight rows and differ in their tokens
+// Work items of a launch, identical for every cluster: cluster c takes items c, c + clusters, ...
+// Tiles are numbered with the token tile running fastest (token tile = tile % t_tiles, weight-row pair =
+// tile / t_tiles), so the clusters that run at the same time share weight rows and differ in their tokens.
+// Items [0, split_from) are whole tiles of 256 tokens; each later tile is two items of 128 tokens, which
+// lets a last, sparsely filled round of tiles spread over twice as many clusters.
 struct Schedule {
-    int w_pairs, t_tiles, k_tiles, clusters;
+    int w_pairs, t_tiles, k_tiles, clusters, split_from;
 };
-__device__ __forceinline__ bool next_tile(const Schedule &sc, int c, int i, int &w_pair, int &t_tile) {
-    const int tile = i * sc.clusters + c;
-    t_tile = tile % sc.t_tiles;
-    w_pair = tile / sc.t_tiles;
-    return tile < sc.w_pairs * sc.t_tiles;
+struct Tile {
+    int w_pair;      // weight rows [256 * w_pair, + 256)
+    int t_start;     // first token
+    int tokens;      // 256 or 128: the N of the MMA
+};
+__device__ __forceinline__ bool next_tile(const Schedule &sc, int c, int i, Tile &t) {
+    const int item = i * sc.clusters + c, tiles = sc.w_pairs * sc.t_tiles;
+    int tile = item, half = 0;
+    t.tokens = 256;
+    if (item >= sc.split_from) {
+        tile = sc.split_from + ((item - sc.split_from) >> 1);
+        half = (item - sc.split_from) & 1;
+        t.tokens = 128;
+    }
+    t.w_pair = tile / sc.t_tiles;
+    t.t_start = (tile % sc.t_tiles) * 256 + half * 128;
+    return tile < tiles;
 }
 
 __device__ __forceinline__ void tcgen05_mma_mxf8_pair_atmem(uint32_t d, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
@@ -205,8 +220,52 @@ __device__ __forceinline__ void mbar_arrive_local(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+// bf16 epilogue of one warp: its 32 * CHUNKS token columns go to registers first, packed as bf16 pairs of
+// neighbouring tokens (16 * CHUNKS registers), so the accumulator is free again after CHUNKS TMEM round trips;
+// then, 64 tokens at a time, lanes 2m and 2m + 1 trade halves so that each writes one 32-bit word of two
+// neighbouring output columns (the even lane the row of token t, the odd lane the row of token t + 1) into the
+// staging tile, which a TMA tensor store writes out as 64 rows x 32 columns.
+template <int CHUNKS, typename Release, typename StagingFree>
+__device__ __forceinline__ void epilogue_bf16(uint32_t t_base, uint8_t *stage_ptr, uint32_t stage_out, const CUtensorMap *mapY,
+                                              int n0, int t0, int lane, volatile uint32_t *abort_flag, Release release_accumulator,
+                                              StagingFree staging_free) {
+    uint32_t p[16 * CHUNKS];
+#pragma unroll
+    for (int c = 0; c < CHUNKS; c++) {
+        uint32_t r[32];
+        tcgen05_ld_32x32b_x32(t_base + c * 32, r);
+        tcgen05_wait_ld();
+#pragma unroll
+        for (int q = 0; q < 16; q++) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * q]), __uint_as_float(r[2 * q + 1]));
+            p[c * 16 + q] = *(uint32_t *)&h;                      // tokens 32 c + 2 q and + 1 of my column
+        }
+    }
+    release_accumulator();
+#pragma unroll
+    for (int pass = 0; pass < CHUNKS / 2; pass++) {
+        staging_free();
+#pragma unroll
+        for (int q = 0; q < 32; q++) {
+            const uint32_t mine = p[32 * pass + q];
+            const uint32_t other = __shfl_xor_sync(0xffffffffu, mine, 1);
+            const uint32_t word = (lane & 1) ? prmt_b32(other, mine, 0x7632u)   // (col - 1, col) of token t + 1
+                                             : prmt_b32(mine, other, 0x5410u);  // (col, col + 1) of token t
+            *(uint32_t *)(stage_ptr + (2 * q + (lane & 1)) * 64 + (lane >> 1) * 4) = word;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0 && !*abort_flag) {
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                         ::"l"(mapY), "r"(n0), "r"(t0 + pass * 64), "r"(stage_out) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+    }
+}
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapCodes,
+gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapXhalf,
+                  const __grid_constant__ CUtensorMap mapCodes,
                   const __grid_constant__ CUtensorMap mapSfW, const __grid_constant__ CUtensorMap mapSfX,
                   const uint8_t *__restrict__ idsW, const Schedule sc, int M, int N, int row_tiles_x, int row_tiles_w,
                   void *__restrict__ Y, int64_t ldy, int out_bf16, const __grid_constant__ CUtensorMap mapY, int use_tma_store) {
@@ -273,20 +332,24 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
 
     if (warp == 0) {
         // ---- TMA producer of the activation tile and the scale atoms (one elected lane issues) ----
-        constexpr uint32_t tx_pair = 2u * (kXTile + 3u * kScaleAtomBytes);
-        int s = 0, w_pair, t_tile;
+        int s = 0;
         uint32_t ph = 1;
-        for (int i = 0; next_tile(sc, cluster, i, w_pair, t_tile); i++) {
-            const int t0 = t_tile * 256 + (int)rank * 128;
+        Tile t;
+        for (int i = 0; next_tile(sc, cluster, i, t); i++) {
+            // each CTA holds half of the tile's tokens; a 128-token item loads 64 rows through its own tensor map
+            const int per_cta = t.tokens / 2, t0 = t.t_start + (int)rank * per_cta;
+            const CUtensorMap *map = t.tokens == 256 ? &mapX : &mapXhalf;
+            const uint32_t tx_pair = 2u * ((uint32_t)per_cta * BK + 3u * kScaleAtomBytes);
             for (int kt = 0; kt < sc.k_tiles; kt++) {
                 mbar_wait(x_empty(s), ph, abort_flag);
                 if (*abort_flag) break;
                 const uint32_t fb = map_to_cta(x_full(s), 0);
                 if (elect_one()) {
                     if (rank == 0) mbar_expect_tx(x_full(s), tx_pair);
-                    tma_load_2d_pair(x_tile(s), &mapX, kt * BK, t0, fb);
-                    tma_load_2d_pair(sfw_tile(s), &mapSfW, 0, kt * row_tiles_w + w_pair * 2 + (int)rank, fb);
-                    tma_load_2d_pair(sfx_tile(s), &mapSfX, 0, kt * row_tiles_x + t_tile * 2, fb);
+                    tma_load_2d_pair(x_tile(s), map, kt * BK, t0, fb);
+                    tma_load_2d_pair(sfw_tile(s), &mapSfW, 0, kt * row_tiles_w + t.w_pair * 2 + (int)rank, fb);
+                    // two scale atoms = 256 tokens from the item's first token (a 128-token item uses the first)
+                    tma_load_2d_pair(sfx_tile(s), &mapSfX, 0, kt * row_tiles_x + t.t_start / 128, fb);
                 }
                 __syncwarp();
                 if (++s == kXStages) { s = 0; ph ^= 1u; }
@@ -295,11 +358,12 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         }
     } else if (warp == 2) {
         // ---- TMA producer of this CTA's packed codes and ids ----
-        int s = 0, w_pair, t_tile;
+        int s = 0;
         uint32_t ph = 1;
-        for (int i = 0; next_tile(sc, cluster, i, w_pair, t_tile); i++) {
-            const int w0 = w_pair * 256 + (int)rank * 128;
-            const int my_row_tile = w_pair * 2 + (int)rank;
+        Tile t;
+        for (int i = 0; next_tile(sc, cluster, i, t); i++) {
+            const int w0 = t.w_pair * 256 + (int)rank * 128;
+            const int my_row_tile = t.w_pair * 2 + (int)rank;
             const bool have_ids = my_row_tile < row_tiles_w;
             for (int kt = 0; kt < sc.k_tiles; kt++) {
                 mbar_wait(c_empty(s), ph, abort_flag);
@@ -324,12 +388,14 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             const uint32_t lo_sfw0 = sfw_tile(0) >> 4, lo_sfx0 = sfx_tile(0) >> 4;
             // block-scaled E4M3 x E4M3 (formats 0), B K-major, UE8M0 scales (bit 23), N >> 3 at bit 17 (256 tokens),
             // M >> 4 at bit 24 (256 weight rows across the pair); scale byte selectors at bits 4 (B) and 29 (A)
-            const uint32_t idesc0 = (uint32_t)(256 >> 3) << 17 | 1u << 23 | (uint32_t)(256 >> 4) << 24;
+            const uint32_t idesc_m = 1u << 23 | (uint32_t)(256 >> 4) << 24;
             const uint32_t t_d = tmem + kColD, t_sfw = tmem + kColSfW, t_sfx = tmem + kColSfX;
-            int s = 0, b = 0, w_pair, t_tile;
+            int s = 0, b = 0;
             uint32_t ph_s = 0, ph_b = 0;
             bool ready = false;
-            for (int i = 0; next_tile(sc, cluster, i, w_pair, t_tile); i++) {
+            Tile t;
+            for (int i = 0; next_tile(sc, cluster, i, t); i++) {
+                const uint32_t idesc0 = idesc_m | (uint32_t)(t.tokens >> 3) << 17;
                 if (i > 0) mbar_wait(tmem_empty_bar, (uint32_t)(i - 1) & 1u, abort_flag);
                 tcgen05_fence_after();
                 for (int kt = 0; kt < sc.k_tiles; kt++) {
@@ -382,8 +448,8 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16) + kColA;
         int total_k = 0;
         {
-            int w_pair, t_tile;
-            for (int i = 0; next_tile(sc, cluster, i, w_pair, t_tile); i++) total_k += sc.k_tiles;
+            Tile t;
+            for (int i = 0; next_tile(sc, cluster, i, t); i++) total_k += sc.k_tiles;
         }
         for (int g = group; g < total_k; g += kDecodeGroups) {
             const int s = g % kCodeStages, b = g % kABufs;
@@ -435,56 +501,24 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             __syncwarp();
         };
-        int w_pair, t_tile;
-        for (int i = 0; next_tile(sc, cluster, i, w_pair, t_tile); i++) {
-            const int n0 = w_pair * 256 + (int)rank * 128 + quad * 32;      // this warp's 32 output columns
-            const int t0 = t_tile * 256 + half * 128;                       // and its 128 output rows
+        Tile t;
+        for (int i = 0; next_tile(sc, cluster, i, t); i++) {
+            const int cols = t.tokens / 2;                                  // token columns of this warp: 128 or 64
+            const int n0 = t.w_pair * 256 + (int)rank * 128 + quad * 32;    // this warp's 32 output columns
+            const int t0 = t.t_start + half * cols;                         // and its first output row
             mbar_wait(tmem_full_bar, (uint32_t)i & 1u, abort_flag, 256);
             tcgen05_fence_after();
-            const uint32_t t_base = tmem + ((uint32_t)(quad * 32) << 16) + kColD + half * 128;
+            const uint32_t t_base = tmem + ((uint32_t)(quad * 32) << 16) + kColD + half * cols;
             if (use_tma_store && out_bf16) {
-                // all 128 token columns of this warp go to registers first, packed as bf16 pairs of neighbouring
-                // tokens (64 registers), so the accumulator is free again after four TMEM round trips
-                uint32_t p[64];
-#pragma unroll
-                for (int c = 0; c < 4; c++) {
-                    uint32_t r[32];
-                    tcgen05_ld_32x32b_x32(t_base + c * 32, r);
-                    tcgen05_wait_ld();
-#pragma unroll
-                    for (int q = 0; q < 16; q++) {
-                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[2 * q]), __uint_as_float(r[2 * q + 1]));
-                        p[c * 16 + q] = *(uint32_t *)&h;                  // tokens 32 c + 2 q and + 1 of my column
-                    }
-                }
-                release_accumulator();
-                for (int pass = 0; pass < 2; pass++) {
-                    staging_free();
-                    // lanes 2m and 2m + 1 trade halves so that each writes one 32-bit word of two neighbouring
-                    // output columns: the even lane the row of token t, the odd lane the row of token t + 1
-#pragma unroll
-                    for (int q = 0; q < 32; q++) {
-                        const uint32_t mine = pass == 0 ? p[q] : p[32 + q];
-                        const uint32_t other = __shfl_xor_sync(0xffffffffu, mine, 1);
-                        const uint32_t word = (lane & 1) ? prmt_b32(other, mine, 0x7632u)   // (col - 1, col) of token t + 1
-                                                         : prmt_b32(mine, other, 0x5410u);  // (col, col + 1) of token t
-                        *(uint32_t *)(stage_ptr + (2 * q + (lane & 1)) * 64 + (lane >> 1) * 4) = word;
-                    }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0 && !*abort_flag) {
-                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                                     ::"l"(&mapY), "r"(n0), "r"(t0 + pass * 64), "r"(stage_out) : "memory");
-                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    }
-                }
+                if (cols == 128) epilogue_bf16<4>(t_base, stage_ptr, stage_out, &mapY, n0, t0, lane, abort_flag, release_accumulator, staging_free);
+                else epilogue_bf16<2>(t_base, stage_ptr, stage_out, &mapY, n0, t0, lane, abort_flag, release_accumulator, staging_free);
             } else if (use_tma_store) {
-                for (int pass = 0; pass < 4; pass++) {                // fp32: 32 tokens x 32 columns per pass
+                for (int pass = 0; pass * 32 < cols; pass++) {        // fp32: 32 tokens x 32 columns per pass
                     uint32_t r[2][16];
 #pragma unroll
                     for (int c = 0; c < 2; c++) tcgen05_ld_32x32b_x16(t_base + pass * 32 + c * 16, r[c]);
                     tcgen05_wait_ld();
-                    if (pass == 3) release_accumulator();
+                    if ((pass + 1) * 32 >= cols) release_accumulator();
                     staging_free();
 #pragma unroll
                     for (int c = 0; c < 2; c++)
@@ -502,17 +536,17 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 // plain stores: for one token the 32 lanes write 32 neighbouring output columns
                 const int n = n0 + lane;
 #pragma unroll 1
-                for (int c = 0; c < 8; c++) {
+                for (int c = 0; c * 16 < cols; c++) {
                     uint32_t r[16];
                     tcgen05_ld_32x32b_x16(t_base + c * 16, r);
                     tcgen05_wait_ld();
                     if (n < N && !*abort_flag) {
 #pragma unroll
                         for (int q = 0; q < 16; q++) {
-                            const int t = t0 + c * 16 + q;
-                            if (t < M) {
-                                if (out_bf16) ((__nv_bfloat16 *)Y)[(int64_t)t * ldy + n] = __float2bfloat16_rn(__uint_as_float(r[q]));
-                                else ((float *)Y)[(int64_t)t * ldy + n] = __uint_as_float(r[q]);
+                            const int tok = t0 + c * 16 + q;
+                            if (tok < M) {
+                                if (out_bf16) ((__nv_bfloat16 *)Y)[(int64_t)tok * ldy + n] = __float2bfloat16_rn(__uint_as_float(r[q]));
+                                else ((float *)Y)[(int64_t)tok * ldy + n] = __uint_as_float(r[q]);
                             }
                         }
                     }
@@ -555,9 +589,10 @@ inline int max_resident_clusters() {
 // X as operand bytes + scale atoms (the quantizer's second output form), W as a packed operand.
 inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, const QView &W, int64_t K, void *Y,
                           bool out_bf16, int64_t ldy, cudaStream_t st) {
-    CUtensorMap mapX, mapCodes, mapSfW, mapSfX, mapY;
+    CUtensorMap mapX, mapXhalf, mapCodes, mapSfW, mapSfX, mapY;
     const int64_t N = W.rows, rtx = row_tiles(M), rtw = row_tiles(N), kg = k_groups(K);
     if (!make_map_2d(&mapX, CU_TENSOR_MAP_DATA_TYPE_UINT8, x8, K, M, K, BK, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_2d(&mapXhalf, CU_TENSOR_MAP_DATA_TYPE_UINT8, x8, K, M, K, BK, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !make_map_2d(&mapCodes, CU_TENSOR_MAP_DATA_TYPE_UINT8, W.codes, K / 2, N, K / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_64B) ||
         !make_map_2d(&mapSfW, CU_TENSOR_MAP_DATA_TYPE_UINT32, W.scales, 128, rtw * kg, kScaleAtomBytes, 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE) ||
         !make_map_2d(&mapSfX, CU_TENSOR_MAP_DATA_TYPE_UINT32, sfx, 128, rtx * kg, kScaleAtomBytes, 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE))
@@ -583,7 +618,13 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
     sc.k_tiles = (int)((K + BK - 1) / BK);
     const int tiles = sc.w_pairs * sc.t_tiles;
     const int resident = max_resident_clusters();
-    sc.clusters = tiles < resident ? tiles : resident;
+    // a last round that fills at most half of the clusters is cut into 128-token items (twice as many, half as
+    // long), unless the second half of the last token tile would be empty
+    const int rest = tiles % resident, m_tail = (int)(M % 256);
+    sc.split_from = tiles;
+    if (rest > 0 && 2 * rest <= resident && (m_tail == 0 || m_tail > 128)) sc.split_from = tiles - rest;
+    const int items = tiles + (tiles - sc.split_from);
+    sc.clusters = items < resident ? items : resident;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * sc.clusters);
     cfg.blockDim = dim3(kThreads);
@@ -594,7 +635,7 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_wtmem_kernel, mapX, mapCodes, mapSfW, mapSfX, (const uint8_t *)W.ids, sc, (int)M,
+    return cudaLaunchKernelEx(&cfg, gemm_wtmem_kernel, mapX, mapXhalf, mapCodes, mapSfW, mapSfX, (const uint8_t *)W.ids, sc, (int)M,
                               (int)N, (int)rtx, (int)rtw, Y, ldy, out_bf16 ? 1 : 0, mapY, use_tma_store);
 }
 
