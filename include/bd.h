@@ -172,6 +172,18 @@ bd_status bd_dequantize(const bd_qtensor *q, float *out, int64_t ld, void *strea
  * of 0.5, ascending. */
 bd_status bd_get_formatbook(uint8_t out[16][8]);
 
+/* Replaces the formatbook (HOST table, same form; NULL restores the built-in one) on the
+ * current device.  The paper shows its table only as a figure (Fig. 4); the built-in table
+ * is reconstructed from the rules of Sec. 3.1 and the printed values of dialects 4 and 5,
+ * so this call is how a caller supplies other values.  Accepted tables keep the structure
+ * the two-stage selection relies on (Sec. 3.2): every row strictly ascending from 0, values
+ * <= 15; rows 2p and 2p + 1 share all values but the one at index 6, the even row holding
+ * the larger; the pair's maximum is 15 - p.  Anything else returns BD_ERR_INVALID_ARG and
+ * changes nothing.  Synchronises the device first; operands quantised under another table
+ * keep their codes but decode through the new one, so requantise them.  Not thread-safe
+ * against other calls of the library. */
+bd_status bd_set_formatbook(const uint8_t in[16][8]);
+
 /* Synchronises `stream`, then returns and clears the device status word:
  * BD_OK, BD_ERR_NONFINITE or BD_ERR_TIMEOUT (or BD_ERR_CUDA). */
 bd_status bd_poll_status(void *stream);

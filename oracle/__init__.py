@@ -43,6 +43,7 @@ def lib():
         _lib.bdo_beneficial_range.argtypes = [ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
         _lib.bdo_round_code.argtypes = [ci, ci]
         _lib.bdo_formatbook.argtypes = [vp]
+        _lib.bdo_set_formatbook.argtypes = [vp]
     return _lib
 
 
@@ -59,6 +60,18 @@ def formatbook():
     out = np.zeros((16, 8), np.uint8)
     lib().bdo_formatbook(_ptr(out))
     return out
+
+
+def set_formatbook(table=None):
+    """Replace the table in use (None restores the reconstruction of Fig. 4).  Raises on a table without
+    the pair structure of Sec. 3.1 / 3.2."""
+    if table is None:
+        rc = lib().bdo_set_formatbook(None)
+    else:
+        t = np.ascontiguousarray(np.asarray(table, np.uint8).reshape(16, 8))
+        rc = lib().bdo_set_formatbook(_ptr(t))
+    if rc:
+        raise ValueError("formatbook rejected")
 
 
 def beneficial_range(dialect):

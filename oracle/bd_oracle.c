@@ -50,19 +50,49 @@ enum { BDO_SELECT_TWO_STAGE = 0, BDO_SELECT_MSE = 1 };
  * Dialect 4 = 0.5*{0,1,2,3,4,6,10,13} is printed in Sec. 3.3; dialect 5 swaps
  * 5.0 for 4.0 (Sec. 3.2).
  * ------------------------------------------------------------------------- */
-static const uint8_t FORMATBOOK[16][8] = {
-    {0, 1, 2, 3, 4, 6, 12, 15}, {0, 1, 2, 3, 4, 6, 10, 15}, /* max 7.5 */
-    {0, 1, 2, 3, 4, 6, 11, 14}, {0, 1, 2, 3, 4, 6, 9, 14},  /* max 7.0 */
-    {0, 1, 2, 3, 4, 6, 10, 13}, {0, 1, 2, 3, 4, 6, 8, 13},  /* max 6.5 */
-    {0, 1, 2, 3, 4, 6, 9, 12},  {0, 1, 2, 3, 4, 6, 8, 12},  /* max 6.0 (odd = FP4 E2M1) */
-    {0, 1, 2, 3, 4, 6, 9, 11},  {0, 1, 2, 3, 4, 6, 8, 11},  /* max 5.5 */
-    {0, 1, 2, 3, 4, 6, 8, 10},  {0, 1, 2, 3, 4, 6, 7, 10},  /* max 5.0 */
-    {0, 1, 2, 3, 4, 6, 8, 9},   {0, 1, 2, 3, 4, 6, 7, 9},   /* max 4.5 */
-    {0, 1, 2, 3, 4, 5, 7, 8},   {0, 1, 2, 3, 4, 5, 6, 8},   /* max 4.0 */
-};
+#define BDO_DEFAULT_FORMATBOOK { \
+    {0, 1, 2, 3, 4, 6, 12, 15}, {0, 1, 2, 3, 4, 6, 10, 15}, /* max 7.5 */ \
+    {0, 1, 2, 3, 4, 6, 11, 14}, {0, 1, 2, 3, 4, 6, 9, 14},  /* max 7.0 */ \
+    {0, 1, 2, 3, 4, 6, 10, 13}, {0, 1, 2, 3, 4, 6, 8, 13},  /* max 6.5 */ \
+    {0, 1, 2, 3, 4, 6, 9, 12},  {0, 1, 2, 3, 4, 6, 8, 12},  /* max 6.0 (odd = FP4 E2M1) */ \
+    {0, 1, 2, 3, 4, 6, 9, 11},  {0, 1, 2, 3, 4, 6, 8, 11},  /* max 5.5 */ \
+    {0, 1, 2, 3, 4, 6, 8, 10},  {0, 1, 2, 3, 4, 6, 7, 10},  /* max 5.0 */ \
+    {0, 1, 2, 3, 4, 6, 8, 9},   {0, 1, 2, 3, 4, 6, 7, 9},   /* max 4.5 */ \
+    {0, 1, 2, 3, 4, 5, 7, 8},   {0, 1, 2, 3, 4, 5, 6, 8},   /* max 4.0 */ \
+}
+static const uint8_t DEFAULT_FORMATBOOK[16][8] = BDO_DEFAULT_FORMATBOOK;
+
+
+/* The table in use.  It starts as the reconstruction above; bdo_set_formatbook replaces it so that a
+ * test can run the same alternative table through the oracle and through the library. */
+static uint8_t FORMATBOOK[16][8] = BDO_DEFAULT_FORMATBOOK;
 
 int bdo_formatbook(uint8_t out[16][8]) {
     memcpy(out, FORMATBOOK, sizeof(FORMATBOOK));
+    return BDO_OK;
+}
+
+/* in == NULL restores the default.  A table is taken only if it has the shape Sec. 3.1 and 3.2 describe:
+ * ascending magnitudes from 0 up to at most 7.5, eight pairs in descending order of their shared maximum
+ * 7.5 ... 4.0, the two members of a pair equal except for the value below the maximum, the even one larger. */
+int bdo_set_formatbook(const uint8_t in[16][8]) {
+    if (!in) {
+        memcpy(FORMATBOOK, DEFAULT_FORMATBOOK, sizeof(FORMATBOOK));
+        return BDO_OK;
+    }
+    for (int d = 0; d < 16; d++) {
+        if (in[d][0] != 0 || in[d][7] > 15) return BDO_ERR_ARG;
+        for (int j = 1; j < 8; j++)
+            if (in[d][j] <= in[d][j - 1]) return BDO_ERR_ARG;
+    }
+    for (int p = 0; p < 8; p++) {
+        const uint8_t *even = in[2 * p], *odd = in[2 * p + 1];
+        if (even[7] != 15 - p || odd[7] != 15 - p) return BDO_ERR_ARG;
+        for (int j = 0; j < 6; j++)
+            if (even[j] != odd[j]) return BDO_ERR_ARG;
+        if (even[6] <= odd[6]) return BDO_ERR_ARG;
+    }
+    memcpy(FORMATBOOK, in, sizeof(FORMATBOOK));
     return BDO_OK;
 }
 

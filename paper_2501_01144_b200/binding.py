@@ -71,6 +71,7 @@ def load():
     lib.bd_import_canonical.argtypes = [vp, vp, vp, qp, vp]
     lib.bd_dequantize.argtypes = [qp, vp, i64, vp]
     lib.bd_get_formatbook.argtypes = [vp]
+    lib.bd_set_formatbook.argtypes = [vp]
     lib.bd_poll_status.argtypes = [vp]
     lib.bd_set_gemm_impl.argtypes = [ci]
     lib.bd_launch_count.restype = ctypes.c_uint64
@@ -112,6 +113,18 @@ def get_formatbook():
     buf = (ctypes.c_uint8 * 128)()
     _check(load().bd_get_formatbook(buf))
     return torch.tensor(list(buf), dtype=torch.uint8).reshape(16, 8)
+
+
+def set_formatbook(table=None):
+    """Replace the DialectFP4 table on the current device (None restores the built-in one)."""
+    if table is None:
+        _check(load().bd_set_formatbook(None))
+        return
+    vals = [int(v) for v in torch.as_tensor(table).reshape(-1).tolist()]
+    if len(vals) != 128:
+        raise ValueError("formatbook must be 16 x 8")
+    buf = (ctypes.c_uint8 * 128)(*vals)
+    _check(load().bd_set_formatbook(buf))
 
 
 def poll_status(stream=None):

@@ -41,9 +41,9 @@ constexpr Formatbook kBook = {{
 // index j or above exactly when q5 >= v[j-1] + v[j] (midpoint of two multiples
 // of 0.5, ties to the larger magnitude; Sec. 3.3).  Stored as a bit mask with
 // bit t set for each threshold t, so that index = popcount(mask & ((2 << q5) - 1)).
-constexpr uint32_t round_mask(int d) {
+constexpr uint32_t round_mask(const Formatbook &b, int d) {
     uint32_t m = 0;
-    for (int j = 1; j < 8; j++) m |= 1u << (kBook.v[d][j - 1] + kBook.v[d][j]);
+    for (int j = 1; j < 8; j++) m |= 1u << (b.v[d][j - 1] + b.v[d][j]);
     return m;
 }
 
@@ -55,11 +55,11 @@ constexpr uint32_t range_bits(int lo, int hi) {
     for (int q = lo; q < hi && q < 32; q++) m |= 1u << q;
     return m;
 }
-constexpr uint32_t even_range_mask(int p) {
-    return range_bits(kBook.v[2 * p][6] + kBook.v[2 * p + 1][6], kBook.v[2 * p][6] + kBook.v[2 * p][7]);
+constexpr uint32_t even_range_mask(const Formatbook &b, int p) {
+    return range_bits(b.v[2 * p][6] + b.v[2 * p + 1][6], b.v[2 * p][6] + b.v[2 * p][7]);
 }
-constexpr uint32_t odd_range_mask(int p) {
-    return range_bits(kBook.v[2 * p + 1][6] + kBook.v[2 * p + 1][5], kBook.v[2 * p][6] + kBook.v[2 * p + 1][6]);
+constexpr uint32_t odd_range_mask(const Formatbook &b, int p) {
+    return range_bits(b.v[2 * p + 1][6] + b.v[2 * p + 1][5], b.v[2 * p][6] + b.v[2 * p + 1][6]);
 }
 
 // E4M3 encoding of the magnitude 0.5 * h, h in 0..15 (exact: four significant bits).
@@ -73,14 +73,14 @@ constexpr uint8_t e4m3_of_half_units(int h) {
     return (uint8_t)(exp_field << 3 | mant);
 }
 // Eight-byte decode tables of a dialect: byte i = operand byte of index i.
-constexpr uint64_t e4m3_lut(int d) {
+constexpr uint64_t e4m3_lut(const Formatbook &b, int d) {
     uint64_t t = 0;
-    for (int i = 0; i < 8; i++) t |= (uint64_t)e4m3_of_half_units(kBook.v[d][i]) << (8 * i);
+    for (int i = 0; i < 8; i++) t |= (uint64_t)e4m3_of_half_units(b.v[d][i]) << (8 * i);
     return t;
 }
-constexpr uint64_t int_lut(int d) {
+constexpr uint64_t int_lut(const Formatbook &b, int d) {
     uint64_t t = 0;
-    for (int i = 0; i < 8; i++) t |= (uint64_t)kBook.v[d][i] << (8 * i);
+    for (int i = 0; i < 8; i++) t |= (uint64_t)b.v[d][i] << (8 * i);
     return t;
 }
 
@@ -171,8 +171,8 @@ __host__ __device__ inline uint32_t word_insert(uint32_t idx, uint32_t sign, int
 //   index under the odd member  = u - [u>=7] - [u>=8] - [u>=10].
 // pair_tables_ok() checks all of this against the plain definitions for every code.
 // ---------------------------------------------------------------------------
-constexpr uint32_t merged_mask(int p) {
-    const uint8_t *ev = kBook.v[2 * p], *od = kBook.v[2 * p + 1];
+constexpr uint32_t merged_mask(const Formatbook &b, int p) {
+    const uint8_t *ev = b.v[2 * p], *od = b.v[2 * p + 1];
     uint32_t m = 0;
     for (int j = 1; j <= 5; j++) m |= 1u << (ev[j - 1] + ev[j]);
     m |= 1u << (od[5] + od[6]);
@@ -187,25 +187,43 @@ constexpr int popcount32(uint32_t x) {
     for (; x; x &= x - 1) c++;
     return c;
 }
-constexpr bool pair_tables_ok() {
+constexpr bool pair_tables_ok(const Formatbook &b) {
     for (int p = 0; p < 8; p++) {
-        const uint32_t mm = merged_mask(p);
+        const uint32_t mm = merged_mask(b, p);
         if (popcount32(mm) != 10) return false;
         for (int j = 0; j < 6; j++)
-            if (kBook.v[2 * p][j] != kBook.v[2 * p + 1][j]) return false;
+            if (b.v[2 * p][j] != b.v[2 * p + 1][j]) return false;
         for (int q = 0; q < 32; q++) {
             const int u = popcount32(mm & ((2u << q) - 1u));
             const int idx_e = u - (u >= 6) - (u >= 8) - (u >= 9);
             const int idx_o = u - (u >= 7) - (u >= 8) - (u >= 10);
-            if (idx_e != popcount32(round_mask(2 * p) & ((2u << q) - 1u))) return false;
-            if (idx_o != popcount32(round_mask(2 * p + 1) & ((2u << q) - 1u))) return false;
-            if (((even_range_mask(p) >> q) & 1u) != (uint32_t)(u == 8 || u == 9)) return false;
-            if (((odd_range_mask(p) >> q) & 1u) != (uint32_t)(u == 6 || u == 7)) return false;
+            if (idx_e != popcount32(round_mask(b, 2 * p) & ((2u << q) - 1u))) return false;
+            if (idx_o != popcount32(round_mask(b, 2 * p + 1) & ((2u << q) - 1u))) return false;
+            if (((even_range_mask(b, p) >> q) & 1u) != (uint32_t)(u == 8 || u == 9)) return false;
+            if (((odd_range_mask(b, p) >> q) & 1u) != (uint32_t)(u == 6 || u == 7)) return false;
         }
     }
     return true;
 }
-static_assert(pair_tables_ok(), "merged-threshold shortcut does not match the formatbook");
+static_assert(pair_tables_ok(kBook), "merged-threshold shortcut does not match the formatbook");
+
+// What the kernels assume of a formatbook (bd_set_formatbook checks it before it replaces the tables):
+// every row strictly ascending from 0 with values <= 15; pair p = rows 2p, 2p + 1 shares every value but
+// the one at index 6, where the even row holds the larger; the pair's maximum is 15 - p (stage 1 maps the
+// rounded block maximum straight to the pair); and the merged-threshold shortcut reproduces the plain
+// definitions of rounding and beneficial ranges for every 5-bit code.
+constexpr bool formatbook_ok(const Formatbook &b) {
+    for (int d = 0; d < 16; d++) {
+        if (b.v[d][0] != 0 || b.v[d][7] > 15) return false;
+        for (int j = 1; j < 8; j++)
+            if (b.v[d][j] <= b.v[d][j - 1]) return false;
+    }
+    for (int p = 0; p < 8; p++) {
+        if (b.v[2 * p][7] != 15 - p || b.v[2 * p + 1][7] != 15 - p) return false;
+        if (b.v[2 * p][6] <= b.v[2 * p + 1][6]) return false;
+    }
+    return pair_tables_ok(b);
+}
 
 struct DeviceTables {
     uint32_t round_mask[16];
@@ -215,23 +233,23 @@ struct DeviceTables {
     uint32_t int_lo[16], int_hi[16];
     uint32_t merged_above[8];     // merged_mask(p) >> 1: popcount(x >> q5) = thresholds above q5
 };
-constexpr DeviceTables make_tables() {
+constexpr DeviceTables make_tables(const Formatbook &b) {
     DeviceTables t{};
     for (int d = 0; d < 16; d++) {
-        t.round_mask[d] = round_mask(d);
-        t.e4m3_lo[d] = (uint32_t)e4m3_lut(d);
-        t.e4m3_hi[d] = (uint32_t)(e4m3_lut(d) >> 32);
-        t.int_lo[d] = (uint32_t)int_lut(d);
-        t.int_hi[d] = (uint32_t)(int_lut(d) >> 32);
+        t.round_mask[d] = round_mask(b, d);
+        t.e4m3_lo[d] = (uint32_t)e4m3_lut(b, d);
+        t.e4m3_hi[d] = (uint32_t)(e4m3_lut(b, d) >> 32);
+        t.int_lo[d] = (uint32_t)int_lut(b, d);
+        t.int_hi[d] = (uint32_t)(int_lut(b, d) >> 32);
     }
     for (int p = 0; p < 8; p++) {
-        t.even_mask[p] = even_range_mask(p);
-        t.odd_mask[p] = odd_range_mask(p);
-        t.merged_above[p] = merged_mask(p) >> 1;
+        t.even_mask[p] = even_range_mask(b, p);
+        t.odd_mask[p] = odd_range_mask(b, p);
+        t.merged_above[p] = merged_mask(b, p) >> 1;
     }
     return t;
 }
-constexpr DeviceTables kTables = make_tables();
+constexpr DeviceTables kTables = make_tables(kBook);
 
 // Bits of the device status word (defined in quantize.cuh; the library is one
 // translation unit).  bd_poll_status reads and clears it.

@@ -18,6 +18,7 @@ namespace {
 int g_last_cuda_error = 0;
 uint64_t g_launches = 0;
 bd_gemm_impl g_gemm_impl = BD_GEMM_AUTO;
+Formatbook g_book = kBook;            // the table bd_get_formatbook reports (host copy of what the device uses)
 
 bd_status cuda_result(cudaError_t e) {
     if (e == cudaSuccess) return BD_OK;
@@ -340,7 +341,23 @@ bd_status bd_dequantize(const bd_qtensor *q, float *out, int64_t ld, void *strea
 bd_status bd_get_formatbook(uint8_t out[16][8]) {
     if (!out) return BD_ERR_INVALID_ARG;
     for (int d = 0; d < 16; d++)
-        for (int i = 0; i < 8; i++) out[d][i] = kBook.v[d][i];
+        for (int i = 0; i < 8; i++) out[d][i] = g_book.v[d][i];
+    return BD_OK;
+}
+
+bd_status bd_set_formatbook(const uint8_t in[16][8]) {
+    Formatbook b = kBook;                                        // NULL restores the built-in table
+    if (in)
+        for (int d = 0; d < 16; d++)
+            for (int i = 0; i < 8; i++) b.v[d][i] = in[d][i];
+    if (!formatbook_ok(b)) return BD_ERR_INVALID_ARG;
+    // the tables live in constant memory of the current device: nothing of the library may be in flight
+    bd_status s = cuda_result(cudaDeviceSynchronize());
+    if (s) return s;
+    const DeviceTables t = make_tables(b);
+    s = cuda_result(cudaMemcpyToSymbol(c_tables, &t, sizeof(t)));
+    if (s) return s;
+    g_book = b;
     return BD_OK;
 }
 

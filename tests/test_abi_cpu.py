@@ -39,6 +39,28 @@ def test_formatbook_matches_independent_oracle_table():
     assert (bd.get_formatbook().numpy() == oracle.formatbook()).all()
 
 
+def test_set_formatbook_rejects_tables_without_the_pair_structure():
+    # validation is host arithmetic and comes before any device call; accepted tables are a GPU test
+    lib = bd.load()
+    good = bd.get_formatbook().numpy().copy()
+
+    def rc(table):
+        buf = (ctypes.c_uint8 * 128)(*[int(v) for v in table.reshape(-1)])
+        return lib.bd_set_formatbook(buf)
+
+    t = good.copy(); t[3, 4] = t[3, 3]                       # a row that is not strictly ascending
+    assert rc(t) == 1
+    t = good.copy(); t[6, 7] = 13; t[7, 7] = 13              # pair 3 must have maximum 15 - 3
+    assert rc(t) == 1
+    t = good.copy(); t[2, 6], t[3, 6] = good[3, 6], good[2, 6]   # the even member must hold the larger value
+    assert rc(t) == 1
+    t = good.copy(); t[8, 2] = 3; t[8, 3] = 4; t[8, 4] = 5   # members of a pair may differ at index 6 only
+    assert rc(t) == 1
+    t = good.copy(); t[0, 0] = 1                             # every dialect contains zero
+    assert rc(t) == 1
+    assert (bd.get_formatbook().numpy() == good).all()       # nothing changed
+
+
 def test_qtensor_sizes_and_argument_errors():
     lib = bd.load()
     c, i, s = (ctypes.c_size_t() for _ in range(3))

@@ -356,3 +356,44 @@ def test_gemm_against_rational_brute_force_and_block_mac():
     assert np.abs(Yb - Y).max() <= 1e-13 * T.max()
     # a transposed operand would be caught: result is not symmetric in general
     assert Y.shape == (3, 5)
+
+
+def test_alternative_formatbook_in_the_oracle():
+    """bdo_set_formatbook: the selection and rounding follow whatever table is loaded (checked against the
+    plain definitions on that table), malformed tables are refused, None restores the default."""
+    default = oracle.formatbook()
+    alt = default.copy()
+    alt[0, 6], alt[1, 6] = 13, 11                       # other slot-6 values for pair 0
+    alt[6] = [0, 1, 2, 3, 5, 7, 10, 12]                 # another common set for pair 3
+    alt[7] = [0, 1, 2, 3, 5, 7, 8, 12]
+    try:
+        oracle.set_formatbook(alt)
+        assert (oracle.formatbook() == alt).all()
+        # beneficial ranges from the definition (Sec. 3.2): even [ (dE+dO)/2, (dE+max)/2 ), odd [ (v5+dO)/2, (dE+dO)/2 )
+        for p in (0, 3):
+            ev, od = [int(v) for v in alt[2 * p]], [int(v) for v in alt[2 * p + 1]]
+            assert oracle.beneficial_range(2 * p) == (ev[6] + od[6], ev[6] + ev[7])
+            assert oracle.beneficial_range(2 * p + 1) == (od[5] + od[6], ev[6] + od[6])
+        # rounding = nearest value of the loaded table, ties toward the larger magnitude
+        for d in (0, 1, 6, 7):
+            vals = [Fraction(int(v), 2) for v in alt[d]]
+            for q5 in range(32):
+                x = Fraction(q5, 4)
+                best = min(range(8), key=lambda j: (abs(vals[j] - x), -vals[j]))
+                assert oracle.round_code(d, q5) == best, (d, q5)
+        # a block whose maximum rounds to 6.0 lands in pair 3 and is quantised with the new values
+        x = np.zeros((1, 32), np.float32)
+        x[0, :4] = [6.0, 5.1, 3.4, -2.6]                # e = 0; 5.1 -> 5.0 exists only in the even member
+        codes, ids, scales = oracle.quantize(x)
+        assert int(ids[0, 0]) in (6, 7) and int(scales[0, 0]) == 127
+        deq = oracle.dequantize(codes, ids, scales)[0, :4]
+        allowed = set(float(v) / 2 for v in alt[int(ids[0, 0])])
+        assert all(abs(float(v)) in allowed for v in deq)
+        bad = alt.copy()
+        bad[6, 7] = 11
+        with pytest.raises(ValueError):
+            oracle.set_formatbook(bad)
+        assert (oracle.formatbook() == alt).all()
+    finally:
+        oracle.set_formatbook(None)
+    assert (oracle.formatbook() == default).all()
