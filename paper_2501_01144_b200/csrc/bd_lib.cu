@@ -80,9 +80,15 @@ bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out
                 attr[0].val.programmaticStreamSerializationAllowed = 1;
                 cfg.attrs = attr;
                 cfg.numAttrs = 1;
-                cudaLaunchKernelEx(&cfg, quantize_bf16_kernel<WC, WE>, (const uint16_t *)X, ld, out, e4m3, chunks,
-                                   (uint32_t)nb, (uint32_t)(nb_pad / kBlocksPerAtom),
-                                   make_fast_div((uint32_t)(nb_pad / kBlocksPerAtom)));
+                const bool regular = out.rows % 64 == 0 && nb % kBlocksPerAtom == 0;
+                if (regular)
+                    cudaLaunchKernelEx(&cfg, quantize_bf16_kernel<WC, WE, true>, (const uint16_t *)X, ld, out, e4m3, chunks,
+                                       (uint32_t)nb, (uint32_t)(nb_pad / kBlocksPerAtom),
+                                       make_fast_div((uint32_t)(nb_pad / kBlocksPerAtom)));
+                else
+                    cudaLaunchKernelEx(&cfg, quantize_bf16_kernel<WC, WE, false>, (const uint16_t *)X, ld, out, e4m3, chunks,
+                                       (uint32_t)nb, (uint32_t)(nb_pad / kBlocksPerAtom),
+                                       make_fast_div((uint32_t)(nb_pad / kBlocksPerAtom)));
             }
             else
                 quantize_contig_kernel<BD_BF16, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad);

@@ -329,7 +329,8 @@ __device__ __forceinline__ void quantize_bf16_block(const uint32_t (&R)[16], con
 // one contiguous 32- or 16-byte piece.  The four lanes of a row read 256 contiguous bytes.
 // A CTA takes chunks blockIdx.x, blockIdx.x + gridDim.x, ... (consecutive chunks walk along K) and
 // loads the next chunk's elements before it works on the current ones.
-template <bool WRITE_CODES, bool WRITE_E4M3>
+// REGULAR: rows is a multiple of 64 and K a multiple of 128, so no chunk has padding rows or blocks.
+template <bool WRITE_CODES, bool WRITE_E4M3, bool REGULAR>
 __global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel(const uint16_t *__restrict__ X, int64_t ld, QView out,
                                                             uint8_t *__restrict__ e4m3, uint32_t chunks, uint32_t nb,
                                                             uint32_t kgroups, FastDiv div_kgroups) {
@@ -339,43 +340,40 @@ __global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel
     const uint32_t rows = (uint32_t)out.rows, tiles = (rows + kRowTile - 1) / kRowTile, half_k = (uint32_t)(out.K / 2);
     const uint32_t lane = threadIdx.x % 32u, b4 = lane & 3u, j = (lane >> 2) & 3u;
     const uint32_t row_in_half = 2u * (threadIdx.x / 32u) + (lane >> 4) + 32u * j;      // + 16 * half
-    uint32_t c = blockIdx.x;
-    uint32_t r = 0, b = 0, kg = 0, th = 0;
-    bool valid = false;
-    uint4 l0 = make_uint4(0, 0, 0, 0), l1 = l0, l2 = l0, l3 = l0;
-    auto locate = [&]() {
-        th = fast_div(c, div_kgroups);
-        kg = c - th * kgroups;
-        r = (th >> 1) * kRowTile + (th & 1u) * 16u + row_in_half;
-        b = kg * kBlocksPerAtom + b4;
-        valid = r < rows && b < nb;
-        if (valid) {
-            const uint4 *src = (const uint4 *)(X + (int64_t)r * ld + b * 32u);
-            l0 = __ldg(src); l1 = __ldg(src + 1); l2 = __ldg(src + 2); l3 = __ldg(src + 3);
+    struct Chunk {
+        uint4 l0, l1, l2, l3;          // the block's 32 elements
+        uint32_t r, b, kg, th;         // row, block, k-group, 2 * tile + half
+        bool valid;
+    };
+    // where chunk c is, and its loads
+    auto fetch = [&](Chunk &k, uint32_t c) {
+        k.th = fast_div(c, div_kgroups);
+        k.kg = c - k.th * kgroups;
+        k.r = (k.th >> 1) * kRowTile + (k.th & 1u) * 16u + row_in_half;
+        k.b = k.kg * kBlocksPerAtom + b4;
+        k.valid = REGULAR || (k.r < rows && k.b < nb);
+        if (k.valid) {
+            const uint4 *src = (const uint4 *)(X + (int64_t)k.r * ld + k.b * 32u);
+            k.l0 = __ldg(src); k.l1 = __ldg(src + 1); k.l2 = __ldg(src + 2); k.l3 = __ldg(src + 3);
         }
     };
-    if (c < chunks) locate();
-    while (c < chunks) {                                         // the same trip count for the whole CTA
-        const uint32_t R[16] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w,
-                                l2.x, l2.y, l2.z, l2.w, l3.x, l3.y, l3.z, l3.w};
-        const uint32_t cr = r, cb = b, ckg = kg, cth = th;
-        const bool cvalid = valid;
-        c += gridDim.x;
-        if (c < chunks) locate();
+    auto process = [&](const Chunk &k) {
         BlockResult res;
         res.id = 0; res.scale = 0;
         res.words[0] = res.words[1] = res.words[2] = res.words[3] = 0;
-        if (cvalid) {
+        if (k.valid) {
+            const uint32_t R[16] = {k.l0.x, k.l0.y, k.l0.z, k.l0.w, k.l1.x, k.l1.y, k.l1.z, k.l1.w,
+                                    k.l2.x, k.l2.y, k.l2.z, k.l2.w, k.l3.x, k.l3.y, k.l3.z, k.l3.w};
             quantize_bf16_block(R, tab, res);
             if (WRITE_CODES)
-                *(uint4 *)(out.codes + (uint64_t)cr * half_k + cb * 16u) =
+                *(uint4 *)(out.codes + (uint64_t)k.r * half_k + k.b * 16u) =
                     make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
             if (WRITE_E4M3) {
                 uint32_t lo = tab.e4m3_lo[res.id], hi = tab.e4m3_hi[res.id];
                 uint32_t o[8];
 #pragma unroll
                 for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, o[2 * w], o[2 * w + 1]);
-                uint4 *dst = (uint4 *)(e4m3 + (uint64_t)cr * (2u * half_k) + cb * 32u);
+                uint4 *dst = (uint4 *)(e4m3 + (uint64_t)k.r * (2u * half_k) + k.b * 32u);
                 dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
             }
@@ -388,10 +386,27 @@ __global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel
         sc |= __shfl_xor_sync(0xffffffffu, sc, 2);
         idn |= __shfl_xor_sync(0xffffffffu, idn, 2);
         if (b4 == 0) {
-            const uint32_t atom = ckg * tiles + (cth >> 1), r32 = cr % 32u;
+            const uint32_t atom = k.kg * tiles + (k.th >> 1), r32 = k.r % 32u;
             *(uint32_t *)(out.scales + (size_t)atom * kScaleAtomBytes + r32 * 16u + j * 4u) = sc;
             if (WRITE_CODES) *(uint16_t *)(out.ids + (size_t)atom * kIdAtomBytes + r32 * 8u + j * 2u) = (uint16_t)idn;
         }
+    };
+    // two register sets take turns, so the prefetched chunk is never copied; the trip count is the same for
+    // the whole CTA (the shuffles in process() need every lane)
+    Chunk ka, kb;
+    ka.valid = kb.valid = false;
+    uint32_t c = blockIdx.x;
+    if (c >= chunks) return;
+    fetch(ka, c);
+    while (true) {
+        c += gridDim.x;
+        if (c < chunks) fetch(kb, c);
+        process(ka);
+        if (c >= chunks) break;
+        c += gridDim.x;
+        if (c < chunks) fetch(ka, c);
+        process(kb);
+        if (c >= chunks) break;
     }
 }
 
