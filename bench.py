@@ -249,19 +249,25 @@ def run_gpu(args, rank, world, local_rank):
             dist.barrier()
         torch.cuda.synchronize()
 
+    per_step = []                                        # device time of each step of the last timed() call
+
     def timed(fn, steps, warmup, finish=None):
         for _ in range(warmup):
             fn()
         barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        e0, e1 = marks[0], marks[-1]
         e0.record()
-        for _ in range(steps):
+        for i in range(steps):
             fn()
+            if i + 1 < steps:
+                marks[i + 1].record()                      # a marker in the stream; the host does not wait on it
         if finish:
             finish()
         e1.record()
         barrier()
         ms = e0.elapsed_time(e1)
+        per_step[:] = [marks[i].elapsed_time(marks[i + 1]) for i in range(steps)]
         if world > 1:
             t = torch.tensor([ms], device=dev)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -281,6 +287,7 @@ def run_gpu(args, rank, world, local_rank):
     clocks = sampler.stop(t_begin, t_end)
     launches = bd.launch_count() - launches_warm
     ms_per_step = total_ms / args.steps
+    step_median, step_best = float(np.median(per_step)), float(np.min(per_step))
     value = world * step_flops / (ms_per_step * 1e-3) / 1e12
 
     e2e_ms = timed(step_e2e, args.steps, min(args.warmup, 3), finish_e2e) / args.steps
@@ -368,6 +375,51 @@ def run_gpu(args, rank, world, local_rank):
                               "gbs": nbytes / us / 1e3, "frac_of_roofline": flops / us / 1e6 / bound_tf})
         bd.poll_status()
 
+    # ---- attention products with both operands quantised online (Mistral-7B shapes: 32 heads, 8 KV heads,
+    # 4096 tokens, head_dim 128; reported, not part of the timed step).  QK^T is bound by the write of the
+    # scores, PV by the read of the fp32 probabilities. ----
+    attention = None
+    if rank == 0:
+        heads, kvh, S, hd = 32, 8, 4096, 128
+        torch.manual_seed(4)
+        Aq = [bd.quantize_act(torch.randn(S, hd, device=dev).to(torch.bfloat16)) for _ in range(heads)]
+        Bk = [bd.quantize_act(torch.randn(S, hd, device=dev).to(torch.bfloat16)) for _ in range(kvh)]
+        scores = torch.empty(heads, S, S, dtype=torch.bfloat16, device=dev)          # 1 GiB: L2-cold by size
+        gws = torch.empty(max(1, bd.gemm_workspace_size(S, S, hd)), dtype=torch.uint8, device=dev)
+
+        def time_us(fn, n_rep):
+            fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(n_rep):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / n_rep * 1e3
+
+        qk_us = time_us(lambda: bd.gemm_batched(Aq, Bk, b_group=heads // kvh, out=scores, workspace=gws), 3)
+        del scores
+        P = [torch.rand(S, S, device=dev) for _ in range(3)]                       # 3 x 64 MiB of fp32 > L2
+        Bv = bd.quantize_act(torch.randn(S, hd, device=dev).to(torch.bfloat16), axis=bd.AXIS_STRIDED)
+        O = torch.empty(S, hd, dtype=torch.bfloat16, device=dev)
+        lws = torch.empty(bd.linear_workspace_size(S, hd, S), dtype=torch.uint8, device=dev)
+        turn = [0]
+
+        def pv():
+            bd.linear(P[turn[0] % 3], Bv, out=O, workspace=lws)
+            turn[0] += 1
+
+        pv_us = time_us(pv, 9)
+        qk_bytes, pv_bytes = heads * S * S * 2.0, S * S * 4.0
+        attention = {"workload": "QK^T: 32 heads x [4096,128] x [4096,128]^T, bf16 scores; PV: per head fp32 P [4096,4096] "
+                                 "quantised online x V (token-axis blocks) [128,4096]^T",
+                     "qk_us_32_heads": qk_us, "qk_write_gbs": qk_bytes / qk_us / 1e3,
+                     "qk_frac_of_hbm": qk_bytes / qk_us / 1e3 / peaks["hbm_gbs"],
+                     "pv_us_per_head": pv_us, "pv_read_gbs": pv_bytes / pv_us / 1e3,
+                     "pv_frac_of_hbm": pv_bytes / pv_us / 1e3 / peaks["hbm_gbs"]}
+        del P, Aq, Bk
+        bd.poll_status()
+
     if rank != 0:
         return
     cpu = None
@@ -387,7 +439,8 @@ def run_gpu(args, rank, world, local_rank):
 
     line = {
         "metric": "bd_linear_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "ms_per_step_median": step_median,
+        "ms_per_step_best": step_best, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "e4m3 x e4m3 (exact DialectFP4 decode), fp32 accumulate", "data": "synthetic",
         "config": {"workload": "llama3-8b linear layers (q/o, k/v, gate/up, down), M=2048 tokens per GPU, "
                                "fused online quantise + W4A4 product, bf16 out",
@@ -402,6 +455,7 @@ def run_gpu(args, rank, world, local_rank):
         "cpu_baseline": cpu,
         "per_layer_gflop": {l["name"]: l["flops"] / 1e9 for l in layers},
         "llama2_mlp_m_sweep": sweep,
+        "attention_mistral7b": attention,
     }
     print(json.dumps(line))
     if world > 1:
