@@ -178,27 +178,29 @@ static_assert(Smem::total <= 227 * 1024, "shared memory budget");
 // Work items of a launch, identical for every cluster: cluster c takes items c, c + clusters, ...
 // Tiles are numbered with the token tile running fastest (token tile = tile % t_tiles, weight-row pair =
 // tile / t_tiles), so the clusters that run at the same time share weight rows and differ in their tokens.
-// Items [0, split_from) are whole tiles of 256 tokens; each later tile is two items of 128 tokens, which
-// lets a last, sparsely filled round of tiles spread over twice as many clusters.
+// Items [0, split_from) are whole tiles of 256 tokens.  Each later tile is cut into `parts` items of
+// `part_tokens` tokens: two of 128, which lets a last, sparsely filled round of tiles spread over twice as
+// many clusters; or, when the whole problem has at most 128 tokens, one item of just those tokens (rounded up
+// to the MMA's step of 16), so that a decode-sized call does not pay for 256 columns per k-step.
 struct Schedule {
-    int w_pairs, t_tiles, k_tiles, clusters, split_from;
+    int w_pairs, t_tiles, k_tiles, clusters, split_from, parts, part_tokens;
 };
 struct Tile {
     int w_pair;      // weight rows [256 * w_pair, + 256)
     int t_start;     // first token
-    int tokens;      // 256 or 128: the N of the MMA
+    int tokens;      // the N of the MMA: 256, or the schedule's part_tokens
 };
 __device__ __forceinline__ bool next_tile(const Schedule &sc, int c, int i, Tile &t) {
     const int item = i * sc.clusters + c, tiles = sc.w_pairs * sc.t_tiles;
-    int tile = item, half = 0;
+    int tile = item, part = 0;
     t.tokens = 256;
     if (item >= sc.split_from) {
-        tile = sc.split_from + ((item - sc.split_from) >> 1);
-        half = (item - sc.split_from) & 1;
-        t.tokens = 128;
+        tile = sc.split_from + (item - sc.split_from) / sc.parts;
+        part = (item - sc.split_from) % sc.parts;
+        t.tokens = sc.part_tokens;
     }
     t.w_pair = tile / sc.t_tiles;
-    t.t_start = (tile % sc.t_tiles) * 256 + half * 128;
+    t.t_start = (tile % sc.t_tiles) * 256 + part * 128;
     return tile < tiles;
 }
 
@@ -264,7 +266,7 @@ __device__ __forceinline__ void epilogue_bf16(uint32_t t_base, uint8_t *stage_pt
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapXhalf,
+gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapXpart,
                   const __grid_constant__ CUtensorMap mapCodes,
                   const __grid_constant__ CUtensorMap mapSfW, const __grid_constant__ CUtensorMap mapSfX,
                   const uint8_t *__restrict__ idsW, const Schedule sc, int M, int N, int row_tiles_x, int row_tiles_w,
@@ -336,9 +338,9 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         uint32_t ph = 1;
         Tile t;
         for (int i = 0; next_tile(sc, cluster, i, t); i++) {
-            // each CTA holds half of the tile's tokens; a 128-token item loads 64 rows through its own tensor map
+            // each CTA holds half of the item's tokens; smaller items load their rows through a tensor map of their own
             const int per_cta = t.tokens / 2, t0 = t.t_start + (int)rank * per_cta;
-            const CUtensorMap *map = t.tokens == 256 ? &mapX : &mapXhalf;
+            const CUtensorMap *map = t.tokens == 256 ? &mapX : &mapXpart;
             const uint32_t tx_pair = 2u * ((uint32_t)per_cta * BK + 3u * kScaleAtomBytes);
             for (int kt = 0; kt < sc.k_tiles; kt++) {
                 mbar_wait(x_empty(s), ph, abort_flag);
@@ -348,7 +350,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                     if (rank == 0) mbar_expect_tx(x_full(s), tx_pair);
                     tma_load_2d_pair(x_tile(s), map, kt * BK, t0, fb);
                     tma_load_2d_pair(sfw_tile(s), &mapSfW, 0, kt * row_tiles_w + t.w_pair * 2 + (int)rank, fb);
-                    // two scale atoms = 256 tokens from the item's first token (a 128-token item uses the first)
+                    // two scale atoms = 256 tokens from the item's first token (a smaller item uses the first)
                     tma_load_2d_pair(sfx_tile(s), &mapSfX, 0, kt * row_tiles_x + t.t_start / 128, fb);
                 }
                 __syncwarp();
@@ -503,13 +505,18 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         };
         Tile t;
         for (int i = 0; next_tile(sc, cluster, i, t); i++) {
-            const int cols = t.tokens / 2;                                  // token columns of this warp: 128 or 64
+            // token columns of this warp: the two warps of a quadrant share items of 128 tokens or more; a smaller
+            // item goes to the first of them, rounded up to whole passes of 64 tokens (the columns past the item
+            // hold stale sums of tokens that do not exist, and the stores clip them)
+            const int cols = t.tokens >= 128 ? t.tokens / 2 : (half == 0 ? (t.tokens + 63) / 64 * 64 : 0);
             const int n0 = t.w_pair * 256 + (int)rank * 128 + quad * 32;    // this warp's 32 output columns
             const int t0 = t.t_start + half * cols;                         // and its first output row
             mbar_wait(tmem_full_bar, (uint32_t)i & 1u, abort_flag, 256);
             tcgen05_fence_after();
             const uint32_t t_base = tmem + ((uint32_t)(quad * 32) << 16) + kColD + half * cols;
-            if (use_tma_store && out_bf16) {
+            if (cols == 0) {
+                release_accumulator();
+            } else if (use_tma_store && out_bf16) {
                 if (cols == 128) epilogue_bf16<4>(t_base, stage_ptr, stage_out, &mapY, n0, t0, lane, abort_flag, release_accumulator, staging_free);
                 else epilogue_bf16<2>(t_base, stage_ptr, stage_out, &mapY, n0, t0, lane, abort_flag, release_accumulator, staging_free);
             } else if (use_tma_store) {
@@ -589,10 +596,12 @@ inline int max_resident_clusters() {
 // X as operand bytes + scale atoms (the quantizer's second output form), W as a packed operand.
 inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, const QView &W, int64_t K, void *Y,
                           bool out_bf16, int64_t ldy, cudaStream_t st) {
-    CUtensorMap mapX, mapXhalf, mapCodes, mapSfW, mapSfX, mapY;
+    CUtensorMap mapX, mapXpart, mapCodes, mapSfW, mapSfX, mapY;
     const int64_t N = W.rows, rtx = row_tiles(M), rtw = row_tiles(N), kg = k_groups(K);
+    // items smaller than a whole tile: the whole problem when it has at most 128 tokens, else halves of 128
+    const int part_tokens = M <= 128 ? (int)((M + 15) / 16 * 16) : 128;
     if (!make_map_2d(&mapX, CU_TENSOR_MAP_DATA_TYPE_UINT8, x8, K, M, K, BK, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map_2d(&mapXhalf, CU_TENSOR_MAP_DATA_TYPE_UINT8, x8, K, M, K, BK, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_2d(&mapXpart, CU_TENSOR_MAP_DATA_TYPE_UINT8, x8, K, M, K, BK, part_tokens / 2, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !make_map_2d(&mapCodes, CU_TENSOR_MAP_DATA_TYPE_UINT8, W.codes, K / 2, N, K / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_64B) ||
         !make_map_2d(&mapSfW, CU_TENSOR_MAP_DATA_TYPE_UINT32, W.scales, 128, rtw * kg, kScaleAtomBytes, 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE) ||
         !make_map_2d(&mapSfX, CU_TENSOR_MAP_DATA_TYPE_UINT32, sfx, 128, rtx * kg, kScaleAtomBytes, 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE))
@@ -618,12 +627,20 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
     sc.k_tiles = (int)((K + BK - 1) / BK);
     const int tiles = sc.w_pairs * sc.t_tiles;
     const int resident = max_resident_clusters();
-    // a last round that fills at most half of the clusters is cut into 128-token items (twice as many, half as
-    // long), unless the second half of the last token tile would be empty
-    const int rest = tiles % resident, m_tail = (int)(M % 256);
     sc.split_from = tiles;
-    if (rest > 0 && 2 * rest <= resident && (m_tail == 0 || m_tail > 128)) sc.split_from = tiles - rest;
-    const int items = tiles + (tiles - sc.split_from);
+    sc.parts = 2;
+    sc.part_tokens = part_tokens;
+    if (M <= 128) {
+        // one token tile: every item is the whole (short) token range
+        sc.split_from = 0;
+        sc.parts = 1;
+    } else {
+        // a last round that fills at most half of the clusters is cut into 128-token items (twice as many, half
+        // as long), unless the second half of the last token tile would be empty
+        const int rest = tiles % resident, m_tail = (int)(M % 256);
+        if (rest > 0 && 2 * rest <= resident && (m_tail == 0 || m_tail > 128)) sc.split_from = tiles - rest;
+    }
+    const int items = sc.split_from + (tiles - sc.split_from) * sc.parts;
     sc.clusters = items < resident ? items : resident;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * sc.clusters);
@@ -635,7 +652,7 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemm_wtmem_kernel, mapX, mapXhalf, mapCodes, mapSfW, mapSfX, (const uint8_t *)W.ids, sc, (int)M,
+    return cudaLaunchKernelEx(&cfg, gemm_wtmem_kernel, mapX, mapXpart, mapCodes, mapSfW, mapSfX, (const uint8_t *)W.ids, sc, (int)M,
                               (int)N, (int)rtx, (int)rtw, Y, ldy, out_bf16 ? 1 : 0, mapY, use_tma_store);
 }
 
