@@ -176,15 +176,13 @@ def run_reference(args, rank):
 # ---------------------------------------------------------------------------
 def run_gpu(args, rank, world, local_rank):
     import torch
-    import torch.distributed as dist
 
     import paper_2501_01144_b200 as bd
-    from paper_2501_01144_b200 import inputs
+    from paper_2501_01144_b200 import inputs, replicas
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init("nccl", dev)
     bd.load()
     peaks = measured_peaks()
 
@@ -194,7 +192,7 @@ def run_gpu(args, rank, world, local_rank):
     # resident state: offline-quantised weights, device activations, outputs, workspaces
     layers = []
     for i, (name, K, N) in enumerate(LAYERS):
-        xb = inputs.act_student_t(M_TOKENS, K, seed=2 + i + 100 * rank)
+        xb = inputs.act_student_t(M_TOKENS, K, seed=replicas.rank_seed(2 + i, rank))
         wq = bd.quantize_weights(dev_bf16(inputs.weights_normal(N, K, seed=2 + i)), bd.SELECT_TWO_STAGE)
         x_host = torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16).pin_memory()
         layers.append({
@@ -245,9 +243,7 @@ def run_gpu(args, rank, world, local_rank):
             compute.wait_event(l["y_free"])
 
     def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        replicas.barrier(torch.cuda.synchronize)
 
     per_step = []                                        # device time of each step of the last timed() call
 
@@ -266,13 +262,8 @@ def run_gpu(args, rank, world, local_rank):
             finish()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
         per_step[:] = [marks[i].elapsed_time(marks[i + 1]) for i in range(steps)]
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return replicas.max_over_ranks(e0.elapsed_time(e1), dev)   # the job's time is the slowest rank's
 
     sampler = ClockSampler(local_rank)
     sampler.start()                                        # runs through warm-up and the timed region
@@ -288,10 +279,10 @@ def run_gpu(args, rank, world, local_rank):
     launches = bd.launch_count() - launches_warm
     ms_per_step = total_ms / args.steps
     step_median, step_best = float(np.median(per_step)), float(np.min(per_step))
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    value = replicas.whole_job_rate(step_flops, ms_per_step * 1e-3, world) / 1e12
 
     e2e_ms = timed(step_e2e, args.steps, min(args.warmup, 3), finish_e2e) / args.steps
-    e2e_value = world * step_flops / (e2e_ms * 1e-3) / 1e12
+    e2e_value = replicas.whole_job_rate(step_flops, e2e_ms * 1e-3, world) / 1e12
     h2d = sum(l["X_host"].numel() * 2 for l in layers)
     d2h = sum(l["Y_host"].numel() * 2 for l in layers)
 
@@ -458,8 +449,7 @@ def run_gpu(args, rank, world, local_rank):
         "attention_mistral7b": attention,
     }
     print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.shutdown()
 
 
 def run_case(args):
