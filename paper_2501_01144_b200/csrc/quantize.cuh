@@ -329,27 +329,29 @@ __device__ __forceinline__ void quantize_bf16_block(const uint32_t (&R)[16], con
 // one contiguous 32- or 16-byte piece.  The four lanes of a row read 256 contiguous bytes.
 // A CTA takes chunks blockIdx.x, blockIdx.x + gridDim.x, ... (consecutive chunks walk along K) and
 // loads the next chunk's elements before it works on the current ones.
+// The loop of one warp over its share of the chunks' eight warp-parts (warp-part wp = 8 * chunk + w, w the
+// warp's place in the chunk): parts first, first + stride, ...  Two register sets take turns, so the
+// prefetched part is never copied.  Every lane of the warp must call this (shuffles).
 // REGULAR: rows is a multiple of 64 and K a multiple of 128, so no chunk has padding rows or blocks.
 template <bool WRITE_CODES, bool WRITE_E4M3, bool REGULAR>
-__global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel(const uint16_t *__restrict__ X, int64_t ld, QView out,
-                                                            uint8_t *__restrict__ e4m3, uint32_t chunks, uint32_t nb,
-                                                            uint32_t kgroups, FastDiv div_kgroups) {
-    __shared__ SmemTables tab;
-    load_tables(tab);
-    asm volatile("griddepcontrol.wait;" ::: "memory");           // the source may be the previous kernel's output
+__device__ __forceinline__ void quantize_bf16_parts(const uint16_t *__restrict__ X, int64_t ld, const QView &out,
+                                                    uint8_t *__restrict__ e4m3, const SmemTables &tab, uint32_t first,
+                                                    uint32_t stride, uint32_t parts, uint32_t nb, uint32_t kgroups,
+                                                    FastDiv div_kgroups) {
     const uint32_t rows = (uint32_t)out.rows, tiles = (rows + kRowTile - 1) / kRowTile, half_k = (uint32_t)(out.K / 2);
     const uint32_t lane = threadIdx.x % 32u, b4 = lane & 3u, j = (lane >> 2) & 3u;
-    const uint32_t row_in_half = 2u * (threadIdx.x / 32u) + (lane >> 4) + 32u * j;      // + 16 * half
-    struct Chunk {
+    const uint32_t row_in_part = (lane >> 4) + 32u * j;           // + 2 * w + 16 * half
+    struct Part {
         uint4 l0, l1, l2, l3;          // the block's 32 elements
         uint32_t r, b, kg, th;         // row, block, k-group, 2 * tile + half
         bool valid;
     };
-    // where chunk c is, and its loads
-    auto fetch = [&](Chunk &k, uint32_t c) {
+    // where part wp is, and its loads
+    auto fetch = [&](Part &k, uint32_t wp) {
+        const uint32_t c = wp >> 3;
         k.th = fast_div(c, div_kgroups);
         k.kg = c - k.th * kgroups;
-        k.r = (k.th >> 1) * kRowTile + (k.th & 1u) * 16u + row_in_half;
+        k.r = (k.th >> 1) * kRowTile + (k.th & 1u) * 16u + 2u * (wp & 7u) + row_in_part;
         k.b = k.kg * kBlocksPerAtom + b4;
         k.valid = REGULAR || (k.r < rows && k.b < nb);
         if (k.valid) {
@@ -357,7 +359,7 @@ __global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel
             k.l0 = __ldg(src); k.l1 = __ldg(src + 1); k.l2 = __ldg(src + 2); k.l3 = __ldg(src + 3);
         }
     };
-    auto process = [&](const Chunk &k) {
+    auto process = [&](const Part &k) {
         BlockResult res;
         res.id = 0; res.scale = 0;
         res.words[0] = res.words[1] = res.words[2] = res.words[3] = 0;
@@ -391,23 +393,33 @@ __global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel
             if (WRITE_CODES) *(uint16_t *)(out.ids + (size_t)atom * kIdAtomBytes + r32 * 8u + j * 2u) = (uint16_t)idn;
         }
     };
-    // two register sets take turns, so the prefetched chunk is never copied; the trip count is the same for
-    // the whole CTA (the shuffles in process() need every lane)
-    Chunk ka, kb;
+    Part ka, kb;
     ka.valid = kb.valid = false;
-    uint32_t c = blockIdx.x;
-    if (c >= chunks) return;
-    fetch(ka, c);
+    uint32_t wp = first;
+    if (wp >= parts) return;
+    fetch(ka, wp);
     while (true) {
-        c += gridDim.x;
-        if (c < chunks) fetch(kb, c);
+        wp += stride;
+        if (wp < parts) fetch(kb, wp);
         process(ka);
-        if (c >= chunks) break;
-        c += gridDim.x;
-        if (c < chunks) fetch(ka, c);
+        if (wp >= parts) break;
+        wp += stride;
+        if (wp < parts) fetch(ka, wp);
         process(kb);
-        if (c >= chunks) break;
+        if (wp >= parts) break;
     }
+}
+
+// Persistent CTAs of eight warps: CTA x takes chunks x, x + gridDim.x, ...
+template <bool WRITE_CODES, bool WRITE_E4M3, bool REGULAR>
+__global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel(const uint16_t *__restrict__ X, int64_t ld, QView out,
+                                                            uint8_t *__restrict__ e4m3, uint32_t chunks, uint32_t nb,
+                                                            uint32_t kgroups, FastDiv div_kgroups) {
+    __shared__ SmemTables tab;
+    load_tables(tab);
+    asm volatile("griddepcontrol.wait;" ::: "memory");           // the source may be the previous kernel's output
+    quantize_bf16_parts<WRITE_CODES, WRITE_E4M3, REGULAR>(X, ld, out, e4m3, tab, 8u * blockIdx.x + threadIdx.x / 32u,
+                                                          8u * gridDim.x, 8u * chunks, nb, kgroups, div_kgroups);
 }
 
 // ---------------------------------------------------------------------------
