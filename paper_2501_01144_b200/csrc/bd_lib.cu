@@ -62,16 +62,16 @@ template <int SELECT, bool WC, bool WE>
 bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out, uint8_t *e4m3, cudaStream_t st) {
     const int nb = (int)(out.K / kBlock), nb_pad = (int)k_groups(out.K) * kBlocksPerAtom;
     const int64_t rows_pad = row_tiles(out.rows) * kRowTile;
-    const unsigned grid = grid_for(rows_pad * nb_pad, 256);
+    const unsigned chunks = (unsigned)(rows_pad / 64) * (unsigned)(nb_pad / kBlocksPerAtom);     // 64 rows x one k-group
+    const unsigned gen_grid = chunks;                                                            // generic kernel: one CTA each
     switch (dt) {
-        case BD_F32: quantize_contig_kernel<BD_F32, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad); break;
+        case BD_F32: quantize_contig_kernel<BD_F32, SELECT, WC, WE><<<gen_grid, 256, 0, st>>>(X, ld, out, e4m3, nb, nb_pad / kBlocksPerAtom); break;
         case BD_BF16:
             if (SELECT == BD_SELECT_TWO_STAGE && rows_pad * nb_pad < (1ll << 31))
             {
                 // programmatic dependent launch: the blocks may be scheduled while the previous kernel of the
                 // stream drains; the kernel waits for that kernel's results before it touches global memory
                 cudaLaunchConfig_t cfg = {};
-                const unsigned chunks = (unsigned)(rows_pad / 64) * (unsigned)(nb_pad / kBlocksPerAtom);
                 cfg.gridDim = dim3(std::min(chunks, quant_bf16_grid_limit()));
                 cfg.blockDim = dim3(256);
                 cfg.stream = st;
@@ -91,9 +91,9 @@ bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out
                                        make_fast_div((uint32_t)(nb_pad / kBlocksPerAtom)));
             }
             else
-                quantize_contig_kernel<BD_BF16, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad);
+                quantize_contig_kernel<BD_BF16, SELECT, WC, WE><<<gen_grid, 256, 0, st>>>(X, ld, out, e4m3, nb, nb_pad / kBlocksPerAtom);
             break;
-        case BD_F16: quantize_contig_kernel<BD_F16, SELECT, WC, WE><<<grid, 256, 0, st>>>(X, ld, out, e4m3, rows_pad, nb, nb_pad); break;
+        case BD_F16: quantize_contig_kernel<BD_F16, SELECT, WC, WE><<<gen_grid, 256, 0, st>>>(X, ld, out, e4m3, nb, nb_pad / kBlocksPerAtom); break;
         default: return BD_ERR_INVALID_ARG;
     }
     return launch_result();

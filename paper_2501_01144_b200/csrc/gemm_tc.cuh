@@ -575,9 +575,18 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
 }
 
 // ---- host side --------------------------------------------------------------
+// Per-device state of the launcher (one process may drive several devices).
+constexpr int kMaxDevices = 64;
+inline int current_device() {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    return dev >= 0 && dev < kMaxDevices ? dev : 0;
+}
+
 inline int max_resident_clusters() {
-    static int cached = 0;
-    if (cached) return cached;
+    static int cached[kMaxDevices] = {};
+    const int dev = current_device();
+    if (cached[dev]) return cached[dev];
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * 128);
     cfg.blockDim = dim3(kThreads);
@@ -586,11 +595,11 @@ inline int max_resident_clusters() {
     if (cudaOccupancyMaxActiveClusters(&n, gemm_wtmem_kernel, &cfg) != cudaSuccess || n <= 0) {
         cudaGetLastError();
         int sms = 0;
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         n = sms / 2;
     }
-    cached = n;
-    return cached;
+    cached[dev] = n;
+    return n;
 }
 
 // X as operand bytes + scale atoms (the quantizer's second output form), W as a packed operand.
@@ -615,11 +624,12 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
                      (uint64_t)ldy * esz, 32, out_bf16 ? 64 : 32, CU_TENSOR_MAP_SWIZZLE_NONE))
         use_tma_store = 0;
     if (!use_tma_store) mapY = mapX;                                   // unused, but must be a valid object
-    static bool configured = false;
-    if (!configured) {
+    static bool configured[kMaxDevices] = {};
+    const int dev = current_device();
+    if (!configured[dev]) {
         cudaError_t e = cudaFuncSetAttribute(gemm_wtmem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured[dev] = true;
     }
     Schedule sc;
     sc.w_pairs = (int)((N + 255) / 256);

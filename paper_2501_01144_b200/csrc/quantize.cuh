@@ -423,25 +423,25 @@ __global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel
 }
 
 // ---------------------------------------------------------------------------
-// Contiguous-axis quantizer.  Thread t of the grid owns block (r, b) with
-// t = r * nb_pad + b, nb_pad = 4 * k_groups: four neighbouring lanes share one
-// row and one scale/id atom, so they merge their scale bytes into one 32-bit
-// store and their id nibbles into one 16-bit store.  Threads past the real rows
-// or blocks write the zero padding of the atoms.
-// Optional second output: the decoded operand bytes (E4M3 of 0.5 * value, sign in
-// bit 7) as a plain [rows][K] byte matrix, the form the tensor-core GEMM loads.
+// Contiguous-axis quantizer for every source type and both selection rules (the bf16 two-stage
+// case has the faster kernel above).  One CTA per chunk of 64 rows x one k-group, with the same
+// thread-to-block map as above: the four lanes of a row read neighbouring blocks, sixteen lanes
+// assemble one 16-byte scale unit, and the stores of scales and ids are whole sectors.  Threads
+// past the real rows or blocks write the zero padding of the atoms.
+// Optional second output: the decoded operand bytes (E4M3 of 0.5 * value, sign in bit 7) as a
+// plain [rows][K] byte matrix, the form the tensor-core GEMM loads.
 // ---------------------------------------------------------------------------
 template <int DT, int SELECT, bool WRITE_CODES, bool WRITE_E4M3>
 __global__ void __launch_bounds__(256) quantize_contig_kernel(const void *__restrict__ X, int64_t ld, QView out,
-                                                              uint8_t *__restrict__ e4m3, int64_t rows_pad,
-                                                              int nb, int nb_pad) {
+                                                              uint8_t *__restrict__ e4m3, int nb, int kgroups) {
     __shared__ SmemTables tab;
     load_tables(tab);
-    int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= rows_pad * nb_pad) return;                          // whole groups of 4 lanes leave together
-    int64_t r = t / nb_pad;
-    int b = (int)(t - r * nb_pad);
-    bool valid = r < out.rows && b < nb;
+    const uint32_t lane = threadIdx.x % 32u, b4 = lane & 3u, j = (lane >> 2) & 3u;
+    const int64_t th = blockIdx.x / (uint32_t)kgroups;           // 2 * tile + half
+    const uint32_t kg = blockIdx.x % (uint32_t)kgroups;
+    const int64_t r = (th >> 1) * kRowTile + (th & 1) * 16 + 2 * (threadIdx.x / 32u) + (lane >> 4) + 32 * j;
+    const int b = (int)(kg * kBlocksPerAtom + b4);
+    const bool valid = r < out.rows && b < nb;
     BlockResult res;
     res.id = 0; res.scale = 0;
     res.words[0] = res.words[1] = res.words[2] = res.words[3] = 0;
@@ -465,14 +465,14 @@ __global__ void __launch_bounds__(256) quantize_contig_kernel(const void *__rest
             dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
         }
     }
-    // merge the four lanes of a k-group (lane & 3 = b % 4)
-    uint32_t sc = res.scale << (8 * (b & 3));
-    uint32_t idn = res.id << (4 * (b & 3));
+    // the four lanes of a row merge their scale bytes and id nibbles
+    uint32_t sc = res.scale << (8 * b4);
+    uint32_t idn = res.id << (4 * b4);
     sc |= __shfl_xor_sync(0xffffffffu, sc, 1);
     idn |= __shfl_xor_sync(0xffffffffu, idn, 1);
     sc |= __shfl_xor_sync(0xffffffffu, sc, 2);
     idn |= __shfl_xor_sync(0xffffffffu, idn, 2);
-    if ((b & 3) == 0) {
+    if (b4 == 0) {
         *(uint32_t *)(out.scales + scale_offset(out.rows, r, b)) = sc;
         if (WRITE_CODES) *(uint16_t *)(out.ids + id_byte_offset(out.rows, r, b)) = (uint16_t)idn;
     }
