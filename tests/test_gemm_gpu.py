@@ -47,7 +47,9 @@ def test_tiny_case(impl):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-@pytest.mark.parametrize("M,N,K", [(1, 8, 32), (5, 130, 96), (128, 128, 128), (130, 257, 352), (200, 384, 1024)])
+@pytest.mark.parametrize("M,N,K", [(1, 8, 32), (5, 130, 96), (128, 128, 128), (130, 257, 352), (200, 384, 1024),
+                                   # token tiles cut into 128-token items, with and without a ragged last tile
+                                   (448, 512, 256), (640, 300, 160), (512, 1024, 128)])
 def test_ragged_shapes(impl, M, N, K):
     rng = np.random.default_rng(M + 31 * N + 977 * K)
     a = rng.standard_t(4, (M, K)).astype(np.float32)
@@ -58,6 +60,14 @@ def test_ragged_shapes(impl, M, N, K):
     Y = _run(impl, qa, qb).cpu().numpy()
     ok, ratio = gemm_tolerance_ok(Y, Yref, T)
     assert ok, f"max err / bound = {ratio}"
+
+
+def _run_into(qa_ref, qb_ref, out):
+    """Tensor-core product written into a caller's (possibly strided) view."""
+    bd.set_gemm_impl(bd.GEMM_TCGEN05)
+    A = bd.import_canonical(*(torch.from_numpy(t).cuda() for t in qa_ref))
+    B = bd.import_canonical(*(torch.from_numpy(t).cuda() for t in qb_ref))
+    return bd.gemm(A, B, out=out)
 
 
 def _wide_range_case():
@@ -100,6 +110,25 @@ def test_bf16_output_is_rounded_fp32_result(impl):
     y32 = _run(impl, qa, qb, torch.float32)
     y16 = _run(impl, qa, qb, torch.bfloat16)
     assert torch.equal(y16, y32.to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 264, 256), (100, 520, 96), (448, 512, 256), (700, 256, 512)])
+def test_bf16_output_all_item_widths(M, N, K):
+    """bf16 results of the tensor-core kernel for every kind of work item (a short token range, 128-token
+    halves, whole tiles) equal the rounded fp32 results, through tensor stores and through plain stores."""
+    rng = np.random.default_rng(M * 13 + N)
+    qa = oracle.quantize(rng.standard_t(4, (M, K)).astype(np.float32))
+    qb = oracle.quantize((0.02 * rng.standard_normal((N, K))).astype(np.float32))
+    y32 = _run(bd.GEMM_TCGEN05, qa, qb, torch.float32)
+    y16 = _run(bd.GEMM_TCGEN05, qa, qb, torch.bfloat16)
+    assert torch.equal(y16, y32.to(torch.bfloat16))
+    Yref, T = _ref(qa, qb)
+    ok, ratio = gemm_tolerance_ok(y32.cpu().numpy(), Yref, T)
+    assert ok, f"max err / bound = {ratio}"
+    # a row pitch that is no multiple of 16 bytes takes the kernel's plain-store path
+    wide = torch.zeros(M, N + 3, dtype=torch.bfloat16, device="cuda")
+    out = _run_into(qa, qb, wide[:, :N])
+    assert torch.equal(out, y16) and not wide[:, N:].any()
 
 
 def test_linear_tiny_case_end_to_end():
