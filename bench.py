@@ -42,6 +42,8 @@ BYTES_PER_ELEM_QUANT = 2 + 0.5 + 1.5 / 32           # bf16 read + 4-bit code + (
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
 QUANT_DRAM_BYTES = 67.13e6 + 3.28e6                 # quantize_bf16_kernel on bf16 [8192, 4096]
 GEMM_GATE_UP_DRAM_BYTES = 40.82e6 + 18.31e6         # tc::gemm_wtmem_kernel on the gate/up layer
+QUANT_WARP_INSTRUCTIONS = 14.1e6                    # smsp__inst_executed.sum of the same quantizer launch
+SM_COUNT, ISSUE_PER_SM_CLK = 148, 4                 # warp instructions per clock an SM can issue (4 schedulers)
 MLP_SWEEP = [(4096, 11008), (11008, 4096)]
 MLP_SWEEP_M = [1, 16, 128, 1024, 8192]
 
@@ -336,7 +338,12 @@ def run_gpu(args, rank, world, local_rank):
                      "bound": "hbm", "achieved": q_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": q_gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": q_gbs / 8000.0,
                      "us_per_launch": q_ms * 1e3, "algorithmic_bytes": q_bytes, "traffic": QUANT_DRAM_BYTES,
-                     "peak_source": peaks["source"]}
+                     "peak_source": peaks["source"],
+                     # the kernel is held by instruction issue, not by HBM: its warp instructions per second against
+                     # what 148 SMs x 4 schedulers issue at the maximum SM clock
+                     "alu": {"bound": "alu", "achieved": QUANT_WARP_INSTRUCTIONS / (q_ms * 1e-3) / 1e9,
+                             "peak": SM_COUNT * ISSUE_PER_SM_CLK * 1.965, "unit": "G warp-instructions/s",
+                             "frac": QUANT_WARP_INSTRUCTIONS / (q_ms * 1e-3) / 1e9 / (SM_COUNT * ISSUE_PER_SM_CLK * 1.965)}}
     bd.poll_status()
 
     # ---- LLaMA2-7B MLP shapes, decode to prefill (reported per M; not part of the timed step) ----
