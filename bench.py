@@ -383,7 +383,7 @@ def run_gpu(args, rank, world, local_rank):
         Aq = [bd.quantize_act(torch.randn(S, hd, device=dev).to(torch.bfloat16)) for _ in range(heads)]
         Bk = [bd.quantize_act(torch.randn(S, hd, device=dev).to(torch.bfloat16)) for _ in range(kvh)]
         scores = torch.empty(heads, S, S, dtype=torch.bfloat16, device=dev)          # 1 GiB: L2-cold by size
-        gws = torch.empty(max(1, bd.gemm_workspace_size(S, S, hd)), dtype=torch.uint8, device=dev)
+        gws = torch.empty(max(1, bd.gemm_batched_workspace_size(S, S, hd, heads // kvh)), dtype=torch.uint8, device=dev)
 
         def time_us(fn, n_rep):
             fn()

@@ -117,7 +117,12 @@ bd_status bd_gemm(const bd_qtensor *A, const bd_qtensor *B, void *Y, bd_dtype yd
  * independent products; operand b of A uses operand b / b_group of B (grouped-query
  * attention shares one K/V head among b_group query heads).  A points to `batch`
  * descriptors, B to batch / b_group descriptors (host arrays); Y + b * stride_y
- * elements is product b. */
+ * elements is product b.  All operands of A share one shape, all of B another.
+ * With a workspace of bd_gemm_batched_workspace_size bytes, results of a group that
+ * are contiguous in Y (stride_y == M * ldy) and M a multiple of 128, the b_group
+ * products of a group run as one stacked launch; otherwise (any workspace of at
+ * least bd_gemm_workspace_size bytes) one launch per product. */
+bd_status bd_gemm_batched_workspace_size(int64_t M, int64_t N, int64_t K, int64_t b_group, size_t *bytes);
 bd_status bd_gemm_batched(const bd_qtensor *A, const bd_qtensor *B, int64_t batch, int64_t b_group,
                           void *Y, bd_dtype ydtype, int64_t ldy, int64_t stride_y, void *workspace,
                           size_t workspace_bytes, void *stream);

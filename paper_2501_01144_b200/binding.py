@@ -63,6 +63,7 @@ def load():
     lib.bd_quantize_act.argtypes = [vp, ci, i64, i64, i64, ci, qp, vp]
     lib.bd_gemm_workspace_size.argtypes = [i64, i64, i64, szp]
     lib.bd_gemm.argtypes = [qp, qp, vp, ci, i64, vp, sz, vp]
+    lib.bd_gemm_batched_workspace_size.argtypes = [i64, i64, i64, i64, szp]
     lib.bd_gemm_batched.argtypes = [qp, qp, i64, i64, vp, ci, i64, i64, vp, sz, vp]
     lib.bd_linear_workspace_size.argtypes = [i64, i64, i64, szp]
     lib.bd_linear.argtypes = [vp, ci, i64, i64, i64, qp, vp, ci, i64, vp, sz, vp]
@@ -212,13 +213,19 @@ def gemm(A, B, out=None, dtype=torch.float32, workspace=None, stream=None):
     return out
 
 
+def gemm_batched_workspace_size(M, N, K, b_group):
+    b = ctypes.c_size_t()
+    _check(load().bd_gemm_batched_workspace_size(M, N, K, b_group, ctypes.byref(b)))
+    return b.value
+
+
 def gemm_batched(As, Bs, b_group=1, out=None, dtype=torch.float32, workspace=None, stream=None):
     """Batched product; A[b] pairs with B[b // b_group] (grouped-query attention)."""
     batch = len(As)
     M, N, K = As[0].rows, Bs[0].rows, As[0].K
     if out is None:
         out = torch.empty(batch, M, N, dtype=dtype, device=As[0].codes.device)
-    workspace, wptr, wbytes = _ws(workspace, gemm_workspace_size(M, N, K), As[0].codes.device)
+    workspace, wptr, wbytes = _ws(workspace, gemm_batched_workspace_size(M, N, K, b_group), As[0].codes.device)
     ca = (_CQTensor * batch)(*[a.c_struct() for a in As])
     cb = (_CQTensor * len(Bs))(*[b.c_struct() for b in Bs])
     _check(load().bd_gemm_batched(ca, cb, batch, b_group, ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),

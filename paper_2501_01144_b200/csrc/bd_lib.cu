@@ -226,6 +226,20 @@ bd_status bd_gemm(const bd_qtensor *A, const bd_qtensor *B, void *Y, bd_dtype yd
     return gemm_dispatch(view_of(A), view_of(B), Y, ydtype, ldy, workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
+bd_status bd_gemm_batched_workspace_size(int64_t M, int64_t N, int64_t K, int64_t b_group, size_t *bytes) {
+    if (!bytes || M <= 0 || N <= 0 || K <= 0 || b_group <= 0) return BD_ERR_INVALID_ARG;
+    if (K % kBlock) return BD_ERR_SHAPE;
+    size_t single = 0;
+    bd_status s = bd_gemm_workspace_size(M, N, K, &single);
+    if (s) return s;
+    const int64_t count = std::min<int64_t>(b_group, kStackMax);
+    size_t c, i, sc;
+    bd_qtensor_sizes(M * count, K, &c, &i, &sc);
+    const size_t stacked = b_group > 1 ? align256(sc) + tc_operand_bytes(M * count, K) : 0;
+    *bytes = std::max(single, stacked);
+    return BD_OK;
+}
+
 bd_status bd_gemm_batched(const bd_qtensor *A, const bd_qtensor *B, int64_t batch, int64_t b_group, void *Y,
                           bd_dtype ydtype, int64_t ldy, int64_t stride_y, void *workspace, size_t workspace_bytes,
                           void *stream) {
@@ -235,6 +249,43 @@ bd_status bd_gemm_batched(const bd_qtensor *A, const bd_qtensor *B, int64_t batc
         if (s) return s;
     }
     const int ysz = ydtype == BD_F32 ? 4 : 2;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t M = A[0].rows, N = B[0].rows, K = A[0].K;
+    size_t stacked_need = 0;
+    bd_gemm_batched_workspace_size(M, N, K, b_group, &stacked_need);
+    // Grouped products share their B operand: when the group's results are contiguous in Y and the operands are
+    // whole row tiles, the group's A operands are decoded into one stacked matrix and the group is one launch.
+    const bool stack = b_group > 1 && M % kRowTile == 0 && stride_y == M * ldy && use_tc(M * b_group, N, K) &&
+                       tc_supported(M * b_group, N, K) && workspace && workspace_bytes >= stacked_need &&
+                       !((uintptr_t)workspace & 255u);
+    if (stack) {
+        const int nb = (int)(K / kBlock);
+        for (int64_t g0 = 0; g0 < batch; g0 += b_group) {
+            uint8_t *y = (uint8_t *)Y + g0 * stride_y * ysz;
+            for (int64_t c0 = 0; c0 < b_group; c0 += kStackMax) {            // at most kStackMax operands per launch
+                const int count = (int)std::min<int64_t>(kStackMax, b_group - c0);
+                size_t sc_bytes, dummy_c, dummy_i;
+                bd_qtensor_sizes(M * count, K, &dummy_c, &dummy_i, &sc_bytes);
+                uint8_t *sf = (uint8_t *)workspace, *a8 = sf + align256(sc_bytes);
+                StackedViews v = {};
+                for (int h = 0; h < count; h++) {
+                    const bd_qtensor &a = A[g0 + c0 + h];
+                    v.codes[h] = (const uint8_t *)a.codes;
+                    v.ids[h] = (const uint8_t *)a.ids;
+                    v.scales[h] = (const uint8_t *)a.scales;
+                }
+                dim3 grid(grid_for(M * nb, 256), (unsigned)count);
+                decode_e4m3_stacked_kernel<<<grid, 256, 0, st>>>(v, count, M, K, a8, sf, nb);
+                bd_status s = launch_result(1);
+                if (s) return s;
+                g_launches += 1;
+                s = cuda_result(tc::launch(a8, sf, M * count, view_of(&B[g0 / b_group]), K, y + c0 * stride_y * ysz,
+                                           ydtype == BD_BF16, ldy, st));
+                if (s) return s;
+            }
+        }
+        return BD_OK;
+    }
     for (int64_t i = 0; i < batch; i++) {
         bd_status s = gemm_dispatch(view_of(&A[i]), view_of(&B[i / b_group]), (char *)Y + i * stride_y * ysz, ydtype,
                                     ldy, workspace, workspace_bytes, (cudaStream_t)stream);

@@ -615,4 +615,41 @@ __global__ void decode_e4m3_kernel(QView q, uint8_t *__restrict__ out, int nb) {
     dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
+// Decode up to kStackMax packed operands of the same shape into one stacked operand-byte matrix
+// [count * rows][K] and gather their scale atoms in the stacked operand's atom order
+// (k-group-major over count * row_tiles row tiles), so that one GEMM launch serves them all.
+// rows must be a multiple of 128 (whole row tiles per operand).  blockIdx.y = operand.
+constexpr int kStackMax = 8;
+struct StackedViews {
+    const uint8_t *codes[kStackMax], *ids[kStackMax], *scales[kStackMax];
+};
+__global__ void decode_e4m3_stacked_kernel(StackedViews v, int count, int64_t rows, int64_t K, uint8_t *__restrict__ out,
+                                           uint8_t *__restrict__ out_scales, int nb) {
+    const int h = blockIdx.y;
+    const int64_t tiles = rows / kRowTile, kgs = (nb + kBlocksPerAtom - 1) / kBlocksPerAtom;
+    QView q{(uint8_t *)v.codes[h], (uint8_t *)v.ids[h], (uint8_t *)v.scales[h], rows, K};
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < rows * nb) {
+        const int64_t r = t / nb;
+        const int b = (int)(t - r * nb);
+        uint4 u = *(const uint4 *)(q.codes + r * (K / 2) + (int64_t)b * 16);
+        uint32_t w[4] = {u.x, u.y, u.z, u.w}, o[8];
+        uint32_t id = (q.ids[id_byte_offset(rows, r, b)] >> (4 * (b & 1))) & 15;
+        uint32_t lo = c_tables.e4m3_lo[id], hi = c_tables.e4m3_hi[id];
+#pragma unroll
+        for (int i = 0; i < 4; i++) decode_word(w[i], lo, hi, o[2 * i], o[2 * i + 1]);
+        uint4 *dst = (uint4 *)(out + ((int64_t)h * rows + r) * K + (int64_t)b * 32);
+        dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+    // scale atoms, 16 bytes per thread: atom (kg, rt) of operand h goes to (kg, h * tiles + rt)
+    const int64_t vecs = kgs * tiles * (kScaleAtomBytes / 16);
+    for (int64_t i = t; i < vecs; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t atom = i / (kScaleAtomBytes / 16), within = i % (kScaleAtomBytes / 16);
+        const int64_t kg = atom / tiles, rt = atom % tiles;
+        const uint4 val = *(const uint4 *)(q.scales + atom * kScaleAtomBytes + within * 16);
+        *(uint4 *)(out_scales + (kg * (count * tiles) + h * tiles + rt) * kScaleAtomBytes + within * 16) = val;
+    }
+}
+
 }  // namespace bd

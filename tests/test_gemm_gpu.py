@@ -153,3 +153,28 @@ def test_batched_grouped_query_product():
         Yref, T = _ref(oracle_quantize(q[h], torch.bfloat16), oracle_quantize(k[h // 2], torch.bfloat16))
         ok, ratio = gemm_tolerance_ok(Y[h], Yref, T)
         assert ok, f"head {h}: max err / bound = {ratio}"
+
+
+def test_batched_groups_as_stacked_launches():
+    """With whole row tiles per operand and contiguous results, a group's products run as one stacked launch:
+    the result must equal the product-by-product route bit for bit, for both output types."""
+    rng = np.random.default_rng(22)
+    heads, kv, S, d = 6, 2, 256, 160                       # b_group = 3, K = 160: two k-groups, the second ragged
+    q = inputs.to_bf16_bits(rng.standard_normal((heads, S, d)).astype(np.float32))
+    k = inputs.to_bf16_bits(rng.standard_normal((kv, 200, d)).astype(np.float32))
+    As = [bd.quantize_act(to_device(q[h], torch.bfloat16)) for h in range(heads)]
+    Bs = [bd.quantize_act(to_device(k[g], torch.bfloat16)) for g in range(kv)]
+    bd.set_gemm_impl(bd.GEMM_TCGEN05)
+    for dt in (torch.float32, torch.bfloat16):
+        stacked = bd.gemm_batched(As, Bs, b_group=3, dtype=dt)
+        single = torch.stack([bd.gemm(As[h], Bs[h // 3], dtype=dt) for h in range(heads)])
+        assert torch.equal(stacked, single)
+    # a workspace that only fits one product falls back to one launch per product
+    small = torch.empty(bd.gemm_workspace_size(S, 200, d), dtype=torch.uint8, device="cuda")
+    assert small.numel() < bd.gemm_batched_workspace_size(S, 200, d, 3)
+    fallback = bd.gemm_batched(As, Bs, b_group=3, dtype=torch.float32, workspace=small)
+    assert torch.equal(fallback, bd.gemm_batched(As, Bs, b_group=3, dtype=torch.float32))
+    Yref, T = _ref(oracle_quantize(q[4], torch.bfloat16), oracle_quantize(k[1], torch.bfloat16))
+    ok, ratio = gemm_tolerance_ok(fallback[4].cpu().numpy(), Yref, T)
+    assert ok, f"max err / bound = {ratio}"
+    bd.poll_status()
