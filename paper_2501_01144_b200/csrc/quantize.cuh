@@ -445,9 +445,40 @@ __global__ void __launch_bounds__(256) quantize_contig_kernel(const void *__rest
     BlockResult res;
     res.id = 0; res.scale = 0;
     res.words[0] = res.words[1] = res.words[2] = res.words[3] = 0;
+    // fp32 blocks are 128 bytes, one cache line each: read thread by thread, every 16-byte load of a warp
+    // would touch 32 lines.  Instead the warp copies its eight rows line by line (the four blocks of a row
+    // are 512 contiguous bytes, 16 per lane) into shared memory, asynchronously, and each thread then
+    // picks up its own block; an xor of the chunk index keeps both sides free of bank conflicts.
+    __shared__ __align__(128) uint8_t stage[DT == BD_F32 ? 8 * 4096 : 16];
+    if (DT == BD_F32) {
+        const uint32_t warp = threadIdx.x / 32u;
+        const int64_t row0 = (th >> 1) * kRowTile + (th & 1) * 16 + 2 * warp;
+        const int cb = (int)(kg * kBlocksPerAtom) + (int)(lane >> 3);            // the block this lane copies from
+#pragma unroll
+        for (int i = 0; i < 8; i++) {
+            const int64_t ri = row0 + (i >> 2) + 32 * (i & 3);
+            const bool ok = ri < out.rows && cb < nb;
+            const char *src = ok ? (const char *)X + (ri * ld + (int64_t)cb * 32) * 4 + (lane & 7u) * 16 : (const char *)X;
+            const uint32_t owner = 4u * i + (lane >> 3);
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(stage) + warp * 4096u + owner * 128u +
+                                 (((lane & 7u) ^ (owner & 7u)) * 16u);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(ok ? 16 : 0) : "memory");
+        }
+        asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+        __syncwarp();
+    }
     if (valid) {
         uint32_t bits[32];
-        Loader<DT>::contiguous((const char *)X + (r * ld + (int64_t)b * 32) * Loader<DT>::kElemBytes, bits);
+        if (DT == BD_F32) {
+            const uint8_t *mine = stage + (threadIdx.x / 32u) * 4096u + lane * 128u;
+#pragma unroll
+            for (int k = 0; k < 8; k++) {
+                const uint4 u = *(const uint4 *)(mine + ((k ^ (lane & 7u)) * 16u));
+                bits[4 * k] = u.x; bits[4 * k + 1] = u.y; bits[4 * k + 2] = u.z; bits[4 * k + 3] = u.w;
+            }
+        } else {
+            Loader<DT>::contiguous((const char *)X + (r * ld + (int64_t)b * 32) * Loader<DT>::kElemBytes, bits);
+        }
         bool nonfinite;
         if (SELECT == BD_SELECT_MSE) res = quantize_mse(bits, tab, nonfinite);
         else res = quantize_two_stage(bits, tab, nonfinite);
