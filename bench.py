@@ -445,6 +445,11 @@ def run_gpu(args, rank, world, local_rank):
                    "l2": f"working set {footprint / 2**20:.0f} MiB per step cycles through 4 layers (> 126 MB L2)",
                    "weights": "offline two-stage rule", "block": 32},
         "clocks": clocks,
+        # the whole step (quantizers included, per GPU) against dense-FP8 figures derived from the bf16 peaks:
+        # twice the burst and twice the sustained (seconds-long, power-capped) measured bf16 rate, and the nominal 4500
+        "step_vs_fp8_peaks": {"of_2x_bf16_burst": value / world / (2.0 * peaks["bf16_tflops"]),
+                              "of_2x_bf16_sustained": value / world / (2.0 * peaks["bf16_tflops_sustained"]),
+                              "of_nominal_4500": value / world / 4500.0, "peak_source": peaks["source"]},
         "e2e": {"value": e2e_value, "unit": "TFLOP/s", "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches),
