@@ -397,3 +397,62 @@ def test_alternative_formatbook_in_the_oracle():
     finally:
         oracle.set_formatbook(None)
     assert (oracle.formatbook() == default).all()
+
+
+def test_power_of_two_scaling_moves_only_the_exponent():
+    """Scaling a block by 2^k is exact in binary floating point, so codes and dialect must not change and the
+    stored exponent moves by k (Sec. 3.2: the shared exponent absorbs the block's magnitude); flipping every
+    sign flips every sign bit and nothing else; permuting the elements of a block permutes its codes."""
+    rng = np.random.default_rng(31)
+    x = (rng.standard_t(4, (6, 96)) * np.exp2(rng.integers(-3, 4, (6, 1)))).astype(np.float32)
+    codes, ids, scales = oracle.quantize(x)
+    for k in (-9, -1, 3, 17):
+        c2, i2, s2 = oracle.quantize(np.ldexp(x, k).astype(np.float32))
+        assert np.array_equal(c2, codes) and np.array_equal(i2, ids)
+        assert np.array_equal(s2.astype(int), scales.astype(int) + k)
+    cn, in_, sn = oracle.quantize(-x)
+    assert np.array_equal(in_, ids) and np.array_equal(sn, scales)
+    assert np.array_equal(cn ^ 0x88, codes)                       # bit 3 of each nibble is the sign
+    perm = rng.permutation(32)
+    xp = x.reshape(6, 3, 32)[:, :, perm].reshape(6, 96)
+    cp, ip, sp = oracle.quantize(xp)
+    assert np.array_equal(ip, ids) and np.array_equal(sp, scales)
+    nib = lambda c: np.stack([c & 15, c >> 4], -1).reshape(6, 3, 32)
+    assert np.array_equal(nib(cp), nib(codes)[:, :, perm])
+    for select in (oracle.SELECT_MSE,):
+        a = oracle.quantize(x, select)
+        b = oracle.quantize(np.ldexp(x, 5).astype(np.float32), select)
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+def test_error_bound_and_idempotence():
+    """Within a block the dequantised value lies within half a grid step of the input, where the step between the
+    chosen dialect's neighbouring values is at most 2.5 units above the common values (Sec. 3.1: granularity 0.5
+    below, one differing large value above), and never exceeds the rounded block maximum; quantising the
+    dequantised values again reproduces codes, dialect and exponent (the grid points are fixed points)."""
+    rng = np.random.default_rng(32)
+    x = (rng.standard_normal((40, 64)) * np.exp2(rng.integers(-8, 8, (40, 1)))).astype(np.float32)
+    x[:, 5] *= 13
+    FB = oracle.formatbook()
+    for select in (oracle.SELECT_TWO_STAGE, oracle.SELECT_MSE):
+        codes, ids, scales = oracle.quantize(x, select)
+        deq = oracle.dequantize(codes, ids, scales)
+        for r in range(x.shape[0]):
+            for b in range(2):
+                seg = slice(32 * b, 32 * b + 32)
+                e = int(scales[r, b]) - 127
+                vals = FB[ids[r, b]].astype(np.float64) / 2
+                gaps = np.diff(vals)
+                scaled_in = np.abs(x[r, seg].astype(np.float64)) / 2.0 ** e
+                scaled_out = np.abs(deq[r, seg]) / 2.0 ** e
+                assert np.all(np.isin(scaled_out, vals))
+                # the truncated 5-bit magnitude is what gets rounded: up to 0.25 lost, then half the local gap,
+                # and values beyond the dialect's maximum saturate at it
+                inside = scaled_in <= vals[-1]
+                assert np.all(np.abs(scaled_out - scaled_in)[inside] <= 0.25 + gaps.max() / 2 + 1e-12)
+                assert np.all(scaled_out[~inside] == vals[-1])
+                assert np.all(scaled_in < 8.0)
+        c2, i2, s2 = oracle.quantize(deq.astype(np.float32), oracle.SELECT_TWO_STAGE)
+        if select == oracle.SELECT_TWO_STAGE:
+            assert np.array_equal(s2, scales)
+            assert np.array_equal(oracle.dequantize(c2, i2, s2), deq)
