@@ -178,3 +178,38 @@ def test_batched_groups_as_stacked_launches():
     ok, ratio = gemm_tolerance_ok(fallback[4].cpu().numpy(), Yref, T)
     assert ok, f"max err / bound = {ratio}"
     bd.poll_status()
+
+
+@pytest.mark.parametrize("kind", [torch.float32, torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("M,N,K", [(37, 300, 224), (300, 130, 96), (520, 264, 1056)])
+def test_linear_source_types_pitches_and_ragged_shapes(kind, M, N, K):
+    """bd_linear through the tensor-core path for every source type, with a source pitch larger than K, an output
+    pitch larger than N and shapes that fill no tile or atom: the result matches the oracle's two-stage
+    quantisation of the same bytes followed by the fp64 product, and nothing is written beside the output."""
+    rng = np.random.default_rng(M + N + K)
+    x = (rng.standard_t(4, (M, K)) * np.exp2(rng.integers(-4, 5, (M, 1)))).astype(np.float32)
+    x[:, rng.integers(0, K)] *= 40
+    if kind == torch.float32:
+        host, odt = x, oracle.F32
+    elif kind == torch.bfloat16:
+        host, odt = inputs.to_bf16_bits(x), oracle.BF16
+    else:
+        host, odt = inputs.to_f16_bits(np.clip(x, -6e4, 6e4)), oracle.F16
+    wb = inputs.weights_normal(N, K, seed=K)
+    Wq = bd.quantize_weights(to_device(wb, torch.bfloat16), bd.SELECT_TWO_STAGE)
+    wide_x = torch.zeros(M, K + 64, dtype=kind, device="cuda")
+    wide_x[:, :K] = to_device(host, kind)
+    bd.set_gemm_impl(bd.GEMM_TCGEN05)
+    Yref, T = _ref(oracle.quantize(host, dtype=odt), oracle.quantize(wb, dtype=oracle.BF16))
+    for ydt in (torch.float32, torch.bfloat16):
+        wide_y = torch.full((M, N + 8), -7.0, dtype=ydt, device="cuda")
+        bd.linear(wide_x[:, :K], Wq, out=wide_y[:, :N])
+        assert (wide_y[:, N:] == -7.0).all()
+        y = wide_y[:, :N].float().cpu().numpy()
+        if ydt == torch.float32:
+            ok, ratio = gemm_tolerance_ok(y, Yref, T)
+            assert ok, f"{kind} -> fp32: max err / bound = {ratio}"
+            y32 = wide_y[:, :N].clone()
+        else:
+            assert torch.equal(wide_y[:, :N], y32.to(torch.bfloat16))
+    bd.poll_status()
