@@ -359,7 +359,8 @@ def run_gpu(args, rank, world, local_rank):
                 for _ in range(3):
                     bd.linear(x, wq, out=y, workspace=ws)
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                n_rep = 10
+                n_rep = 20
+                torch.cuda._sleep(2_000_000)                  # GPU head start: the events see kernel time, not launch rate
                 a.record()
                 for _ in range(n_rep):
                     bd.linear(x, wq, out=y, workspace=ws)
