@@ -182,16 +182,30 @@ static_assert(Smem::total <= 227 * 1024, "shared memory budget");
 // `part_tokens` tokens: two of 128, which lets a last, sparsely filled round of tiles spread over twice as
 // many clusters; or, when the whole problem has at most 128 tokens, one item of just those tokens (rounded up
 // to the MMA's step of 16), so that a decode-sized call does not pay for 256 columns per k-step.
+// A decode-sized call (at most 16 tokens) has few tiles (one per 256 weight rows); with k_splits > 1 each is
+// further cut along K into k_splits items of k_per k-steps whose partial sums meet in global memory (see the
+// epilogue), so that more SMs pull weights.
 struct Schedule {
-    int w_pairs, t_tiles, k_tiles, clusters, split_from, parts, part_tokens;
+    int w_pairs, t_tiles, k_tiles, clusters, split_from, parts, part_tokens, k_splits, k_per;
 };
 struct Tile {
     int w_pair;      // weight rows [256 * w_pair, + 256)
     int t_start;     // first token
     int tokens;      // the N of the MMA: 256, or the schedule's part_tokens
+    int k_begin, k_end, split;   // k-steps of this item; which split of its tile it is
 };
 __device__ __forceinline__ bool next_tile(const Schedule &sc, int c, int i, Tile &t) {
-    const int item = i * sc.clusters + c, tiles = sc.w_pairs * sc.t_tiles;
+    int item = i * sc.clusters + c;
+    const int tiles = sc.w_pairs * sc.t_tiles;
+    t.k_begin = 0;
+    t.k_end = sc.k_tiles;
+    t.split = 0;
+    if (sc.k_splits > 1) {                                        // every tile is k_splits consecutive items
+        t.split = item % sc.k_splits;
+        item /= sc.k_splits;
+        t.k_begin = t.split * sc.k_per;
+        t.k_end = min(sc.k_tiles, t.k_begin + sc.k_per);
+    }
     int tile = item, part = 0;
     t.tokens = 256;
     if (item >= sc.split_from) {
@@ -203,6 +217,12 @@ __device__ __forceinline__ bool next_tile(const Schedule &sc, int c, int i, Tile
     t.t_start = (tile % sc.t_tiles) * 256 + part * 128;
     return tile < tiles;
 }
+
+// Split-K bookkeeping: arrival counters of the slices (weight-row pair x CTA x lane quadrant) of a launch, all
+// zero between launches (the last arriver resets its counter).  Launches take the slots in turn, so launches
+// that overlap in time (other streams) do not share counters unless more than kArrivalSlots do.
+constexpr int kMaxKSplits = 4, kMinKPerSplit = 8, kSplitMaxTokens = 16, kArrivalSlots = 16, kArrivalWords = 4096;
+__device__ unsigned int g_splitk_arrivals[kArrivalSlots * kArrivalWords];
 
 __device__ __forceinline__ void tcgen05_mma_mxf8_pair_atmem(uint32_t d, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
                                                             uint32_t sfa, uint32_t sfb, uint32_t accumulate) {
@@ -270,7 +290,8 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                   const __grid_constant__ CUtensorMap mapCodes,
                   const __grid_constant__ CUtensorMap mapSfW, const __grid_constant__ CUtensorMap mapSfX,
                   const uint8_t *__restrict__ idsW, const Schedule sc, int M, int N, int row_tiles_x, int row_tiles_w,
-                  void *__restrict__ Y, int64_t ldy, int out_bf16, const __grid_constant__ CUtensorMap mapY, int use_tma_store) {
+                  void *__restrict__ Y, int64_t ldy, int out_bf16, const __grid_constant__ CUtensorMap mapY, int use_tma_store,
+                  float *__restrict__ partials, unsigned int *__restrict__ arrivals) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *const base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -342,7 +363,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             const int per_cta = t.tokens / 2, t0 = t.t_start + (int)rank * per_cta;
             const CUtensorMap *map = t.tokens == 256 ? &mapX : &mapXpart;
             const uint32_t tx_pair = 2u * ((uint32_t)per_cta * BK + 3u * kScaleAtomBytes);
-            for (int kt = 0; kt < sc.k_tiles; kt++) {
+            for (int kt = t.k_begin; kt < t.k_end; kt++) {
                 mbar_wait(x_empty(s), ph, abort_flag);
                 if (*abort_flag) break;
                 const uint32_t fb = map_to_cta(x_full(s), 0);
@@ -367,7 +388,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             const int w0 = t.w_pair * 256 + (int)rank * 128;
             const int my_row_tile = t.w_pair * 2 + (int)rank;
             const bool have_ids = my_row_tile < row_tiles_w;
-            for (int kt = 0; kt < sc.k_tiles; kt++) {
+            for (int kt = t.k_begin; kt < t.k_end; kt++) {
                 mbar_wait(c_empty(s), ph, abort_flag);
                 if (*abort_flag) break;
                 if (elect_one()) {
@@ -400,7 +421,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 const uint32_t idesc0 = idesc_m | (uint32_t)(t.tokens >> 3) << 17;
                 if (i > 0) mbar_wait(tmem_empty_bar, (uint32_t)(i - 1) & 1u, abort_flag);
                 tcgen05_fence_after();
-                for (int kt = 0; kt < sc.k_tiles; kt++) {
+                for (int kt = t.k_begin; kt < t.k_end; kt++) {
                     if (!ready) {
                         // slow path: the probe at the end of the previous k-step found a barrier open
                         mbar_wait(x_full(s), ph_s, abort_flag);
@@ -412,7 +433,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                     const uint32_t lo_sfx = lo_sfx0 + (uint32_t)s * (2 * kScaleAtomBytes >> 4);
                     const uint32_t lo_x = lo_x0 + (uint32_t)s * (kXTile >> 4);
                     const uint32_t t_a = tmem + kColA + 32u * (uint32_t)b;
-                    const uint32_t first = kt == 0 ? 0u : 1u;
+                    const uint32_t first = kt == t.k_begin ? 0u : 1u;
                     if (elect_one()) {
                         tcgen05_cp_pair(t_sfw, desc_join(lo_sfw, hi_sf));
                         tcgen05_cp_pair(t_sfx, desc_join(lo_sfx, hi_sf));
@@ -451,7 +472,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         int total_k = 0;
         {
             Tile t;
-            for (int i = 0; next_tile(sc, cluster, i, t); i++) total_k += sc.k_tiles;
+            for (int i = 0; next_tile(sc, cluster, i, t); i++) total_k += t.k_end - t.k_begin;
         }
         for (int g = group; g < total_k; g += kDecodeGroups) {
             const int s = g % kCodeStages, b = g % kABufs;
@@ -516,6 +537,54 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             const uint32_t t_base = tmem + ((uint32_t)(quad * 32) << 16) + kColD + half * cols;
             if (cols == 0) {
                 release_accumulator();
+            } else if (sc.k_splits > 1) {
+                // split along K: this item's sums are partial.  Each warp writes its 32 weight rows x tokens to
+                // partials[split][token][weight row]; the warp that arrives last for this slice (an atomic count,
+                // nobody waits) adds the splits in their fixed order and writes Y, so the result does not depend
+                // on who came last.
+                const int n = n0 + lane, np = sc.w_pairs * 256, toks = sc.part_tokens;
+                const int tok0 = t.tokens >= 128 ? half * cols : 0;          // this warp's first token
+                float *mine = partials + ((size_t)t.split * toks + tok0) * np + n;
+#pragma unroll 1
+                for (int c = 0; c * 16 < cols; c++) {
+                    uint32_t r[16];
+                    tcgen05_ld_32x32b_x16(t_base + c * 16, r);
+                    tcgen05_wait_ld();
+#pragma unroll
+                    for (int q = 0; q < 16; q++)
+                        if (tok0 + c * 16 + q < toks) __stcg(mine + (size_t)(c * 16 + q) * np, __uint_as_float(r[q]));
+                }
+                release_accumulator();
+                __threadfence();
+                __syncwarp();
+                unsigned int *count = arrivals + ((t.w_pair * 2 + (int)rank) * 2 + half) * 4 + quad;
+                unsigned int seen = 0;
+                if (lane == 0) seen = atomicAdd(count, 1u);
+                seen = __shfl_sync(0xffffffffu, seen, 0);
+                if (seen == (unsigned)sc.k_splits - 1) {
+                    __threadfence();
+                    if (lane == 0) *count = 0;                      // ready for the next launch that uses this slot
+                    const int tok_end = min(min(tok0 + cols, toks), M);
+                    for (int tok = tok0; tok < tok_end; tok += 8) {
+                        float v[8][kMaxKSplits];                    // all loads of eight tokens in flight at once
+#pragma unroll
+                        for (int u = 0; u < 8; u++)
+#pragma unroll
+                            for (int sp = 0; sp < kMaxKSplits; sp++)
+                                v[u][sp] = (sp < sc.k_splits && tok + u < tok_end)
+                                               ? __ldcg(partials + ((size_t)sp * toks + tok + u) * np + n) : 0.0f;
+#pragma unroll
+                        for (int u = 0; u < 8; u++) {
+                            float sum = 0.0f;
+#pragma unroll
+                            for (int sp = 0; sp < kMaxKSplits; sp++) sum += v[u][sp];      // fixed order: split 0, 1, ...
+                            if (tok + u < tok_end && n < N && !*abort_flag) {
+                                if (out_bf16) ((__nv_bfloat16 *)Y)[(int64_t)(tok + u) * ldy + n] = __float2bfloat16_rn(sum);
+                                else ((float *)Y)[(int64_t)(tok + u) * ldy + n] = sum;
+                            }
+                        }
+                    }
+                }
             } else if (use_tma_store && out_bf16) {
                 if (cols == 128) epilogue_bf16<4>(t_base, stage_ptr, stage_out, &mapY, n0, t0, lane, abort_flag, release_accumulator, staging_free);
                 else epilogue_bf16<2>(t_base, stage_ptr, stage_out, &mapY, n0, t0, lane, abort_flag, release_accumulator, staging_free);
@@ -603,8 +672,16 @@ inline int max_resident_clusters() {
 }
 
 // X as operand bytes + scale atoms (the quantizer's second output form), W as a packed operand.
+// Scratch a short call (M <= 128) can use to split K over more clusters: bytes of fp32 partial sums.
+inline size_t splitk_workspace(int64_t M, int64_t N, int64_t K) {
+    if (M > kSplitMaxTokens) return 0;
+    const int64_t toks = (M + 15) / 16 * 16, np = (N + 255) / 256 * 256;
+    return (size_t)kMaxKSplits * toks * np * sizeof(float);
+}
+
+// `scratch` (optional): splitk_workspace bytes, 256-byte aligned.
 inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, const QView &W, int64_t K, void *Y,
-                          bool out_bf16, int64_t ldy, cudaStream_t st) {
+                          bool out_bf16, int64_t ldy, cudaStream_t st, void *scratch = nullptr, size_t scratch_bytes = 0) {
     CUtensorMap mapX, mapXpart, mapCodes, mapSfW, mapSfX, mapY;
     const int64_t N = W.rows, rtx = row_tiles(M), rtw = row_tiles(N), kg = k_groups(K);
     // items smaller than a whole tile: the whole problem when it has at most 128 tokens, else halves of 128
@@ -640,17 +717,35 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
     sc.split_from = tiles;
     sc.parts = 2;
     sc.part_tokens = part_tokens;
+    sc.k_splits = 1;
+    sc.k_per = sc.k_tiles;
+    unsigned int *arrivals = nullptr;
     if (M <= 128) {
         // one token tile: every item is the whole (short) token range
         sc.split_from = 0;
         sc.parts = 1;
+        // few tiles: cut K so that about all clusters have an item of at least kMinKPerSplit k-steps
+        int want = resident / tiles;
+        if (want > kMaxKSplits) want = kMaxKSplits;
+        if (want > sc.k_tiles / kMinKPerSplit) want = sc.k_tiles / kMinKPerSplit;
+        if (want > 1 && M <= kSplitMaxTokens && scratch && scratch_bytes >= splitk_workspace(M, N, K) &&
+            tiles * 16 <= kArrivalWords) {
+            sc.k_per = (sc.k_tiles + want - 1) / want;
+            sc.k_splits = (sc.k_tiles + sc.k_per - 1) / sc.k_per;      // no empty split
+            static unsigned int turn[kMaxDevices] = {};
+            unsigned int *base_words = nullptr;
+            if (sc.k_splits > 1 && cudaGetSymbolAddress((void **)&base_words, g_splitk_arrivals) == cudaSuccess)
+                arrivals = base_words + (size_t)(turn[dev]++ % kArrivalSlots) * kArrivalWords;
+            else
+                sc.k_splits = 1, sc.k_per = sc.k_tiles;
+        }
     } else {
         // a last round that fills at most half of the clusters is cut into 128-token items (twice as many, half
         // as long), unless the second half of the last token tile would be empty
         const int rest = tiles % resident, m_tail = (int)(M % 256);
         if (rest > 0 && 2 * rest <= resident && (m_tail == 0 || m_tail > 128)) sc.split_from = tiles - rest;
     }
-    const int items = sc.split_from + (tiles - sc.split_from) * sc.parts;
+    const int items = (sc.split_from + (tiles - sc.split_from) * sc.parts) * sc.k_splits;
     sc.clusters = items < resident ? items : resident;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * sc.clusters);
@@ -663,7 +758,7 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, gemm_wtmem_kernel, mapX, mapXpart, mapCodes, mapSfW, mapSfX, (const uint8_t *)W.ids, sc, (int)M,
-                              (int)N, (int)rtx, (int)rtw, Y, ldy, out_bf16 ? 1 : 0, mapY, use_tma_store);
+                              (int)N, (int)rtx, (int)rtw, Y, ldy, out_bf16 ? 1 : 0, mapY, use_tma_store, (float *)scratch, arrivals);
 }
 
 }  // namespace tc
@@ -672,7 +767,8 @@ inline bool tc_supported(int64_t M, int64_t N, int64_t K) {
     return K % kBlock == 0 && M >= 1 && N >= 1 && M < (1ll << 31) && N < (1ll << 31) && K < (1ll << 31);
 }
 inline size_t tc_operand_bytes(int64_t rows, int64_t K) { return ((size_t)rows * (size_t)K + 255) & ~(size_t)255; }
-// workspace of the tensor-core path given A as a packed operand: its operand bytes
-inline size_t tc_gemm_workspace(int64_t M, int64_t, int64_t K) { return tc_operand_bytes(M, K); }
+// workspace of the tensor-core path given A as a packed operand: its operand bytes, then (short calls) the
+// split-K scratch
+inline size_t tc_gemm_workspace(int64_t M, int64_t N, int64_t K) { return tc_operand_bytes(M, K) + tc::splitk_workspace(M, N, K); }
 
 }  // namespace bd

@@ -49,7 +49,9 @@ def test_tiny_case(impl):
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("M,N,K", [(1, 8, 32), (5, 130, 96), (128, 128, 128), (130, 257, 352), (200, 384, 1024),
                                    # token tiles cut into 128-token items, with and without a ragged last tile
-                                   (448, 512, 256), (640, 300, 160), (512, 1024, 128)])
+                                   (448, 512, 256), (640, 300, 160), (512, 1024, 128),
+                                   # decode-sized calls whose K is cut over several clusters (ragged last k-step)
+                                   (5, 300, 2144), (16, 520, 4128), (1, 256, 8192)])
 def test_ragged_shapes(impl, M, N, K):
     rng = np.random.default_rng(M + 31 * N + 977 * K)
     a = rng.standard_t(4, (M, K)).astype(np.float32)
@@ -112,7 +114,7 @@ def test_bf16_output_is_rounded_fp32_result(impl):
     assert torch.equal(y16, y32.to(torch.bfloat16))
 
 
-@pytest.mark.parametrize("M,N,K", [(16, 264, 256), (100, 520, 96), (448, 512, 256), (700, 256, 512)])
+@pytest.mark.parametrize("M,N,K", [(16, 264, 256), (100, 520, 96), (448, 512, 256), (700, 256, 512), (9, 264, 4096)])
 def test_bf16_output_all_item_widths(M, N, K):
     """bf16 results of the tensor-core kernel for every kind of work item (a short token range, 128-token
     halves, whole tiles) equal the rounded fp32 results, through tensor stores and through plain stores."""
