@@ -319,7 +319,8 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     const int cluster = blockIdx.x / 2;
 
     if (threadIdx.x == 0) {
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;                                        // set once the previous kernel has completed
         for (int s = 0; s < kXStages; s++) {
             mbar_init(x_full(s), 1);
             mbar_init(x_empty(s), 1);
@@ -348,13 +349,17 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     cluster_sync_all();                                           // both CTAs: barriers initialised, TMEM allocated
     tcgen05_fence_after();
     const uint32_t tmem = *tmem_slot;
-    // programmatic dependent launch: everything above overlapped the tail of the previous kernel in the
-    // stream; its results (the operand bytes the quantizer wrote) are read only after this point
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ---- TMA producer of the activation tile and the scale atoms (one elected lane issues) ----
+        // Programmatic dependent launch: the previous kernel of the stream is the one that wrote the activation
+        // operand, and only this warp reads it, so only this warp waits for that kernel.  The weights are older
+        // than that kernel (it started its own dependents only after everything before it had completed), so
+        // the code producer and the decode warps fill their rings while it drains.  Every store of this kernel
+        // follows an MMA that consumed a tile loaded here, i.e. follows the wait.
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        if (lane == 0) abort_flag[1] = 1;                         // from here on every bounded wait counts its polls
         int s = 0;
         uint32_t ph = 1;
         Tile t;

@@ -45,13 +45,19 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  `abort_flag` (shared memory) is raised by the first wait that runs out;
 // later waits return at once so that the CTA drains quickly.  After a few failed polls the
 // warp sleeps between polls (`sleep_ns`), so that a long wait does not take issue slots
-// from the warps that are working.
+// from the warps that are working.  abort_flag[1] is the CTA's "earlier kernels of the stream
+// have completed" word: while it is zero the polls are not counted, because the wait then
+// includes the rest of the previous kernel, whose length is not this kernel's to bound (the
+// warp that waits for that kernel does so in hardware, without a limit, and sets the word).
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
                                           uint32_t sleep_ns = 32) {
     for (uint32_t spin = 0; spin < kSpinLimit; spin++) {
         if (mbar_try_wait(bar, parity)) return;
         if (spin >= 8) __nanosleep(sleep_ns);
-        if ((spin & 1023u) == 1023u && *abort_flag) return;
+        if ((spin & 1023u) == 1023u) {
+            if (*abort_flag) return;
+            if (!abort_flag[1]) spin = 0;
+        }
     }
     *abort_flag = 1;
     atomicOr(&g_status_word, kStatusTimeout);

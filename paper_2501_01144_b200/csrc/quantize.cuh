@@ -418,6 +418,9 @@ __global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel
     __shared__ SmemTables tab;
     load_tables(tab);
     asm volatile("griddepcontrol.wait;" ::: "memory");           // the source may be the previous kernel's output
+    // everything earlier in the stream is complete now: the next kernel may take the processors this grid
+    // leaves and set itself up; it waits for this grid's results in the same way
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     quantize_bf16_parts<WRITE_CODES, WRITE_E4M3, REGULAR>(X, ld, out, e4m3, tab, 8u * blockIdx.x + threadIdx.x / 32u,
                                                           8u * gridDim.x, 8u * chunks, nb, kgroups, div_kgroups);
 }
