@@ -362,6 +362,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         if (lane == 0) abort_flag[1] = 1;                         // from here on every bounded wait counts its polls
         int s = 0;
         uint32_t ph = 1;
+        const uint32_t x_full_leader = map_to_cta(x_full(0), 0);
         Tile t;
         for (int i = 0; next_tile(sc, cluster, i, t); i++) {
             // each CTA holds half of the item's tokens; smaller items load their rows through a tensor map of their own
@@ -369,9 +370,8 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             const CUtensorMap *map = t.tokens == 256 ? &mapX : &mapXpart;
             const uint32_t tx_pair = 2u * ((uint32_t)per_cta * BK + 3u * kScaleAtomBytes);
             for (int kt = t.k_begin; kt < t.k_end; kt++) {
-                mbar_wait(x_empty(s), ph, abort_flag);
-                if (*abort_flag) break;
-                const uint32_t fb = map_to_cta(x_full(s), 0);
+                if (!mbar_wait(x_empty(s), ph, abort_flag)) break;
+                const uint32_t fb = x_full_leader + 8u * (uint32_t)s;
                 if (elect_one()) {
                     if (rank == 0) mbar_expect_tx(x_full(s), tx_pair);
                     tma_load_2d_pair(x_tile(s), map, kt * BK, t0, fb);
@@ -394,8 +394,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             const int my_row_tile = t.w_pair * 2 + (int)rank;
             const bool have_ids = my_row_tile < row_tiles_w;
             for (int kt = t.k_begin; kt < t.k_end; kt++) {
-                mbar_wait(c_empty(s), ph, abort_flag);
-                if (*abort_flag) break;
+                if (!mbar_wait(c_empty(s), ph, abort_flag)) break;
                 if (elect_one()) {
                     mbar_expect_tx(c_full(s), kCodeTile + (have_ids ? kIdAtomBytes : 0));
                     tma_load_2d(code_tile(s), &mapCodes, kt * (BK / 2), w0, c_full(s));
@@ -429,9 +428,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 for (int kt = t.k_begin; kt < t.k_end; kt++) {
                     if (!ready) {
                         // slow path: the probe at the end of the previous k-step found a barrier open
-                        mbar_wait(x_full(s), ph_s, abort_flag);
-                        mbar_wait(a_full(b), ph_b, abort_flag);
-                        if (*abort_flag) break;
+                        if (!mbar_wait(x_full(s), ph_s, abort_flag) || !mbar_wait(a_full(b), ph_b, abort_flag)) break;
                     }
                     tcgen05_fence_after();
                     const uint32_t lo_sfw = lo_sfw0 + (uint32_t)s * (kScaleAtomBytes >> 4);
@@ -479,10 +476,13 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             Tile t;
             for (int i = 0; next_tile(sc, cluster, i, t); i++) total_k += t.k_end - t.k_begin;
         }
+        // ring positions of this group's k-step, kept by increments (the step, the number of groups, is smaller
+        // than either ring): code stage s with the parity to wait for, operand buffer b likewise
+        int s = group % kCodeStages, b = group % kABufs;
+        uint32_t s_par = 0, b_par = 1;
+        static_assert(kDecodeGroups <= kCodeStages && kDecodeGroups <= kABufs, "one wrap per step at most");
         for (int g = group; g < total_k; g += kDecodeGroups) {
-            const int s = g % kCodeStages, b = g % kABufs;
-            mbar_wait(c_full(s), (uint32_t)(g / kCodeStages) & 1u, abort_flag);
-            if (*abort_flag) break;
+            if (!mbar_wait(c_full(s), s_par, abort_flag)) break;
             const uint8_t *codes = base_ptr + Smem::codes + s * kCodeTile + j * 64;
             const uint32_t ids16 = *(const uint16_t *)(base_ptr + Smem::ids + s * kIdAtomBytes + (j % 32) * 8 + (j / 32) * 2);
             uint4 w[4];
@@ -491,8 +491,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             // the codes are in registers: hand the stage back to its producer
             __syncwarp();
             if (lane == 0) mbar_arrive_local(c_empty(s));
-            mbar_wait(a_empty(b), ((uint32_t)(g / kABufs) & 1u) ^ 1u, abort_flag);
-            if (*abort_flag) break;
+            if (!mbar_wait(a_empty(b), b_par, abort_flag)) break;
             tcgen05_fence_after();                                // the MMAs that read this buffer have completed
 #pragma unroll
             for (int c = 0; c < 4; c++) {
@@ -509,6 +508,10 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             tcgen05_fence_before();
             asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");   // the four warps of this group are done
             if (group_leader) mbar_arrive_cluster(a_full_leader + 8u * b);
+            s += kDecodeGroups;
+            if (s >= kCodeStages) { s -= kCodeStages; s_par ^= 1u; }
+            b += kDecodeGroups;
+            if (b >= kABufs) { b -= kABufs; b_par ^= 1u; }
         }
     } else {
         // ---- epilogue: warp w reads the TMEM lanes 32 * (w % 4) .. + 31 (weight rows) of this CTA's

@@ -49,18 +49,21 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // have completed" word: while it is zero the polls are not counted, because the wait then
 // includes the rest of the previous kernel, whose length is not this kernel's to bound (the
 // warp that waits for that kernel does so in hardware, without a limit, and sets the word).
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
+// Returns false when the CTA is aborting (this wait or an earlier one ran out), so that a caller
+// in a hot loop need not read the flag again after every wait.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
                                           uint32_t sleep_ns = 32) {
     for (uint32_t spin = 0; spin < kSpinLimit; spin++) {
-        if (mbar_try_wait(bar, parity)) return;
+        if (mbar_try_wait(bar, parity)) return true;
         if (spin >= 8) __nanosleep(sleep_ns);
         if ((spin & 1023u) == 1023u) {
-            if (*abort_flag) return;
+            if (*abort_flag) return false;
             if (!abort_flag[1]) spin = 0;
         }
     }
     *abort_flag = 1;
     atomicOr(&g_status_word, kStatusTimeout);
+    return false;
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
     asm volatile(
