@@ -638,7 +638,8 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 release_accumulator();
             }
         }
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");    // staging buffers must outlive the stores
+        // the staging buffers must outlive the stores' reads of them; the writes themselves complete with the grid
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
         __syncwarp();
     }
 
