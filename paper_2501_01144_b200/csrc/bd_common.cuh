@@ -78,6 +78,15 @@ constexpr uint64_t e4m3_lut(const Formatbook &b, int d) {
     for (int i = 0; i < 8; i++) t |= (uint64_t)e4m3_of_half_units(b.v[d][i]) << (8 * i);
     return t;
 }
+// The one-pass quantizer knows an element by u = the number of merged thresholds of its dialect pair at or
+// below its 5-bit code (0..10, see merged_mask).  Its index in the chosen dialect: the pair's members skip
+// different thresholds of the merged list.
+constexpr int index_of_count(int u, bool odd) { return u - (u >= (odd ? 7 : 6)) - (u >= 8) - (u >= (odd ? 10 : 9)); }
+// Operand bytes of a dialect by v = 10 - u (what the quantizer accumulates): bytes 0..7 are v = 0..7, bytes
+// 8..10 are v = 8..10 (the three smallest magnitudes); all have a clear top bit.
+constexpr uint8_t direct_byte(const Formatbook &b, int d, int v) {
+    return e4m3_of_half_units(b.v[d][index_of_count(10 - v, (d & 1) != 0)]);
+}
 constexpr uint64_t int_lut(const Formatbook &b, int d) {
     uint64_t t = 0;
     for (int i = 0; i < 8; i++) t |= (uint64_t)b.v[d][i] << (8 * i);
@@ -232,6 +241,7 @@ struct DeviceTables {
     uint32_t e4m3_lo[16], e4m3_hi[16];
     uint32_t int_lo[16], int_hi[16];
     uint32_t merged_above[8];     // merged_mask(p) >> 1: popcount(x >> q5) = thresholds above q5
+    uint32_t direct_lo[16], direct_hi[16], direct_top[16];   // direct_byte for v = 0..3, 4..7, 8..10
 };
 constexpr DeviceTables make_tables(const Formatbook &b) {
     DeviceTables t{};
@@ -241,6 +251,11 @@ constexpr DeviceTables make_tables(const Formatbook &b) {
         t.e4m3_hi[d] = (uint32_t)(e4m3_lut(b, d) >> 32);
         t.int_lo[d] = (uint32_t)int_lut(b, d);
         t.int_hi[d] = (uint32_t)(int_lut(b, d) >> 32);
+        for (int v = 0; v < 4; v++) {
+            t.direct_lo[d] |= (uint32_t)direct_byte(b, d, v) << (8 * v);
+            t.direct_hi[d] |= (uint32_t)direct_byte(b, d, 4 + v) << (8 * v);
+            if (v < 3) t.direct_top[d] |= (uint32_t)direct_byte(b, d, 8 + v) << (8 * v);
+        }
     }
     for (int p = 0; p < 8; p++) {
         t.even_mask[p] = even_range_mask(b, p);

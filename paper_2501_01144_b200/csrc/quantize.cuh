@@ -31,12 +31,16 @@ struct SmemTables {
     uint32_t odd_mask[8];
     uint32_t e4m3_lo[16], e4m3_hi[16];
     uint32_t merged_above[8];
+    uint32_t direct_lo[16], direct_hi[16], direct_top[16];
 };
 __device__ __forceinline__ void load_tables(SmemTables &s) {
     for (int i = threadIdx.x; i < 16; i += blockDim.x) {
         s.round_mask[i] = c_tables.round_mask[i];
         s.e4m3_lo[i] = c_tables.e4m3_lo[i];
         s.e4m3_hi[i] = c_tables.e4m3_hi[i];
+        s.direct_lo[i] = c_tables.direct_lo[i];
+        s.direct_hi[i] = c_tables.direct_hi[i];
+        s.direct_top[i] = c_tables.direct_top[i];
         if (i < 8) {
             s.even_mask[i] = c_tables.even_mask[i];
             s.odd_mask[i] = c_tables.odd_mask[i];
@@ -183,6 +187,28 @@ __device__ __forceinline__ void finish_two_stage(const uint32_t (&v)[4], const u
     }
 }
 
+// The same selection, emitting operand bytes (E4M3) instead of indices: with the dialect known, the byte of an
+// element is a function of its v alone, an eleven-entry table.  Two byte permutes read it: entries 0..7 with v
+// as the selector (v >= 8 selects "replicate the top bit" of a byte whose top bit is clear: zero), entries 8..10
+// with v ^ 8 (now v < 8 gives zero).  s03 / s47 hold the high bytes of elements 0..3 / 4..7 of each group.
+__device__ __forceinline__ void finish_two_stage_e4m3(const uint32_t (&v)[4], const uint32_t (&s03)[4],
+                                                      const uint32_t (&s47)[4], uint32_t pair, const SmemTables &tab,
+                                                      uint32_t &id, uint32_t (&out)[8]) {
+    uint32_t acc = 0;
+#pragma unroll
+    for (int w = 0; w < 4; w++)
+        acc += prmt_b32(0x10010100u, 0x00000010u, v[w]) + prmt_b32(0x10010100u, 0x00000010u, v[w] >> 16);
+    const uint32_t cnt_even = byte_sum(acc & 0x0f0f0f0fu), cnt_odd = byte_sum((acc >> 4) & 0x0f0f0f0fu);
+    id = 2u * pair + (cnt_odd > cnt_even ? 1u : 0u);              // equal counts: the even member
+    const uint32_t lo = tab.direct_lo[id], hi = tab.direct_hi[id], top = tab.direct_top[id];
+#pragma unroll
+    for (int w = 0; w < 4; w++) {
+        const uint32_t x = v[w] ^ 0x88888888u;
+        out[2 * w] = (prmt_b32(lo, hi, v[w]) | prmt_b32(top, 0u, x)) | (s03[w] & 0x80808080u);
+        out[2 * w + 1] = (prmt_b32(lo, hi, v[w] >> 16) | prmt_b32(top, 0u, x >> 16)) | (s47[w] & 0x80808080u);
+    }
+}
+
 // Two-stage rule (Sec. 3.2) for a block given as fp32 bit patterns.
 __device__ __forceinline__ BlockResult quantize_two_stage(const uint32_t (&bits)[32], const SmemTables &tab,
                                                           bool &nonfinite) {
@@ -273,15 +299,17 @@ __device__ __noinline__ void quantize_bf16_clamped_block(const uint32_t (&R)[16]
     res = quantize_two_stage(bits, tab, nonfinite);
 }
 
-// Two-stage rule on one block held as sixteen packed bf16 pairs.
-__device__ __forceinline__ void quantize_bf16_block(const uint32_t (&R)[16], const SmemTables &tab, BlockResult &res) {
-    uint32_t a[16], signs[4];
+// Two-stage rule on one block held as sixteen packed bf16 pairs.  BYTES: emit the operand bytes (e4m3[0..7],
+// eight elements per pair of words) instead of the packed indices (res.words).
+template <bool BYTES>
+__device__ __forceinline__ void quantize_bf16_block(const uint32_t (&R)[16], const SmemTables &tab, BlockResult &res,
+                                                    uint32_t (&e4m3)[8]) {
+    uint32_t a[16], s03[4], s47[4];
 #pragma unroll
     for (int w = 0; w < 4; w++) {
-        // the high byte of each bf16 carries its sign in bit 7: elements 0..3 of the group keep it there,
-        // elements 4..7 move it to bit 3 of the same bytes
-        const uint32_t s03 = prmt_b32(R[4 * w], R[4 * w + 1], 0x7531u), s47 = prmt_b32(R[4 * w + 2], R[4 * w + 3], 0x7531u);
-        signs[w] = (s03 & 0x80808080u) | ((s47 >> 4) & 0x08080808u);
+        // the high byte of each bf16 carries its sign in bit 7
+        s03[w] = prmt_b32(R[4 * w], R[4 * w + 1], 0x7531u);
+        s47[w] = prmt_b32(R[4 * w + 2], R[4 * w + 3], 0x7531u);
     }
 #pragma unroll
     for (int i = 0; i < 16; i++) {
@@ -311,12 +339,25 @@ __device__ __forceinline__ void quantize_bf16_block(const uint32_t (&R)[16], con
             v[i / 4] = v_hi * (1u << (4 * slot_of(2 * (i % 4) + 1))) + v[i / 4];
         }
         res.scale = eadj - 2u;
-        finish_two_stage(v, signs, pair, res.id, res.words);
+        if (BYTES) {
+            finish_two_stage_e4m3(v, s03, s47, pair, tab, res.id, e4m3);
+        } else {
+            uint32_t signs[4];
+#pragma unroll
+            for (int w = 0; w < 4; w++)                           // elements 4..7 carry their sign in bit 3 of the same bytes
+                signs[w] = (s03[w] & 0x80808080u) | ((s47[w] >> 4) & 0x08080808u);
+            finish_two_stage(v, signs, pair, res.id, res.words);
+        }
     } else {
         uint32_t copy[16];                                       // only this branch spills the block to local memory
 #pragma unroll
         for (int i = 0; i < 16; i++) copy[i] = R[i];
         quantize_bf16_clamped_block(copy, tab, res);
+        if (BYTES) {
+            const uint32_t lo = tab.e4m3_lo[res.id], hi = tab.e4m3_hi[res.id];
+#pragma unroll
+            for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, e4m3[2 * w], e4m3[2 * w + 1]);
+        }
     }
 }
 
@@ -366,15 +407,17 @@ __device__ __forceinline__ void quantize_bf16_parts(const uint16_t *__restrict__
         if (k.valid) {
             const uint32_t R[16] = {k.l0.x, k.l0.y, k.l0.z, k.l0.w, k.l1.x, k.l1.y, k.l1.z, k.l1.w,
                                     k.l2.x, k.l2.y, k.l2.z, k.l2.w, k.l3.x, k.l3.y, k.l3.z, k.l3.w};
-            quantize_bf16_block(R, tab, res);
+            uint32_t o[8];
+            quantize_bf16_block<WRITE_E4M3 && !WRITE_CODES>(R, tab, res, o);
             if (WRITE_CODES)
                 *(uint4 *)(out.codes + (uint64_t)k.r * half_k + k.b * 16u) =
                     make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
             if (WRITE_E4M3) {
-                uint32_t lo = tab.e4m3_lo[res.id], hi = tab.e4m3_hi[res.id];
-                uint32_t o[8];
+                if (WRITE_CODES) {                                // both forms: the bytes from the indices
+                    uint32_t lo = tab.e4m3_lo[res.id], hi = tab.e4m3_hi[res.id];
 #pragma unroll
-                for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, o[2 * w], o[2 * w + 1]);
+                    for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, o[2 * w], o[2 * w + 1]);
+                }
                 uint4 *dst = (uint4 *)(e4m3 + (uint64_t)k.r * (2u * half_k) + k.b * 32u);
                 dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
