@@ -304,16 +304,12 @@ __device__ __noinline__ void quantize_bf16_clamped_block(const uint32_t (&R)[16]
 template <bool BYTES>
 __device__ __forceinline__ void quantize_bf16_block(const uint32_t (&R)[16], const SmemTables &tab, BlockResult &res,
                                                     uint32_t (&e4m3)[8]) {
-    uint32_t a[16], s03[4], s47[4];
+    uint32_t s03[4], s47[4];
 #pragma unroll
     for (int w = 0; w < 4; w++) {
         // the high byte of each bf16 carries its sign in bit 7
         s03[w] = prmt_b32(R[4 * w], R[4 * w + 1], 0x7531u);
         s47[w] = prmt_b32(R[4 * w + 2], R[4 * w + 3], 0x7531u);
-    }
-#pragma unroll
-    for (int i = 0; i < 16; i++) {
-        a[i] = R[i] & 0x7fff7fffu;
     }
     uint32_t m = R[0];
 #pragma unroll
@@ -330,8 +326,10 @@ __device__ __forceinline__ void quantize_bf16_block(const uint32_t (&R)[16], con
         uint32_t v[4] = {0, 0, 0, 0};
 #pragma unroll
         for (int i = 0; i < 16; i++) {
-            const uint32_t t_lo = __float_as_uint(__fmaf_rz(__uint_as_float(a[i] << 16), scale, 8388608.0f));
-            const uint32_t t_hi = __float_as_uint(__fmaf_rz(__uint_as_float(a[i]), scale, 8388608.0f));
+            // magnitudes through the multiplier's |.| operand modifier; the upper element keeps the lower one's
+            // bits below its own last place (less than one bf16 ulp, sign bit of the lower element included)
+            const uint32_t t_lo = __float_as_uint(__fmaf_rz(fabsf(__uint_as_float(R[i] << 16)), scale, 8388608.0f));
+            const uint32_t t_hi = __float_as_uint(__fmaf_rz(fabsf(__uint_as_float(R[i])), scale, 8388608.0f));
             // funnel shift in wrap mode uses only the low five bits of the count, i.e. q5
             const uint32_t v_lo = __popc(__funnelshift_r(above, 0u, t_lo));
             const uint32_t v_hi = __popc(__funnelshift_r(above, 0u, t_hi));
