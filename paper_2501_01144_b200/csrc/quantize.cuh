@@ -285,32 +285,18 @@ __device__ __forceinline__ BlockResult quantize_mse(const uint32_t (&bits)[32], 
 //               nibbles, then finish_two_stage;
 //   signs       two byte permutes gather the high bytes of a group's eight elements; one shift by 4
 //               puts elements 4..7 on their sign bits.
-// Blocks whose exponent is clamped (maximum below 2^-123) take the generic routine.
 // ---------------------------------------------------------------------------
-__device__ __noinline__ void quantize_bf16_clamped_block(const uint32_t (&R)[16], const SmemTables &tab,
-                                                         BlockResult &res) {
-    uint32_t bits[32];
-#pragma unroll
-    for (int i = 0; i < 16; i++) {
-        bits[2 * i] = R[i] << 16;
-        bits[2 * i + 1] = R[i] & 0xffff0000u;
-    }
-    bool nonfinite;
-    res = quantize_two_stage(bits, tab, nonfinite);
-}
-
 // Two-stage rule on one block held as sixteen packed bf16 pairs.  BYTES: emit the operand bytes (e4m3[0..7],
 // eight elements per pair of words) instead of the packed indices (res.words).
+// A block whose exponent is clamped (maximum below 2^-123, eadj < 4) would need a scale of 2^128 or more: its
+// elements are first multiplied by 2^64 (exact for a power of two, subnormal inputs included) and the scale
+// shrinks by the same factor, so the common arithmetic serves it too, with no call and no local memory.
 template <bool BYTES>
-__device__ __forceinline__ void quantize_bf16_block(const uint32_t (&R)[16], const SmemTables &tab, BlockResult &res,
+__device__ __forceinline__ void quantize_bf16_block(const uint32_t (&Rin)[16], const SmemTables &tab, BlockResult &res,
                                                     uint32_t (&e4m3)[8]) {
-    uint32_t s03[4], s47[4];
+    uint32_t R[16], s03[4], s47[4];
 #pragma unroll
-    for (int w = 0; w < 4; w++) {
-        // the high byte of each bf16 carries its sign in bit 7
-        s03[w] = prmt_b32(R[4 * w], R[4 * w + 1], 0x7531u);
-        s47[w] = prmt_b32(R[4 * w + 2], R[4 * w + 3], 0x7531u);
-    }
+    for (int i = 0; i < 16; i++) R[i] = Rin[i];
     // |.| maximum per half as a tree (four levels instead of a chain of fifteen); NaN wins; the sign bits are noise
     uint32_t t8[8], m;
 #pragma unroll
@@ -322,44 +308,47 @@ __device__ __forceinline__ void quantize_bf16_block(const uint32_t (&R)[16], con
     const uint32_t amax = max(m & 0xffffu, m >> 16);              // bf16 magnitude bits of the block maximum
     if (amax >= 0x7f80u) atomicOr(&g_status_word, kStatusNonfinite);
     const uint32_t eadj = max(amax >> 7, 2u);
-    if (eadj >= 4u) {
-        const float scale = __uint_as_float((258u - eadj) << 23);         // 2^(2 - e), e = eadj - 129
-        const uint32_t m5 = __float_as_uint(__fmaf_rz(__uint_as_float(amax << 16), scale, 8388608.0f)) & 63u;
-        const uint32_t pair = min(7u, 15u - min(15u, (m5 + 1u) >> 1));
-        const uint32_t above = tab.merged_above[pair];
-        uint32_t v[4] = {0, 0, 0, 0};
+    float amax_f = __uint_as_float(amax << 16);
+    uint32_t eadj_eff = eadj;
+    if (eadj < 4u) {
+        const uint32_t two64 = 0x5f805f80u;                      // 2^64 in both halves
 #pragma unroll
-        for (int i = 0; i < 16; i++) {
-            // magnitudes through the multiplier's |.| operand modifier; the upper element keeps the lower one's
-            // bits below its own last place (less than one bf16 ulp, sign bit of the lower element included)
-            const uint32_t t_lo = __float_as_uint(__fmaf_rz(fabsf(__uint_as_float(R[i] << 16)), scale, 8388608.0f));
-            const uint32_t t_hi = __float_as_uint(__fmaf_rz(fabsf(__uint_as_float(R[i])), scale, 8388608.0f));
-            // funnel shift in wrap mode uses only the low five bits of the count, i.e. q5
-            const uint32_t v_lo = __popc(__funnelshift_r(above, 0u, t_lo));
-            const uint32_t v_hi = __popc(__funnelshift_r(above, 0u, t_hi));
-            v[i / 4] = v_lo * (1u << (4 * slot_of(2 * (i % 4)))) + v[i / 4];
-            v[i / 4] = v_hi * (1u << (4 * slot_of(2 * (i % 4) + 1))) + v[i / 4];
-        }
-        res.scale = eadj - 2u;
-        if (BYTES) {
-            finish_two_stage_e4m3(v, s03, s47, pair, tab, res.id, e4m3);
-        } else {
-            uint32_t signs[4];
+        for (int i = 0; i < 16; i++) asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(R[i]) : "r"(R[i]), "r"(two64));
+        amax_f *= 18446744073709551616.0f;
+        eadj_eff = eadj + 64u;
+    }
 #pragma unroll
-            for (int w = 0; w < 4; w++)                           // elements 4..7 carry their sign in bit 3 of the same bytes
-                signs[w] = (s03[w] & 0x80808080u) | ((s47[w] >> 4) & 0x08080808u);
-            finish_two_stage(v, signs, pair, res.id, res.words);
-        }
+    for (int w = 0; w < 4; w++) {
+        // the high byte of each bf16 carries its sign in bit 7
+        s03[w] = prmt_b32(R[4 * w], R[4 * w + 1], 0x7531u);
+        s47[w] = prmt_b32(R[4 * w + 2], R[4 * w + 3], 0x7531u);
+    }
+    const float scale = __uint_as_float((258u - eadj_eff) << 23);        // 2^(2 - e) (over 2^64 for a clamped block), e = eadj - 129
+    const uint32_t m5 = __float_as_uint(__fmaf_rz(amax_f, scale, 8388608.0f)) & 63u;
+    const uint32_t pair = min(7u, 15u - min(15u, (m5 + 1u) >> 1));
+    const uint32_t above = tab.merged_above[pair];
+    uint32_t v[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int i = 0; i < 16; i++) {
+        // magnitudes through the multiplier's |.| operand modifier; the upper element keeps the lower one's
+        // bits below its own last place (less than one bf16 ulp, sign bit of the lower element included)
+        const uint32_t t_lo = __float_as_uint(__fmaf_rz(fabsf(__uint_as_float(R[i] << 16)), scale, 8388608.0f));
+        const uint32_t t_hi = __float_as_uint(__fmaf_rz(fabsf(__uint_as_float(R[i])), scale, 8388608.0f));
+        // funnel shift in wrap mode uses only the low five bits of the count, i.e. q5
+        const uint32_t v_lo = __popc(__funnelshift_r(above, 0u, t_lo));
+        const uint32_t v_hi = __popc(__funnelshift_r(above, 0u, t_hi));
+        v[i / 4] = v_lo * (1u << (4 * slot_of(2 * (i % 4)))) + v[i / 4];
+        v[i / 4] = v_hi * (1u << (4 * slot_of(2 * (i % 4) + 1))) + v[i / 4];
+    }
+    res.scale = eadj - 2u;
+    if (BYTES) {
+        finish_two_stage_e4m3(v, s03, s47, pair, tab, res.id, e4m3);
     } else {
-        uint32_t copy[16];                                       // only this branch spills the block to local memory
+        uint32_t signs[4];
 #pragma unroll
-        for (int i = 0; i < 16; i++) copy[i] = R[i];
-        quantize_bf16_clamped_block(copy, tab, res);
-        if (BYTES) {
-            const uint32_t lo = tab.e4m3_lo[res.id], hi = tab.e4m3_hi[res.id];
-#pragma unroll
-            for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, e4m3[2 * w], e4m3[2 * w + 1]);
-        }
+        for (int w = 0; w < 4; w++)                               // elements 4..7 carry their sign in bit 3 of the same bytes
+            signs[w] = (s03[w] & 0x80808080u) | ((s47[w] >> 4) & 0x08080808u);
+        finish_two_stage(v, signs, pair, res.id, res.words);
     }
 }
 

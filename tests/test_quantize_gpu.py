@@ -71,6 +71,43 @@ def test_degenerate_blocks():
     assert_bit_exact(q, oracle_quantize(hb, torch.float16), "fp16 subnormal")
 
 
+def _bf16_clamped_rows():
+    """bf16 bit patterns whose blocks sit at and below the exponent clamp (block maximum under 2^-123)."""
+    rng = np.random.default_rng(17)
+    b = np.zeros((8, 128), np.uint16)
+    b[0, 3] = 0x8000                                              # all-zero block with a negative zero
+    b[1, :32] = np.arange(32)                                     # the smallest subnormals
+    b[1, 32:64] = rng.integers(1, 0x80, 32)                       # any subnormal
+    b[1, 64:96] = rng.integers(1, 0x80, 32) | 0x8000              # negative subnormals
+    b[2, :32] = 0x0100; b[2, 5] = 0x0033                          # maximum 2^-125 (exponent field 2)
+    b[2, 32:64] = rng.integers(0, 0x0180, 32)                     # fields 0..2
+    b[3, :64] = rng.integers(0, 0x0200, 64)                       # fields 0..3: the last clamped exponent
+    b[3, 64:] = rng.integers(0, 0x0280, 64)                       # field 4: the first regular one
+    b[4] = rng.integers(0, 0x0300, 128) | (rng.integers(0, 2, 128) << 15)
+    b[5, :32] = 0x01ff; b[5, 32:64] = 0x017f; b[5, 64:96] = 0x00ff; b[5, 96:] = 0x007f   # all-ones mantissas
+    b[6, ::2] = 0x0150; b[6, 1::2] = 0x8140; b[6, 0] = 0x0168    # equal beneficial-range counts at the clamp
+    b[7] = rng.integers(0, 0x0400, 128) | (rng.integers(0, 2, 128) << 15)
+    return b
+
+
+def test_bf16_blocks_at_the_exponent_clamp():
+    b = _bf16_clamped_rows()
+    q = bd.quantize_act(to_device(b, torch.bfloat16))
+    ref = oracle_quantize(b, torch.bfloat16)
+    assert_bit_exact(q, ref, "bf16 clamp")
+    # the form bd_linear quantises to (operand bytes) through a product with large weights: 2^-125 x 2^100
+    # lands in the normal fp32 range, so the 1e-6 bound is not hidden by the underflow floor
+    rng = np.random.default_rng(18)
+    W = (rng.standard_normal((96, 128)) * 2.0 ** 100).astype(np.float32)
+    Wq = bd.quantize_weights(to_device(W, torch.float32), bd.SELECT_TWO_STAGE)
+    Y = bd.linear(to_device(b, torch.bfloat16), Wq, dtype=torch.float32).cpu().numpy()
+    Yref, T = oracle.gemm(oracle.dequantize(*ref), oracle.dequantize(*oracle.quantize(W)))
+    err = np.abs(Y.astype(np.float64) - Yref)
+    assert (err <= 1e-6 * T).all(), float((err / np.maximum(1e-6 * T, 1e-300)).max())
+    assert np.abs(Yref).max() > 2.0 ** -40                        # the check above is not vacuous
+    bd.poll_status()
+
+
 def test_leading_dimension_and_output_guard_bands():
     rng = np.random.default_rng(5)
     big = rng.standard_normal((40, 512)).astype(np.float32)
