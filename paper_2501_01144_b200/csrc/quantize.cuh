@@ -668,6 +668,9 @@ __global__ void dequantize_kernel(QView q, float *__restrict__ out, int64_t ld, 
 
 // Decode a packed operand into the plain [rows][K] operand-byte matrix (E4M3).
 __global__ void decode_e4m3_kernel(QView q, uint8_t *__restrict__ out, int nb) {
+    // launched in plain stream order, so everything earlier has completed: the GEMM that follows may set itself
+    // up and fetch its weights while this grid runs (it waits for this grid before it reads `out`)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= q.rows * nb) return;
     int64_t r = t / nb;
@@ -693,6 +696,7 @@ struct StackedViews {
 };
 __global__ void decode_e4m3_stacked_kernel(StackedViews v, int count, int64_t rows, int64_t K, uint8_t *__restrict__ out,
                                            uint8_t *__restrict__ out_scales, int nb) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see decode_e4m3_kernel
     const int h = blockIdx.y;
     const int64_t tiles = rows / kRowTile, kgs = (nb + kBlocksPerAtom - 1) / kBlocksPerAtom;
     QView q{(uint8_t *)v.codes[h], (uint8_t *)v.ids[h], (uint8_t *)v.scales[h], rows, K};
