@@ -58,42 +58,68 @@ unsigned quant_bf16_grid_limit() {
     return limit[dev];
 }
 
+// Launch with programmatic stream serialisation: the blocks may be scheduled while the previous kernel of the
+// stream drains; such a kernel waits for that kernel's results before it touches global memory.
+template <typename... Params, typename... Args>
+void launch_serialized(void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
+}
+
 template <int SELECT, bool WC, bool WE>
 bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out, uint8_t *e4m3, cudaStream_t st) {
     const int nb = (int)(out.K / kBlock), nb_pad = (int)k_groups(out.K) * kBlocksPerAtom;
     const int64_t rows_pad = row_tiles(out.rows) * kRowTile;
     const unsigned chunks = (unsigned)(rows_pad / 64) * (unsigned)(nb_pad / kBlocksPerAtom);     // 64 rows x one k-group
-    const unsigned gen_grid = chunks;                                                            // generic kernel: one CTA each
+    // generic kernel: its CTAs loop over the chunks; three per SM fit with the fp32 staging buffers, and the
+    // other source types are served well enough by the same number
+    const unsigned gen_grid = std::min(chunks, quant_bf16_grid_limit());
+    const int kgs = nb_pad / kBlocksPerAtom;
+    const FastDiv div_kgs = make_fast_div((uint32_t)kgs);
+    const bool regular = out.rows % 64 == 0 && nb % kBlocksPerAtom == 0;
     switch (dt) {
-        case BD_F32: quantize_contig_kernel<BD_F32, SELECT, WC, WE><<<gen_grid, 256, 0, st>>>(X, ld, out, e4m3, nb, nb_pad / kBlocksPerAtom); break;
+        case BD_F32: {
+            static bool configured[64] = {};                      // per instantiation and device
+            int dev = 0;
+            cudaGetDevice(&dev);
+            if (dev >= 0 && dev < 64 && !configured[dev]) {
+                if (cudaFuncSetAttribute(quantize_contig_kernel<BD_F32, SELECT, WC, WE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kContigStageBytes) != cudaSuccess ||
+                    cudaFuncSetAttribute(quantize_contig_kernel<BD_F32, SELECT, WC, WE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kContigStageBytes) != cudaSuccess)
+                    return launch_result();
+                configured[dev] = true;
+            }
+            if (regular)
+                launch_serialized(quantize_contig_kernel<BD_F32, SELECT, WC, WE, true>, gen_grid, 256, kContigStageBytes, st, X, ld, out, e4m3, nb, kgs, chunks, div_kgs);
+            else
+                launch_serialized(quantize_contig_kernel<BD_F32, SELECT, WC, WE, false>, gen_grid, 256, kContigStageBytes, st, X, ld, out, e4m3, nb, kgs, chunks, div_kgs);
+            break;
+        }
         case BD_BF16:
             if (SELECT == BD_SELECT_TWO_STAGE && rows_pad * nb_pad < (1ll << 31))
             {
-                // programmatic dependent launch: the blocks may be scheduled while the previous kernel of the
-                // stream drains; the kernel waits for that kernel's results before it touches global memory
-                cudaLaunchConfig_t cfg = {};
-                cfg.gridDim = dim3(std::min(chunks, quant_bf16_grid_limit()));
-                cfg.blockDim = dim3(256);
-                cfg.stream = st;
-                cudaLaunchAttribute attr[1];
-                attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-                attr[0].val.programmaticStreamSerializationAllowed = 1;
-                cfg.attrs = attr;
-                cfg.numAttrs = 1;
-                const bool regular = out.rows % 64 == 0 && nb % kBlocksPerAtom == 0;
+                const unsigned grid = std::min(chunks, quant_bf16_grid_limit());
                 if (regular)
-                    cudaLaunchKernelEx(&cfg, quantize_bf16_kernel<WC, WE, true>, (const uint16_t *)X, ld, out, e4m3, chunks,
-                                       (uint32_t)nb, (uint32_t)(nb_pad / kBlocksPerAtom),
-                                       make_fast_div((uint32_t)(nb_pad / kBlocksPerAtom)));
+                    launch_serialized(quantize_bf16_kernel<WC, WE, true>, grid, 256, 0, st, (const uint16_t *)X, ld, out, e4m3, chunks,
+                                      (uint32_t)nb, (uint32_t)kgs, div_kgs);
                 else
-                    cudaLaunchKernelEx(&cfg, quantize_bf16_kernel<WC, WE, false>, (const uint16_t *)X, ld, out, e4m3, chunks,
-                                       (uint32_t)nb, (uint32_t)(nb_pad / kBlocksPerAtom),
-                                       make_fast_div((uint32_t)(nb_pad / kBlocksPerAtom)));
+                    launch_serialized(quantize_bf16_kernel<WC, WE, false>, grid, 256, 0, st, (const uint16_t *)X, ld, out, e4m3, chunks,
+                                      (uint32_t)nb, (uint32_t)kgs, div_kgs);
             }
             else
-                quantize_contig_kernel<BD_BF16, SELECT, WC, WE><<<gen_grid, 256, 0, st>>>(X, ld, out, e4m3, nb, nb_pad / kBlocksPerAtom);
+                launch_serialized(quantize_contig_kernel<BD_BF16, SELECT, WC, WE, false>, gen_grid, 256, 0, st, X, ld, out, e4m3, nb, kgs, chunks, div_kgs);
             break;
-        case BD_F16: quantize_contig_kernel<BD_F16, SELECT, WC, WE><<<gen_grid, 256, 0, st>>>(X, ld, out, e4m3, nb, nb_pad / kBlocksPerAtom); break;
+        case BD_F16: launch_serialized(quantize_contig_kernel<BD_F16, SELECT, WC, WE, false>, gen_grid, 256, 0, st, X, ld, out, e4m3, nb, kgs, chunks, div_kgs); break;
         default: return BD_ERR_INVALID_ARG;
     }
     return launch_result();

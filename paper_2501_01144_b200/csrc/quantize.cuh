@@ -274,6 +274,66 @@ __device__ __forceinline__ BlockResult quantize_mse(const uint32_t (&bits)[32], 
     return r;
 }
 
+// max(|a|, |b|) of two fp32 values (the result's sign is the xor of the inputs'); a NaN input gives NaN.
+__device__ __forceinline__ uint32_t absmax_f32(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.NaN.xorsign.abs.f32 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// Two-stage rule on a block of 32 fp32 bit patterns with the arithmetic of the bf16 fast path below: the
+// maximum as a tree of |.|-maxima, one fma.rz per element on |x| for its 5-bit code (a clamped block is
+// prescaled by 2^64 first), popcount of the shifted merged threshold mask, signs gathered with byte permutes
+// (three per four elements).  BYTES: operand bytes in e4m3[0..7] instead of indices in res.words.
+template <bool BYTES>
+__device__ __forceinline__ void quantize_two_stage_f32(const uint32_t (&bits_in)[32], const SmemTables &tab, BlockResult &res,
+                                                       uint32_t (&e4m3)[8], bool &nonfinite) {
+    uint32_t bits[32], t16[16];
+#pragma unroll
+    for (int k = 0; k < 32; k++) bits[k] = bits_in[k];
+#pragma unroll
+    for (int i = 0; i < 16; i++) t16[i] = absmax_f32(bits[2 * i], bits[2 * i + 1]);
+#pragma unroll
+    for (int i = 0; i < 8; i++) t16[i] = absmax_f32(t16[2 * i], t16[2 * i + 1]);
+#pragma unroll
+    for (int i = 0; i < 4; i++) t16[i] = absmax_f32(t16[2 * i], t16[2 * i + 1]);
+    const uint32_t amax = absmax_f32(absmax_f32(t16[0], t16[1]), absmax_f32(t16[2], t16[3])) & 0x7fffffffu;
+    nonfinite = amax >= 0x7f800000u;
+    const uint32_t eadj = max(amax >> 23, 2u);
+    float amax_f = __uint_as_float(amax);
+    uint32_t eadj_eff = eadj;
+    if (eadj < 4u) {                                              // 2^(131 - eadj) would overflow: move 2^64 into the data
+#pragma unroll
+        for (int k = 0; k < 32; k++) bits[k] = __float_as_uint(__uint_as_float(bits[k]) * 18446744073709551616.0f);
+        amax_f *= 18446744073709551616.0f;
+        eadj_eff = eadj + 64u;
+    }
+    const float scale = __uint_as_float((258u - eadj_eff) << 23);
+    const uint32_t m5 = __float_as_uint(__fmaf_rz(amax_f, scale, 8388608.0f)) & 63u;
+    const uint32_t pair = min(7u, 15u - min(15u, (m5 + 1u) >> 1));
+    const uint32_t above = tab.merged_above[pair];
+    uint32_t v[4] = {0, 0, 0, 0}, s03[4], s47[4];
+#pragma unroll
+    for (int k = 0; k < 32; k++) {
+        const uint32_t t = __float_as_uint(__fmaf_rz(fabsf(__uint_as_float(bits[k])), scale, 8388608.0f));
+        v[k / 8] = (uint32_t)__popc(__funnelshift_r(above, 0u, t)) * (1u << (4 * slot_of(k % 8))) + v[k / 8];
+    }
+#pragma unroll
+    for (int w = 0; w < 4; w++) {                                 // the top bytes of the group's eight elements
+        s03[w] = prmt_b32(prmt_b32(bits[8 * w], bits[8 * w + 1], 0x0073u), prmt_b32(bits[8 * w + 2], bits[8 * w + 3], 0x0073u), 0x5410u);
+        s47[w] = prmt_b32(prmt_b32(bits[8 * w + 4], bits[8 * w + 5], 0x0073u), prmt_b32(bits[8 * w + 6], bits[8 * w + 7], 0x0073u), 0x5410u);
+    }
+    res.scale = eadj - 2u;
+    if (BYTES) {
+        finish_two_stage_e4m3(v, s03, s47, pair, tab, res.id, e4m3);
+    } else {
+        uint32_t signs[4];
+#pragma unroll
+        for (int w = 0; w < 4; w++) signs[w] = (s03[w] & 0x80808080u) | ((s47[w] >> 4) & 0x08080808u);
+        finish_two_stage(v, signs, pair, res.id, res.words);
+    }
+}
+
 // ---------------------------------------------------------------------------
 // bf16 fast path of the contiguous-axis quantizer (same thread-to-block map and outputs
 // as quantize_contig_kernel).  The 32 elements stay packed two per register:
@@ -468,81 +528,109 @@ __global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel
 // Optional second output: the decoded operand bytes (E4M3 of 0.5 * value, sign in bit 7) as a
 // plain [rows][K] byte matrix, the form the tensor-core GEMM loads.
 // ---------------------------------------------------------------------------
-template <int DT, int SELECT, bool WRITE_CODES, bool WRITE_E4M3>
+constexpr int kContigStageBytes = 2 * 8 * 4096;               // two buffers of 4 KiB per warp
+// REGULAR: rows is a multiple of 64 and K a multiple of 128, so no chunk has padding rows or blocks.
+template <int DT, int SELECT, bool WRITE_CODES, bool WRITE_E4M3, bool REGULAR>
 __global__ void __launch_bounds__(256) quantize_contig_kernel(const void *__restrict__ X, int64_t ld, QView out,
-                                                              uint8_t *__restrict__ e4m3, int nb, int kgroups) {
+                                                              uint8_t *__restrict__ e4m3, int nb, int kgroups, uint32_t chunks,
+                                                              FastDiv div_kgroups) {
     __shared__ SmemTables tab;
     load_tables(tab);
-    const uint32_t lane = threadIdx.x % 32u, b4 = lane & 3u, j = (lane >> 2) & 3u;
-    const int64_t th = blockIdx.x / (uint32_t)kgroups;           // 2 * tile + half
-    const uint32_t kg = blockIdx.x % (uint32_t)kgroups;
-    const int64_t r = (th >> 1) * kRowTile + (th & 1) * 16 + 2 * (threadIdx.x / 32u) + (lane >> 4) + 32 * j;
-    const int b = (int)(kg * kBlocksPerAtom + b4);
-    const bool valid = r < out.rows && b < nb;
-    BlockResult res;
-    res.id = 0; res.scale = 0;
-    res.words[0] = res.words[1] = res.words[2] = res.words[3] = 0;
+    // launched with programmatic stream serialisation, like the bf16 kernel below: wait for the previous
+    // kernel's results, then let the next kernel set itself up on the processors this grid leaves
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const uint32_t lane = threadIdx.x % 32u, b4 = lane & 3u, j = (lane >> 2) & 3u, warp = threadIdx.x / 32u;
     // fp32 blocks are 128 bytes, one cache line each: read thread by thread, every 16-byte load of a warp
     // would touch 32 lines.  Instead the warp copies its eight rows line by line (the four blocks of a row
     // are 512 contiguous bytes, 16 per lane) into shared memory, asynchronously, and each thread then
-    // picks up its own block; an xor of the chunk index keeps both sides free of bank conflicts.
-    __shared__ __align__(128) uint8_t stage[DT == BD_F32 ? 8 * 4096 : 16];
-    if (DT == BD_F32) {
-        const uint32_t warp = threadIdx.x / 32u;
-        const int64_t row0 = (th >> 1) * kRowTile + (th & 1) * 16 + 2 * warp;
+    // picks up its own block; an xor of the chunk index keeps both sides free of bank conflicts.  Two such
+    // buffers per warp: the copy of the CTA's next chunk runs while the current one is quantised.
+    // (dynamic shared memory: kContigStageBytes for fp32 sources, none otherwise)
+    extern __shared__ __align__(128) uint8_t stage[];
+    // the copy's addresses: per chunk one 64-bit base; the eight rows of a lane are 0 or 1 and 0, 32, 64 or 96 rows
+    // further on, and their places in the buffer differ by constants (the xor term depends on the parity of i only)
+    const int64_t ld_bytes = ld * 4;
+    const uint32_t stage_base = (uint32_t)__cvta_generic_to_shared(stage) + warp * 4096u + (lane >> 3) * 128u;
+    const uint32_t swz_even = ((lane & 7u) ^ ((lane >> 3) & 7u)) * 16u, swz_odd = ((lane & 7u) ^ ((4u + (lane >> 3)) & 7u)) * 16u;
+    auto copy_in = [&](uint32_t chunk, uint32_t buf) {
+        const uint32_t th = fast_div(chunk, div_kgroups), kg = chunk - th * (uint32_t)kgroups;
+        const int64_t row0 = (int64_t)(th >> 1) * kRowTile + (th & 1u) * 16 + 2 * warp;
         const int cb = (int)(kg * kBlocksPerAtom) + (int)(lane >> 3);            // the block this lane copies from
+        const char *src0 = (const char *)X + (row0 * ld + (int64_t)cb * 32) * 4 + (lane & 7u) * 16;
+        const uint32_t dst0 = stage_base + buf * 32768u;
 #pragma unroll
         for (int i = 0; i < 8; i++) {
-            const int64_t ri = row0 + (i >> 2) + 32 * (i & 3);
-            const bool ok = ri < out.rows && cb < nb;
-            const char *src = ok ? (const char *)X + (ri * ld + (int64_t)cb * 32) * 4 + (lane & 7u) * 16 : (const char *)X;
-            const uint32_t owner = 4u * i + (lane >> 3);
-            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(stage) + warp * 4096u + owner * 128u +
-                                 (((lane & 7u) ^ (owner & 7u)) * 16u);
+            const bool ok = REGULAR || (row0 + (i >> 2) + 32 * (i & 3) < out.rows && cb < nb);
+            const char *src = ok ? src0 + ((i >> 2) + 32 * (i & 3)) * ld_bytes : (const char *)X;
+            const uint32_t dst = dst0 + 512u * i + ((i & 1) ? swz_odd : swz_even);
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(ok ? 16 : 0) : "memory");
         }
-        asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-        __syncwarp();
+    };
+    // CTA x takes chunks x, x + gridDim.x, ...
+    uint32_t chunk = blockIdx.x, buf = 0;
+    if (DT == BD_F32) {
+        if (chunk < chunks) copy_in(chunk, 0);
+        asm volatile("cp.async.commit_group;" ::: "memory");
     }
-    if (valid) {
-        uint32_t bits[32];
+    for (; chunk < chunks; chunk += gridDim.x, buf ^= 1u) {
+        const uint32_t th = fast_div(chunk, div_kgroups);        // 2 * tile + half
+        const uint32_t kg = chunk - th * (uint32_t)kgroups;
+        const int64_t r = (int64_t)(th >> 1) * kRowTile + (th & 1u) * 16 + 2 * warp + (lane >> 4) + 32 * j;
+        const int b = (int)(kg * kBlocksPerAtom + b4);
+        const bool valid = REGULAR || (r < out.rows && b < nb);
+        BlockResult res;
+        res.id = 0; res.scale = 0;
+        res.words[0] = res.words[1] = res.words[2] = res.words[3] = 0;
         if (DT == BD_F32) {
-            const uint8_t *mine = stage + (threadIdx.x / 32u) * 4096u + lane * 128u;
+            if (chunk + gridDim.x < chunks) copy_in(chunk + gridDim.x, buf ^ 1u);
+            asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 1;" ::: "memory");   // all but the newest group: this chunk is in
+            __syncwarp();
+        }
+        if (valid) {
+            uint32_t bits[32];
+            if (DT == BD_F32) {
+                const uint8_t *mine = stage + buf * 32768u + warp * 4096u + lane * 128u;
 #pragma unroll
-            for (int k = 0; k < 8; k++) {
-                const uint4 u = *(const uint4 *)(mine + ((k ^ (lane & 7u)) * 16u));
-                bits[4 * k] = u.x; bits[4 * k + 1] = u.y; bits[4 * k + 2] = u.z; bits[4 * k + 3] = u.w;
+                for (int k = 0; k < 8; k++) {
+                    const uint4 u = *(const uint4 *)(mine + ((k ^ (lane & 7u)) * 16u));
+                    bits[4 * k] = u.x; bits[4 * k + 1] = u.y; bits[4 * k + 2] = u.z; bits[4 * k + 3] = u.w;
+                }
+            } else {
+                Loader<DT>::contiguous((const char *)X + (r * ld + (int64_t)b * 32) * Loader<DT>::kElemBytes, bits);
             }
-        } else {
-            Loader<DT>::contiguous((const char *)X + (r * ld + (int64_t)b * 32) * Loader<DT>::kElemBytes, bits);
-        }
-        bool nonfinite;
-        if (SELECT == BD_SELECT_MSE) res = quantize_mse(bits, tab, nonfinite);
-        else res = quantize_two_stage(bits, tab, nonfinite);
-        if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
-        if (WRITE_CODES)
-            *(uint4 *)(out.codes + r * (out.K / 2) + (int64_t)b * 16) =
-                make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
-        if (WRITE_E4M3) {
-            uint32_t lo = tab.e4m3_lo[res.id], hi = tab.e4m3_hi[res.id];
+            bool nonfinite;
             uint32_t o[8];
+            constexpr bool kBytesOnly = WRITE_E4M3 && !WRITE_CODES && SELECT != BD_SELECT_MSE;
+            if (SELECT == BD_SELECT_MSE) res = quantize_mse(bits, tab, nonfinite);
+            else quantize_two_stage_f32<kBytesOnly>(bits, tab, res, o, nonfinite);
+            if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
+            if (WRITE_CODES)
+                *(uint4 *)(out.codes + r * (out.K / 2) + (int64_t)b * 16) =
+                    make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
+            if (WRITE_E4M3) {
+                if (!kBytesOnly) {
+                    uint32_t lo = tab.e4m3_lo[res.id], hi = tab.e4m3_hi[res.id];
 #pragma unroll
-            for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, o[2 * w], o[2 * w + 1]);
-            uint4 *dst = (uint4 *)(e4m3 + r * out.K + (int64_t)b * 32);
-            dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
-            dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                    for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, o[2 * w], o[2 * w + 1]);
+                }
+                uint4 *dst = (uint4 *)(e4m3 + r * out.K + (int64_t)b * 32);
+                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+            }
         }
-    }
-    // the four lanes of a row merge their scale bytes and id nibbles
-    uint32_t sc = res.scale << (8 * b4);
-    uint32_t idn = res.id << (4 * b4);
-    sc |= __shfl_xor_sync(0xffffffffu, sc, 1);
-    idn |= __shfl_xor_sync(0xffffffffu, idn, 1);
-    sc |= __shfl_xor_sync(0xffffffffu, sc, 2);
-    idn |= __shfl_xor_sync(0xffffffffu, idn, 2);
-    if (b4 == 0) {
-        *(uint32_t *)(out.scales + scale_offset(out.rows, r, b)) = sc;
-        if (WRITE_CODES) *(uint16_t *)(out.ids + id_byte_offset(out.rows, r, b)) = (uint16_t)idn;
+        // the four lanes of a row merge their scale bytes and id nibbles
+        uint32_t sc = res.scale << (8 * b4);
+        uint32_t idn = res.id << (4 * b4);
+        sc |= __shfl_xor_sync(0xffffffffu, sc, 1);
+        idn |= __shfl_xor_sync(0xffffffffu, idn, 1);
+        sc |= __shfl_xor_sync(0xffffffffu, sc, 2);
+        idn |= __shfl_xor_sync(0xffffffffu, idn, 2);
+        if (b4 == 0) {
+            *(uint32_t *)(out.scales + scale_offset(out.rows, r, b)) = sc;
+            if (WRITE_CODES) *(uint16_t *)(out.ids + id_byte_offset(out.rows, r, b)) = (uint16_t)idn;
+        }
+        __syncwarp();                                            // the buffer read above is the next iteration's copy target
     }
 }
 
