@@ -40,9 +40,9 @@ M_TOKENS = 2048
 QUANT_SHAPE = (8192, 4096)
 BYTES_PER_ELEM_QUANT = 2 + 0.5 + 1.5 / 32           # bf16 read + 4-bit code + (4-bit id + 8-bit scale) / 32
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
-QUANT_DRAM_BYTES = 67.59e6 + 4.05e6                 # quantize_bf16_kernel on bf16 [8192, 4096]
-GEMM_GATE_UP_DRAM_BYTES = 40.86e6 + 18.90e6         # tc::gemm_wtmem_kernel on the gate/up layer
-QUANT_WARP_INSTRUCTIONS = 14.1e6                    # smsp__inst_executed.sum of the same quantizer launch
+QUANT_DRAM_BYTES = 67.13e6 + 4.82e6                 # quantize_bf16_kernel on bf16 [8192, 4096]
+GEMM_GATE_UP_DRAM_BYTES = 40.84e6 + 20.82e6         # tc::gemm_wtmem_kernel on the gate/up layer
+QUANT_WARP_INSTRUCTIONS = 12.9e6                    # smsp__inst_executed.sum of the same quantizer launch
 SM_COUNT, ISSUE_PER_SM_CLK = 148, 4                 # warp instructions per clock an SM can issue (4 schedulers)
 MLP_SWEEP = [(4096, 11008), (11008, 4096)]
 MLP_SWEEP_M = [1, 16, 128, 1024, 8192]
