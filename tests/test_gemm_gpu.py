@@ -215,3 +215,27 @@ def test_linear_source_types_pitches_and_ragged_shapes(kind, M, N, K):
         else:
             assert torch.equal(wide_y[:, :N], y32.to(torch.bfloat16))
     bd.poll_status()
+
+
+def test_two_streams_of_decode_sized_calls_do_not_disturb_each_other():
+    # calls whose K is cut over several clusters keep arrival counters in device memory and start before the
+    # kernel ahead of them has finished; two streams of them, interleaved, must give what each gives alone
+    rng = np.random.default_rng(77)
+    shapes = [(4, 4096, 11008), (16, 520, 4128)]
+    work = []
+    for M, N, K in shapes:
+        x = to_device(inputs.to_bf16_bits(rng.standard_normal((M, K)).astype(np.float32)), torch.bfloat16)
+        w = to_device(inputs.to_bf16_bits((0.02 * rng.standard_normal((N, K))).astype(np.float32)), torch.bfloat16)
+        wq = bd.quantize_weights(w, bd.SELECT_TWO_STAGE)
+        ws = torch.empty(bd.linear_workspace_size(M, N, K), dtype=torch.uint8, device="cuda")
+        alone = bd.linear(x, wq, dtype=torch.float32, workspace=ws).clone()
+        work.append((x, wq, ws, alone, torch.empty_like(alone), torch.cuda.Stream()))
+    torch.cuda.synchronize()
+    for it in range(200):
+        for x, wq, ws, alone, out, stream in work:
+            bd.linear(x, wq, out=out, workspace=ws, stream=stream)
+        if it % 50 == 49:
+            torch.cuda.synchronize()
+            for x, wq, ws, alone, out, stream in work:
+                assert torch.equal(out, alone), f"iteration {it}"
+    bd.poll_status()
