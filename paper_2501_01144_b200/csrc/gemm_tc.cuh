@@ -267,13 +267,20 @@ __device__ __forceinline__ void epilogue_bf16(uint32_t t_base, uint8_t *stage_pt
 #pragma unroll
     for (int pass = 0; pass < CHUNKS / 2; pass++) {
         staging_free();
+        // the exchanges of eight registers go out together, so that their latencies overlap
 #pragma unroll
-        for (int q = 0; q < 32; q++) {
-            const uint32_t mine = p[32 * pass + q];
-            const uint32_t other = __shfl_xor_sync(0xffffffffu, mine, 1);
-            const uint32_t word = (lane & 1) ? prmt_b32(other, mine, 0x7632u)   // (col - 1, col) of token t + 1
-                                             : prmt_b32(mine, other, 0x5410u);  // (col, col + 1) of token t
-            *(uint32_t *)(stage_ptr + (2 * q + (lane & 1)) * 64 + (lane >> 1) * 4) = word;
+        for (int q0 = 0; q0 < 32; q0 += 8) {
+            uint32_t other[8];
+#pragma unroll
+            for (int u = 0; u < 8; u++) other[u] = __shfl_xor_sync(0xffffffffu, p[32 * pass + q0 + u], 1);
+#pragma unroll
+            for (int u = 0; u < 8; u++) {
+                const int q = q0 + u;
+                const uint32_t mine = p[32 * pass + q];
+                const uint32_t word = (lane & 1) ? prmt_b32(other[u], mine, 0x7632u)   // (col - 1, col) of token t + 1
+                                                 : prmt_b32(mine, other[u], 0x5410u);  // (col, col + 1) of token t
+                *(uint32_t *)(stage_ptr + (2 * q + (lane & 1)) * 64 + (lane >> 1) * 4) = word;
+            }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
