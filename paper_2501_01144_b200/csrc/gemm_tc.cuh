@@ -151,7 +151,8 @@ constexpr int kCodeTile = 128 * 64;          // 8 KiB: 128 weight rows x 64 byte
 constexpr int kDecodeWarp0 = 3, kDecodeGroups = 3, kDecodeWarps = 4 * kDecodeGroups;
 constexpr int kEpilogueWarp0 = kDecodeWarp0 + kDecodeWarps, kEpilogueWarps = 8;
 constexpr int kThreads = 32 * (kEpilogueWarp0 + kEpilogueWarps);
-constexpr int kStageOut = 4096;            // per epilogue warp: 64 tokens x 32 bf16 or 32 tokens x 32 fp32
+constexpr int kStageOut = 2048;            // one staging buffer: 32 tokens x 32 bf16 or 16 tokens x 32 fp32
+constexpr int kStageBufs = 2;               // per epilogue warp, used in turn: a store reads one while the next is filled
 
 // tensor-memory columns
 constexpr int kColD = 0;                     // accumulator: 256 token columns
@@ -170,7 +171,7 @@ struct Smem {
     static constexpr int words = bars + 512;
     static constexpr int luts = words + 64;
     static constexpr int out = ((luts + 128 + 1023) / 1024) * 1024;
-    static constexpr int total = out + kEpilogueWarps * kStageOut + 1024 /* alignment slack */;
+    static constexpr int total = out + kEpilogueWarps * kStageBufs * kStageOut + 1024 /* alignment slack */;
 };
 static_assert((2 * kXStages + 2 * kCodeStages + 2 * kABufs + 2) * 8 <= 512, "barrier area too small");
 static_assert(Smem::total <= 227 * 1024, "shared memory budget");
@@ -244,9 +245,10 @@ __device__ __forceinline__ void mbar_arrive_local(uint32_t bar) {
 
 // bf16 epilogue of one warp: its 32 * CHUNKS token columns go to registers first, packed as bf16 pairs of
 // neighbouring tokens (16 * CHUNKS registers), so the accumulator is free again after CHUNKS TMEM round trips;
-// then, 64 tokens at a time, lanes 2m and 2m + 1 trade halves so that each writes one 32-bit word of two
-// neighbouring output columns (the even lane the row of token t, the odd lane the row of token t + 1) into the
-// staging tile, which a TMA tensor store writes out as 64 rows x 32 columns.
+// then, 32 tokens at a time, lanes 2m and 2m + 1 trade halves so that each writes one 32-bit word of two
+// neighbouring output columns (the even lane the row of token t, the odd lane the row of token t + 1) into one
+// of the warp's two staging buffers, which a TMA tensor store writes out as 32 rows x 32 columns while the
+// other buffer is filled.
 template <int CHUNKS, typename Release, typename StagingFree>
 __device__ __forceinline__ void epilogue_bf16(uint32_t t_base, uint8_t *stage_ptr, uint32_t stage_out, const CUtensorMap *mapY,
                                               int n0, int t0, int lane, volatile uint32_t *abort_flag, Release release_accumulator,
@@ -265,28 +267,28 @@ __device__ __forceinline__ void epilogue_bf16(uint32_t t_base, uint8_t *stage_pt
     }
     release_accumulator();
 #pragma unroll
-    for (int pass = 0; pass < CHUNKS / 2; pass++) {
-        staging_free();
+    for (int pass = 0; pass < CHUNKS; pass++) {                   // 32 tokens per pass
+        const uint32_t sb = staging_free();                       // offset of the staging buffer whose turn it is
         // the exchanges of eight registers go out together, so that their latencies overlap
 #pragma unroll
-        for (int q0 = 0; q0 < 32; q0 += 8) {
+        for (int q0 = 0; q0 < 16; q0 += 8) {
             uint32_t other[8];
 #pragma unroll
-            for (int u = 0; u < 8; u++) other[u] = __shfl_xor_sync(0xffffffffu, p[32 * pass + q0 + u], 1);
+            for (int u = 0; u < 8; u++) other[u] = __shfl_xor_sync(0xffffffffu, p[16 * pass + q0 + u], 1);
 #pragma unroll
             for (int u = 0; u < 8; u++) {
                 const int q = q0 + u;
-                const uint32_t mine = p[32 * pass + q];
+                const uint32_t mine = p[16 * pass + q];
                 const uint32_t word = (lane & 1) ? prmt_b32(other[u], mine, 0x7632u)   // (col - 1, col) of token t + 1
                                                  : prmt_b32(mine, other[u], 0x5410u);  // (col, col + 1) of token t
-                *(uint32_t *)(stage_ptr + (2 * q + (lane & 1)) * 64 + (lane >> 1) * 4) = word;
+                *(uint32_t *)(stage_ptr + sb + (2 * q + (lane & 1)) * 64 + (lane >> 1) * 4) = word;
             }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (lane == 0 && !*abort_flag) {
             asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                         ::"l"(mapY), "r"(n0), "r"(t0 + pass * 64), "r"(stage_out) : "memory");
+                         ::"l"(mapY), "r"(n0), "r"(t0 + pass * 32), "r"(stage_out + sb) : "memory");
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
     }
@@ -525,19 +527,23 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         // accumulator, token columns [128 * half, + 128), and writes them transposed: Y[token][weight row] ----
         const int quad = warp % 4, ew = warp - kEpilogueWarp0, half = ew / 4;
         const uint32_t tmem_empty_leader = map_to_cta(tmem_empty_bar, 0);
-        const uint32_t stage_out = base + Smem::out + (uint32_t)ew * kStageOut;
-        uint8_t *const stage_ptr = base_ptr + Smem::out + ew * kStageOut;
-        // 4 KiB of staging per warp: 64 tokens x 32 bf16 or 32 tokens x 32 fp32 per tensor store
+        const uint32_t stage_out = base + Smem::out + (uint32_t)ew * (kStageBufs * kStageOut);
+        uint8_t *const stage_ptr = base_ptr + Smem::out + ew * (kStageBufs * kStageOut);
+        // 4 KiB of staging per warp, two buffers: 32 tokens x 32 bf16 or 16 tokens x 32 fp32 per tensor store
         // accumulator read out (all of this warp's columns are in registers): the MMA issuer may start the next tile
         auto release_accumulator = [&]() {
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(tmem_empty_leader);
         };
-        // the previous pass's tensor store must have finished reading the staging buffer
-        auto staging_free = [&]() {
-            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        // the two staging buffers take turns: before one is filled again, the tensor store issued two passes ago
+        // (the one that read it) must have finished reading; the latest store may still be in flight
+        uint32_t stage_turn = 0;
+        auto staging_free = [&]() -> uint32_t {
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
             __syncwarp();
+            stage_turn ^= 1u;
+            return stage_turn * kStageOut;
         };
         Tile t;
         for (int i = 0; next_tile(sc, cluster, i, t); i++) {
@@ -604,22 +610,19 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 if (cols == 128) epilogue_bf16<4>(t_base, stage_ptr, stage_out, &mapY, n0, t0, lane, abort_flag, release_accumulator, staging_free);
                 else epilogue_bf16<2>(t_base, stage_ptr, stage_out, &mapY, n0, t0, lane, abort_flag, release_accumulator, staging_free);
             } else if (use_tma_store) {
-                for (int pass = 0; pass * 32 < cols; pass++) {        // fp32: 32 tokens x 32 columns per pass
-                    uint32_t r[2][16];
-#pragma unroll
-                    for (int c = 0; c < 2; c++) tcgen05_ld_32x32b_x16(t_base + pass * 32 + c * 16, r[c]);
+                for (int pass = 0; pass * 16 < cols; pass++) {        // fp32: 16 tokens x 32 columns per pass
+                    uint32_t r[16];
+                    tcgen05_ld_32x32b_x16(t_base + pass * 16, r);
                     tcgen05_wait_ld();
-                    if ((pass + 1) * 32 >= cols) release_accumulator();
-                    staging_free();
+                    if ((pass + 1) * 16 >= cols) release_accumulator();
+                    const uint32_t sb = staging_free();
 #pragma unroll
-                    for (int c = 0; c < 2; c++)
-#pragma unroll
-                        for (int q = 0; q < 16; q++) *(uint32_t *)(stage_ptr + (c * 16 + q) * 128 + lane * 4) = r[c][q];
+                    for (int q = 0; q < 16; q++) *(uint32_t *)(stage_ptr + sb + q * 128 + lane * 4) = r[q];
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     if (lane == 0 && !*abort_flag) {
                         asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                                     ::"l"(&mapY), "r"(n0), "r"(t0 + pass * 32), "r"(stage_out) : "memory");
+                                     ::"l"(&mapY), "r"(n0), "r"(t0 + pass * 16), "r"(stage_out + sb) : "memory");
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                 }
@@ -708,13 +711,13 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
         !make_map_2d(&mapSfW, CU_TENSOR_MAP_DATA_TYPE_UINT32, W.scales, 128, rtw * kg, kScaleAtomBytes, 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE) ||
         !make_map_2d(&mapSfX, CU_TENSOR_MAP_DATA_TYPE_UINT32, sfx, 128, rtx * kg, kScaleAtomBytes, 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE))
         return cudaErrorInvalidValue;
-    // output through TMA tensor stores (32 columns x 64 or 32 rows per box) when Y is 16-byte aligned with a
+    // output through TMA tensor stores (32 columns x 32 or 16 rows per box) when Y is 16-byte aligned with a
     // row pitch that is a multiple of 16 bytes; otherwise plain stores
     const int esz = out_bf16 ? 2 : 4;
     int use_tma_store = (((uintptr_t)Y & 15u) == 0 && (ldy * esz) % 16 == 0) ? 1 : 0;
     if (use_tma_store &&
         !make_map_2d(&mapY, out_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Y, N, M,
-                     (uint64_t)ldy * esz, 32, out_bf16 ? 64 : 32, CU_TENSOR_MAP_SWIZZLE_NONE))
+                     (uint64_t)ldy * esz, 32, out_bf16 ? 32 : 16, CU_TENSOR_MAP_SWIZZLE_NONE))
         use_tma_store = 0;
     if (!use_tma_store) mapY = mapX;                                   // unused, but must be a valid object
     static bool configured[kMaxDevices] = {};
