@@ -73,7 +73,7 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "10",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "25",
                  "-i", str(self.gpu_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
@@ -249,12 +249,16 @@ def run_gpu(args, rank, world, local_rank):
 
     per_step = []                                        # device time of each step of the last timed() call
 
-    def timed(fn, steps, warmup, finish=None):
+    def timed(fn, steps, warmup, finish=None, head_start=False):
         for _ in range(warmup):
             fn()
         barrier()
         marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
         e0, e1 = marks[0], marks[-1]
+        if head_start:
+            # the GPU spins for a few milliseconds while the host queues the first steps behind it, so that a
+            # host hiccup (interpreter, sampler thread) does not starve the GPU inside the timed region
+            torch.cuda._sleep(10_000_000)
         e0.record()
         for i in range(steps):
             fn()
@@ -275,7 +279,7 @@ def run_gpu(args, rank, world, local_rank):
     barrier()
     launches_warm = bd.launch_count()
     t_begin = time.time()
-    total_ms = timed(step, args.steps, 0)
+    total_ms = timed(step, args.steps, 0, head_start=True)
     t_end = time.time()
     clocks = sampler.stop(t_begin, t_end)
     launches = bd.launch_count() - launches_warm
