@@ -401,6 +401,10 @@ def run_gpu(args, rank, world, local_rank):
             return a.elapsed_time(b) / n_rep * 1e3
 
         qk_us = time_us(lambda: bd.gemm_batched(Aq, Bk, b_group=heads // kvh, out=scores, workspace=gws), 3)
+        # context for the write-bound product: what a plain write-only stream reaches on this GPU (the measured
+        # peak is a copy, half reads and half writes)
+        fill_us = time_us(lambda: scores.fill_(0), 5)
+        write_stream_gbs = scores.numel() * 2.0 / fill_us / 1e3
         del scores
         # the four query heads of a KV group share V, so their probabilities go through one call as one
         # [4 * 4096, 4096] matrix (contiguous heads): one quantizer launch and one product per group
@@ -421,6 +425,8 @@ def run_gpu(args, rank, world, local_rank):
                                  "quantised online x V (token-axis blocks) [128,4096]^T, the 4 heads of a KV group per call",
                      "qk_us_32_heads": qk_us, "qk_write_gbs": qk_bytes / qk_us / 1e3,
                      "qk_frac_of_hbm": qk_bytes / qk_us / 1e3 / peaks["hbm_gbs"],
+                     "write_only_stream_gbs": write_stream_gbs,
+                     "qk_frac_of_write_only_stream": qk_bytes / qk_us / 1e3 / write_stream_gbs,
                      "pv_us_per_head": pv_us, "pv_read_gbs": pv_bytes / pv_us / 1e3,
                      "pv_frac_of_hbm": pv_bytes / pv_us / 1e3 / peaks["hbm_gbs"]}
         del P, Aq, Bk
