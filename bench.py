@@ -420,6 +420,28 @@ def run_gpu(args, rank, world, local_rank):
             turn[0] += 1
 
         pv_us = time_us(pv, 6) / grp
+        # the KV groups are independent problems: on two streams the quantizer of one group's probabilities (HBM)
+        # runs beside the product of the previous group's (tensor cores)
+        side = [torch.cuda.Stream(), torch.cuda.Stream()]
+        O2 = [O, torch.empty_like(O)]
+        lws2 = [lws, torch.empty_like(lws)]
+
+        def pv_two_streams(n_rep):
+            cur = torch.cuda.current_stream()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for st in side:
+                st.wait_event(a)
+            for i in range(n_rep):
+                bd.linear(P[i % 3], Bv, out=O2[i % 2], workspace=lws2[i % 2], stream=side[i % 2])
+            for st in side:
+                cur.wait_stream(st)
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / n_rep * 1e3
+
+        pv_two_streams(2)
+        pv2_us = pv_two_streams(8) / grp
         qk_bytes, pv_bytes = heads * S * S * 2.0, S * S * 4.0
         attention = {"workload": "QK^T: 32 heads x [4096,128] x [4096,128]^T, bf16 scores; PV: fp32 P [4096,4096] per head "
                                  "quantised online x V (token-axis blocks) [128,4096]^T, the 4 heads of a KV group per call",
@@ -428,7 +450,9 @@ def run_gpu(args, rank, world, local_rank):
                      "write_only_stream_gbs": write_stream_gbs,
                      "qk_frac_of_write_only_stream": qk_bytes / qk_us / 1e3 / write_stream_gbs,
                      "pv_us_per_head": pv_us, "pv_read_gbs": pv_bytes / pv_us / 1e3,
-                     "pv_frac_of_hbm": pv_bytes / pv_us / 1e3 / peaks["hbm_gbs"]}
+                     "pv_frac_of_hbm": pv_bytes / pv_us / 1e3 / peaks["hbm_gbs"],
+                     "pv_two_streams_us_per_head": pv2_us, "pv_two_streams_read_gbs": pv_bytes / pv2_us / 1e3,
+                     "pv_two_streams_frac_of_hbm": pv_bytes / pv2_us / 1e3 / peaks["hbm_gbs"]}
         del P, Aq, Bk
         bd.poll_status()
 
