@@ -169,9 +169,11 @@ bd_status gemm_dispatch(const QView &A, const QView &B, void *Y, bd_dtype ydt, i
         decode_e4m3_kernel<<<grid_for(A.rows * nb, 256), 256, 0, st>>>(A, a8, nb);
         bd_status s = launch_result(1);
         if (s) return s;
-        g_launches += 1;
-        return cuda_result(tc::launch(a8, A.scales, A.rows, B, A.K, Y, ydt == BD_BF16, ldy, st,
-                                      a8 + tc_operand_bytes(A.rows, A.K), tc::splitk_workspace(A.rows, B.rows, A.K)));
+        int kernels = 1;
+        s = cuda_result(tc::launch(a8, A.scales, A.rows, B, A.K, Y, ydt == BD_BF16, ldy, st,
+                                   a8 + tc_operand_bytes(A.rows, A.K), tc::splitk_workspace(A.rows, B.rows, A.K), &kernels));
+        g_launches += (uint64_t)kernels;
+        return s;
     }
     if (ydt == BD_F32) return launch_simt<float>(A, B, Y, ldy, st);
     return launch_simt<__nv_bfloat16>(A, B, Y, ldy, st);
@@ -359,9 +361,11 @@ bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_
         bd_qtensor xq{nullptr, nullptr, sfa, M, K};
         s = launch_contig<BD_SELECT_TWO_STAGE, false, true>(X, xdtype, ldx, view_of(&xq), a8, st);
         if (s) return s;
-        g_launches += 1;
-        return cuda_result(tc::launch(a8, sfa, M, view_of(Wq), K, Y, ydtype == BD_BF16, ldy, st,
-                                      a8 + tc_operand_bytes(M, K), tc::splitk_workspace(M, N, K)));
+        int kernels = 1;
+        s = cuda_result(tc::launch(a8, sfa, M, view_of(Wq), K, Y, ydtype == BD_BF16, ldy, st,
+                                   a8 + tc_operand_bytes(M, K), tc::splitk_workspace(M, N, K), &kernels));
+        g_launches += (uint64_t)kernels;
+        return s;
     }
     bd_qtensor xq{p, p + align256(c), p + align256(c) + align256(i), M, K};
     s = launch_contig<BD_SELECT_TWO_STAGE, true, false>(X, xdtype, ldx, view_of(&xq), nullptr, st);

@@ -51,7 +51,9 @@ def test_tiny_case(impl):
                                    # token tiles cut into 128-token items, with and without a ragged last tile
                                    (448, 512, 256), (640, 300, 160), (512, 1024, 128),
                                    # decode-sized calls whose K is cut over several clusters (ragged last k-step)
-                                   (5, 300, 2144), (16, 520, 4128), (1, 256, 8192)])
+                                   (5, 300, 2144), (16, 520, 4128), (1, 256, 8192),
+                                   # 17 to 128 tokens with few tiles: K cut likewise, the partial sums added by a second kernel
+                                   (17, 300, 2144), (100, 520, 4128), (128, 1024, 4096)])
 def test_ragged_shapes(impl, M, N, K):
     rng = np.random.default_rng(M + 31 * N + 977 * K)
     a = rng.standard_t(4, (M, K)).astype(np.float32)
