@@ -53,7 +53,9 @@ def test_tiny_case(impl):
                                    # decode-sized calls whose K is cut over several clusters (ragged last k-step)
                                    (5, 300, 2144), (16, 520, 4128), (1, 256, 8192),
                                    # 17 to 128 tokens with few tiles: K cut likewise, the partial sums added by a second kernel
-                                   (17, 300, 2144), (100, 520, 4128), (128, 1024, 4096)])
+                                   (17, 300, 2144), (100, 520, 4128), (128, 1024, 4096),
+                                   # a few hundred tokens against few weight rows, ragged last tile
+                                   (300, 520, 2144), (512, 256, 4096), (257, 1024, 1056)])
 def test_ragged_shapes(impl, M, N, K):
     rng = np.random.default_rng(M + 31 * N + 977 * K)
     a = rng.standard_t(4, (M, K)).astype(np.float32)
