@@ -209,32 +209,6 @@ __device__ __forceinline__ void finish_two_stage_e4m3(const uint32_t (&v)[4], co
     }
 }
 
-// Two-stage rule (Sec. 3.2) for a block given as fp32 bit patterns.
-__device__ __forceinline__ BlockResult quantize_two_stage(const uint32_t (&bits)[32], const SmemTables &tab,
-                                                          bool &nonfinite) {
-    uint32_t amax = 0;
-#pragma unroll
-    for (int k = 0; k < 32; k++) amax = max(amax, bits[k] & 0x7fffffffu);
-    nonfinite = amax >= 0x7f800000u;
-    uint32_t eadj = max(amax >> 23, 2u);
-    Scaler sc(eadj);
-    uint32_t m5 = sc.q5(amax);
-    uint32_t max_hu = min(15u, (m5 + 1u) >> 1);
-    uint32_t pair = min(7u, 15u - max_hu);                       // pair maxima are 15 - pair
-    const uint32_t above = tab.merged_above[pair];
-    uint32_t v[4] = {0, 0, 0, 0}, signs[4] = {0, 0, 0, 0};
-#pragma unroll
-    for (int k = 0; k < 32; k++) {
-        const uint32_t q = sc.q5(bits[k] & 0x7fffffffu);
-        v[k / 8] += (uint32_t)__popc(above >> q) << (4 * slot_of(k % 8));
-        signs[k / 8] |= (bits[k] >> 31) << sign_bit_of_slot(slot_of(k % 8));
-    }
-    BlockResult r;
-    r.scale = eadj - 2u;                                         // (eadj - 129) + 127
-    finish_two_stage(v, signs, pair, r.id, r.words);
-    return r;
-}
-
 // Exact-MSE rule (Sec. 3.2 first paragraph; Sec. 4.3): all 16 dialects, squared
 // error against the untruncated scaled magnitude, fp64, element order, no
 // contraction; the lowest id wins equal sums.
@@ -661,7 +635,8 @@ __global__ void __launch_bounds__(256) quantize_strided_kernel(const void *__res
             for (int k = 0; k < 32; k++)
                 bits[k] = Loader<DT>::one((const char *)X + (((int64_t)b * 32 + k) * ld + r) * Loader<DT>::kElemBytes);
             bool nonfinite;
-            res = quantize_two_stage(bits, tab, nonfinite);
+            uint32_t unused[8];
+            quantize_two_stage_f32<false>(bits, tab, res, unused, nonfinite);
             if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
             *(uint4 *)(out.codes + r * (out.K / 2) + (int64_t)b * 16) =
                 make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
