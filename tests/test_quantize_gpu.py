@@ -108,6 +108,34 @@ def test_bf16_blocks_at_the_exponent_clamp():
     bd.poll_status()
 
 
+@pytest.mark.parametrize("kind", [torch.bfloat16, torch.float32, torch.float16])
+def test_random_bit_patterns_every_finite_exponent(kind):
+    # inputs drawn as bit patterns, so that every exponent (subnormals and the top of the range included) and every
+    # mantissa meets the quantizer; row i keeps its exponents within a window that moves with i, so that blocks
+    # at the clamp, blocks of one exponent and blocks spanning many all occur.  Inf and NaN are left out.
+    rng = np.random.default_rng(23)
+    rows, K = 192, 256
+    if kind == torch.float32:
+        ebits, mbits, word = 8, 23, np.uint32
+    elif kind == torch.bfloat16:
+        ebits, mbits, word = 8, 7, np.uint16
+    else:
+        ebits, mbits, word = 5, 10, np.uint16
+    top = (1 << ebits) - 1                                        # the exponent field of Inf / NaN
+    lo = (np.arange(rows) * (top - 1) // rows)[:, None]           # window start per row
+    width = rng.integers(1, 12, (rows, 1))
+    lo[:8, 0] = [0, 0, 0, 1, 0, 1, 0, 2]                          # the first rows sit at and below the exponent clamp
+    width[:8, 0] = [1, 2, 3, 2, 4, 3, 5, 1]
+    exp = np.minimum(lo + rng.integers(0, 1 << 30, (rows, K)) % width, top - 1)
+    man = rng.integers(0, 1 << mbits, (rows, K))
+    sign = rng.integers(0, 2, (rows, K))
+    bits = ((sign << (ebits + mbits)) | (exp << mbits) | man).astype(word)
+    host = bits.view(np.float32) if kind == torch.float32 else bits
+    q = bd.quantize_act(to_device(host, kind))
+    assert_bit_exact(q, oracle_quantize(host, kind), f"bit patterns {kind}")
+    bd.poll_status()
+
+
 def test_leading_dimension_and_output_guard_bands():
     rng = np.random.default_rng(5)
     big = rng.standard_normal((40, 512)).astype(np.float32)
