@@ -85,7 +85,7 @@ bd_status launch_contig(const void *X, bd_dtype dt, int64_t ld, const QView &out
     const unsigned gen_grid = std::min(chunks, quant_bf16_grid_limit());
     const int kgs = nb_pad / kBlocksPerAtom;
     const FastDiv div_kgs = make_fast_div((uint32_t)kgs);
-    const bool regular = out.rows % 64 == 0 && nb % kBlocksPerAtom == 0;
+    const bool regular = out.rows % kRowTile == 0 && nb % kBlocksPerAtom == 0;
     switch (dt) {
         case BD_F32: {
             static bool configured[64] = {};                      // per instantiation and device

@@ -398,7 +398,8 @@ __device__ __forceinline__ void quantize_bf16_block(const uint32_t (&Rin)[16], c
 // The loop of one warp over its share of the chunks' eight warp-parts (warp-part wp = 8 * chunk + w, w the
 // warp's place in the chunk): parts first, first + stride, ...  Two register sets take turns, so the
 // prefetched part is never copied.  Every lane of the warp must call this (shuffles).
-// REGULAR: rows is a multiple of 64 and K a multiple of 128, so no chunk has padding rows or blocks.
+// REGULAR: rows is a multiple of 128 (a chunk takes its 64 rows from all four quarters of a 128-row tile) and
+// K a multiple of 128, so no chunk has padding rows or blocks.
 template <bool WRITE_CODES, bool WRITE_E4M3, bool REGULAR>
 __device__ __forceinline__ void quantize_bf16_parts(const uint16_t *__restrict__ X, int64_t ld, const QView &out,
                                                     uint8_t *__restrict__ e4m3, const SmemTables &tab, uint32_t first,
@@ -503,7 +504,8 @@ __global__ void __launch_bounds__(256, BD_QUANT_MIN_BLOCKS) quantize_bf16_kernel
 // plain [rows][K] byte matrix, the form the tensor-core GEMM loads.
 // ---------------------------------------------------------------------------
 constexpr int kContigStageBytes = 2 * 8 * 4096;               // two buffers of 4 KiB per warp
-// REGULAR: rows is a multiple of 64 and K a multiple of 128, so no chunk has padding rows or blocks.
+// REGULAR: rows is a multiple of 128 (a chunk takes its 64 rows from all four quarters of a 128-row tile) and
+// K a multiple of 128, so no chunk has padding rows or blocks.
 template <int DT, int SELECT, bool WRITE_CODES, bool WRITE_E4M3, bool REGULAR>
 __global__ void __launch_bounds__(256) quantize_contig_kernel(const void *__restrict__ X, int64_t ld, QView out,
                                                               uint8_t *__restrict__ e4m3, int nb, int kgroups, uint32_t chunks,

@@ -31,7 +31,9 @@ def test_activation_bandwidth_workload_full_size():
     bd.poll_status()
 
 
-@pytest.mark.parametrize("rows,K", [(1, 32), (3, 96), (127, 160), (129, 4096), (300, 352), (16, 11008)])
+@pytest.mark.parametrize("rows,K", [(1, 32), (3, 96), (127, 160), (129, 4096), (300, 352), (16, 11008),
+                                    # whole chunks of 64 rows that do not fill a 128-row tile
+                                    (64, 256), (192, 128), (320, 512)])
 @pytest.mark.parametrize("kind", [torch.float32, torch.bfloat16, torch.float16])
 def test_ragged_shapes_and_dtypes(rows, K, kind):
     rng = np.random.default_rng(rows * 7919 + K)
