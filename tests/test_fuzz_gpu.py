@@ -1,0 +1,121 @@
+"""Seeded sweeps of shapes through the quantizers and the linear layer against the CPU oracle.  Every output
+and the workspace sit between pattern-filled guard bands, so a store outside a buffer shows as a changed guard
+byte even where it would not change a result."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2501_01144_b200 as bd
+from paper_2501_01144_b200 import inputs
+from util import assert_bit_exact, gemm_tolerance_ok, to_device
+
+pytestmark = pytest.mark.gpu
+
+GUARD = 4096
+EDGES = [1, 15, 16, 17, 31, 32, 33, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 320, 384, 448, 512]
+
+
+@pytest.fixture(autouse=True)
+def _reset_impl():
+    yield
+    bd.set_gemm_impl(bd.GEMM_AUTO)
+
+
+def _guarded(n_bytes):
+    raw = torch.full((n_bytes + 2 * GUARD,), 0xA5, dtype=torch.uint8, device="cuda")
+    return raw, raw[GUARD:GUARD + n_bytes]
+
+
+def _intact(raw, n_bytes):
+    return bool((raw[:GUARD] == 0xA5).all()) and bool((raw[GUARD + n_bytes:] == 0xA5).all())
+
+
+def _host(x, kind):
+    if kind == torch.float32:
+        return x, oracle.F32
+    if kind == torch.bfloat16:
+        return inputs.to_bf16_bits(x), oracle.BF16
+    return inputs.to_f16_bits(np.clip(x, -6e4, 6e4)), oracle.F16
+
+
+def _quantizer_cases():
+    rng = np.random.default_rng(101)
+    kinds = [torch.bfloat16, torch.float32, torch.float16]
+    cases = []
+    for i in range(36):
+        rows = int(rng.choice(EDGES)) if i % 3 else int(rng.integers(1, 520))
+        K = 32 * int(rng.choice([1, 2, 3, 4, 5, 8, 12, 16, 17, 32]) if i % 2 else rng.integers(1, 48))
+        cases.append((rows, K, kinds[i % 3], int(rng.choice([0, 32, 64])), int(i % 5 == 4)))
+    return cases
+
+
+@pytest.mark.parametrize("rows,K,kind,ld_extra,mse", _quantizer_cases())
+def test_quantizer_shapes_with_guard_bands(rows, K, kind, ld_extra, mse):
+    rng = np.random.default_rng(rows * 131 + K)
+    x = (rng.standard_t(4, (rows, K)) * np.exp2(rng.integers(-8, 9, (rows, 1)))).astype(np.float32)
+    host, odt = _host(x, kind)
+    wide = torch.zeros(rows, K + ld_extra, dtype=kind, device="cuda")
+    wide[:, :K] = to_device(host, kind)
+    q = bd.QTensor(rows, K)
+    raws = {}
+    for name in ("codes", "ids", "scales"):
+        n = getattr(q, name).numel()
+        raws[name], view = _guarded(n)
+        setattr(q, name, view)
+    if mse:
+        bd.quantize_weights(wide[:, :K], bd.SELECT_MSE, out=q)
+        ref = oracle.quantize(host, oracle.SELECT_MSE, dtype=odt)
+    else:
+        bd.quantize_act(wide[:, :K], out=q)
+        ref = oracle.quantize(host, dtype=odt)
+    assert_bit_exact(q, ref, f"{rows}x{K} {kind} ld+{ld_extra} mse={mse}")
+    for name, raw in raws.items():
+        assert _intact(raw, raw.numel() - 2 * GUARD), f"{name}: write outside the buffer"
+    bd.poll_status()
+
+
+def _linear_cases():
+    rng = np.random.default_rng(202)
+    cases = []
+    for i in range(30):
+        M = int(rng.choice(EDGES)) if i % 2 else int(rng.integers(1, 300))
+        N = int(rng.choice([8, 127, 128, 129, 255, 256, 257, 384])) if i % 3 == 0 else int(rng.integers(8, 400))
+        K = 32 * int(rng.integers(1, 33))
+        cases.append((M, N, K, [torch.bfloat16, torch.float32, torch.float16][i % 3], i % 2))
+    return cases
+
+
+@pytest.mark.parametrize("M,N,K,kind,forced", _linear_cases())
+def test_linear_shapes_with_guard_bands(M, N, K, kind, forced):
+    rng = np.random.default_rng(M * 7 + N * 131 + K)
+    x = (rng.standard_t(4, (M, K)) * np.exp2(rng.integers(-4, 5, (M, 1)))).astype(np.float32)
+    host, odt = _host(x, kind)
+    wb = inputs.to_bf16_bits((0.02 * rng.standard_normal((N, K))).astype(np.float32))
+    Wq = bd.quantize_weights(to_device(wb, torch.bfloat16), bd.SELECT_TWO_STAGE)
+    Yref, T = oracle.gemm(oracle.dequantize(*oracle.quantize(host, dtype=odt)),
+                          oracle.dequantize(*oracle.quantize(wb, dtype=oracle.BF16)))
+    if forced:
+        bd.set_gemm_impl(bd.GEMM_TCGEN05)                         # otherwise the library's own choice by shape
+    xd = to_device(host, kind)
+    ws_bytes = bd.linear_workspace_size(M, N, K)
+    for ydt in (torch.float32, torch.bfloat16):
+        esz = 4 if ydt == torch.float32 else 2
+        ldy = N + 8
+        raw_y, ybytes = _guarded(M * ldy * esz)
+        y = ybytes.view(ydt).view(M, ldy)
+        y.fill_(-7.0)
+        raw_ws, ws = _guarded(ws_bytes)
+        bd.linear(xd, Wq, out=y[:, :N], workspace=ws)
+        torch.cuda.synchronize()
+        assert _intact(raw_y, M * ldy * esz) and _intact(raw_ws, ws_bytes), "write outside a buffer"
+        assert (y[:, N:] == -7.0).all(), "write into the padding columns"
+        got = y[:, :N].float().cpu().numpy()
+        if ydt == torch.float32:
+            ok, ratio = gemm_tolerance_ok(got, Yref, T)
+        else:
+            err = np.abs(got.astype(np.float64) - Yref)
+            bound = 1e-6 * T + 2.0 ** -8 * np.abs(Yref) + 2.0 ** -120
+            ok, ratio = bool((err <= bound).all()), float((err / bound).max())
+        assert ok, f"{M}x{N}x{K} {kind} -> {ydt}: max err / bound = {ratio}"
+    bd.poll_status()

@@ -222,8 +222,9 @@ def test_linear_source_types_pitches_and_ragged_shapes(kind, M, N, K):
 
 
 def test_two_streams_of_decode_sized_calls_do_not_disturb_each_other():
-    # calls whose K is cut over several clusters keep arrival counters in device memory and start before the
-    # kernel ahead of them has finished; two streams of them, interleaved, must give what each gives alone
+    # calls whose K is cut over several clusters keep their partial sums in the caller's workspace, run two
+    # kernels each and start before the kernel ahead of them has finished; two streams of them, interleaved,
+    # must give what each gives alone
     rng = np.random.default_rng(77)
     shapes = [(4, 4096, 11008), (16, 520, 4128)]
     work = []
