@@ -119,3 +119,27 @@ def test_linear_shapes_with_guard_bands(M, N, K, kind, forced):
             ok, ratio = bool((err <= bound).all()), float((err / bound).max())
         assert ok, f"{M}x{N}x{K} {kind} -> {ydt}: max err / bound = {ratio}"
     bd.poll_status()
+
+
+@pytest.mark.parametrize("tokens,dim,kind", [(32, 8, torch.bfloat16), (64, 128, torch.float32), (96, 33, torch.float16),
+                                             (320, 128, torch.bfloat16), (4096, 128, torch.bfloat16), (160, 257, torch.float32),
+                                             (1024, 64, torch.float16), (32, 1, torch.bfloat16)])
+def test_token_axis_quantizer_shapes(tokens, dim, kind):
+    # V [tokens, dim] with blocks of 32 along the tokens: equals quantising the transpose along its rows
+    rng = np.random.default_rng(tokens + 977 * dim)
+    v = (rng.standard_normal((tokens, dim)) * np.exp2(rng.integers(-6, 7, (1, dim)))).astype(np.float32)
+    host, odt = _host(v, kind)
+    pad = (-dim) % 8                                              # a row pitch of whole 16 bytes
+    wide = torch.zeros(tokens, dim + pad, dtype=kind, device="cuda")
+    wide[:, :dim] = to_device(host, kind)
+    q = bd.QTensor(dim, tokens)
+    raws = {}
+    for name in ("codes", "ids", "scales"):
+        n = getattr(q, name).numel()
+        raws[name], view = _guarded(n)
+        setattr(q, name, view)
+    bd.quantize_act(wide[:, :dim], axis=bd.AXIS_STRIDED, out=q)
+    assert_bit_exact(q, oracle.quantize(np.ascontiguousarray(host.T), dtype=odt), f"token axis {tokens}x{dim} {kind}")
+    for name, raw in raws.items():
+        assert _intact(raw, raw.numel() - 2 * GUARD), f"{name}: write outside the buffer"
+    bd.poll_status()
