@@ -143,3 +143,33 @@ def test_token_axis_quantizer_shapes(tokens, dim, kind):
     for name, raw in raws.items():
         assert _intact(raw, raw.numel() - 2 * GUARD), f"{name}: write outside the buffer"
     bd.poll_status()
+
+
+@pytest.mark.parametrize("heads,group,S,T_,d", [(4, 2, 128, 96, 64), (6, 3, 256, 200, 160), (8, 4, 384, 130, 32),
+                                                (3, 1, 100, 257, 96), (4, 4, 128, 512, 128), (2, 2, 130, 64, 64)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_batched_grouped_products(heads, group, S, T_, d, dtype):
+    # queries [heads][S, d] against keys [heads / group][T_, d]: stacked launches where the rows are whole tiles
+    # (S a multiple of 128), one launch per product otherwise; every head against the oracle, guard bands around
+    # the result and the workspace
+    rng = np.random.default_rng(heads + 31 * S + 977 * d)
+    q = inputs.to_bf16_bits(rng.standard_normal((heads, S, d)).astype(np.float32))
+    k = inputs.to_bf16_bits(rng.standard_normal((heads // group, T_, d)).astype(np.float32))
+    As = [bd.quantize_act(to_device(q[h], torch.bfloat16)) for h in range(heads)]
+    Bs = [bd.quantize_act(to_device(k[g], torch.bfloat16)) for g in range(heads // group)]
+    bd.set_gemm_impl(bd.GEMM_TCGEN05)
+    esz = 4 if dtype == torch.float32 else 2
+    raw_y, ybytes = _guarded(heads * S * T_ * esz)
+    out = ybytes.view(dtype).view(heads, S, T_)
+    ws_bytes = bd.gemm_batched_workspace_size(S, T_, d, group)
+    raw_ws, ws = _guarded(ws_bytes)
+    bd.gemm_batched(As, Bs, b_group=group, out=out, workspace=ws)
+    torch.cuda.synchronize()
+    assert _intact(raw_y, heads * S * T_ * esz) and _intact(raw_ws, ws_bytes), "write outside a buffer"
+    for h in range(heads):
+        Yref, T = oracle.gemm(oracle.dequantize(*oracle.quantize(q[h], dtype=oracle.BF16)),
+                              oracle.dequantize(*oracle.quantize(k[h // group], dtype=oracle.BF16)))
+        err = np.abs(out[h].float().cpu().numpy().astype(np.float64) - Yref)
+        bound = 1e-6 * T + (2.0 ** -8 * np.abs(Yref) if dtype == torch.bfloat16 else 0.0) + 2.0 ** -120
+        assert (err <= bound).all(), f"head {h}: max err / bound = {float((err / bound).max())}"
+    bd.poll_status()
