@@ -173,3 +173,41 @@ def test_batched_grouped_products(heads, group, S, T_, d, dtype):
         bound = 1e-6 * T + (2.0 ** -8 * np.abs(Yref) if dtype == torch.bfloat16 else 0.0) + 2.0 ** -120
         assert (err <= bound).all(), f"head {h}: max err / bound = {float((err / bound).max())}"
     bd.poll_status()
+
+
+@pytest.mark.parametrize("M,N,K", [(1280, 3840, 256),      # 75 tiles: one more than the clusters of a round
+                                   (768, 9472, 128),       # 111 tiles: a last round half full (128-token items)
+                                   (1792, 4096, 160),      # 112 tiles: a last round just over half full
+                                   (1700, 5376, 128),      # 147 tiles, ragged last token tile
+                                   (1536, 6400, 96),       # 150 tiles: two items into the third round
+                                   (2304, 1000, 256),      # ragged weight rows, nine token tiles
+                                   (640, 19200, 64)])      # many weight-row pairs, few token tiles
+def test_schedules_over_several_rounds(M, N, K):
+    # tile counts around whole and half rounds of the persistent kernel; sampled rows and columns (tile edges
+    # included) against the oracle, and the bf16 output must be the rounded fp32 one
+    rng = np.random.default_rng(M + 31 * N + K)
+    xb = inputs.to_bf16_bits((rng.standard_t(4, (M, K))).astype(np.float32))
+    wb = inputs.to_bf16_bits((0.02 * rng.standard_normal((N, K))).astype(np.float32))
+    Wq = bd.quantize_weights(to_device(wb, torch.bfloat16), bd.SELECT_TWO_STAGE)
+    xd = to_device(xb, torch.bfloat16)
+    Y32 = bd.linear(xd, Wq, dtype=torch.float32)
+    Y = Y32.cpu().numpy()
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, M - 129, M - 128, M - 1], rng.choice(M, 6, replace=False)]))
+    cols = np.unique(np.concatenate([[0, 127, 128, 255, 256, N - 257, N - 256, N - 1], rng.choice(N, 6, replace=False)]))
+    wdq = oracle.dequantize(*oracle.quantize(wb, dtype=oracle.BF16))
+    Yref, T = oracle.gemm(oracle.dequantize(*oracle.quantize(xb[rows], dtype=oracle.BF16)), wdq)
+    ok, ratio = gemm_tolerance_ok(Y[rows], Yref, T)
+    assert ok, f"rows: max err / bound = {ratio}"
+    Yref, T = oracle.gemm(oracle.dequantize(*oracle.quantize(xb, dtype=oracle.BF16)), wdq[cols])
+    ok, ratio = gemm_tolerance_ok(Y[:, cols], Yref, T)
+    assert ok, f"cols: max err / bound = {ratio}"
+    assert torch.equal(bd.linear(xd, Wq, dtype=torch.bfloat16), Y32.to(torch.bfloat16))
+    # every element, against the library's other product kernel (CUDA cores, exact block sums, fp64 across
+    # blocks): the two share no code path after the quantizer, so a tile one of them misses shows here
+    bd.set_gemm_impl(bd.GEMM_SIMT)
+    Yexact = bd.linear(xd, Wq, dtype=torch.float32)
+    Aabs = bd.dequantize(bd.quantize_act(xd)).abs()
+    Wabs = bd.dequantize(Wq).abs()
+    bound = 2e-6 * (Aabs @ Wabs.T) + 2.0 ** -120
+    assert bool(((Y32 - Yexact).abs() <= bound).all())
+    bd.poll_status()
