@@ -44,6 +44,14 @@ def test_llama3_linear_layers_m2048(K, N):
     # bf16 output (what the benchmark times) is the rounded fp32 result
     Y16 = bd.linear(to_device(xb, torch.bfloat16), Wq, dtype=torch.bfloat16)
     assert torch.equal(Y16.cpu(), torch.from_numpy(Y).to(torch.bfloat16))
+    # every element against the library's CUDA-core product (exact block sums, fp64 across blocks), which
+    # shares no code with the tensor-core kernel after the quantizer
+    xd = to_device(xb, torch.bfloat16)
+    bd.set_gemm_impl(bd.GEMM_SIMT)
+    Yexact = bd.linear(xd, Wq, dtype=torch.float32)
+    bd.set_gemm_impl(bd.GEMM_AUTO)
+    bound = 2e-6 * (bd.dequantize(bd.quantize_act(xd)).abs() @ bd.dequantize(Wq).abs().T) + 2.0 ** -120
+    assert bool(((torch.from_numpy(Y).cuda() - Yexact).abs() <= bound).all())
     bd.poll_status()
 
 
