@@ -64,3 +64,60 @@ def test_alternative_formatbook_end_to_end():
     after = bd.export_canonical(bd.quantize_act(x))
     assert all(torch.equal(a, b) for a, b in zip(before, after))
     bd.poll_status()
+
+
+def _random_book(rng):
+    """A table with the pair structure the library asks for: pair p has maximum 15 - p, its two rows share the
+    six smallest values and differ in the seventh (the even row's is the larger)."""
+    book = np.zeros((16, 8), np.uint8)
+    for p in range(8):
+        mx = 15 - p
+        while True:
+            picks = np.sort(rng.choice(np.arange(1, mx), 7, replace=False))
+            common, d_odd, d_even = picks[:5], picks[5], picks[6]
+            if d_even < mx:
+                break
+        book[2 * p] = [0, *common, d_even, mx]
+        book[2 * p + 1] = [0, *common, d_odd, mx]
+    return book
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_formatbooks(seed):
+    # tables drawn at random within the structure the kernels assume (those the library's own check refuses are
+    # drawn again): quantizer in both output forms, MSE rule and both product kernels against the oracle with
+    # the same table
+    rng = np.random.default_rng(500 + seed)
+    M, K, N = 130, 512, 200
+    xb = inputs.to_bf16_bits((rng.standard_t(4, (M, K)) * np.exp2(rng.integers(-3, 4, (M, 1)))).astype(np.float32))
+    xf = (rng.standard_normal((M, K)) * 3).astype(np.float32)
+    wb = inputs.to_bf16_bits((0.05 * rng.standard_normal((N, K))).astype(np.float32))
+    try:
+        for _ in range(200):
+            book = _random_book(rng)
+            try:
+                bd.set_formatbook(book)
+                break
+            except bd.BdError:
+                continue
+        else:
+            pytest.skip("no acceptable table drawn")
+        oracle.set_formatbook(book)
+        x, w = to_device(xb, torch.bfloat16), to_device(wb, torch.bfloat16)
+        ref_x = oracle_quantize(xb, torch.bfloat16)
+        assert_bit_exact(bd.quantize_act(x), ref_x, "bf16 activations")
+        assert_bit_exact(bd.quantize_act(to_device(xf, torch.float32)), oracle_quantize(xf, torch.float32), "fp32 activations")
+        assert_bit_exact(bd.quantize_weights(w, bd.SELECT_MSE), oracle_quantize(wb, torch.bfloat16, oracle.SELECT_MSE), "MSE")
+        ref_w = oracle_quantize(wb, torch.bfloat16)
+        Wq = bd.quantize_weights(w, bd.SELECT_TWO_STAGE)
+        assert_bit_exact(Wq, ref_w, "weights")
+        Yref, T = oracle.gemm(oracle.dequantize(*ref_x), oracle.dequantize(*ref_w))
+        for impl in (bd.GEMM_SIMT, bd.GEMM_TCGEN05):
+            bd.set_gemm_impl(impl)
+            ok, ratio = gemm_tolerance_ok(bd.linear(x, Wq, dtype=torch.float32).cpu().numpy(), Yref, T)
+            assert ok, f"impl {impl}: max err / bound = {ratio}"
+    finally:
+        bd.set_gemm_impl(bd.GEMM_AUTO)
+        bd.set_formatbook(None)
+        oracle.set_formatbook(None)
+    bd.poll_status()
