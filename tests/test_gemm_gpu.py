@@ -244,3 +244,34 @@ def test_two_streams_of_decode_sized_calls_do_not_disturb_each_other():
             for x, wq, ws, alone, out, stream in work:
                 assert torch.equal(out, alone), f"iteration {it}"
     bd.poll_status()
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 4096, 4096), (16, 520, 4128), (300, 264, 512)])
+def test_linear_calls_replay_from_a_cuda_graph(M, N, K):
+    # after one eager call (which sets function attributes and queries the device) the calls are plain kernel
+    # launches on the given stream: a captured graph of them, dependent-launch edges included, replays to the
+    # same bits, on new inputs written into the captured buffers
+    rng = np.random.default_rng(M + N + K)
+    x = to_device(inputs.to_bf16_bits(rng.standard_normal((M, K)).astype(np.float32)), torch.bfloat16)
+    x2 = to_device(inputs.to_bf16_bits((3 * rng.standard_normal((M, K))).astype(np.float32)), torch.bfloat16)
+    wq = bd.quantize_weights(to_device(inputs.to_bf16_bits((0.02 * rng.standard_normal((N, K))).astype(np.float32)),
+                                       torch.bfloat16), bd.SELECT_TWO_STAGE)
+    ws = torch.empty(bd.linear_workspace_size(M, N, K), dtype=torch.uint8, device="cuda")
+    y = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+    expected = [bd.linear(t, wq, workspace=ws).clone() for t in (x, x2)]
+    xin = x.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(3):
+                bd.linear(xin, wq, out=y, workspace=ws, stream=side)
+    torch.cuda.synchronize()
+    for src, exp in zip((x, x2), expected):
+        xin.copy_(src)
+        y.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(y, exp)
+    bd.poll_status()
