@@ -128,7 +128,15 @@ bd_status bd_gemm_batched(const bd_qtensor *A, const bd_qtensor *B, int64_t batc
                           size_t workspace_bytes, void *stream);
 
 /* The quantised linear layer: quantise X [M,K] online (two-stage rule), then
- * Y = dq(X) * dq(Wq)^T.  The quantised activation lives only in `workspace`. */
+ * Y = dq(X) * dq(Wq)^T.  The quantised activation lives only in `workspace`.
+ * The call is two or three kernel launches on `stream` (quantizer, product, and for
+ * short calls with few weight rows a kernel that adds partial sums kept in the
+ * workspace), linked by programmatic dependent launch: each starts while its
+ * predecessor drains and waits for it before touching its results; work queued
+ * behind the call in the usual way sees it complete.  After one call per device
+ * (which sets function attributes) further calls can be captured into a CUDA graph.
+ * Wq must not be written by the kernel immediately before the call in the stream
+ * unless that kernel is one of this library's. */
 bd_status bd_linear_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes);
 bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx,
                     const bd_qtensor *Wq, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace,
