@@ -134,9 +134,7 @@ bd_status bd_gemm_batched(const bd_qtensor *A, const bd_qtensor *B, int64_t batc
  * workspace), linked by programmatic dependent launch: each starts while its
  * predecessor drains and waits for it before touching its results; work queued
  * behind the call in the usual way sees it complete.  After one call per device
- * (which sets function attributes) further calls can be captured into a CUDA graph.
- * Wq must not be written by the kernel immediately before the call in the stream
- * unless that kernel is one of this library's. */
+ * (which sets function attributes) further calls can be captured into a CUDA graph. */
 bd_status bd_linear_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes);
 bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx,
                     const bd_qtensor *Wq, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace,
