@@ -505,6 +505,7 @@ def run_gpu(args, rank, world, local_rank):
 def run_case(args):
     """A few launches of one kernel family on a small, fixed case (for ncu captures).
     quantizer: bd_quantize_act on bf16 [8192, 4096] (168 MiB of buffers in rotation).
+    quantizer_f32: bd_quantize_act on fp32 [4096, 4096] (three buffer sets in rotation).
     linear_<layer>: bd_linear of one LLaMA3-8B layer at M = 2048 (layer in qo_proj, kv_proj, gate_up, down)."""
     import torch
 
@@ -534,6 +535,23 @@ def run_case(args):
         us = e0.elapsed_time(e1) / reps * 1e3
         print(json.dumps({"case": args.case, "us_per_launch": us,
                           "GB/s": qm * qk * BYTES_PER_ELEM_QUANT / us / 1e3}))
+        return
+    if args.case == "quantizer_f32":
+        # fp32 source (the attention probabilities of the PV product): [4096, 4096], three buffer sets in rotation
+        g = torch.Generator(device=dev)
+        g.manual_seed(1)
+        xs = [torch.rand(4096, 4096, device=dev, generator=g) for _ in range(3)]
+        qs = [bd.QTensor(4096, 4096, dev) for _ in range(3)]
+        for i in range(args.warmup):
+            bd.quantize_act(xs[i % 3], out=qs[i % 3])
+        torch.cuda._sleep(4_000_000)
+        e0.record()
+        for i in range(reps):
+            bd.quantize_act(xs[i % 3], out=qs[i % 3])
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        print(json.dumps({"case": args.case, "us_per_launch": us, "GB/s": 4096 * 4096 * 4.546875 / us / 1e3}))
         return
     if args.case == "step":
         # the benchmark step alone: the four layers through bd_linear, nothing else on the GPU
@@ -576,7 +594,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--case", default=None,
-                    choices=["quantizer", "step"] + ["linear_" + n for n, _, _ in LAYERS],
+                    choices=["quantizer", "quantizer_f32", "step"] + ["linear_" + n for n, _, _ in LAYERS],
                     help="run a few launches of one small case (for profiler captures) instead of the benchmark")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
