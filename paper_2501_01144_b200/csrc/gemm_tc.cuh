@@ -180,7 +180,7 @@ static_assert(Smem::total <= 227 * 1024, "shared memory budget");
 // Tiles are numbered with the token tile running fastest (token tile = tile % t_tiles, weight-row pair =
 // tile / t_tiles), so the clusters that run at the same time share weight rows and differ in their tokens.
 // Items [0, split_from) are whole tiles of 256 tokens.  Each later tile is cut into `parts` items of
-// `part_tokens` tokens: two of 128, which lets a last, sparsely filled round of tiles spread over twice as
+// `part_tokens` tokens: two of 128, which lets a last, sparsely filled wave of tiles spread over twice as
 // many clusters; or, when the whole problem has at most 128 tokens, one item of just those tokens (rounded up
 // to the MMA's step of 16), so that a decode-sized call does not pay for 256 columns per k-step.
 // A call of at most 128 tokens has few tiles (one per 256 weight rows); with k_splits > 1 each is further cut
@@ -756,7 +756,7 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
             sc.k_splits = (sc.k_tiles + sc.k_per - 1) / sc.k_per;      // no empty split
         }
     } else {
-        // a last round that fills at most half of the clusters is cut into 128-token items (twice as many, half
+        // a last wave (one tile per cluster) that fills at most half of the clusters is cut into 128-token items (twice as many, half
         // as long), unless the second half of the last token tile would be empty
         const int rest = tiles % resident, m_tail = (int)(M % 256);
         if (rest > 0 && 2 * rest <= resident && (m_tail == 0 || m_tail > 128)) sc.split_from = tiles - rest;

@@ -175,15 +175,15 @@ def test_batched_grouped_products(heads, group, S, T_, d, dtype):
     bd.poll_status()
 
 
-@pytest.mark.parametrize("M,N,K", [(1280, 3840, 256),      # 75 tiles: one more than the clusters of a round
-                                   (768, 9472, 128),       # 111 tiles: a last round half full (128-token items)
-                                   (1792, 4096, 160),      # 112 tiles: a last round just over half full
+@pytest.mark.parametrize("M,N,K", [(1280, 3840, 256),      # 75 tiles: one more than the clusters of a wave
+                                   (768, 9472, 128),       # 111 tiles: a last wave half full (128-token items)
+                                   (1792, 4096, 160),      # 112 tiles: a last wave just over half full
                                    (1700, 5376, 128),      # 147 tiles, ragged last token tile
-                                   (1536, 6400, 96),       # 150 tiles: two items into the third round
+                                   (1536, 6400, 96),       # 150 tiles: two items into the third wave
                                    (2304, 1000, 256),      # ragged weight rows, nine token tiles
                                    (640, 19200, 64)])      # many weight-row pairs, few token tiles
-def test_schedules_over_several_rounds(M, N, K):
-    # tile counts around whole and half rounds of the persistent kernel; sampled rows and columns (tile edges
+def test_schedules_over_several_waves(M, N, K):
+    # tile counts near whole and half waves of the persistent kernel (a wave = one tile per cluster); sampled rows and columns (tile edges
     # included) against the oracle, and the bf16 output must be the rounded fp32 one
     rng = np.random.default_rng(M + 31 * N + K)
     xb = inputs.to_bf16_bits((rng.standard_t(4, (M, K))).astype(np.float32))
