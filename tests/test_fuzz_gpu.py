@@ -211,3 +211,36 @@ def test_schedules_over_several_waves(M, N, K):
     bound = 2e-6 * (Aabs @ Wabs.T) + 2.0 ** -120
     assert bool(((Y32 - Yexact).abs() <= bound).all())
     bd.poll_status()
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 256, 8192), (5, 300, 2144), (16, 520, 4128), (100, 520, 4128), (128, 1024, 4096),
+                                   (64, 4096, 2048)])
+@pytest.mark.parametrize("ydt", [torch.float32, torch.bfloat16])
+def test_split_k_calls_with_guard_bands(M, N, K, ydt):
+    # short calls against few weight rows: K is cut over several clusters, the partial sums live in the workspace
+    # and a second kernel adds them; guard bands around the workspace and the result, every element against the
+    # oracle
+    rng = np.random.default_rng(M + 31 * N + 977 * K)
+    xb = inputs.to_bf16_bits(rng.standard_t(4, (M, K)).astype(np.float32))
+    wb = inputs.to_bf16_bits((0.02 * rng.standard_normal((N, K))).astype(np.float32))
+    Wq = bd.quantize_weights(to_device(wb, torch.bfloat16), bd.SELECT_TWO_STAGE)
+    Yref, T = oracle.gemm(oracle.dequantize(*oracle.quantize(xb, dtype=oracle.BF16)),
+                          oracle.dequantize(*oracle.quantize(wb, dtype=oracle.BF16)))
+    bd.set_gemm_impl(bd.GEMM_TCGEN05)
+    esz = 4 if ydt == torch.float32 else 2
+    ldy = N + 8
+    raw_y, ybytes = _guarded(M * ldy * esz)
+    y = ybytes.view(ydt).view(M, ldy)
+    y.fill_(-7.0)
+    ws_bytes = bd.linear_workspace_size(M, N, K)
+    raw_ws, ws = _guarded(ws_bytes)
+    before = bd.launch_count()
+    bd.linear(to_device(xb, torch.bfloat16), Wq, out=y[:, :N], workspace=ws)
+    torch.cuda.synchronize()
+    assert bd.launch_count() - before == 3, "expected quantizer, product and the kernel that adds the partial sums"
+    assert _intact(raw_y, M * ldy * esz) and _intact(raw_ws, ws_bytes), "write outside a buffer"
+    assert (y[:, N:] == -7.0).all(), "write into the padding columns"
+    err = np.abs(y[:, :N].float().cpu().numpy().astype(np.float64) - Yref)
+    bound = 1e-6 * T + (2.0 ** -8 * np.abs(Yref) if ydt == torch.bfloat16 else 0.0) + 2.0 ** -120
+    assert (err <= bound).all(), f"max err / bound = {float((err / bound).max())}"
+    bd.poll_status()
