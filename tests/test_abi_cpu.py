@@ -79,6 +79,35 @@ def test_qtensor_sizes_and_argument_errors():
     assert lib.bd_set_gemm_impl(7) == 1 and lib.bd_set_gemm_impl(0) == 0
 
 
+def test_workspace_sizes_follow_the_documented_parts():
+    """Host arithmetic only: the operand bytes of the activations, their scale atoms, and for short calls
+    against few weight rows the fp32 partial sums of a K split."""
+    lib = bd.load()
+    b = ctypes.c_size_t()
+
+    def linear_ws(M, N, K):
+        assert lib.bd_linear_workspace_size(M, N, K, ctypes.byref(b)) == 0
+        return b.value
+
+    def gemm_ws(M, N, K):
+        assert lib.bd_gemm_workspace_size(M, N, K, ctypes.byref(b)) == 0
+        return b.value
+
+    atoms = lambda M, K: ((M + 127) // 128) * ((K // 32 + 3) // 4) * 512
+    # the benchmark's layers: operand bytes + scale atoms, nothing else
+    assert gemm_ws(2048, 14336, 4096) == 2048 * 4096
+    assert linear_ws(2048, 14336, 4096) == atoms(2048, 4096) + 2048 * 4096
+    # up to 128 tokens against at most 37 pairs of 128 weight rows (half of the clusters): room for four splits of
+    # [tokens rounded to 16][weight rows rounded to 256] fp32 partial sums behind the operand bytes
+    assert gemm_ws(16, 4096, 11008) == 16 * 11008 + 4 * 16 * 4096 * 4
+    assert gemm_ws(5, 300, 2144) == 256 * ((5 * 2144 + 255) // 256) + 4 * 16 * 512 * 4
+    assert gemm_ws(128, 9472, 4096) == 128 * 4096 + 4 * 128 * 9472 * 4
+    # more weight rows than that, or more tokens: no split, no scratch
+    assert gemm_ws(16, 11008, 4096) == 16 * 4096
+    assert gemm_ws(128, 9473, 4096) == 128 * 4096
+    assert gemm_ws(129, 4096, 11008) == 256 * ((129 * 11008 + 255) // 256)
+
+
 def test_null_and_misaligned_arguments_rejected_before_any_launch():
     lib = bd.load()
     q = bd.binding._CQTensor(0, 0, 0, 16, 64)
