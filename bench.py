@@ -173,6 +173,59 @@ def run_reference(args, rank):
     print(json.dumps(line))
 
 
+def fp8_dense_probe(dev, n=8192, reps=10):
+    """A dense FP8 yardstick measured in this run: the library GEMM torch._scaled_mm (E4M3 x E4M3 -> bf16,
+    n^3) timed alone, best of `reps`.  It is never on the product path; it only gives the tensor roofline a
+    measured FP8 denominator beside the figure derived from the bf16 peak.  None when the call is unavailable."""
+    import torch
+    try:
+        a = (torch.randn(n, n, device=dev) * 0.5).to(torch.float8_e4m3fn)
+        b = (torch.randn(n, n, device=dev) * 0.5).to(torch.float8_e4m3fn).t()       # column-major second operand
+        one = torch.ones((), device=dev)
+        for _ in range(3):
+            torch._scaled_mm(a, b, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
+        best = None
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            torch._scaled_mm(a, b, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None else min(best, ms)
+        return {"tflops": 2.0 * n ** 3 / (best * 1e-3) / 1e12, "ms": best,
+                "how": f"torch._scaled_mm e4m3 x e4m3 -> bf16, {n}^3, best of {reps}, timed alone (burst)"}
+    except Exception as e:                                  # noqa: BLE001 - a yardstick, not part of the product
+        return {"tflops": None, "how": f"unavailable: {type(e).__name__}: {str(e)[:120]}"}
+
+
+def oracle_quantizer_baseline():
+    """The CPU oracle's two-stage quantizer on the full activation-quantizer workload (bf16 [8192, 4096]),
+    on all host threads and on one, as GB/s of the same algorithmic bytes the GPU figure counts."""
+    import ctypes
+
+    import oracle
+    from paper_2501_01144_b200 import inputs
+    qm, qk = QUANT_SHAPE
+    x = inputs.act_normal_outliers(qm, qk, seed=1)
+    nbytes = qm * qk * BYTES_PER_ELEM_QUANT
+    out = {"workload": "bf16 [8192, 4096], whole tensor", "unit": "GB/s", "kind": "oracle"}
+    threads = oracle.threads()
+    t0 = time.perf_counter()
+    oracle.quantize(x, dtype=oracle.BF16)
+    out["all_threads"] = {"value": nbytes / (time.perf_counter() - t0) / 1e9, "cores": threads}
+    try:
+        gomp = ctypes.CDLL("libgomp.so.1")
+        gomp.omp_set_num_threads(1)
+        t0 = time.perf_counter()
+        oracle.quantize(x, dtype=oracle.BF16)
+        out["one_thread"] = {"value": nbytes / (time.perf_counter() - t0) / 1e9, "cores": 1}
+        gomp.omp_set_num_threads(threads)
+    except OSError:
+        out["one_thread"] = None
+    return out
+
+
 # ---------------------------------------------------------------------------
 # GPU leg
 # ---------------------------------------------------------------------------
@@ -319,12 +372,18 @@ def run_gpu(args, rank, world, local_rank):
     gemm_ms = float(np.mean(durations))
     achieved_tf = big["flops"] / (gemm_ms * 1e-3) / 1e12
     fp8_peak = 2.0 * peaks["bf16_tflops"]                 # dense FP8 = 2 x dense bf16 (nominal ratio), burst: kernel timed alone
+    time.sleep(0.5)
+    fp8_probe = fp8_dense_probe(dev) if rank == 0 else None
+    time.sleep(0.5)                                       # let the clock recover before the other sections
     # DRAM traffic of this launch from the committed ncu capture (profiles/gemm_wtmem_kernel_llama3_gate_up.md)
     roofline = {"bound": "tensor", "kernel": "bd_gemm " + big["name"] + " (decode_e4m3 of the activations + tc::gemm_wtmem_kernel)",
                 "achieved": achieved_tf, "peak": fp8_peak,
                 "unit": "TFLOP/s", "frac": achieved_tf / fp8_peak, "traffic": GEMM_GATE_UP_DRAM_BYTES,
                 "peak_source": f"2 x {peaks['source']} bf16 burst", "ms_per_launch": gemm_ms,
-                "frac_of_nominal_4500": achieved_tf / 4500.0}
+                "frac_of_nominal_4500": achieved_tf / 4500.0,
+                # the same launch against a dense FP8 library GEMM timed in this run (a yardstick only)
+                "fp8_probe": fp8_probe,
+                "frac_of_fp8_probe": (achieved_tf / fp8_probe["tflops"]) if fp8_probe and fp8_probe.get("tflops") else None}
 
     # ---- standalone activation quantizer on bf16 [8192, 4096] (HBM-bound) ----
     qm, qk = QUANT_SHAPE
@@ -357,32 +416,45 @@ def run_gpu(args, rank, world, local_rank):
                              "frac": QUANT_WARP_INSTRUCTIONS / (q_ms * 1e-3) / 1e9 / (SM_COUNT * ISSUE_PER_SM_CLK * 1.965)}}
     bd.poll_status()
 
-    # ---- LLaMA2-7B MLP shapes, decode to prefill (reported per M; not part of the timed step) ----
+    # ---- LLaMA2-7B MLP shapes, decode to prefill (reported per M; not part of the timed step).  Inputs are
+    # the seeded generators the parity tests use (|N| * N products with 1 % outlier channels).  The decode-sized
+    # calls are bound by the weight stream, so the weights rotate over six copies (6 x 24.7 MB > the 126 MB L2):
+    # no call finds its weights in L2. ----
     sweep = []
     if rank == 0:
-        torch.manual_seed(3)
+        n_wsets = 6
         for K, N in MLP_SWEEP:
-            wq = bd.quantize_weights(dev_bf16(inputs.weights_normal(N, K, seed=3)), bd.SELECT_TWO_STAGE)
+            wsrc = dev_bf16(inputs.weights_normal(N, K, seed=3))
+            wqs = [bd.quantize_weights(wsrc, bd.SELECT_TWO_STAGE) for _ in range(n_wsets)]
+            del wsrc
             for M in MLP_SWEEP_M:
-                x = (torch.randn(M, K, device=dev).abs() * torch.randn(M, K, device=dev)).to(torch.bfloat16)
+                x = dev_bf16(inputs.act_post_silu(M, K, seed=3))
                 y = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
                 ws = torch.empty(bd.linear_workspace_size(M, N, K), dtype=torch.uint8, device=dev)
-                for _ in range(3):
-                    bd.linear(x, wq, out=y, workspace=ws)
+                for i in range(n_wsets):
+                    bd.linear(x, wqs[i], out=y, workspace=ws)
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                n_rep = 20
+                n_rep = 24 if M <= 1024 else 6
                 torch.cuda._sleep(2_000_000)                  # GPU head start: the events see kernel time, not launch rate
                 a.record()
-                for _ in range(n_rep):
-                    bd.linear(x, wq, out=y, workspace=ws)
+                for i in range(n_rep):
+                    bd.linear(x, wqs[i % n_wsets], out=y, workspace=ws)
                 b.record()
                 torch.cuda.synchronize()
                 us = a.elapsed_time(b) / n_rep * 1e3
+                # host time of one call (argument checks, tensor-map encoding, launches), GPU idle
+                t0 = time.perf_counter()
+                for i in range(n_rep):
+                    bd.linear(x, wqs[i % n_wsets], out=y, workspace=ws)
+                host_us = (time.perf_counter() - t0) / n_rep * 1e6
+                torch.cuda.synchronize()
                 flops = 2.0 * M * N * K
                 nbytes = N * K * 0.546875 + M * K * 2 + M * N * 2
                 bound_tf = min(2.0 * peaks["bf16_tflops"], flops / nbytes * peaks["hbm_gbs"] / 1e3)
-                sweep.append({"K": K, "N": N, "M": M, "us": us, "tflops": flops / us / 1e6,
-                              "gbs": nbytes / us / 1e3, "frac_of_roofline": flops / us / 1e6 / bound_tf})
+                sweep.append({"K": K, "N": N, "M": M, "us": us, "host_us_per_call": host_us, "tflops": flops / us / 1e6,
+                              "gbs": nbytes / us / 1e3, "floor_us": flops / bound_tf / 1e6,
+                              "frac_of_roofline": flops / us / 1e6 / bound_tf})
+            del wqs
         bd.poll_status()
 
     # ---- attention products with both operands quantised online (Mistral-7B shapes: 32 heads, 8 KV heads,
@@ -391,9 +463,12 @@ def run_gpu(args, rank, world, local_rank):
     attention = None
     if rank == 0:
         heads, kvh, S, hd = 32, 8, 4096, 128
-        torch.manual_seed(4)
-        Aq = [bd.quantize_act(torch.randn(S, hd, device=dev).to(torch.bfloat16)) for _ in range(heads)]
-        Bk = [bd.quantize_act(torch.randn(S, hd, device=dev).to(torch.bfloat16)) for _ in range(kvh)]
+        grp = heads // kvh
+        n_pheads = 3 * grp                                    # probabilities for three KV groups (each head 64 MiB)
+        # the seeded generator of the parity tests: Q/K with head-dim outlier channels, Dirichlet(0.1) rows of P
+        Qb, Kb, Pn, Vb = inputs.attention_case(heads, kvh, S, hd, seed=4, p_heads=n_pheads)
+        Aq = [bd.quantize_act(dev_bf16(Qb[h])) for h in range(heads)]
+        Bk = [bd.quantize_act(dev_bf16(Kb[g])) for g in range(kvh)]
         scores = torch.empty(heads, S, S, dtype=torch.bfloat16, device=dev)          # 1 GiB: L2-cold by size
         gws = torch.empty(max(1, bd.gemm_batched_workspace_size(S, S, hd, heads // kvh)), dtype=torch.uint8, device=dev)
 
@@ -415,9 +490,9 @@ def run_gpu(args, rank, world, local_rank):
         del scores
         # the four query heads of a KV group share V, so their probabilities go through one call as one
         # [4 * 4096, 4096] matrix (contiguous heads): one quantizer launch and one product per group
-        grp = heads // kvh
-        P = [torch.rand(grp * S, S, device=dev) for _ in range(3)]                 # 3 x 256 MiB of fp32 > L2
-        Bv = bd.quantize_act(torch.randn(S, hd, device=dev).to(torch.bfloat16), axis=bd.AXIS_STRIDED)
+        P = [torch.from_numpy(Pn[g * grp:(g + 1) * grp].reshape(grp * S, S)).to(dev) for g in range(3)]   # 3 x 256 MiB > L2
+        del Pn
+        Bv = bd.quantize_act(dev_bf16(Vb[0]), axis=bd.AXIS_STRIDED)
         O = torch.empty(grp * S, hd, dtype=torch.bfloat16, device=dev)
         lws = torch.empty(bd.linear_workspace_size(grp * S, hd, S), dtype=torch.uint8, device=dev)
         turn = [0]
@@ -450,8 +525,9 @@ def run_gpu(args, rank, world, local_rank):
         pv_two_streams(2)
         pv2_us = pv_two_streams(8) / grp
         qk_bytes, pv_bytes = heads * S * S * 2.0, S * S * 4.0
-        attention = {"workload": "QK^T: 32 heads x [4096,128] x [4096,128]^T, bf16 scores; PV: fp32 P [4096,4096] per head "
-                                 "quantised online x V (token-axis blocks) [128,4096]^T, the 4 heads of a KV group per call",
+        attention = {"workload": "QK^T: 32 heads x [4096,128] x [4096,128]^T (head-dim outlier channels), bf16 scores; "
+                                 "PV: fp32 Dirichlet(0.1) rows P [4096,4096] per head quantised online x V (token-axis "
+                                 "blocks) [128,4096]^T, the 4 heads of a KV group per call; seeded generator, seed 4",
                      "qk_us_32_heads": qk_us, "qk_write_gbs": qk_bytes / qk_us / 1e3,
                      "qk_frac_of_hbm": qk_bytes / qk_us / 1e3 / peaks["hbm_gbs"],
                      "write_only_stream_gbs": write_stream_gbs,
@@ -478,7 +554,8 @@ def run_gpu(args, rank, world, local_rank):
             s += ss
             n += 1
         cpu = {"value": f / s / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
-               "sample": f"{n} passes over 16 tokens x 4 layers (quantise + dequantise + fp64 product)"}
+               "sample": f"{n} passes over 16 tokens x 4 layers (quantise + dequantise + fp64 product)",
+               "act_quantizer": oracle_quantizer_baseline()}
 
     line = {
         "metric": "bd_linear_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
@@ -486,7 +563,8 @@ def run_gpu(args, rank, world, local_rank):
         "ms_per_step_best": step_best, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "e4m3 x e4m3 (exact DialectFP4 decode), fp32 accumulate", "data": "synthetic",
         "config": {"workload": "llama3-8b linear layers (q/o, k/v, gate/up, down), M=2048 tokens per GPU, "
-                               "fused online quantise + W4A4 product, bf16 out",
+                               "online two-stage quantise kernel + W4A4 tensor-core product kernel per layer "
+                               "(linked by programmatic dependent launch), bf16 out",
                    "l2": f"working set {footprint / 2**20:.0f} MiB per step cycles through 4 layers (> 126 MB L2)",
                    "weights": "offline two-stage rule", "block": 32},
         "clocks": clocks,
@@ -596,6 +674,19 @@ def run_case(args):
     print(json.dumps({"case": args.case, "us_per_call": us, "TFLOP/s": 2.0 * M_TOKENS * N * K / us / 1e6}))
 
 
+def spawn_ranks(args):
+    """`python bench.py --gpus N` outside torchrun: re-run this file as N ranks of one node (one process per
+    GPU, rendezvous on 127.0.0.1 at a free port).  Rank 0 prints the JSON line; the exit code is the job's."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__),
+           "--gpus", str(args.gpus), "--steps", str(args.steps), "--warmup", str(args.warmup), "--impl", args.impl]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -606,6 +697,9 @@ def main():
                     choices=["quantizer", "quantizer_f32", "step"] + ["linear_" + n for n, _, _ in LAYERS],
                     help="run a few launches of one small case (for profiler captures) instead of the benchmark")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.case:
+        # started as a plain process: start the N ranks here, one per GPU, the way torchrun would
+        sys.exit(spawn_ranks(args))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

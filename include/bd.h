@@ -10,6 +10,13 @@
  * never allocates or frees device memory on these paths: scratch is passed in as
  * `workspace` (sizes from the *_workspace_size calls).  There is no CPU fallback.
  *
+ * Threads: the library keeps a few unsynchronised host-side globals (launch counter,
+ * last CUDA error, implementation choice, per-device caches filled on first use), so
+ * it is NOT thread-safe: serialise calls into it, or make every call from one thread.
+ * bd_get_formatbook reports the table of the last successful bd_set_formatbook of the
+ * process; the device tables are per device, so set the same table on every device
+ * that is used.
+ *
  * The method (arXiv 2501.01144, "BlockDialect"):
  *   - operands are cut into blocks of 32 consecutive elements along the
  *     multiplication dimension K (Sec. 3.1; Appendix "Quantization Dimension");
@@ -108,7 +115,23 @@ bd_status bd_quantize_act(const void *X, bd_dtype dtype, int64_t M, int64_t K, i
 /* Y[M,N] = dq(A)[M,K] * dq(B)[N,K]^T (Sec. 3.3, Fig. 6).  ydtype is BD_F32 or BD_BF16
  * (bf16 = round-to-nearest-even of the fp32 accumulator); ldy = row stride of Y in
  * elements.  workspace: bd_gemm_workspace_size bytes, 256-byte aligned, or NULL when
- * that size is 0. */
+ * that size is 0.
+ *
+ * Accuracy of the fp32 result against the exact product, per output element, with
+ * S = sum_k |a_k| |b_k| over the dequantised operands (bd_gemm, bd_gemm_batched and
+ * bd_linear alike):
+ *   BD_GEMM_SIMT      in-block sums are exact integers and blocks are added in fp64:
+ *                     |err| <= 2^-24 * |y| (the final rounding to fp32) for any input.
+ *   BD_GEMM_TCGEN05   one block-scaled tensor-core instruction per block of 32; each
+ *                     aligns its 32 products and the running fp32 sum to the largest
+ *                     exponent among them, drops bits below 2^-25 of it and truncates
+ *                     the sum to fp32.  When the block scales met along a row of K lie
+ *                     within a factor 2^24 of each other, as activations and weights
+ *                     of a layer do, the result is exact or within about 1e-8 * S;
+ *                     the guaranteed bound for ANY input is (K / 32) * 2^-21 * S (an
+ *                     operand with blocks 2^28 apart and opposite signs gets close to
+ *                     it).  Callers who need 1e-6 * S on such inputs select BD_GEMM_SIMT.
+ *   BD_GEMM_AUTO      picks BD_GEMM_TCGEN05 except for tiny problems; its bound applies. */
 bd_status bd_gemm_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes);
 bd_status bd_gemm(const bd_qtensor *A, const bd_qtensor *B, void *Y, bd_dtype ydtype, int64_t ldy,
                   void *workspace, size_t workspace_bytes, void *stream);
@@ -117,7 +140,8 @@ bd_status bd_gemm(const bd_qtensor *A, const bd_qtensor *B, void *Y, bd_dtype yd
  * independent products; operand b of A uses operand b / b_group of B (grouped-query
  * attention shares one K/V head among b_group query heads).  A points to `batch`
  * descriptors, B to batch / b_group descriptors (host arrays); Y + b * stride_y
- * elements is product b.  All operands of A share one shape, all of B another.
+ * elements is product b.  All operands of A share one shape, all of B another
+ * (checked: BD_ERR_SHAPE otherwise).
  * With a workspace of bd_gemm_batched_workspace_size bytes, results of a group that
  * are contiguous in Y (stride_y == M * ldy) and M a multiple of 128, the b_group
  * products of a group run as one stacked launch; otherwise (any workspace of at

@@ -276,6 +276,8 @@ bd_status bd_gemm_batched(const bd_qtensor *A, const bd_qtensor *B, int64_t batc
     for (int64_t i = 0; i < batch; i++) {
         bd_status s = check_gemm(&A[i], &B[i / b_group], Y, ydtype, ldy);
         if (s) return s;
+        // one shape per side: the stacked route reads A[0]'s row count and K from every operand
+        if (A[i].rows != A[0].rows || A[i].K != A[0].K || B[i / b_group].rows != B[0].rows) return BD_ERR_SHAPE;
     }
     const int ysz = ydtype == BD_F32 ? 4 : 2;
     cudaStream_t st = (cudaStream_t)stream;

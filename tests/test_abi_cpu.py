@@ -124,3 +124,13 @@ def test_null_and_misaligned_arguments_rejected_before_any_launch():
     qb = bd.binding._CQTensor(base, base + 1024, base + 2048, 16, 96)
     assert lib.bd_gemm(ctypes.byref(qa), ctypes.byref(qb), ctypes.c_void_p(base), bd.F32, 16, None, 0, None) == 2
     assert lib.bd_gemm(ctypes.byref(qa), ctypes.byref(qa), ctypes.c_void_p(base), bd.F16, 16, None, 0, None) == 1
+
+
+def test_batched_product_rejects_operands_of_different_shapes():
+    # argument checks come before any launch, so made-up (aligned, non-null) addresses are enough here
+    lib = bd.load()
+    Q = bd.binding._CQTensor
+    a = (Q * 2)(Q(0x1000, 0x2000, 0x3000, 128, 128), Q(0x1000, 0x2000, 0x3000, 64, 128))
+    b = (Q * 1)(Q(0x1000, 0x2000, 0x3000, 256, 128))
+    rc = lib.bd_gemm_batched(a, b, 2, 2, ctypes.c_void_p(0x4000), 0, 256, 128 * 256, None, 0, None)
+    assert rc == 2                                            # BD_ERR_SHAPE: A[1] is shorter than A[0]

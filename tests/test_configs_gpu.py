@@ -67,11 +67,34 @@ def test_llama2_mlp_m_sweep(K, N, M):
     xb = inputs.act_post_silu(M, K, seed=3)
     wb = inputs.weights_normal(N, K, seed=3)
     Wq = bd.quantize_weights(to_device(wb, torch.bfloat16), bd.SELECT_TWO_STAGE)
-    Y = bd.linear(to_device(xb, torch.bfloat16), Wq, dtype=torch.float32).cpu().numpy()
+    xd = to_device(xb, torch.bfloat16)
+    Yd = bd.linear(xd, Wq, dtype=torch.float32)
+    Y = Yd.cpu().numpy()
     rng = np.random.default_rng(M)
-    rows = np.unique(np.concatenate([[0, M - 1], rng.choice(M, min(M, 6), replace=False)]))
-    cols = np.array([0, N - 1, 255, 256]) if M <= 1024 else np.array([], int)
+    # rows and columns at the tile boundaries of the tensor-core kernel (256 tokens x 256 weight rows, items of
+    # 128 tokens) plus random ones: eight or more whole rows and eight or more whole columns at every M
+    edge_rows = [r for r in (0, 127, 128, 255, 256, M - 129, M - 128, M - 1) if 0 <= r < M]
+    rows = np.unique(np.concatenate([edge_rows, rng.choice(M, min(M, 8), replace=False)]))
+    cols = np.unique(np.concatenate([[0, 127, 128, 255, 256, N - 257, N - 256, N - 1], rng.choice(N, 8, replace=False)]))
     _check_rows_cols(Y, xb, wb, rows, cols, f"M={M} K={K} N={N}")
+    if M >= 1024:
+        # 4096 further entries: a random 64 x 64 sub-grid of the result
+        r64, c64 = rng.choice(M, 64, replace=False), rng.choice(N, 64, replace=False)
+        qa = oracle.quantize(xb[r64], dtype=oracle.BF16)
+        qb = oracle.quantize(wb[c64], dtype=oracle.BF16)
+        Yref, T = oracle.gemm(oracle.dequantize(*qa), oracle.dequantize(*qb))
+        ok, ratio = gemm_tolerance_ok(Y[np.ix_(r64, c64)], Yref, T)
+        assert ok, f"M={M} K={K} N={N} sub-grid: max err / bound = {ratio}"
+    # every element against the library's CUDA-core product (exact block sums, fp64 across blocks), which shares
+    # no code with the tensor-core kernel after the quantizer
+    bd.set_gemm_impl(bd.GEMM_SIMT)
+    Yexact = bd.linear(xd, Wq, dtype=torch.float32)
+    bd.set_gemm_impl(bd.GEMM_AUTO)
+    wabs = bd.dequantize(Wq).abs()
+    xabs = bd.dequantize(bd.quantize_act(xd)).abs()
+    for r0 in range(0, M, 2048):                              # the bound in slabs of 2048 tokens
+        bound = 2e-6 * (xabs[r0:r0 + 2048] @ wabs.T) + 2.0 ** -120
+        assert bool(((Yd[r0:r0 + 2048] - Yexact[r0:r0 + 2048]).abs() <= bound).all()), f"tokens from {r0}"
     bd.poll_status()
 
 

@@ -31,6 +31,14 @@ def test_dialect4_and_5_match_printed_values(golden_dialect4):
     assert FB[4][7] == FB[5][7] == int(2 * g["pair_shared_max_real"][0])
 
 
+def test_formatbook_equals_the_stated_reading():
+    # typo guard, not a paper value: the table as this build's reading of Sec. 3.1 states it, row by row
+    from conftest import read_golden
+    g = read_golden("formatbook_reading.txt")
+    for d in range(16):
+        assert list(FB[d]) == g[f"dialect{d}"], f"dialect {d}"
+
+
 def test_formatbook_structure():
     maxima = []
     for p in range(8):
