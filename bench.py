@@ -457,6 +457,60 @@ def run_gpu(args, rank, world, local_rank):
             del wqs
         bd.poll_status()
 
+    # ---- two chained layers (gate/up then down, M = 2048) with and without the requantising epilogue (Sec. 3.3,
+    # last paragraph).  Without: the first layer writes bf16, the second layer's quantizer reads it back.  With: the
+    # first product's epilogue writes the DialectFP4 operand and the second product takes it (its operand bytes are
+    # expanded by a small kernel).  Three copies of both weight matrices in rotation (186 MB > L2). ----
+    chained = None
+    if rank == 0:
+        d0, d1, d2 = 4096, 14336, 4096
+        xs = dev_bf16(inputs.act_student_t(M_TOKENS, d0, seed=2))
+        w1 = dev_bf16(inputs.weights_normal(d1, d0, seed=4))
+        w2 = dev_bf16(inputs.weights_normal(d2, d1, seed=5))
+        sets = [(bd.quantize_weights(w1, bd.SELECT_TWO_STAGE), bd.quantize_weights(w2, bd.SELECT_TWO_STAGE)) for _ in range(3)]
+        del w1, w2
+        h16 = torch.empty(M_TOKENS, d1, dtype=torch.bfloat16, device=dev)
+        hq = bd.QTensor(M_TOKENS, d1, dev)
+        yo = torch.empty(M_TOKENS, d2, dtype=torch.bfloat16, device=dev)
+        ws1 = torch.empty(max(bd.linear_workspace_size(M_TOKENS, d1, d0), bd.linear_requant_workspace_size(M_TOKENS, d1, d0)),
+                          dtype=torch.uint8, device=dev)
+        ws2 = torch.empty(max(bd.linear_workspace_size(M_TOKENS, d2, d1), bd.gemm_workspace_size(M_TOKENS, d2, d1), 1),
+                          dtype=torch.uint8, device=dev)
+
+        def plain(i):
+            a, b = sets[i % 3]
+            bd.linear(xs, a, out=h16, workspace=ws1)
+            bd.linear(h16, b, out=yo, workspace=ws2)
+
+        def fused(i):
+            a, b = sets[i % 3]
+            bd.linear_requant(xs, a, out=hq, workspace=ws1)
+            bd.gemm(hq, b, out=yo, workspace=ws2)
+
+        def time_chain(fn, n_rep=30):
+            for i in range(3):
+                fn(i)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda._sleep(4_000_000)
+            e0.record()
+            for i in range(n_rep):
+                fn(i)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / n_rep * 1e3
+
+        plain_us = time_chain(plain)
+        time.sleep(0.3)
+        fused_us = time_chain(fused)
+        chain_flops = 2.0 * M_TOKENS * (d0 * d1 + d1 * d2)
+        chained = {"workload": "gate/up (4096 -> 14336) then down (14336 -> 4096), M = 2048, bf16 final result",
+                   "bf16_between_us": plain_us, "requantised_between_us": fused_us,
+                   "bf16_between_tflops": chain_flops / plain_us / 1e6, "requantised_between_tflops": chain_flops / fused_us / 1e6,
+                   "speedup": plain_us / fused_us}
+        del sets, h16, hq, yo, ws1, ws2
+        bd.poll_status()
+        time.sleep(0.5)
+
     # ---- attention products with both operands quantised online (Mistral-7B shapes: 32 heads, 8 KV heads,
     # 4096 tokens, head_dim 128; reported, not part of the timed step).  QK^T is bound by the write of the
     # scores, PV by the read of the fp32 probabilities. ----
@@ -583,6 +637,7 @@ def run_gpu(args, rank, world, local_rank):
         "cpu_baseline": cpu,
         "per_layer_gflop": {l["name"]: l["flops"] / 1e9 for l in layers},
         "llama2_mlp_m_sweep": sweep,
+        "chained_layers": chained,
         "attention_mistral7b": attention,
     }
     print(json.dumps(line))

@@ -164,6 +164,25 @@ bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_
                     const bd_qtensor *Wq, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace,
                     size_t workspace_bytes, void *stream);
 
+/* Products whose result stays in DialectFP4 (Sec. 3.3, last paragraph: the accumulated
+ * partial sums are "requantized into 4-bit DialectFP4 format for the next matrix
+ * multiplication").  Instead of Y [M, N] the call writes Yq, the quantised operand
+ * [M rows, N along its K axis] that quantising the fp32 result row by row with the online
+ * two-stage rule (bd_quantize_act, BD_AXIS_CONTIG) would give: bit for bit the same codes,
+ * ids and scales.  N must be a multiple of 32; Yq->rows = M, Yq->K = N.  Yq then feeds the
+ * next layer through bd_gemm / bd_gemm_requant, and no high-precision Y is written.
+ * With more than 128 tokens on the tensor-core route the requantisation runs in the
+ * product kernel's epilogue on the fp32 accumulators; otherwise the fp32 result is parked
+ * in the workspace and the quantizer kernel follows (same result).  The workspace sizes
+ * depend on the implementation chosen with bd_set_gemm_impl: ask after choosing. */
+bd_status bd_linear_requant_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes);
+bd_status bd_linear_requant(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx,
+                            const bd_qtensor *Wq, bd_qtensor *Yq, void *workspace,
+                            size_t workspace_bytes, void *stream);
+bd_status bd_gemm_requant_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes);
+bd_status bd_gemm_requant(const bd_qtensor *A, const bd_qtensor *B, bd_qtensor *Yq, void *workspace,
+                          size_t workspace_bytes, void *stream);
+
 /* bd_linear for callers that can neither allocate device memory nor hand in a
  * workspace (the paper has no counterpart; this is a convenience of the library).
  * Think of code that runs where cudaMalloc is off limits: inside a region whose

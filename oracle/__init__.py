@@ -112,6 +112,16 @@ def quantize(x, select=SELECT_TWO_STAGE, dtype=None):
     return codes, ids, scales
 
 
+def requantize(y):
+    """A product's fp32 result [M, N] back into DialectFP4 for the next product (Sec. 3.3, last paragraph: the
+    accumulated sums are requantised "for the next matrix multiplication").  The paper defines no separate
+    arithmetic for this step: it is the online two-stage rule applied to the result's rows, blocks of 32 along N."""
+    y = np.ascontiguousarray(y)
+    if y.dtype != np.float32:
+        raise TypeError("requantize takes the fp32 result")
+    return quantize(y, SELECT_TWO_STAGE)
+
+
 def dequantize(codes, ids, scales):
     """Canonical (codes, ids, scales) -> fp64 [rows, K] (Sec. 3.3, Fig. 6)."""
     rows, K = codes.shape[0], codes.shape[1] * 2

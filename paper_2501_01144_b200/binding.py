@@ -68,6 +68,10 @@ def load():
     lib.bd_linear_workspace_size.argtypes = [i64, i64, i64, szp]
     lib.bd_linear.argtypes = [vp, ci, i64, i64, i64, qp, vp, ci, i64, vp, sz, vp]
     lib.bd_linear_noalloc.argtypes = [vp, ci, i64, i64, i64, qp, vp, ci, i64, vp]
+    lib.bd_linear_requant_workspace_size.argtypes = [i64, i64, i64, szp]
+    lib.bd_linear_requant.argtypes = [vp, ci, i64, i64, i64, qp, qp, vp, sz, vp]
+    lib.bd_gemm_requant_workspace_size.argtypes = [i64, i64, i64, szp]
+    lib.bd_gemm_requant.argtypes = [qp, qp, qp, vp, sz, vp]
     lib.bd_export_canonical.argtypes = [qp, vp, vp, vp, vp]
     lib.bd_import_canonical.argtypes = [vp, vp, vp, qp, vp]
     lib.bd_dequantize.argtypes = [qp, vp, i64, vp]
@@ -243,6 +247,39 @@ def linear(X, Wq, out=None, dtype=torch.bfloat16, workspace=None, stream=None):
     cw = Wq.c_struct()
     _check(load().bd_linear(ptr, dt, M, K, ld, ctypes.byref(cw), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
                             out.stride(0), wptr, wbytes, _stream(stream)))
+    return out
+
+
+def linear_requant_workspace_size(M, N, K):
+    b = ctypes.c_size_t()
+    _check(load().bd_linear_requant_workspace_size(M, N, K, ctypes.byref(b)))
+    return b.value
+
+
+def gemm_requant_workspace_size(M, N, K):
+    b = ctypes.c_size_t()
+    _check(load().bd_gemm_requant_workspace_size(M, N, K, ctypes.byref(b)))
+    return b.value
+
+
+def linear_requant(X, Wq, out=None, workspace=None, stream=None):
+    """The quantised linear layer with its result requantised for the next product (Sec. 3.3, last
+    paragraph): returns the QTensor [M, N] instead of Y."""
+    ptr, dt, ld = _src(X)
+    M, K = X.shape
+    out = out or QTensor(M, Wq.rows, X.device)
+    workspace, wptr, wbytes = _ws(workspace, linear_requant_workspace_size(M, Wq.rows, K), X.device)
+    cw, cy = Wq.c_struct(), out.c_struct()
+    _check(load().bd_linear_requant(ptr, dt, M, K, ld, ctypes.byref(cw), ctypes.byref(cy), wptr, wbytes, _stream(stream)))
+    return out
+
+
+def gemm_requant(A, B, out=None, workspace=None, stream=None):
+    """dq(A) dq(B)^T requantised along N for the next product (Sec. 3.3, last paragraph)."""
+    out = out or QTensor(A.rows, B.rows, A.codes.device)
+    workspace, wptr, wbytes = _ws(workspace, gemm_requant_workspace_size(A.rows, B.rows, A.K), A.codes.device)
+    ca, cb, cy = A.c_struct(), B.c_struct(), out.c_struct()
+    _check(load().bd_gemm_requant(ctypes.byref(ca), ctypes.byref(cb), ctypes.byref(cy), wptr, wbytes, _stream(stream)))
     return out
 
 

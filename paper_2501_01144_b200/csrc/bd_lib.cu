@@ -375,6 +375,107 @@ bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_
     return gemm_dispatch(view_of(&xq), view_of(Wq), Y, ydtype, ldy, nullptr, 0, st);
 }
 
+// ---- products whose result is requantised for the next product (Sec. 3.3, last paragraph) ----
+namespace {
+bool requant_fused(int64_t M, int64_t N, int64_t K) {
+    // the tensor-core kernel's requantising epilogue serves items of 128 or 256 tokens
+    return g_gemm_impl != BD_GEMM_SIMT && tc_supported(M, N, K) && M > tc::kSplitMaxTokens;
+}
+size_t requant_extra(int64_t M, int64_t N, int64_t K) {            // fp32 result in scratch when the epilogue cannot requantise
+    return requant_fused(M, N, K) ? 0 : align256((size_t)M * (size_t)N * sizeof(float));
+}
+bd_status check_requant_out(const bd_qtensor *Yq, int64_t M, int64_t N) {
+    bd_status s = check_qtensor(Yq);
+    if (s) return s;
+    if (Yq->rows != M || Yq->K != N) return BD_ERR_SHAPE;          // (N % 32 is part of check_qtensor)
+    return BD_OK;
+}
+}  // namespace
+
+bd_status bd_linear_requant_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes) {
+    bd_status s = bd_linear_workspace_size(M, N, K, bytes);
+    if (s) return s;
+    if (N % kBlock) return BD_ERR_SHAPE;
+    *bytes = align256(*bytes) + requant_extra(M, N, K);
+    return BD_OK;
+}
+
+bd_status bd_gemm_requant_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes) {
+    bd_status s = bd_gemm_workspace_size(M, N, K, bytes);
+    if (s) return s;
+    if (N % kBlock) return BD_ERR_SHAPE;
+    *bytes = align256(*bytes) + requant_extra(M, N, K);
+    return BD_OK;
+}
+
+bd_status bd_linear_requant(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, const bd_qtensor *Wq,
+                            bd_qtensor *Yq, void *workspace, size_t workspace_bytes, void *stream) {
+    bd_status s = check_source(X, xdtype, M, K, ldx, K);
+    if (s) return s;
+    s = check_qtensor(Wq);
+    if (s) return s;
+    if (Wq->K != K) return BD_ERR_SHAPE;
+    const int64_t N = Wq->rows;
+    s = check_requant_out(Yq, M, N);
+    if (s) return s;
+    size_t need, base;
+    bd_linear_requant_workspace_size(M, N, K, &need);
+    bd_linear_workspace_size(M, N, K, &base);
+    if (!workspace || workspace_bytes < need) return BD_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 255u) return BD_ERR_ALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (requant_fused(M, N, K)) {
+        size_t c, i, sc;
+        bd_qtensor_sizes(M, K, &c, &i, &sc);
+        uint8_t *sfa = (uint8_t *)workspace, *a8 = sfa + align256(sc);
+        bd_qtensor xq{nullptr, nullptr, sfa, M, K};
+        s = launch_contig<BD_SELECT_TWO_STAGE, false, true>(X, xdtype, ldx, view_of(&xq), a8, st);
+        if (s) return s;
+        const QView out = view_of(Yq);
+        s = cuda_result(tc::launch(a8, sfa, M, view_of(Wq), K, nullptr, false, N, st, nullptr, 0, nullptr, &out));
+        g_launches += 1;
+        return s;
+    }
+    // short calls and the CUDA-core route: the fp32 result goes to scratch and the quantizer reads it from there
+    float *y32 = (float *)((char *)workspace + align256(base));
+    s = bd_linear(X, xdtype, M, K, ldx, Wq, y32, BD_F32, N, workspace, base, stream);
+    if (s) return s;
+    return launch_contig<BD_SELECT_TWO_STAGE, true, false>(y32, BD_F32, N, view_of(Yq), nullptr, st);
+}
+
+bd_status bd_gemm_requant(const bd_qtensor *A, const bd_qtensor *B, bd_qtensor *Yq, void *workspace, size_t workspace_bytes,
+                          void *stream) {
+    bd_status s = check_qtensor(A);
+    if (s) return s;
+    s = check_qtensor(B);
+    if (s) return s;
+    if (A->K != B->K) return BD_ERR_SHAPE;
+    const int64_t M = A->rows, N = B->rows, K = A->K;
+    s = check_requant_out(Yq, M, N);
+    if (s) return s;
+    size_t need, base;
+    bd_gemm_requant_workspace_size(M, N, K, &need);
+    bd_gemm_workspace_size(M, N, K, &base);
+    if (need && (!workspace || workspace_bytes < need)) return BD_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 255u) return BD_ERR_ALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (requant_fused(M, N, K)) {
+        const QView a = view_of(A), out = view_of(Yq);
+        uint8_t *a8 = (uint8_t *)workspace;
+        const int nb = (int)(K / kBlock);
+        decode_e4m3_kernel<<<grid_for(M * nb, 256), 256, 0, st>>>(a, a8, nb);
+        s = launch_result(1);
+        if (s) return s;
+        s = cuda_result(tc::launch(a8, a.scales, M, view_of(B), K, nullptr, false, N, st, nullptr, 0, nullptr, &out));
+        g_launches += 1;
+        return s;
+    }
+    float *y32 = (float *)((char *)workspace + align256(base));
+    s = gemm_dispatch(view_of(A), view_of(B), y32, BD_F32, N, workspace, base, st);
+    if (s) return s;
+    return launch_contig<BD_SELECT_TWO_STAGE, true, false>(y32, BD_F32, N, view_of(Yq), nullptr, st);
+}
+
 bd_status bd_linear_noalloc(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, const bd_qtensor *Wq,
                             void *Y, bd_dtype ydtype, int64_t ldy, void *stream) {
     if (!Wq || M <= 0 || K <= 0 || Wq->rows <= 0) return BD_ERR_INVALID_ARG;

@@ -170,7 +170,9 @@ struct Smem {
     static constexpr int bars = ids + kCodeStages * kIdAtomBytes;
     static constexpr int words = bars + 512;
     static constexpr int luts = words + 64;
-    static constexpr int out = ((luts + 128 + 1023) / 1024) * 1024;
+    static constexpr int qtab = luts + 128;                      // the quantizer's tables (requantising epilogue)
+    static constexpr int idx = qtab + (int)sizeof(SmemTables);   // dialect ids traded between the four warps of an epilogue half
+    static constexpr int out = ((idx + 512 + 1023) / 1024) * 1024;
     static constexpr int total = out + kEpilogueWarps * kStageBufs * kStageOut + 1024 /* alignment slack */;
 };
 static_assert((2 * kXStages + 2 * kCodeStages + 2 * kABufs + 2) * 8 <= 512, "barrier area too small");
@@ -294,13 +296,16 @@ __device__ __forceinline__ void epilogue_bf16(uint32_t t_base, uint8_t *stage_pt
     }
 }
 
+// REQUANT: the instantiation whose epilogue requantises the result (its quantizer arithmetic costs registers that the
+// plain instantiation keeps for the main loop).
+template <bool REQUANT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapXpart,
                   const __grid_constant__ CUtensorMap mapCodes,
                   const __grid_constant__ CUtensorMap mapSfW, const __grid_constant__ CUtensorMap mapSfX,
                   const uint8_t *__restrict__ idsW, const Schedule sc, int M, int N, int row_tiles_x, int row_tiles_w,
                   void *__restrict__ Y, int64_t ldy, int out_bf16, const __grid_constant__ CUtensorMap mapY, int use_tma_store,
-                  float *__restrict__ partials) {
+                  float *__restrict__ partials, const QView yq) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *const base_ptr = smem_raw + (base - smem_u32(smem_raw));
@@ -348,6 +353,8 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     }
     if (threadIdx.x < 32)
         luts[threadIdx.x] = threadIdx.x < 16 ? c_tables.e4m3_lo[threadIdx.x] : c_tables.e4m3_hi[threadIdx.x - 16];
+    SmemTables &qtab = *(SmemTables *)(base_ptr + Smem::qtab);
+    if (REQUANT) load_tables(qtab);                               // (ends with __syncthreads())
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32((const void *)tmem_slot)), "r"(512u) : "memory");
@@ -574,6 +581,56 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                         if (tok0 + c * 16 + q < toks && !*abort_flag) __stcg(mine + (size_t)(c * 16 + q) * np, __uint_as_float(r[q]));
                 }
                 release_accumulator();
+            } else if (REQUANT) {
+                // Requantising epilogue (Sec. 3.3, last paragraph: the accumulated result is "requantized into 4-bit
+                // DialectFP4 format for the next matrix multiplication").  The result row of a token is the next
+                // product's operand row, cut into blocks of 32 along N; this warp's 32 weight rows are one such
+                // block (number n0 / 32) of every token.  32 tokens per pass: each lane stores its row's fp32 sums
+                // into a 32 x 32 staging tile (element (token q, row n) at q * 32 + (n ^ q): both the row-wise
+                // stores and the token-wise loads touch 32 banks), then lane q owns token q's block and runs the
+                // two-stage rule of Sec. 3.2 on it, exactly as the standalone quantizer does on fp32 sources.
+                // Codes and scale bytes go out per lane; the four dialect ids of a token's four blocks (the four
+                // warps of this epilogue half) share two bytes of the id atom, so they meet in shared memory and
+                // the first warp stores them.
+                uint32_t *const tile = (uint32_t *)stage_ptr;     // 4 KiB: both staging buffers of this warp
+                const int b = n0 / kBlock, nb_out = (int)(yq.K / kBlock);
+                const int atoms_rows = (int)row_tiles(yq.rows) * kRowTile, atoms_blocks = (int)k_groups(yq.K) * kBlocksPerAtom;
+                for (int pass = 0; pass * 32 < cols; pass++) {
+                    uint32_t r[32];
+                    tcgen05_ld_32x32b_x32(t_base + pass * 32, r);
+                    tcgen05_wait_ld();
+                    if ((pass + 1) * 32 >= cols) release_accumulator();
+                    __syncwarp();                                 // the previous pass's loads of the tile are done
+#pragma unroll
+                    for (int q = 0; q < 32; q++) tile[q * 32 + (lane ^ q)] = r[q];
+                    __syncwarp();
+                    uint32_t bits[32];
+#pragma unroll
+                    for (int k = 0; k < 32; k++) bits[k] = tile[lane * 32 + (k ^ lane)];
+                    const int tok = t0 + pass * 32 + lane;
+                    const bool valid = tok < M && b < nb_out;
+                    BlockResult res;
+                    res.id = 0; res.scale = 0;
+                    if (valid) {
+                        bool nonfinite;
+                        uint32_t unused[8];
+                        quantize_two_stage_f32<false>(bits, qtab, res, unused, nonfinite);
+                        if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
+                        if (!*abort_flag)
+                            *(uint4 *)(yq.codes + (int64_t)tok * (yq.K / 2) + (int64_t)b * 16) =
+                                make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
+                    }
+                    // scale bytes and ids of the atoms' padding (tokens past M, blocks past N / 32) are written as zeros
+                    const bool in_atoms = tok < atoms_rows && b < atoms_blocks;
+                    if (in_atoms && !*abort_flag) yq.scales[scale_offset(yq.rows, tok, b)] = (uint8_t)res.scale;
+                    uint8_t *const trade = base_ptr + Smem::idx + (half * 2 + (pass & 1)) * 128;
+                    trade[quad * 32 + lane] = (uint8_t)res.id;
+                    asm volatile("bar.sync %0, 128;" ::"r"(4 + half) : "memory");   // the four warps of this half
+                    if (quad == 0 && in_atoms && !*abort_flag) {
+                        const uint32_t id16 = trade[lane] | trade[32 + lane] << 4 | trade[64 + lane] << 8 | trade[96 + lane] << 12;
+                        *(uint16_t *)(yq.ids + id_byte_offset(yq.rows, tok, b)) = (uint16_t)id16;
+                    }
+                }
             } else if (use_tma_store && out_bf16) {
                 if (cols == 128) epilogue_bf16<4>(t_base, stage_ptr, stage_out, &mapY, n0, t0, lane, abort_flag, release_accumulator, staging_free);
                 else epilogue_bf16<2>(t_base, stage_ptr, stage_out, &mapY, n0, t0, lane, abort_flag, release_accumulator, staging_free);
@@ -679,7 +736,7 @@ inline int max_resident_clusters() {
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = Smem::total;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, gemm_wtmem_kernel, &cfg) != cudaSuccess || n <= 0) {
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_wtmem_kernel<false>, &cfg) != cudaSuccess || n <= 0) {
         cudaGetLastError();
         int sms = 0;
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -702,9 +759,11 @@ inline size_t splitk_workspace(int64_t M, int64_t N, int64_t K) {
 
 // `scratch` (optional): splitk_workspace bytes, 256-byte aligned.
 // `kernels` (optional) receives the number of kernels launched: one, or two when K was split.
+// `requant` (optional; more than 128 tokens, N a multiple of 32): instead of writing Y, the epilogue quantises each
+// token's result row along N with the two-stage rule and writes it as the packed operand [M, N] given here.
 inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, const QView &W, int64_t K, void *Y,
                           bool out_bf16, int64_t ldy, cudaStream_t st, void *scratch = nullptr, size_t scratch_bytes = 0,
-                          int *kernels = nullptr) {
+                          int *kernels = nullptr, const QView *requant = nullptr) {
     if (kernels) *kernels = 1;
     CUtensorMap mapX, mapXpart, mapCodes, mapSfW, mapSfX, mapY;
     const int64_t N = W.rows, rtx = row_tiles(M), rtw = row_tiles(N), kg = k_groups(K);
@@ -719,7 +778,7 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
     // output through TMA tensor stores (32 columns x 32 or 16 rows per box) when Y is 16-byte aligned with a
     // row pitch that is a multiple of 16 bytes; otherwise plain stores
     const int esz = out_bf16 ? 2 : 4;
-    int use_tma_store = (((uintptr_t)Y & 15u) == 0 && (ldy * esz) % 16 == 0) ? 1 : 0;
+    int use_tma_store = (!requant && ((uintptr_t)Y & 15u) == 0 && (ldy * esz) % 16 == 0) ? 1 : 0;
     if (use_tma_store &&
         !make_map_2d(&mapY, out_bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Y, N, M,
                      (uint64_t)ldy * esz, 32, out_bf16 ? 32 : 16, CU_TENSOR_MAP_SWIZZLE_NONE))
@@ -728,7 +787,9 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
     static bool configured[kMaxDevices] = {};
     const int dev = current_device();
     if (!configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_wtmem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total);
+        cudaError_t e = cudaFuncSetAttribute(gemm_wtmem_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(gemm_wtmem_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem::total);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -773,9 +834,12 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_wtmem_kernel, mapX, mapXpart, mapCodes, mapSfW, mapSfX, (const uint8_t *)W.ids, sc,
-                                       (int)M, (int)N, (int)rtx, (int)rtw, Y, ldy, out_bf16 ? 1 : 0, mapY, use_tma_store,
-                                       (float *)scratch);
+    const QView none{nullptr, nullptr, nullptr, 0, 0};
+    cudaError_t e = requant
+        ? cudaLaunchKernelEx(&cfg, gemm_wtmem_kernel<true>, mapX, mapXpart, mapCodes, mapSfW, mapSfX, (const uint8_t *)W.ids, sc,
+                             (int)M, (int)N, (int)rtx, (int)rtw, Y, ldy, 0, mapY, use_tma_store, (float *)scratch, *requant)
+        : cudaLaunchKernelEx(&cfg, gemm_wtmem_kernel<false>, mapX, mapXpart, mapCodes, mapSfW, mapSfX, (const uint8_t *)W.ids, sc,
+                             (int)M, (int)N, (int)rtx, (int)rtw, Y, ldy, out_bf16 ? 1 : 0, mapY, use_tma_store, (float *)scratch, none);
     if (e != cudaSuccess || sc.k_splits == 1) return e;
     if (kernels) *kernels = 2;
     const int np = sc.w_pairs * 256;
