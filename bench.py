@@ -644,6 +644,13 @@ def run_gpu(args, rank, world, local_rank):
     replicas.shutdown()
 
 
+def _lib_override():
+    """BDLIB=<path>: load another build of the library (A/B timing of work-in-progress kernels)."""
+    if os.environ.get("BDLIB"):
+        from paper_2501_01144_b200 import binding
+        binding._LIB_PATH = os.environ["BDLIB"]
+
+
 def run_case(args):
     """A few launches of one kernel family on a small, fixed case (for ncu captures).
     quantizer: bd_quantize_act on bf16 [8192, 4096] (168 MiB of buffers in rotation).
@@ -752,6 +759,7 @@ def main():
                     choices=["quantizer", "quantizer_f32", "step"] + ["linear_" + n for n, _, _ in LAYERS],
                     help="run a few launches of one small case (for profiler captures) instead of the benchmark")
     args = ap.parse_args()
+    _lib_override()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.case:
         # started as a plain process: start the N ranks here, one per GPU, the way torchrun would
         sys.exit(spawn_ranks(args))

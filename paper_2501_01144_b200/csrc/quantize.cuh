@@ -423,7 +423,7 @@ __device__ __forceinline__ void quantize_bf16_parts(const uint16_t *__restrict__
         k.valid = REGULAR || (k.r < rows && k.b < nb);
         if (k.valid) {
             const uint4 *src = (const uint4 *)(X + (int64_t)k.r * ld + k.b * 32u);
-            k.l0 = __ldg(src); k.l1 = __ldg(src + 1); k.l2 = __ldg(src + 2); k.l3 = __ldg(src + 3);
+            k.l0 = __ldcs(src); k.l1 = __ldcs(src + 1); k.l2 = __ldcs(src + 2); k.l3 = __ldcs(src + 3);   // read once: streaming
         }
     };
     auto process = [&](const Part &k) {
