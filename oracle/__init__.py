@@ -37,6 +37,9 @@ def lib():
         _lib = ctypes.CDLL(build())
         i64, vp, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_int
         _lib.bdo_quantize.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp]
+        _lib.bdo_quantize_bs.argtypes = [vp, ci, i64, i64, i64, ci, ci, vp, vp, vp]
+        _lib.bdo_dequantize_bs.argtypes = [vp, vp, vp, i64, i64, ci, vp]
+        _lib.bdo_gemm_blockmac_bs.argtypes = [vp] * 6 + [i64] * 3 + [ci, vp]
         _lib.bdo_dequantize.argtypes = [vp, vp, vp, i64, i64, vp]
         _lib.bdo_gemm.argtypes = [vp, vp, i64, i64, i64, vp, vp]
         _lib.bdo_gemm_blockmac.argtypes = [vp] * 6 + [i64] * 3 + [vp]
@@ -95,16 +98,17 @@ def _dtype_of(x):
     raise TypeError(f"unsupported input dtype {x.dtype}")
 
 
-def quantize(x, select=SELECT_TWO_STAGE, dtype=None):
-    """Quantise a [rows, K] array along K.  Returns canonical (codes, ids, scales)."""
+def quantize(x, select=SELECT_TWO_STAGE, dtype=None, block=BLOCK):
+    """Quantise a [rows, K] array along K in blocks of `block` elements (32 unless the block-size study of
+    Sec. 4.2 / Table 3 is meant: 16 or 64).  Returns canonical (codes, ids, scales)."""
     x = np.ascontiguousarray(x)
     if dtype is None:
         dtype = _dtype_of(x)
     rows, K = x.shape
     codes = np.zeros((rows, K // 2), np.uint8)
-    ids = np.zeros((rows, K // BLOCK), np.uint8)
-    scales = np.zeros((rows, K // BLOCK), np.uint8)
-    st = lib().bdo_quantize(_ptr(x), dtype, rows, K, K, select, _ptr(codes), _ptr(ids), _ptr(scales))
+    ids = np.zeros((rows, K // block), np.uint8)
+    scales = np.zeros((rows, K // block), np.uint8)
+    st = lib().bdo_quantize_bs(_ptr(x), dtype, rows, K, K, select, block, _ptr(codes), _ptr(ids), _ptr(scales))
     if st == 2:
         raise FloatingPointError("non-finite input")
     if st:
@@ -123,11 +127,13 @@ def requantize(y):
 
 
 def dequantize(codes, ids, scales):
-    """Canonical (codes, ids, scales) -> fp64 [rows, K] (Sec. 3.3, Fig. 6)."""
+    """Canonical (codes, ids, scales) -> fp64 [rows, K] (Sec. 3.3, Fig. 6); the block size follows from the
+    shapes (K / number of ids per row)."""
     rows, K = codes.shape[0], codes.shape[1] * 2
+    block = K // ids.shape[1]
     out = np.zeros((rows, K), np.float64)
-    if lib().bdo_dequantize(_ptr(np.ascontiguousarray(codes)), _ptr(np.ascontiguousarray(ids)),
-                            _ptr(np.ascontiguousarray(scales)), rows, K, _ptr(out)):
+    if lib().bdo_dequantize_bs(_ptr(np.ascontiguousarray(codes)), _ptr(np.ascontiguousarray(ids)),
+                               _ptr(np.ascontiguousarray(scales)), rows, K, block, _ptr(out)):
         raise ValueError("bad arguments")
     return out
 
@@ -151,7 +157,9 @@ def gemm_blockmac(qa, qb):
     cb, ib, sb = (np.ascontiguousarray(t) for t in qb)
     M, K = ca.shape[0], ca.shape[1] * 2
     N = cb.shape[0]
+    block = K // ia.shape[1]
+    assert K // ib.shape[1] == block, "both operands of a product use one block size"
     Y = np.zeros((M, N), np.float64)
-    if lib().bdo_gemm_blockmac(_ptr(ca), _ptr(ia), _ptr(sa), _ptr(cb), _ptr(ib), _ptr(sb), M, N, K, _ptr(Y)):
+    if lib().bdo_gemm_blockmac_bs(_ptr(ca), _ptr(ia), _ptr(sa), _ptr(cb), _ptr(ib), _ptr(sb), M, N, K, block, _ptr(Y)):
         raise ValueError("bad arguments")
     return Y

@@ -21,17 +21,20 @@
  * All floating point is fp64; every quantity that decides an integer result is
  * an exact integer or an exactly representable double.
  *
- * Canonical output layout (rows x K operand, blocks of 32 along K):
+ * Canonical output layout (rows x K operand, blocks of B = 32 elements along K;
+ * the *_bs entry points take B = 16, 32 or 64, the block sizes of the paper's
+ * block-size study, Sec. 4.2 and its Table 3):
  *   codes  [rows][K/2]  byte j: element 2j in bits 3:0, element 2j+1 in bits 7:4,
  *                        nibble = sign<<3 | idx
- *   ids    [rows][K/32] one byte per block, 0..15
- *   scales [rows][K/32] one byte per block, e + 127
+ *   ids    [rows][K/B]  one byte per block, 0..15
+ *   scales [rows][K/B]  one byte per block, e + 127
  */
 #include <math.h>
 #include <stdint.h>
 #include <string.h>
 
 #define BDO_BLOCK 32
+#define BDO_MAX_BLOCK 64
 #define BDO_OK 0
 #define BDO_ERR_ARG 1
 #define BDO_ERR_NONFINITE 2
@@ -135,9 +138,9 @@ static double load_elem(const void *p, int dtype, int64_t i) {
  *   q5[k] = the scaled magnitude |x_k| * 2^-e with three integer and two
  *           fractional bits, lower bits truncated: floor(4 * |x_k| * 2^-e)
  * ------------------------------------------------------------------------- */
-static int shared_exponent(const double *mag) {
+static int shared_exponent(const double *mag, int bs) {
     double amax = 0.0;
-    for (int k = 0; k < BDO_BLOCK; k++)
+    for (int k = 0; k < bs; k++)
         if (mag[k] > amax) amax = mag[k];
     if (amax == 0.0) return -127;
     int ex;
@@ -157,9 +160,9 @@ static int mag_trunc(double mag, int e) {
  * pair of dialects whose maximum equals it.  A maximum below 4.0 (only after
  * the exponent clamp) takes the last pair.
  * ------------------------------------------------------------------------- */
-static int stage1_pair(const int *q5) {
+static int stage1_pair(const int *q5, int bs) {
     int m5 = 0;
-    for (int k = 0; k < BDO_BLOCK; k++)
+    for (int k = 0; k < bs; k++)
         if (q5[k] > m5) m5 = q5[k];
     int max_hu = (m5 + 1) / 2; /* half-units */
     if (max_hu > 15) max_hu = 15;
@@ -192,11 +195,11 @@ int bdo_beneficial_range(int dialect, int *lo, int *hi) {
 
 /* Stage 2: the dialect of the pair with more block elements inside its
  * beneficial range; on equal counts the even one (larger magnitudes first). */
-static int stage2_pick(const int *q5, int pair) {
+static int stage2_pick(const int *q5, int pair, int bs) {
     int lo_e, hi_e, lo_o, hi_o, cnt_e = 0, cnt_o = 0;
     bdo_beneficial_range(2 * pair, &lo_e, &hi_e);
     bdo_beneficial_range(2 * pair + 1, &lo_o, &hi_o);
-    for (int k = 0; k < BDO_BLOCK; k++) {
+    for (int k = 0; k < bs; k++) {
         if (q5[k] >= lo_e && q5[k] < hi_e) cnt_e++;
         if (q5[k] >= lo_o && q5[k] < hi_o) cnt_o++;
     }
@@ -225,12 +228,12 @@ int bdo_round_code(int dialect, int q5) {
  * the 16 dialects with the block's shared exponent and keep the dialect with
  * the smallest sum of squared errors against the untruncated scaled
  * magnitudes; the lowest number wins equal sums. */
-static int select_mse(const double *mag, const int *q5, int e) {
+static int select_mse(const double *mag, const int *q5, int e, int bs) {
     int best = 0;
     double best_err = INFINITY;
     for (int d = 0; d < 16; d++) {
         double err = 0.0;
-        for (int k = 0; k < BDO_BLOCK; k++) {
+        for (int k = 0; k < bs; k++) {
             double t = ldexp(mag[k], -e) - 0.5 * (double)FORMATBOOK[d][bdo_round_code(d, q5[k])];
             err = err + t * t;
         }
@@ -242,20 +245,21 @@ static int select_mse(const double *mag, const int *q5, int e) {
     return best;
 }
 
-/* One block: 32 reals -> 32 nibbles, dialect id, shared exponent. */
-static int quantize_block(const double *x, int select, uint8_t *nib, int *id_out, int *e_out) {
-    double mag[BDO_BLOCK];
-    int q5[BDO_BLOCK];
-    for (int k = 0; k < BDO_BLOCK; k++) {
+/* One block: bs reals -> bs nibbles, dialect id, shared exponent.  The block size only sets how many elements
+ * share the exponent and the dialect (Sec. 4.2, Table 3); every step is the same. */
+static int quantize_block(const double *x, int select, int bs, uint8_t *nib, int *id_out, int *e_out) {
+    double mag[BDO_MAX_BLOCK];
+    int q5[BDO_MAX_BLOCK];
+    for (int k = 0; k < bs; k++) {
         if (!isfinite(x[k])) return BDO_ERR_NONFINITE;
         mag[k] = fabs(x[k]);
     }
-    int e = shared_exponent(mag);
-    for (int k = 0; k < BDO_BLOCK; k++) q5[k] = mag_trunc(mag[k], e);
+    int e = shared_exponent(mag, bs);
+    for (int k = 0; k < bs; k++) q5[k] = mag_trunc(mag[k], e);
     int id;
-    if (select == BDO_SELECT_MSE) id = select_mse(mag, q5, e);
-    else id = stage2_pick(q5, stage1_pair(q5));
-    for (int k = 0; k < BDO_BLOCK; k++) {
+    if (select == BDO_SELECT_MSE) id = select_mse(mag, q5, e, bs);
+    else id = stage2_pick(q5, stage1_pair(q5, bs), bs);
+    for (int k = 0; k < bs; k++) {
         int sign = signbit(x[k]) ? 1 : 0;
         nib[k] = (uint8_t)(sign << 3 | bdo_round_code(id, q5[k]));
     }
@@ -267,27 +271,29 @@ static int quantize_block(const double *x, int select, uint8_t *nib, int *id_out
 /* Quantise a [rows, K] operand whose blocks run along the contiguous K axis.
  * ld = row stride in elements.  Returns BDO_ERR_NONFINITE if any element is
  * Inf or NaN (outputs then unspecified). */
-int bdo_quantize(const void *x, int dtype, int64_t rows, int64_t K, int64_t ld, int select,
-                 uint8_t *codes, uint8_t *ids, uint8_t *scales) {
-    if (K % BDO_BLOCK || rows < 0 || K < 0 || ld < K) return BDO_ERR_ARG;
+static int block_size_ok(int bs) { return bs == 16 || bs == 32 || bs == 64; }
+
+int bdo_quantize_bs(const void *x, int dtype, int64_t rows, int64_t K, int64_t ld, int select, int bs,
+                    uint8_t *codes, uint8_t *ids, uint8_t *scales) {
+    if (!block_size_ok(bs) || K % bs || rows < 0 || K < 0 || ld < K) return BDO_ERR_ARG;
     int status = BDO_OK;
-    int64_t nb = K / BDO_BLOCK;
+    int64_t nb = K / bs;
 #ifdef _OPENMP
 #pragma omp parallel for schedule(static) reduction(max : status)
 #endif
     for (int64_t r = 0; r < rows; r++) {
         for (int64_t b = 0; b < nb; b++) {
-            double xb[BDO_BLOCK];
-            uint8_t nib[BDO_BLOCK];
+            double xb[BDO_MAX_BLOCK];
+            uint8_t nib[BDO_MAX_BLOCK];
             int id, e;
-            for (int k = 0; k < BDO_BLOCK; k++) xb[k] = load_elem(x, dtype, r * ld + b * BDO_BLOCK + k);
-            int st = quantize_block(xb, select, nib, &id, &e);
+            for (int k = 0; k < bs; k++) xb[k] = load_elem(x, dtype, r * ld + b * bs + k);
+            int st = quantize_block(xb, select, bs, nib, &id, &e);
             if (st != BDO_OK) {
                 status = st;
                 continue;
             }
-            for (int k = 0; k < BDO_BLOCK; k += 2)
-                codes[r * (K / 2) + b * 16 + k / 2] = (uint8_t)(nib[k] | nib[k + 1] << 4);
+            for (int k = 0; k < bs; k += 2)
+                codes[r * (K / 2) + b * (bs / 2) + k / 2] = (uint8_t)(nib[k] | nib[k + 1] << 4);
             ids[r * nb + b] = (uint8_t)id;
             scales[r * nb + b] = (uint8_t)(e + 127);
         }
@@ -295,15 +301,20 @@ int bdo_quantize(const void *x, int dtype, int64_t rows, int64_t K, int64_t ld, 
     return status;
 }
 
+int bdo_quantize(const void *x, int dtype, int64_t rows, int64_t K, int64_t ld, int select,
+                 uint8_t *codes, uint8_t *ids, uint8_t *scales) {
+    return bdo_quantize_bs(x, dtype, rows, K, ld, select, BDO_BLOCK, codes, ids, scales);
+}
+
 /* Dequantisation (Sec. 3.3, Fig. 6): index -> 4-bit unsigned integer through
  * the dialect's table, times 0.5, times 2^e, with the stored sign. */
-int bdo_dequantize(const uint8_t *codes, const uint8_t *ids, const uint8_t *scales, int64_t rows,
-                   int64_t K, double *out) {
-    if (K % BDO_BLOCK) return BDO_ERR_ARG;
-    int64_t nb = K / BDO_BLOCK;
+int bdo_dequantize_bs(const uint8_t *codes, const uint8_t *ids, const uint8_t *scales, int64_t rows,
+                      int64_t K, int bs, double *out) {
+    if (!block_size_ok(bs) || K % bs) return BDO_ERR_ARG;
+    int64_t nb = K / bs;
     for (int64_t r = 0; r < rows; r++)
         for (int64_t k = 0; k < K; k++) {
-            int64_t b = k / BDO_BLOCK;
+            int64_t b = k / bs;
             uint8_t byte = codes[r * (K / 2) + k / 2];
             int nib = (k % 2) ? byte >> 4 : byte & 15;
             int h = FORMATBOOK[ids[r * nb + b]][nib & 7];
@@ -311,6 +322,11 @@ int bdo_dequantize(const uint8_t *codes, const uint8_t *ids, const uint8_t *scal
             out[r * K + k] = (nib & 8) ? -v : v;
         }
     return BDO_OK;
+}
+
+int bdo_dequantize(const uint8_t *codes, const uint8_t *ids, const uint8_t *scales, int64_t rows,
+                   int64_t K, double *out) {
+    return bdo_dequantize_bs(codes, ids, scales, rows, K, BDO_BLOCK, out);
 }
 
 /* Reference product Y = dq(A) dq(B)^T in fp64 over the dequantised operands
@@ -339,18 +355,18 @@ int bdo_gemm(const double *a, const double *b, int64_t M, int64_t N, int64_t K, 
  * products with the sign applied separately, exact integer sums inside a block,
  * one conversion per block: S_b * 2^(eA + eB - 2), accumulated in fp64.
  * Used by the tests to check that this route equals bdo_gemm. */
-int bdo_gemm_blockmac(const uint8_t *codesA, const uint8_t *idsA, const uint8_t *scalesA,
-                      const uint8_t *codesB, const uint8_t *idsB, const uint8_t *scalesB,
-                      int64_t M, int64_t N, int64_t K, double *Y) {
-    if (K % BDO_BLOCK) return BDO_ERR_ARG;
-    int64_t nb = K / BDO_BLOCK;
+int bdo_gemm_blockmac_bs(const uint8_t *codesA, const uint8_t *idsA, const uint8_t *scalesA,
+                         const uint8_t *codesB, const uint8_t *idsB, const uint8_t *scalesB,
+                         int64_t M, int64_t N, int64_t K, int bs, double *Y) {
+    if (!block_size_ok(bs) || K % bs) return BDO_ERR_ARG;
+    int64_t nb = K / bs;
     for (int64_t m = 0; m < M; m++)
         for (int64_t n = 0; n < N; n++) {
             double y = 0.0;
             for (int64_t blk = 0; blk < nb; blk++) {
                 int64_t s = 0;
-                for (int k = 0; k < BDO_BLOCK; k++) {
-                    int64_t kk = blk * BDO_BLOCK + k;
+                for (int k = 0; k < bs; k++) {
+                    int64_t kk = blk * bs + k;
                     uint8_t ba = codesA[m * (K / 2) + kk / 2], bb = codesB[n * (K / 2) + kk / 2];
                     int na = (kk % 2) ? ba >> 4 : ba & 15, nbv = (kk % 2) ? bb >> 4 : bb & 15;
                     int64_t prod = (int64_t)FORMATBOOK[idsA[m * nb + blk]][na & 7] *
@@ -363,6 +379,12 @@ int bdo_gemm_blockmac(const uint8_t *codesA, const uint8_t *idsA, const uint8_t 
             Y[m * N + n] = y;
         }
     return BDO_OK;
+}
+
+int bdo_gemm_blockmac(const uint8_t *codesA, const uint8_t *idsA, const uint8_t *scalesA,
+                      const uint8_t *codesB, const uint8_t *idsB, const uint8_t *scalesB,
+                      int64_t M, int64_t N, int64_t K, double *Y) {
+    return bdo_gemm_blockmac_bs(codesA, idsA, scalesA, codesB, idsB, scalesB, M, N, K, BDO_BLOCK, Y);
 }
 
 /* Number of threads the row loops above run on (1 without OpenMP). */

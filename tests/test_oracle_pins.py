@@ -464,3 +464,58 @@ def test_error_bound_and_idempotence():
         if select == oracle.SELECT_TWO_STAGE:
             assert np.array_equal(s2, scales)
             assert np.array_equal(oracle.dequantize(c2, i2, s2), deq)
+
+
+# ----------------------------------------------------------------------------
+# Block sizes 16 and 64 (the block-size study of Sec. 4.2, Table 3): the same steps over a block of another length
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("block", [16, 64])
+def test_other_block_sizes_against_rational_brute_force(block):
+    rng = np.random.default_rng(300 + block)
+    x = rng.standard_normal((12, 4 * block)).astype(np.float32)
+    x[::3, 5] *= 60.0                                            # an outlier in the first block of some rows
+    x[1::4] = np.round(x[1::4] * 4) / 4                          # exact ties on the grid
+    x[2] *= 2.0 ** -30
+    codes, ids, scales = oracle.quantize(x, block=block)
+    assert ids.shape == scales.shape == (12, 4)
+    for r in range(x.shape[0]):
+        nib = _unpack(codes[r])
+        for b in range(4):
+            seg = x[r, b * block:(b + 1) * block]
+            e, d, idx = _exact_block_two_stage(seg)              # the restatement takes any block length
+            assert int(scales[r, b]) - 127 == e
+            assert int(ids[r, b]) == d
+            assert [n & 7 for n in nib[b * block:(b + 1) * block]] == idx
+            assert [n >> 3 for n in nib[b * block:(b + 1) * block]] == [int(np.signbit(v)) for v in seg]
+
+
+@pytest.mark.parametrize("block", [16, 64])
+def test_other_block_sizes_mse_rule_and_product(block):
+    rng = np.random.default_rng(310 + block)
+    x = rng.standard_normal((6, 2 * block)).astype(np.float32)
+    x[:, 3] *= 25.0
+    codes, ids, scales = oracle.quantize(x, oracle.SELECT_MSE, block=block)
+    for r in range(x.shape[0]):
+        for b in range(2):
+            errs = _exact_mse_errors(x[r, b * block:(b + 1) * block], int(scales[r, b]) - 127)
+            assert int(ids[r, b]) == errs.index(min(errs))       # lowest id among exact minima
+    # dequantised values sit on the block's grid, and the block MAC with one rescale per block equals the fp64 product
+    w = (0.02 * rng.standard_normal((5, 2 * block))).astype(np.float32)
+    qa, qb = oracle.quantize(x, block=block), oracle.quantize(w, block=block)
+    da, db = oracle.dequantize(*qa), oracle.dequantize(*qb)
+    for r in range(x.shape[0]):
+        for b in range(2):
+            grid = {float(v) * 0.5 * 2.0 ** (int(qa[2][r, b]) - 127) for v in FB[qa[1][r, b]]}
+            assert set(np.abs(da[r, b * block:(b + 1) * block]).tolist()) <= grid
+    Y, T = oracle.gemm(da, db)
+    assert np.abs(oracle.gemm_blockmac(qa, qb) - Y).max() <= 1e-13 * T.max()
+
+
+def test_smaller_blocks_never_share_an_exponent_across_their_border():
+    # two halves of a 32-element row six binades apart: block 16 gives each half its own exponent, block 32 one
+    x = np.concatenate([np.full(16, 5.0), np.full(16, 5.0 / 64)]).astype(np.float32)[None, :]
+    s16 = oracle.quantize(x, block=16)[2]
+    s32 = oracle.quantize(x, block=32)[2]
+    assert s16.tolist() == [[127, 121]] and s32.tolist() == [[127]]
+    assert np.array_equal(oracle.dequantize(*oracle.quantize(x, block=16)), x.astype(np.float64))   # both halves exact
+    assert np.abs(oracle.dequantize(*oracle.quantize(x, block=32))[0, 16:]).max() == 0.0            # the small half is lost
