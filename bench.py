@@ -511,6 +511,47 @@ def run_gpu(args, rank, world, local_rank):
         bd.poll_status()
         time.sleep(0.5)
 
+    # ---- block sizes 16 / 32 / 64 (Sec. 4.2, Table 3; e.g. block 16 for the down projection): the quantizer on the
+    # activation-quantizer workload and the down projection at M = 2048.  Block 64 is stored as pairs of 32-blocks
+    # (same product kernel, same time); block 16 is stored zero-padded to 32-blocks: twice the code bytes and MMA work ----
+    block_sizes = None
+    if rank == 0:
+        block_sizes = []
+        xq_src = dev_bf16(inputs.act_normal_outliers(qm, qk, seed=1))
+        Kd, Nd = 14336, 4096
+        xd_src = dev_bf16(inputs.act_student_t(M_TOKENS, Kd, seed=5))
+        wd_src = dev_bf16(inputs.weights_normal(Nd, Kd, seed=5))
+        yd = torch.empty(M_TOKENS, Nd, dtype=torch.bfloat16, device=dev)
+        for block in (16, 32, 64):
+            qo = bd.QTensor(qm, bd.physical_k(qk, block), dev)
+            for _ in range(3):
+                bd.quantize_bs(xq_src, block, out=qo)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(10):
+                bd.quantize_bs(xq_src, block, out=qo)
+            e1.record()
+            torch.cuda.synchronize()
+            q_us = e0.elapsed_time(e1) / 10 * 1e3
+            q_bytes_b = qm * qk * (2 + 0.5 + 1.5 / block)
+            wq_b = bd.quantize_bs(wd_src, block)
+            ws_b = torch.empty(bd.linear_bs_workspace_size(M_TOKENS, Nd, Kd, block), dtype=torch.uint8, device=dev)
+            for _ in range(3):
+                bd.linear_bs(xd_src, wq_b, block, out=yd, workspace=ws_b)
+            e0.record()
+            for _ in range(10):
+                bd.linear_bs(xd_src, wq_b, block, out=yd, workspace=ws_b)
+            e1.record()
+            torch.cuda.synchronize()
+            l_us = e0.elapsed_time(e1) / 10 * 1e3
+            block_sizes.append({"block": block, "quantizer_us": q_us, "quantizer_gbs_algorithmic": q_bytes_b / q_us / 1e3,
+                                "bits_per_element_paper_accounting": 4 + 9 / block, "bits_per_element_stored": 8.75 if block == 16 else 4.375,
+                                "linear_down_proj_us": l_us, "linear_down_proj_tflops": 2.0 * M_TOKENS * Nd * Kd / l_us / 1e6})
+            del qo, wq_b, ws_b
+        del xq_src, xd_src, wd_src, yd
+        bd.poll_status()
+        time.sleep(0.3)
+
     # ---- attention products with both operands quantised online (Mistral-7B shapes: 32 heads, 8 KV heads,
     # 4096 tokens, head_dim 128; reported, not part of the timed step).  QK^T is bound by the write of the
     # scores, PV by the read of the fp32 probabilities. ----
@@ -638,6 +679,7 @@ def run_gpu(args, rank, world, local_rank):
         "per_layer_gflop": {l["name"]: l["flops"] / 1e9 for l in layers},
         "llama2_mlp_m_sweep": sweep,
         "chained_layers": chained,
+        "block_sizes": block_sizes,
         "attention_mistral7b": attention,
     }
     print(json.dumps(line))

@@ -183,6 +183,30 @@ bd_status bd_gemm_requant_workspace_size(int64_t M, int64_t N, int64_t K, size_t
 bd_status bd_gemm_requant(const bd_qtensor *A, const bd_qtensor *B, bd_qtensor *Yq, void *workspace,
                           size_t workspace_bytes, void *stream);
 
+/* Block sizes 16 and 64 beside the default 32 (the block-size study of Sec. 4.2 and its
+ * Table 3, including per-sublayer mixes such as block 16 for the down projection: the block
+ * size is chosen per call).  `block` is 16, 32 or 64 and must divide K; both operands of a
+ * product use the same block size.  The tensor-core product scales per 32 elements, so other
+ * block sizes are STORED in the ordinary 32-block form and every product entry point
+ * (bd_gemm, bd_gemm_batched, bd_gemm_requant) takes such operands as they are, exactly:
+ *   block 64: two neighbouring 32-blocks with the same scale and id; physical K' = K;
+ *   block 16: one 32-block per block, its second half zero codes; physical K' = 2 K
+ *             (twice the code bytes and twice the MMA work of the same K at block 32).
+ * bd_qtensor_sizes_bs gives the buffer sizes; out->K must be the physical K'.
+ * bd_export_canonical_bs gives the canonical view: codes [rows][K/2], ids and scales
+ * [rows][K/block].  bd_linear_bs = two-stage quantisation of X with that block size
+ * (into the workspace) followed by the product with Wq (quantised with the same block size). */
+bd_status bd_qtensor_sizes_bs(int64_t rows, int64_t K, int block, size_t *codes_bytes, size_t *ids_bytes,
+                              size_t *scales_bytes);
+bd_status bd_quantize_bs(const void *X, bd_dtype dtype, int64_t rows, int64_t K, int64_t ld, bd_select select,
+                         int block, bd_qtensor *out, void *stream);
+bd_status bd_export_canonical_bs(const bd_qtensor *q, int block, uint8_t *codes, uint8_t *ids, uint8_t *scales,
+                                 void *stream);
+bd_status bd_linear_bs_workspace_size(int64_t M, int64_t N, int64_t K, int block, size_t *bytes);
+bd_status bd_linear_bs(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, int block,
+                       const bd_qtensor *Wq, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace,
+                       size_t workspace_bytes, void *stream);
+
 /* bd_linear for callers that can neither allocate device memory nor hand in a
  * workspace (the paper has no counterpart; this is a convenience of the library).
  * Think of code that runs where cudaMalloc is off limits: inside a region whose

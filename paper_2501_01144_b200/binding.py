@@ -68,6 +68,11 @@ def load():
     lib.bd_linear_workspace_size.argtypes = [i64, i64, i64, szp]
     lib.bd_linear.argtypes = [vp, ci, i64, i64, i64, qp, vp, ci, i64, vp, sz, vp]
     lib.bd_linear_noalloc.argtypes = [vp, ci, i64, i64, i64, qp, vp, ci, i64, vp]
+    lib.bd_qtensor_sizes_bs.argtypes = [i64, i64, ci, szp, szp, szp]
+    lib.bd_quantize_bs.argtypes = [vp, ci, i64, i64, i64, ci, ci, qp, vp]
+    lib.bd_export_canonical_bs.argtypes = [qp, ci, vp, vp, vp, vp]
+    lib.bd_linear_bs_workspace_size.argtypes = [i64, i64, i64, ci, szp]
+    lib.bd_linear_bs.argtypes = [vp, ci, i64, i64, i64, ci, qp, vp, ci, i64, vp, sz, vp]
     lib.bd_linear_requant_workspace_size.argtypes = [i64, i64, i64, szp]
     lib.bd_linear_requant.argtypes = [vp, ci, i64, i64, i64, qp, qp, vp, sz, vp]
     lib.bd_gemm_requant_workspace_size.argtypes = [i64, i64, i64, szp]
@@ -280,6 +285,54 @@ def gemm_requant(A, B, out=None, workspace=None, stream=None):
     workspace, wptr, wbytes = _ws(workspace, gemm_requant_workspace_size(A.rows, B.rows, A.K), A.codes.device)
     ca, cb, cy = A.c_struct(), B.c_struct(), out.c_struct()
     _check(load().bd_gemm_requant(ctypes.byref(ca), ctypes.byref(cb), ctypes.byref(cy), wptr, wbytes, _stream(stream)))
+    return out
+
+
+def physical_k(K, block):
+    """K of the stored operand for a block size: block 16 is stored zero-padded to 32-element blocks."""
+    return 2 * K if block == 16 else K
+
+
+def quantize_bs(X, block, select=SELECT_TWO_STAGE, out=None, stream=None):
+    """Quantise X [rows, K] along K in blocks of 16, 32 or 64 elements (Sec. 4.2, Table 3).  The result is an
+    ordinary QTensor with K' = physical_k(K, block) that every product takes as it is."""
+    ptr, dt, ld = _src(X)
+    rows, K = X.shape
+    out = out or QTensor(rows, physical_k(K, block), X.device)
+    cq = out.c_struct()
+    _check(load().bd_quantize_bs(ptr, dt, rows, K, ld, select, block, ctypes.byref(cq), _stream(stream)))
+    return out
+
+
+def export_canonical_bs(q, block, stream=None):
+    """(codes [rows, K/2], ids [rows, K/block], scales [rows, K/block]) of an operand stored for `block`."""
+    dev = q.codes.device
+    K = q.K // 2 if block == 16 else q.K
+    codes = torch.empty(q.rows, K // 2, dtype=torch.uint8, device=dev)
+    ids = torch.empty(q.rows, K // block, dtype=torch.uint8, device=dev)
+    scales = torch.empty(q.rows, K // block, dtype=torch.uint8, device=dev)
+    cq = q.c_struct()
+    _check(load().bd_export_canonical_bs(ctypes.byref(cq), block, ctypes.c_void_p(codes.data_ptr()),
+                                         ctypes.c_void_p(ids.data_ptr()), ctypes.c_void_p(scales.data_ptr()), _stream(stream)))
+    return codes, ids, scales
+
+
+def linear_bs_workspace_size(M, N, K, block):
+    b = ctypes.c_size_t()
+    _check(load().bd_linear_bs_workspace_size(M, N, K, block, ctypes.byref(b)))
+    return b.value
+
+
+def linear_bs(X, Wq, block, out=None, dtype=torch.bfloat16, workspace=None, stream=None):
+    """The quantised linear layer with blocks of 16, 32 or 64 elements; Wq from quantize_bs with the same block."""
+    ptr, dt, ld = _src(X)
+    M, K = X.shape
+    if out is None:
+        out = torch.empty(M, Wq.rows, dtype=dtype, device=X.device)
+    workspace, wptr, wbytes = _ws(workspace, linear_bs_workspace_size(M, Wq.rows, K, block), X.device)
+    cw = Wq.c_struct()
+    _check(load().bd_linear_bs(ptr, dt, M, K, ld, block, ctypes.byref(cw), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
+                               out.stride(0), wptr, wbytes, _stream(stream)))
     return out
 
 

@@ -9,6 +9,7 @@
 #include "bd_common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "blocksize.cuh"
 #include "quantize.cuh"
 
 using namespace bd;
@@ -191,6 +192,27 @@ static __device__ __align__(256) uint8_t g_noalloc_scratch[BD_NOALLOC_SCRATCH_BY
 namespace {
 constexpr int kMaxDevices = 64;
 void *g_noalloc_ptr[kMaxDevices] = {};
+}  // namespace
+
+// launchers of the quantizer for block sizes 16 and 64
+namespace {
+template <int DT, int BS>
+void launch_quantize_bs(const void *X, int64_t ld, bd_select select, const QView &v, cudaStream_t st) {
+    const int nbp = (int)(v.K / kBlock), nbp_pad = (int)k_groups(v.K) * kBlocksPerAtom;
+    const int64_t rows_pad = row_tiles(v.rows) * kRowTile;
+    const unsigned grid = grid_for(rows_pad * nbp_pad, 256);
+    if (select == BD_SELECT_MSE) quantize_bs_kernel<DT, BS, BD_SELECT_MSE><<<grid, 256, 0, st>>>(X, ld, v, rows_pad, nbp, nbp_pad);
+    else quantize_bs_kernel<DT, BS, BD_SELECT_TWO_STAGE><<<grid, 256, 0, st>>>(X, ld, v, rows_pad, nbp, nbp_pad);
+}
+template <int BS>
+bd_status quantize_bs_dtype(const void *X, bd_dtype dt, int64_t ld, bd_select select, const QView &v, cudaStream_t st) {
+    switch (dt) {
+        case BD_F32: launch_quantize_bs<BD_F32, BS>(X, ld, select, v, st); break;
+        case BD_BF16: launch_quantize_bs<BD_BF16, BS>(X, ld, select, v, st); break;
+        default: launch_quantize_bs<BD_F16, BS>(X, ld, select, v, st); break;
+    }
+    return launch_result();
+}
 }  // namespace
 
 extern "C" {
@@ -494,6 +516,84 @@ bd_status bd_linear_noalloc(const void *X, bd_dtype xdtype, int64_t M, int64_t K
         g_noalloc_ptr[dev] = p;
     }
     return bd_linear(X, xdtype, M, K, ldx, Wq, Y, ydtype, ldy, g_noalloc_ptr[dev], BD_NOALLOC_SCRATCH_BYTES, stream);
+}
+
+// ---- block sizes 16 and 64 (Sec. 4.2, Table 3) ----
+bd_status bd_qtensor_sizes_bs(int64_t rows, int64_t K, int block, size_t *codes_bytes, size_t *ids_bytes, size_t *scales_bytes) {
+    if (!block_size_ok(block)) return BD_ERR_INVALID_ARG;
+    if (rows <= 0 || K <= 0) return BD_ERR_INVALID_ARG;
+    if (K % block) return BD_ERR_SHAPE;
+    return bd_qtensor_sizes(rows, physical_k(K, block), codes_bytes, ids_bytes, scales_bytes);
+}
+
+bd_status bd_quantize_bs(const void *X, bd_dtype dtype, int64_t rows, int64_t K, int64_t ld, bd_select select, int block,
+                         bd_qtensor *out, void *stream) {
+    if (!block_size_ok(block) || (select != BD_SELECT_TWO_STAGE && select != BD_SELECT_MSE)) return BD_ERR_INVALID_ARG;
+    if (!X || rows <= 0 || K <= 0 || (dtype != BD_F32 && dtype != BD_BF16 && dtype != BD_F16)) return BD_ERR_INVALID_ARG;
+    if (K % block || ld < K) return BD_ERR_SHAPE;
+    if (!aligned16(X) || (ld * elem_bytes(dtype)) % 16) return BD_ERR_ALIGN;
+    bd_status s = check_qtensor(out);
+    if (s) return s;
+    if (out->rows != rows || out->K != physical_k(K, block)) return BD_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (block == 32) {
+        if (select == BD_SELECT_MSE) return launch_contig<BD_SELECT_MSE, true, false>(X, dtype, ld, view_of(out), nullptr, st);
+        return launch_contig<BD_SELECT_TWO_STAGE, true, false>(X, dtype, ld, view_of(out), nullptr, st);
+    }
+    if (block == 16) return quantize_bs_dtype<16>(X, dtype, ld, select, view_of(out), st);
+    return quantize_bs_dtype<64>(X, dtype, ld, select, view_of(out), st);
+}
+
+bd_status bd_export_canonical_bs(const bd_qtensor *q, int block, uint8_t *codes, uint8_t *ids, uint8_t *scales, void *stream) {
+    if (!block_size_ok(block)) return BD_ERR_INVALID_ARG;
+    if (block == 32) return bd_export_canonical(q, codes, ids, scales, stream);
+    bd_status s = check_qtensor(q);
+    if (s) return s;
+    if (!codes || !ids || !scales) return BD_ERR_INVALID_ARG;
+    if (!aligned16(codes)) return BD_ERR_ALIGN;
+    if (q->K % 64) return BD_ERR_SHAPE;                            // K' = 2 K with K % 16 == 0 ... K % 64 == 0 for block 64
+    const int nbp = (int)(q->K / kBlock);
+    const unsigned grid = grid_for(q->rows * nbp, 256);
+    if (block == 16) export_canonical_bs_kernel<16><<<grid, 256, 0, (cudaStream_t)stream>>>(view_of(q), codes, ids, scales, nbp);
+    else export_canonical_bs_kernel<64><<<grid, 256, 0, (cudaStream_t)stream>>>(view_of(q), codes, ids, scales, nbp);
+    return launch_result();
+}
+
+bd_status bd_linear_bs_workspace_size(int64_t M, int64_t N, int64_t K, int block, size_t *bytes) {
+    if (!bytes || !block_size_ok(block) || M <= 0 || N <= 0 || K <= 0) return BD_ERR_INVALID_ARG;
+    if (K % block) return BD_ERR_SHAPE;
+    const int64_t Kp = physical_k(K, block);
+    if (block == 32) return bd_linear_workspace_size(M, N, K, bytes);
+    size_t c, i, s, g;
+    bd_qtensor_sizes(M, Kp, &c, &i, &s);
+    bd_gemm_workspace_size(M, N, Kp, &g);
+    *bytes = align256(c) + align256(i) + align256(s) + g;
+    return BD_OK;
+}
+
+bd_status bd_linear_bs(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, int block, const bd_qtensor *Wq, void *Y,
+                       bd_dtype ydtype, int64_t ldy, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!block_size_ok(block)) return BD_ERR_INVALID_ARG;
+    if (block == 32) return bd_linear(X, xdtype, M, K, ldx, Wq, Y, ydtype, ldy, workspace, workspace_bytes, stream);
+    if (K <= 0 || K % block) return BD_ERR_SHAPE;
+    bd_status s = check_qtensor(Wq);
+    if (s) return s;
+    const int64_t Kp = physical_k(K, block), N = Wq->rows;
+    if (Wq->K != Kp || ldy < N) return BD_ERR_SHAPE;
+    if (!Y || (ydtype != BD_F32 && ydtype != BD_BF16)) return BD_ERR_INVALID_ARG;
+    size_t need;
+    s = bd_linear_bs_workspace_size(M, N, K, block, &need);
+    if (s) return s;
+    if (!workspace || workspace_bytes < need) return BD_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 255u) return BD_ERR_ALIGN;
+    size_t c, i, sc, g;
+    bd_qtensor_sizes(M, Kp, &c, &i, &sc);
+    bd_gemm_workspace_size(M, N, Kp, &g);
+    char *p = (char *)workspace;
+    bd_qtensor xq{p, p + align256(c), p + align256(c) + align256(i), M, Kp};
+    s = bd_quantize_bs(X, xdtype, M, K, ldx, BD_SELECT_TWO_STAGE, block, &xq, stream);
+    if (s) return s;
+    return gemm_dispatch(view_of(&xq), view_of(Wq), Y, ydtype, ldy, p + align256(c) + align256(i) + align256(sc), g, (cudaStream_t)stream);
 }
 
 bd_status bd_export_canonical(const bd_qtensor *q, uint8_t *codes, uint8_t *ids, uint8_t *scales, void *stream) {
