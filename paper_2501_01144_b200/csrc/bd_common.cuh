@@ -276,9 +276,11 @@ struct QView {                 // a qtensor as kernels see it
     uint8_t *ids;
     uint8_t *scales;
     int64_t rows, K;
+    int64_t ldc;               // bytes between the code rows: K / 2, or more for a view of the first K elements of
+                               // longer rows (the value cache, whose token axis grows)
 };
 inline QView view_of(const bd_qtensor *q) {
-    return QView{(uint8_t *)q->codes, (uint8_t *)q->ids, (uint8_t *)q->scales, q->rows, q->K};
+    return QView{(uint8_t *)q->codes, (uint8_t *)q->ids, (uint8_t *)q->scales, q->rows, q->K, q->K / 2};
 }
 
 }  // namespace bd

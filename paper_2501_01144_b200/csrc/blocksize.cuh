@@ -143,7 +143,7 @@ __global__ void __launch_bounds__(256) quantize_bs_kernel(const void *__restrict
     if (valid && nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
     if (!valid) { res.id = 0; res.scale = 0; }
     if (valid)
-        *(uint4 *)(out.codes + r * (out.K / 2) + (int64_t)pb * 16) = make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
+        *(uint4 *)(out.codes + r * out.ldc + (int64_t)pb * 16) = make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
     uint32_t scw = res.scale << (8 * (pb & 3)), idn = res.id << (4 * (pb & 3));
     scw |= __shfl_xor_sync(0xffffffffu, scw, 1);
     idn |= __shfl_xor_sync(0xffffffffu, idn, 1);
@@ -164,7 +164,7 @@ __global__ void export_canonical_bs_kernel(QView q, uint8_t *__restrict__ codes,
     if (t >= q.rows * nbp) return;
     const int64_t r = t / nbp;
     const int pb = (int)(t - r * nbp);
-    const uint4 u = *(const uint4 *)(q.codes + r * (q.K / 2) + (int64_t)pb * 16);
+    const uint4 u = *(const uint4 *)(q.codes + r * q.ldc + (int64_t)pb * 16);
     const uint32_t w[4] = {u.x, u.y, u.z, u.w};
     uint32_t o[4];
 #pragma unroll

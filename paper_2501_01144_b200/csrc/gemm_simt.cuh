@@ -27,7 +27,7 @@ __device__ __forceinline__ void simt_decode_block(const QView &q, int64_t row, i
         scale = 0;
         return;
     }
-    uint4 u = *(const uint4 *)(q.codes + row * (q.K / 2) + (int64_t)b * 16);
+    uint4 u = *(const uint4 *)(q.codes + row * q.ldc + (int64_t)b * 16);
     uint32_t w[4] = {u.x, u.y, u.z, u.w};
     uint32_t id = (q.ids[id_byte_offset(q.rows, row, b)] >> (4 * (b & 1))) & 15;
     uint32_t lo = c_tables.int_lo[id], hi = c_tables.int_hi[id];

@@ -617,7 +617,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                         quantize_two_stage_f32<false>(bits, qtab, res, unused, nonfinite);
                         if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
                         if (!*abort_flag)
-                            *(uint4 *)(yq.codes + (int64_t)tok * (yq.K / 2) + (int64_t)b * 16) =
+                            *(uint4 *)(yq.codes + (int64_t)tok * yq.ldc + (int64_t)b * 16) =
                                 make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
                     }
                     // scale bytes and ids of the atoms' padding (tokens past M, blocks past N / 32) are written as zeros
@@ -771,7 +771,7 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
     const int part_tokens = M <= 128 ? (int)((M + 15) / 16 * 16) : 128;
     if (!make_map_2d(&mapX, CU_TENSOR_MAP_DATA_TYPE_UINT8, x8, K, M, K, BK, 128, CU_TENSOR_MAP_SWIZZLE_128B) ||
         !make_map_2d(&mapXpart, CU_TENSOR_MAP_DATA_TYPE_UINT8, x8, K, M, K, BK, part_tokens / 2, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map_2d(&mapCodes, CU_TENSOR_MAP_DATA_TYPE_UINT8, W.codes, K / 2, N, K / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_64B) ||
+        !make_map_2d(&mapCodes, CU_TENSOR_MAP_DATA_TYPE_UINT8, W.codes, K / 2, N, (uint64_t)W.ldc, 64, 128, CU_TENSOR_MAP_SWIZZLE_64B) ||
         !make_map_2d(&mapSfW, CU_TENSOR_MAP_DATA_TYPE_UINT32, W.scales, 128, rtw * kg, kScaleAtomBytes, 128, 1, CU_TENSOR_MAP_SWIZZLE_NONE) ||
         !make_map_2d(&mapSfX, CU_TENSOR_MAP_DATA_TYPE_UINT32, sfx, 128, rtx * kg, kScaleAtomBytes, 128, 2, CU_TENSOR_MAP_SWIZZLE_NONE))
         return cudaErrorInvalidValue;
@@ -834,7 +834,7 @@ inline cudaError_t launch(const uint8_t *x8, const uint8_t *sfx, int64_t M, cons
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const QView none{nullptr, nullptr, nullptr, 0, 0};
+    const QView none{nullptr, nullptr, nullptr, 0, 0, 0};
     cudaError_t e = requant
         ? cudaLaunchKernelEx(&cfg, gemm_wtmem_kernel<true>, mapX, mapXpart, mapCodes, mapSfW, mapSfX, (const uint8_t *)W.ids, sc,
                              (int)M, (int)N, (int)rtx, (int)rtw, Y, ldy, 0, mapY, use_tma_store, (float *)scratch, *requant)

@@ -405,7 +405,7 @@ __device__ __forceinline__ void quantize_bf16_parts(const uint16_t *__restrict__
                                                     uint8_t *__restrict__ e4m3, const SmemTables &tab, uint32_t first,
                                                     uint32_t stride, uint32_t parts, uint32_t nb, uint32_t kgroups,
                                                     FastDiv div_kgroups) {
-    const uint32_t rows = (uint32_t)out.rows, tiles = (rows + kRowTile - 1) / kRowTile, half_k = (uint32_t)(out.K / 2);
+    const uint32_t rows = (uint32_t)out.rows, tiles = (rows + kRowTile - 1) / kRowTile, half_k = (uint32_t)out.ldc, row_k = (uint32_t)out.K;
     const uint32_t lane = threadIdx.x % 32u, b4 = lane & 3u, j = (lane >> 2) & 3u;
     const uint32_t row_in_part = (lane >> 4) + 32u * j;           // + 2 * w + 16 * half
     struct Part {
@@ -444,7 +444,7 @@ __device__ __forceinline__ void quantize_bf16_parts(const uint16_t *__restrict__
 #pragma unroll
                     for (int w = 0; w < 4; w++) decode_word(res.words[w], lo, hi, o[2 * w], o[2 * w + 1]);
                 }
-                uint4 *dst = (uint4 *)(e4m3 + (uint64_t)k.r * (2u * half_k) + k.b * 32u);
+                uint4 *dst = (uint4 *)(e4m3 + (uint64_t)k.r * row_k + k.b * 32u);
                 dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                 dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
             }
@@ -582,7 +582,7 @@ __global__ void __launch_bounds__(256) quantize_contig_kernel(const void *__rest
             else quantize_two_stage_f32<kBytesOnly>(bits, tab, res, o, nonfinite);
             if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
             if (WRITE_CODES)
-                *(uint4 *)(out.codes + r * (out.K / 2) + (int64_t)b * 16) =
+                *(uint4 *)(out.codes + r * out.ldc + (int64_t)b * 16) =
                     make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
             if (WRITE_E4M3) {
                 if (!kBytesOnly) {
@@ -640,7 +640,7 @@ __global__ void __launch_bounds__(256) quantize_strided_kernel(const void *__res
             uint32_t unused[8];
             quantize_two_stage_f32<false>(bits, tab, res, unused, nonfinite);
             if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
-            *(uint4 *)(out.codes + r * (out.K / 2) + (int64_t)b * 16) =
+            *(uint4 *)(out.codes + r * out.ldc + (int64_t)b * 16) =
                 make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
         }
         out.scales[scale_offset(out.rows, r, b)] = (uint8_t)res.scale;
@@ -658,7 +658,7 @@ __global__ void export_canonical_kernel(QView q, uint8_t *__restrict__ codes, ui
     if (t >= q.rows * nb) return;
     int64_t r = t / nb;
     int b = (int)(t - r * nb);
-    uint4 u = *(const uint4 *)(q.codes + r * (q.K / 2) + (int64_t)b * 16);
+    uint4 u = *(const uint4 *)(q.codes + r * q.ldc + (int64_t)b * 16);
     uint32_t w[4] = {u.x, u.y, u.z, u.w}, o[4];
 #pragma unroll
     for (int i = 0; i < 4; i++) {
@@ -695,7 +695,7 @@ __global__ void import_canonical_kernel(const uint8_t *__restrict__ codes, const
             }
             o[i] = w;
         }
-        *(uint4 *)(q.codes + r * (q.K / 2) + (int64_t)b * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+        *(uint4 *)(q.codes + r * q.ldc + (int64_t)b * 16) = make_uint4(o[0], o[1], o[2], o[3]);
         id = ids[r * nb + b] & 15u;
         sc = scales[r * nb + b];
     }
@@ -715,7 +715,7 @@ __global__ void dequantize_kernel(QView q, float *__restrict__ out, int64_t ld, 
     if (t >= q.rows * nb) return;
     int64_t r = t / nb;
     int b = (int)(t - r * nb);
-    uint4 u = *(const uint4 *)(q.codes + r * (q.K / 2) + (int64_t)b * 16);
+    uint4 u = *(const uint4 *)(q.codes + r * q.ldc + (int64_t)b * 16);
     uint32_t w[4] = {u.x, u.y, u.z, u.w};
     uint32_t id = (q.ids[id_byte_offset(q.rows, r, b)] >> (4 * (b & 1))) & 15;
     int e = (int)q.scales[scale_offset(q.rows, r, b)] - 127;
@@ -740,7 +740,7 @@ __global__ void decode_e4m3_kernel(QView q, uint8_t *__restrict__ out, int nb) {
     if (t >= q.rows * nb) return;
     int64_t r = t / nb;
     int b = (int)(t - r * nb);
-    uint4 u = *(const uint4 *)(q.codes + r * (q.K / 2) + (int64_t)b * 16);
+    uint4 u = *(const uint4 *)(q.codes + r * q.ldc + (int64_t)b * 16);
     uint32_t w[4] = {u.x, u.y, u.z, u.w}, o[8];
     uint32_t id = (q.ids[id_byte_offset(q.rows, r, b)] >> (4 * (b & 1))) & 15;
     uint32_t lo = c_tables.e4m3_lo[id], hi = c_tables.e4m3_hi[id];
@@ -764,7 +764,7 @@ __global__ void decode_e4m3_stacked_kernel(StackedViews v, int count, int64_t ro
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // see decode_e4m3_kernel
     const int h = blockIdx.y;
     const int64_t tiles = rows / kRowTile, kgs = (nb + kBlocksPerAtom - 1) / kBlocksPerAtom;
-    QView q{(uint8_t *)v.codes[h], (uint8_t *)v.ids[h], (uint8_t *)v.scales[h], rows, K};
+    QView q{(uint8_t *)v.codes[h], (uint8_t *)v.ids[h], (uint8_t *)v.scales[h], rows, K, K / 2};
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t < rows * nb) {
         const int64_t r = t / nb;
