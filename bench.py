@@ -552,6 +552,56 @@ def run_gpu(args, rank, world, local_rank):
         bd.poll_status()
         time.sleep(0.3)
 
+    # ---- KV cache (appendix "Quantization Dimension", Fig. 9b), Mistral-7B shape: 8 KV heads of head_dim 128 with 4113
+    # tokens each (128 stored chunks + 17 recent tokens in high precision); one decode step = append one token per head,
+    # then scores and P V for the 4 query heads of each KV head.  One cache object per KV head, so a step is dozens of
+    # small launches: the time is launch-bound, far from the 4.6 MB of cache bytes it reads ----
+    kv_cache = None
+    if rank == 0:
+        kvh, grp, hd, n_tok, cap = 8, 4, 128, 4113, 4224
+        rng_kv = np.random.default_rng(6)
+        caches = []
+        for g in range(kvh):
+            cch = bd.KVCache(cap, hd, device=dev)
+            cch.append(dev_bf16(inputs.to_bf16_bits(rng_kv.standard_normal((n_tok, hd)).astype(np.float32))),
+                       dev_bf16(inputs.to_bf16_bits(rng_kv.standard_normal((n_tok, hd)).astype(np.float32))))
+            caches.append(cch)
+        q_rows = [bd.quantize_act(dev_bf16(inputs.to_bf16_bits(rng_kv.standard_normal((grp, hd)).astype(np.float32)))) for _ in range(kvh)]
+        pitch = (n_tok + 3) // 4 * 4
+        probs = [torch.softmax(torch.randn(grp, pitch, device=dev), -1)[:, :n_tok] for _ in range(kvh)]
+        s_out = torch.empty(grp, n_tok, dtype=torch.float32, device=dev)
+        o_out = torch.empty(grp, hd, dtype=torch.bfloat16, device=dev)
+
+        def attend():
+            for g in range(kvh):
+                caches[g].scores(q_rows[g], out=s_out)
+                caches[g].pv(probs[g], out=o_out)
+
+        for _ in range(3):
+            attend()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(10):
+            attend()
+        e1.record()
+        torch.cuda.synchronize()
+        attend_us = e0.elapsed_time(e1) / 10 * 1e3
+        new_k = dev_bf16(inputs.to_bf16_bits(rng_kv.standard_normal((1, hd)).astype(np.float32)))
+        e0.record()
+        for _ in range(10):                                   # ten more tokens per head (27 recent tokens at the end)
+            for g in range(kvh):
+                caches[g].append(new_k, new_k)
+        e1.record()
+        torch.cuda.synchronize()
+        append_us = e0.elapsed_time(e1) / 10 * 1e3
+        cache_bytes = kvh * 2 * n_tok * hd * 0.546875
+        kv_cache = {"workload": "8 KV heads x 4113 tokens x head_dim 128, 4 query heads per KV head, one object per KV head",
+                    "scores_and_pv_us_per_step": attend_us, "append_one_token_us_per_step": append_us,
+                    "cache_bytes_read_per_step": cache_bytes, "cache_read_gbs": cache_bytes / attend_us / 1e3,
+                    "stored_bits_per_value": 4.375, "recent_tokens_in_high_precision": n_tok % 32}
+        del caches, probs
+        bd.poll_status()
+
     # ---- attention products with both operands quantised online (Mistral-7B shapes: 32 heads, 8 KV heads,
     # 4096 tokens, head_dim 128; reported, not part of the timed step).  QK^T is bound by the write of the
     # scores, PV by the read of the fp32 probabilities. ----
@@ -680,6 +730,7 @@ def run_gpu(args, rank, world, local_rank):
         "llama2_mlp_m_sweep": sweep,
         "chained_layers": chained,
         "block_sizes": block_sizes,
+        "kv_cache": kv_cache,
         "attention_mistral7b": attention,
     }
     print(json.dumps(line))

@@ -207,6 +207,43 @@ bd_status bd_linear_bs(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int
                        const bd_qtensor *Wq, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace,
                        size_t workspace_bytes, void *stream);
 
+/* KV cache of one KV head (appendix "Quantization Dimension", Fig. 9b).  Keys are quantised
+ * sub-token-wise (along head_dim) when they arrive and appended as rows of the key operand
+ * k [capacity, head_dim].  Values are quantised sub-channel-wise, along the token axis: the
+ * value operand is v [head_dim, capacity] with blocks of 32 consecutive tokens per channel.
+ * Such a block cannot take a single new token, so the newest (length mod 32) value rows are
+ * kept in high precision in v_recent (the source type, [32, head_dim]) and are quantised
+ * once, as a whole chunk, when 32 are there; nothing stored is requantised.
+ * All buffers are caller-allocated device memory: k and v as bd_qtensor_sizes(capacity,
+ * head_dim) and (head_dim, capacity) say, v_recent as bd_kvcache_recent_bytes.  head_dim is
+ * a multiple of 32, at most 128; capacity a multiple of 32.  `length` is host state that
+ * bd_kvcache_append advances (the struct is not thread-safe).  Call bd_kvcache_reset once
+ * before the first append (it clears scales and ids and sets length = 0).
+ *   bd_kvcache_append   t new tokens: Knew, Vnew [t, head_dim] of the cache's dtype.
+ *   bd_kvcache_scores   S [q, length] = dq(Q) dq(K)^T for a quantised query operand Q [q, head_dim].
+ *   bd_kvcache_pv       O [q, head_dim] = P V for fp32 probabilities P [q, length]: the columns
+ *                       over stored chunks are quantised online along the keys and multiplied with
+ *                       the 4-bit values; the columns of the recent tokens are multiplied in fp32
+ *                       with the high-precision rows.  Once a chunk is stored, P and its row
+ *                       pitch (ldp * 4 bytes) must be 16-byte aligned.
+ * workspace: bd_kvcache_workspace_size(capacity, head_dim, q) bytes, 256-byte aligned. */
+typedef struct {
+    bd_qtensor k;       /* [capacity, head_dim]                      */
+    bd_qtensor v;       /* [head_dim, capacity]                      */
+    void *v_recent;     /* [32, head_dim] elements of `dtype`        */
+    bd_dtype dtype;     /* type of the key / value rows handed in    */
+    int64_t capacity, head_dim, length;
+} bd_kvcache;
+bd_status bd_kvcache_recent_bytes(int64_t head_dim, bd_dtype dtype, size_t *bytes);
+bd_status bd_kvcache_reset(bd_kvcache *c, void *stream);
+bd_status bd_kvcache_append(bd_kvcache *c, const void *Knew, const void *Vnew, int64_t t, int64_t ldk, int64_t ldv,
+                            void *stream);
+bd_status bd_kvcache_workspace_size(int64_t capacity, int64_t head_dim, int64_t q_rows, size_t *bytes);
+bd_status bd_kvcache_scores(const bd_kvcache *c, const bd_qtensor *Q, void *S, bd_dtype sdtype, int64_t lds,
+                            void *workspace, size_t workspace_bytes, void *stream);
+bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int64_t ldp, void *Y, bd_dtype ydtype,
+                        int64_t ldy, void *workspace, size_t workspace_bytes, void *stream);
+
 /* bd_linear for callers that can neither allocate device memory nor hand in a
  * workspace (the paper has no counterpart; this is a convenience of the library).
  * Think of code that runs where cudaMalloc is off limits: inside a region whose

@@ -30,6 +30,11 @@ class _CQTensor(ctypes.Structure):
                 ("rows", ctypes.c_int64), ("K", ctypes.c_int64)]
 
 
+class _CKVCache(ctypes.Structure):
+    _fields_ = [("k", _CQTensor), ("v", _CQTensor), ("v_recent", ctypes.c_void_p), ("dtype", ctypes.c_int),
+                ("capacity", ctypes.c_int64), ("head_dim", ctypes.c_int64), ("length", ctypes.c_int64)]
+
+
 def library_path():
     return _LIB_PATH
 
@@ -68,6 +73,13 @@ def load():
     lib.bd_linear_workspace_size.argtypes = [i64, i64, i64, szp]
     lib.bd_linear.argtypes = [vp, ci, i64, i64, i64, qp, vp, ci, i64, vp, sz, vp]
     lib.bd_linear_noalloc.argtypes = [vp, ci, i64, i64, i64, qp, vp, ci, i64, vp]
+    kp = ctypes.POINTER(_CKVCache)
+    lib.bd_kvcache_recent_bytes.argtypes = [i64, ci, szp]
+    lib.bd_kvcache_reset.argtypes = [kp, vp]
+    lib.bd_kvcache_append.argtypes = [kp, vp, vp, i64, i64, i64, vp]
+    lib.bd_kvcache_workspace_size.argtypes = [i64, i64, i64, szp]
+    lib.bd_kvcache_scores.argtypes = [kp, qp, vp, ci, i64, vp, sz, vp]
+    lib.bd_kvcache_pv.argtypes = [kp, vp, i64, i64, vp, ci, i64, vp, sz, vp]
     lib.bd_qtensor_sizes_bs.argtypes = [i64, i64, ci, szp, szp, szp]
     lib.bd_quantize_bs.argtypes = [vp, ci, i64, i64, i64, ci, ci, qp, vp]
     lib.bd_export_canonical_bs.argtypes = [qp, ci, vp, vp, vp, vp]
@@ -334,6 +346,60 @@ def linear_bs(X, Wq, block, out=None, dtype=torch.bfloat16, workspace=None, stre
     _check(load().bd_linear_bs(ptr, dt, M, K, ld, block, ctypes.byref(cw), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
                                out.stride(0), wptr, wbytes, _stream(stream)))
     return out
+
+
+class KVCache:
+    """KV cache of one KV head (appendix "Quantization Dimension", Fig. 9b): keys quantised per token along
+    head_dim, values in 4-bit chunks of 32 tokens along the token axis, the newest length % 32 value rows in
+    high precision.  Buffers are torch tensors; every step runs in the library."""
+
+    def __init__(self, capacity, head_dim, dtype=torch.bfloat16, device="cuda"):
+        self.capacity, self.head_dim, self.dtype = capacity, head_dim, dtype
+        self.k = QTensor(capacity, head_dim, device)
+        self.v = QTensor(head_dim, capacity, device)
+        self.v_recent = torch.zeros(32, head_dim, dtype=dtype, device=device)
+        self._c = _CKVCache(self.k.c_struct(), self.v.c_struct(), self.v_recent.data_ptr(), _TORCH_DTYPE[dtype], capacity, head_dim, 0)
+        self._ws = None
+        _check(load().bd_kvcache_reset(ctypes.byref(self._c), _stream()))
+
+    @property
+    def length(self):
+        return int(self._c.length)
+
+    def append(self, k_new, v_new, stream=None):
+        kp, kdt, ldk = _src(k_new)
+        vp_, vdt, ldv = _src(v_new)
+        if kdt != self._c.dtype or vdt != self._c.dtype or k_new.shape != v_new.shape or k_new.shape[1] != self.head_dim:
+            raise ValueError("key / value rows must be [t, head_dim] of the cache's dtype")
+        _check(load().bd_kvcache_append(ctypes.byref(self._c), kp, vp_, k_new.shape[0], ldk, ldv, _stream(stream)))
+
+    def _workspace(self, q_rows):
+        b = ctypes.c_size_t()
+        _check(load().bd_kvcache_workspace_size(self.capacity, self.head_dim, q_rows, ctypes.byref(b)))
+        if self._ws is None or self._ws.numel() < b.value:
+            self._ws = torch.empty(max(b.value, 256), dtype=torch.uint8, device=self.k.codes.device)
+        return ctypes.c_void_p(self._ws.data_ptr()), self._ws.numel()
+
+    def scores(self, Q, out=None, dtype=torch.float32, stream=None):
+        """S [q, length] = dq(Q) dq(K)^T for a quantised query operand Q [q, head_dim]."""
+        if out is None:
+            out = torch.empty(Q.rows, self.length, dtype=dtype, device=self.k.codes.device)
+        wptr, wbytes = self._workspace(Q.rows)
+        cq = Q.c_struct()
+        _check(load().bd_kvcache_scores(ctypes.byref(self._c), ctypes.byref(cq), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
+                                        out.stride(0), wptr, wbytes, _stream(stream)))
+        return out
+
+    def pv(self, P, out=None, dtype=torch.float32, stream=None):
+        """O [q, head_dim] = P V for fp32 probabilities P [q, length]."""
+        if P.dtype != torch.float32 or P.dim() != 2 or P.stride(1) != 1 or P.shape[1] != self.length:
+            raise ValueError("P must be fp32 [q, length] with a contiguous last axis")
+        if out is None:
+            out = torch.empty(P.shape[0], self.head_dim, dtype=dtype, device=P.device)
+        wptr, wbytes = self._workspace(P.shape[0])
+        _check(load().bd_kvcache_pv(ctypes.byref(self._c), ctypes.c_void_p(P.data_ptr()), P.shape[0], P.stride(0),
+                                    ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype), out.stride(0), wptr, wbytes, _stream(stream)))
+        return out
 
 
 NOALLOC_SCRATCH_BYTES = 32 << 20

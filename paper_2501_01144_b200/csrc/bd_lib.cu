@@ -10,6 +10,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "blocksize.cuh"
+#include "kvcache.cuh"
 #include "quantize.cuh"
 
 using namespace bd;
@@ -193,6 +194,32 @@ namespace {
 constexpr int kMaxDevices = 64;
 void *g_noalloc_ptr[kMaxDevices] = {};
 }  // namespace
+
+// launchers of the KV-cache kernels per source type
+template <int DT>
+void launch_kv_keys(const void *Knew, int64_t ldk, int64_t t, const QView &k, int64_t row0, cudaStream_t st) {
+    kv_append_keys_kernel<DT><<<grid_for(t * kBlocksPerAtom, 256), 256, 0, st>>>(Knew, ldk, t, k, row0, (int)(k.K / kBlock));
+}
+template <int DT>
+void launch_kv_chunks(const void *src, int64_t ld, int n_chunks, const QView &v, int chunk0, cudaStream_t st) {
+    const int pairs = (chunk0 + n_chunks + 1) / 2 - chunk0 / 2;
+    kv_quantize_chunks_kernel<DT><<<grid_for(v.rows * pairs, 256), 256, 0, st>>>(src, ld, n_chunks, v, chunk0);
+}
+template <int DT>
+void launch_kv_finish(const float *part, int64_t ld_part, const float *P, int64_t ldp, int64_t n_q, int n_recent, const void *recent,
+                      int d, int64_t q_rows, void *Y, bd_dtype ydt, int64_t ldy, cudaStream_t st) {
+    const unsigned grid = grid_for(q_rows * d, 256);
+    if (ydt == BD_BF16)
+        kv_pv_finish_kernel<DT, __nv_bfloat16><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, recent, d, q_rows, (__nv_bfloat16 *)Y, ldy);
+    else
+        kv_pv_finish_kernel<DT, float><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, recent, d, q_rows, (float *)Y, ldy);
+}
+#define BD_KV_DISPATCH(dt, fn, ...)                          \
+    switch (dt) {                                            \
+        case BD_F32: fn<BD_F32>(__VA_ARGS__); break;         \
+        case BD_BF16: fn<BD_BF16>(__VA_ARGS__); break;       \
+        default: fn<BD_F16>(__VA_ARGS__); break;             \
+    }
 
 // launchers of the quantizer for block sizes 16 and 64
 namespace {
@@ -594,6 +621,147 @@ bd_status bd_linear_bs(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int
     s = bd_quantize_bs(X, xdtype, M, K, ldx, BD_SELECT_TWO_STAGE, block, &xq, stream);
     if (s) return s;
     return gemm_dispatch(view_of(&xq), view_of(Wq), Y, ydtype, ldy, p + align256(c) + align256(i) + align256(sc), g, (cudaStream_t)stream);
+}
+
+// ---- KV cache (appendix "Quantization Dimension", Fig. 9b) ----
+static bd_status check_kvcache(const bd_kvcache *c) {
+    if (!c || !c->v_recent) return BD_ERR_INVALID_ARG;
+    bd_status s = check_qtensor(&c->k);
+    if (s) return s;
+    s = check_qtensor(&c->v);
+    if (s) return s;
+    if (c->dtype != BD_F32 && c->dtype != BD_BF16 && c->dtype != BD_F16) return BD_ERR_INVALID_ARG;
+    if (c->head_dim <= 0 || c->head_dim % kBlock || c->head_dim > 128 || c->capacity <= 0 || c->capacity % kBlock) return BD_ERR_SHAPE;
+    if (c->k.rows != c->capacity || c->k.K != c->head_dim || c->v.rows != c->head_dim || c->v.K != c->capacity) return BD_ERR_SHAPE;
+    if (c->length < 0 || c->length > c->capacity) return BD_ERR_SHAPE;
+    if (!aligned16(c->v_recent)) return BD_ERR_ALIGN;
+    return BD_OK;
+}
+
+bd_status bd_kvcache_recent_bytes(int64_t head_dim, bd_dtype dtype, size_t *bytes) {
+    if (!bytes || head_dim <= 0) return BD_ERR_INVALID_ARG;
+    *bytes = (size_t)kBlock * (size_t)head_dim * (size_t)elem_bytes(dtype);
+    return BD_OK;
+}
+
+bd_status bd_kvcache_reset(bd_kvcache *c, void *stream) {
+    bd_status s = check_kvcache(c);
+    if (s) return s;
+    size_t cb, ib, sb;
+    cudaStream_t st = (cudaStream_t)stream;
+    bd_qtensor_sizes(c->capacity, c->head_dim, &cb, &ib, &sb);
+    if ((s = cuda_result(cudaMemsetAsync(c->k.ids, 0, ib, st)))) return s;
+    if ((s = cuda_result(cudaMemsetAsync(c->k.scales, 0, sb, st)))) return s;
+    bd_qtensor_sizes(c->head_dim, c->capacity, &cb, &ib, &sb);
+    if ((s = cuda_result(cudaMemsetAsync(c->v.ids, 0, ib, st)))) return s;
+    if ((s = cuda_result(cudaMemsetAsync(c->v.scales, 0, sb, st)))) return s;
+    c->length = 0;
+    return BD_OK;
+}
+
+bd_status bd_kvcache_append(bd_kvcache *c, const void *Knew, const void *Vnew, int64_t t, int64_t ldk, int64_t ldv, void *stream) {
+    bd_status s = check_kvcache(c);
+    if (s) return s;
+    if (!Knew || !Vnew || t <= 0) return BD_ERR_INVALID_ARG;
+    const int64_t d = c->head_dim;
+    const int esz = elem_bytes(c->dtype);
+    if (ldk < d || ldv < d || c->length + t > c->capacity) return BD_ERR_SHAPE;
+    if (!aligned16(Knew) || !aligned16(Vnew) || (ldk * esz) % 16 || (ldv * esz) % 16) return BD_ERR_ALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    const QView kq = view_of(&c->k), vq = view_of(&c->v);
+    int kernels = 0;
+    // keys: one quantisation per new token, appended as rows
+    BD_KV_DISPATCH(c->dtype, launch_kv_keys, Knew, ldk, t, kq, c->length, st);
+    kernels++;
+    // values: complete the waiting chunk, then whole chunks straight from the source, then the new remainder
+    int64_t done = 0, len = c->length;
+    const int waiting = (int)(len % kBlock);
+    if (waiting) {
+        const int fill = (int)std::min<int64_t>(kBlock - waiting, t);
+        kv_store_recent_kernel<<<grid_for((int64_t)fill * d * esz / 2, 256), 256, 0, st>>>(Vnew, ldv * esz, fill, (int)(d * esz),
+                                                                                         (uint8_t *)c->v_recent, waiting);
+        kernels++;
+        if (waiting + fill == kBlock) {
+            BD_KV_DISPATCH(c->dtype, launch_kv_chunks, c->v_recent, d, 1, vq, (int)(len / kBlock), st);
+            kernels++;
+        }
+        done = fill;
+        len += fill;
+    }
+    const int64_t whole = (t - done) / kBlock;
+    if (whole) {
+        BD_KV_DISPATCH(c->dtype, launch_kv_chunks, (const char *)Vnew + done * ldv * esz, ldv, (int)whole, vq, (int)(len / kBlock), st);
+        kernels++;
+        done += whole * kBlock;
+    }
+    if (done < t) {
+        const int rest = (int)(t - done);
+        kv_store_recent_kernel<<<grid_for((int64_t)rest * d * esz / 2, 256), 256, 0, st>>>((const char *)Vnew + done * ldv * esz, ldv * esz, rest,
+                                                                                         (int)(d * esz), (uint8_t *)c->v_recent, 0);
+        kernels++;
+    }
+    c->length += t;
+    return launch_result(kernels);
+}
+
+bd_status bd_kvcache_workspace_size(int64_t capacity, int64_t head_dim, int64_t q_rows, size_t *bytes) {
+    if (!bytes || capacity <= 0 || head_dim <= 0 || q_rows <= 0) return BD_ERR_INVALID_ARG;
+    if (capacity % kBlock || head_dim % kBlock) return BD_ERR_SHAPE;
+    size_t g1, g2, cb, ib, sb;
+    bd_gemm_workspace_size(q_rows, capacity, head_dim, &g1);       // scores
+    bd_gemm_workspace_size(q_rows, head_dim, capacity, &g2);       // P x V over the stored chunks
+    bd_qtensor_sizes(q_rows, capacity, &cb, &ib, &sb);            // the quantised probabilities
+    const size_t pv = align256(cb) + align256(ib) + align256(sb) + align256(g2) + align256((size_t)q_rows * head_dim * sizeof(float));
+    *bytes = std::max(align256(g1), pv);
+    return BD_OK;
+}
+
+bd_status bd_kvcache_scores(const bd_kvcache *c, const bd_qtensor *Q, void *S, bd_dtype sdtype, int64_t lds, void *workspace,
+                            size_t workspace_bytes, void *stream) {
+    bd_status s = check_kvcache(c);
+    if (s) return s;
+    s = check_qtensor(Q);
+    if (s) return s;
+    if (Q->K != c->head_dim || c->length == 0 || lds < c->length) return BD_ERR_SHAPE;
+    if (!S || (sdtype != BD_F32 && sdtype != BD_BF16)) return BD_ERR_INVALID_ARG;
+    QView keys = view_of(&c->k);
+    keys.rows = c->length;                                        // the rows stored so far (one scale atom along K: the
+    return gemm_dispatch(view_of(Q), keys, S, sdtype, lds, workspace, workspace_bytes, (cudaStream_t)stream);   // atom order ignores the row count)
+}
+
+bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int64_t ldp, void *Y, bd_dtype ydtype, int64_t ldy,
+                        void *workspace, size_t workspace_bytes, void *stream) {
+    bd_status s = check_kvcache(c);
+    if (s) return s;
+    if (!P || !Y || q_rows <= 0 || (ydtype != BD_F32 && ydtype != BD_BF16)) return BD_ERR_INVALID_ARG;
+    if (c->length == 0 || ldp < c->length || ldy < c->head_dim) return BD_ERR_SHAPE;
+    if (c->length >= kBlock && (!aligned16(P) || (ldp * 4) % 16)) return BD_ERR_ALIGN;   // the quantizer reads P in 16-byte pieces
+    size_t need;
+    bd_kvcache_workspace_size(c->capacity, c->head_dim, q_rows, &need);
+    if (!workspace || workspace_bytes < need) return BD_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 255u) return BD_ERR_ALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t d = c->head_dim, n_q = c->length / kBlock * kBlock;
+    const int n_recent = (int)(c->length - n_q);
+    float *part = nullptr;
+    if (n_q) {
+        // probabilities over the stored chunks: quantised online along the keys, then the block-scaled product
+        size_t cb, ib, sb, g2;
+        bd_qtensor_sizes(q_rows, n_q, &cb, &ib, &sb);
+        bd_gemm_workspace_size(q_rows, d, n_q, &g2);
+        char *p = (char *)workspace;
+        bd_qtensor pq{p, p + align256(cb), p + align256(cb) + align256(ib), q_rows, n_q};
+        char *gws = p + align256(cb) + align256(ib) + align256(sb);
+        part = (float *)(gws + align256(g2));
+        s = launch_contig<BD_SELECT_TWO_STAGE, true, false>(P, BD_F32, ldp, view_of(&pq), nullptr, st);
+        if (s) return s;
+        QView vals = view_of(&c->v);
+        vals.K = n_q;                                             // the first n_q tokens of every channel; the pitch stays
+        s = gemm_dispatch(view_of(&pq), vals, part, BD_F32, d, gws, g2, st);
+        if (s) return s;
+    }
+    BD_KV_DISPATCH(c->dtype, launch_kv_finish, part, d, P, ldp, n_q, n_recent, c->v_recent, (int)d, q_rows, Y, ydtype, ldy, st);
+    return launch_result();
 }
 
 bd_status bd_export_canonical(const bd_qtensor *q, uint8_t *codes, uint8_t *ids, uint8_t *scales, void *stream) {

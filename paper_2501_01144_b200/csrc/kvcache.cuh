@@ -1,0 +1,115 @@
+// KV cache of one KV head in DialectFP4 (appendix "Quantization Dimension", Fig. 9b).
+//
+// Keys are quantised sub-token-wise (blocks of 32 along head_dim): a new key vector is quantised once and becomes
+// the next row of the key operand [capacity, head_dim].  Values are quantised sub-channel-wise, along the token
+// axis, which is their multiplication dimension in score x V: the value operand is [head_dim, capacity] and a
+// block is 32 consecutive tokens of one channel.  A single new token cannot extend such a block, so the newest
+// N mod 32 value rows wait in high precision (`recent`, the source type) and are quantised once, as a whole chunk,
+// when there are 32 of them.  Nothing stored is ever requantised.
+//
+// Both operands keep the library's ordinary layout, so the product kernels read them through views: the first
+// `length` rows of the keys, and the first 32 * (length / 32) elements of every value row (code rows keep the
+// pitch of the full capacity).  With head_dim <= 128 the key operand has one scale atom along K and the value
+// operand one row tile, so the atom order of both does not depend on the capacity.
+#pragma once
+#include "bd_common.cuh"
+#include "quantize.cuh"
+
+namespace bd {
+
+// New key rows: thread = (new row i, block b of 4); the four lanes of a row merge scale bytes and id nibbles.
+template <int DT>
+__global__ void __launch_bounds__(256) kv_append_keys_kernel(const void *__restrict__ Knew, int64_t ldk, int64_t t_new, QView k,
+                                                             int64_t row0, int nb) {
+    __shared__ SmemTables tab;
+    load_tables(tab);
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / kBlocksPerAtom;
+    const int b = (int)(t % kBlocksPerAtom);
+    const bool valid = i < t_new && b < nb;
+    BlockResult res;
+    res.id = 0; res.scale = 0;
+    res.words[0] = res.words[1] = res.words[2] = res.words[3] = 0;
+    const int64_t r = row0 + i;
+    if (valid) {
+        uint32_t bits[32], unused[8];
+        Loader<DT>::contiguous((const char *)Knew + (i * ldk + (int64_t)b * 32) * Loader<DT>::kElemBytes, bits);
+        bool nonfinite;
+        quantize_two_stage_f32<false>(bits, tab, res, unused, nonfinite);
+        if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
+        *(uint4 *)(k.codes + r * k.ldc + (int64_t)b * 16) = make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
+    }
+    uint32_t scw = res.scale << (8 * b), idn = res.id << (4 * b);
+    scw |= __shfl_xor_sync(0xffffffffu, scw, 1);
+    idn |= __shfl_xor_sync(0xffffffffu, idn, 1);
+    scw |= __shfl_xor_sync(0xffffffffu, scw, 2);
+    idn |= __shfl_xor_sync(0xffffffffu, idn, 2);
+    if (b == 0 && i < t_new) {
+        *(uint32_t *)(k.scales + scale_offset(k.rows, r, 0)) = scw;
+        *(uint16_t *)(k.ids + id_byte_offset(k.rows, r, 0)) = (uint16_t)idn;
+    }
+}
+
+// Value rows that do not complete a chunk: copied as they are into the high-precision slots.
+__global__ void kv_store_recent_kernel(const void *__restrict__ Vnew, int64_t ldv_bytes, int rows, int row_bytes, uint8_t *__restrict__ recent,
+                                       int slot0) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;          // one 2-byte unit each
+    const int units = row_bytes / 2;
+    if (t >= rows * units) return;
+    const int i = t / units, u = t % units;
+    ((uint16_t *)(recent + (int64_t)(slot0 + i) * row_bytes))[u] = ((const uint16_t *)((const char *)Vnew + i * ldv_bytes))[u];
+}
+
+// Whole chunks of 32 value rows -> one block per channel.  Thread = (channel c, pair of chunks p): the chunks 2p and
+// 2p + 1 of a channel share an id byte, so one thread writes both nibbles; a nibble of an earlier call is kept.
+// src: [32 * n_chunks, ld] elements, the rows of chunks chunk0 .. chunk0 + n_chunks - 1.
+template <int DT>
+__global__ void __launch_bounds__(256) kv_quantize_chunks_kernel(const void *__restrict__ src, int64_t ld, int n_chunks, QView v, int chunk0) {
+    __shared__ SmemTables tab;
+    load_tables(tab);
+    const int d = (int)v.rows;
+    const int pair0 = chunk0 / 2, n_pairs = (chunk0 + n_chunks + 1) / 2 - pair0;
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (int64_t)d * n_pairs) return;
+    const int c = (int)(t % d), p = pair0 + (int)(t / d);          // neighbouring lanes = neighbouring channels
+    uint32_t idbyte = 0;
+    for (int h = 0; h < 2; h++) {
+        const int chunk = 2 * p + h;
+        if (chunk < chunk0) {                                     // stored by an earlier call: keep its nibble
+            idbyte |= v.ids[id_byte_offset(v.rows, c, chunk)] & 0x0fu;
+            continue;
+        }
+        if (chunk >= chunk0 + n_chunks) continue;
+        uint32_t bits[32], unused[8];
+        const char *base = (const char *)src + ((int64_t)(chunk - chunk0) * 32 * ld + c) * Loader<DT>::kElemBytes;
+#pragma unroll
+        for (int k = 0; k < 32; k++) bits[k] = Loader<DT>::one(base + (int64_t)k * ld * Loader<DT>::kElemBytes);
+        BlockResult res;
+        bool nonfinite;
+        quantize_two_stage_f32<false>(bits, tab, res, unused, nonfinite);
+        if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
+        *(uint4 *)(v.codes + (int64_t)c * v.ldc + (int64_t)chunk * 16) = make_uint4(res.words[0], res.words[1], res.words[2], res.words[3]);
+        v.scales[scale_offset(v.rows, c, chunk)] = (uint8_t)res.scale;
+        idbyte |= res.id << (4 * h);
+    }
+    v.ids[id_byte_offset(v.rows, c, 2 * p)] = (uint8_t)idbyte;
+}
+
+// O[q, c] = (product over the stored chunks, fp32, or nothing) + sum over the recent tokens of P[q, n_q + k] * V_recent[k, c],
+// the latter in fp32 on the source values ("maintained in high precision").  Thread = one output.
+template <int DT, typename OutT>
+__global__ void kv_pv_finish_kernel(const float *__restrict__ part, int64_t ld_part, const float *__restrict__ P, int64_t ldp, int64_t n_q,
+                                    int n_recent, const void *__restrict__ recent, int d, int64_t q_rows, OutT *__restrict__ Y, int64_t ldy) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= q_rows * d) return;
+    const int64_t q = t / d;
+    const int c = (int)(t % d);
+    float acc = 0.0f;
+    for (int k = 0; k < n_recent; k++)
+        acc = fmaf(P[q * ldp + n_q + k], __uint_as_float(Loader<DT>::one((const char *)recent + ((int64_t)k * d + c) * Loader<DT>::kElemBytes)), acc);
+    const float y = (part ? part[q * ld_part + c] : 0.0f) + acc;
+    if (sizeof(OutT) == 2) ((__nv_bfloat16 *)Y)[q * ldy + c] = __float2bfloat16_rn(y);
+    else ((float *)Y)[q * ldy + c] = y;
+}
+
+}  // namespace bd

@@ -1,0 +1,108 @@
+"""The KV-cache structure (appendix "Quantization Dimension", Fig. 9b) on the GPU against its oracle: stored keys and
+value chunks bit for bit, the high-precision remainder byte for byte, scores and P V within the product tolerance,
+under token-by-token and bulk appends."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2501_01144_b200 as bd
+from oracle.kvcache import KVCache as OracleCache
+from paper_2501_01144_b200 import inputs
+from util import ORACLE_DTYPE, gemm_tolerance_ok, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def _rows(n, d, kind, seed):
+    rng = np.random.default_rng(seed)
+    k = rng.standard_normal((n, d)).astype(np.float32)
+    k[:, rng.integers(0, d)] *= 12.0
+    v = (rng.standard_normal((n, d)) * np.exp2(rng.integers(-3, 4, (1, d)))).astype(np.float32)
+    if kind == torch.float32:
+        return k, v
+    if kind == torch.bfloat16:
+        return inputs.to_bf16_bits(k), inputs.to_bf16_bits(v)
+    return inputs.to_f16_bits(k), inputs.to_f16_bits(v)
+
+
+def _stored_values(cache, n_q):
+    """Canonical view of the first n_q tokens of the library's value operand [head_dim, n_q]."""
+    codes, ids, scales = (t.cpu().numpy() for t in bd.export_canonical(cache.v))
+    return codes[:, :n_q // 2], ids[:, :n_q // 32], scales[:, :n_q // 32]
+
+
+def _check_state(cache, ref, kind):
+    n, n_q = ref.length, ref.length // 32 * 32
+    assert cache.length == n
+    kc, ki, ks = (t.cpu().numpy()[:n] for t in bd.export_canonical(cache.k))
+    rc, ri, rs = ref.keys()
+    assert np.array_equal(ks, rs) and np.array_equal(ki, ri) and np.array_equal(kc, rc), "stored keys"
+    if n_q:
+        got, want = _stored_values(cache, n_q), ref.values_quantised()
+        assert all(np.array_equal(g, w) for g, w in zip(got, want)), "stored value chunks"
+    r = n - n_q
+    if r:
+        recent = cache.v_recent[:r].float().cpu().numpy().astype(np.float64)
+        assert np.array_equal(recent, ref.values_recent()), "high-precision remainder"
+
+
+@pytest.mark.parametrize("kind", [torch.bfloat16, torch.float32, torch.float16])
+@pytest.mark.parametrize("d", [64, 128])
+def test_appends_in_uneven_pieces_match_the_oracle(kind, d):
+    total, cap = 333, 512
+    k, v = _rows(total, d, kind, seed=d + 1)
+    cache, ref = bd.KVCache(cap, d, dtype=kind), OracleCache(d, dtype=ORACLE_DTYPE[kind])
+    pos = 0
+    for t in (1, 1, 29, 1, 1, 40, 64, 3, 100, 31, 32, 30):            # crossing chunk borders in every way
+        cache.append(to_device(k[pos:pos + t], kind), to_device(v[pos:pos + t], kind))
+        ref.append(k[pos:pos + t], v[pos:pos + t])
+        pos += t
+        _check_state(cache, ref, kind)
+    assert pos == total
+    bd.poll_status()
+
+
+@pytest.mark.parametrize("n,q_rows", [(19, 4), (32, 1), (77, 4), (1000, 8), (4096, 4), (4127, 130)])
+def test_scores_and_pv_match_the_oracle(n, q_rows):
+    d, cap, kind = 128, 4160, torch.bfloat16
+    k, v = _rows(n, d, kind, seed=n)
+    cache, ref = bd.KVCache(cap, d, dtype=kind), OracleCache(d)
+    cache.append(to_device(k, kind), to_device(v, kind))
+    ref.append(k, v)
+    _check_state(cache, ref, kind)
+    rng = np.random.default_rng(n + q_rows)
+    qb = inputs.to_bf16_bits(rng.standard_normal((q_rows, d)).astype(np.float32))
+    Qq = bd.quantize_act(to_device(qb, torch.bfloat16))
+    S = cache.scores(Qq).cpu().numpy()
+    Sref, T = ref.scores(oracle.quantize(qb, dtype=oracle.BF16))
+    ok, ratio = gemm_tolerance_ok(S, Sref, T)
+    assert ok, f"scores: max err / bound = {ratio}"
+    # probabilities: softmax of the library's own scores in fp64, handed in as fp32 (softmax stays in high precision)
+    z = S.astype(np.float64) / np.sqrt(d)
+    P = np.exp(z - z.max(-1, keepdims=True))
+    P = (P / P.sum(-1, keepdims=True)).astype(np.float32)
+    Pd = torch.zeros(q_rows, (n + 3) // 4 * 4, device="cuda")[:, :n]          # a row pitch of whole 16 bytes
+    Pd.copy_(torch.from_numpy(P))
+    O = cache.pv(Pd).cpu().numpy()
+    Oref, To = ref.pv(P)
+    ok, ratio = gemm_tolerance_ok(O, Oref, To)
+    assert ok, f"P V: max err / bound = {ratio}"
+    O16 = cache.pv(Pd, dtype=torch.bfloat16)
+    assert torch.equal(O16.cpu(), torch.from_numpy(O).to(torch.bfloat16))
+    bd.poll_status()
+
+
+def test_decoding_token_by_token_never_changes_a_stored_chunk():
+    d, kind = 64, torch.bfloat16
+    k, v = _rows(100, d, kind, seed=9)
+    cache = bd.KVCache(128, d, dtype=kind)
+    cache.append(to_device(k[:64], kind), to_device(v[:64], kind))
+    before = [np.array(b) for b in _stored_values(cache, 64)]
+    for t in range(64, 100):
+        cache.append(to_device(k[t:t + 1], kind), to_device(v[t:t + 1], kind))
+    after = _stored_values(cache, 64)
+    assert all(np.array_equal(a, b) for a, b in zip(after, before))
+    with pytest.raises(bd.BdError):
+        cache.append(to_device(k[:64], kind), to_device(v[:64], kind))       # beyond the capacity
+    bd.poll_status()
