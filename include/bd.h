@@ -303,6 +303,14 @@ bd_status bd_set_formatbook(const uint8_t in[16][8]);
  * BD_OK, BD_ERR_NONFINITE or BD_ERR_TIMEOUT (or BD_ERR_CUDA). */
 bd_status bd_poll_status(void *stream);
 
+/* Test hook for the bounded device-side waits (every wait on a barrier inside the kernels gives up
+ * after a number of polls, records BD_ERR_TIMEOUT in the status word and lets the kernel drain and
+ * return).  poll_limit > 0 replaces the built-in limit (about a second) on the current device, rounded
+ * up to 1024 polls; skip_first_code_stage != 0 makes the tensor-core product leave out the first copy
+ * of packed weights of every CTA, so that the wait for it runs out: the call then writes no result and
+ * bd_poll_status returns BD_ERR_TIMEOUT.  (0, 0) restores normal operation.  Synchronises the device. */
+bd_status bd_debug_fault(uint32_t poll_limit, int skip_first_code_stage);
+
 bd_status bd_set_gemm_impl(bd_gemm_impl impl);
 /* Number of kernels this library has launched in this process (host counter). */
 uint64_t bd_launch_count(void);

@@ -96,6 +96,7 @@ def load():
     lib.bd_set_formatbook.argtypes = [vp]
     lib.bd_poll_status.argtypes = [vp]
     lib.bd_set_gemm_impl.argtypes = [ci]
+    lib.bd_debug_fault.argtypes = [ctypes.c_uint32, ci]
     lib.bd_launch_count.restype = ctypes.c_uint64
     lib.bd_status_string.argtypes = [ci]
     lib.bd_status_string.restype = ctypes.c_char_p
@@ -124,6 +125,11 @@ def version():
 def launch_count():
     """Kernels launched by the library so far in this process."""
     return int(load().bd_launch_count())
+
+
+def debug_fault(poll_limit=0, skip_first_code_stage=False):
+    """Test hook: shorten the bounded device-side waits and make one of them run out (see bd.h)."""
+    _check(load().bd_debug_fault(ctypes.c_uint32(poll_limit), 1 if skip_first_code_stage else 0))
 
 
 def set_gemm_impl(impl):

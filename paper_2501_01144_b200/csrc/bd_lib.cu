@@ -862,6 +862,15 @@ const char *bd_status_string(bd_status s) {
     return "unknown status";
 }
 
+bd_status bd_debug_fault(uint32_t poll_limit, int skip_first_code_stage) {
+    bd_status s = cuda_result(cudaDeviceSynchronize());
+    if (s) return s;
+    const uint32_t skip = skip_first_code_stage ? 1u : 0u;
+    s = cuda_result(cudaMemcpyToSymbol(g_debug_spin_limit, &poll_limit, sizeof(poll_limit)));
+    if (s) return s;
+    return cuda_result(cudaMemcpyToSymbol(g_debug_skip_first_code_stage, &skip, sizeof(skip)));
+}
+
 int bd_version(void) { return 100; }
 
 }  // extern "C"

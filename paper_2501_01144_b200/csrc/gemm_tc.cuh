@@ -335,6 +335,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     if (threadIdx.x == 0) {
         abort_flag[0] = 0;
         abort_flag[1] = 0;                                        // set once the previous kernel has completed
+        abort_flag[2] = g_debug_spin_limit ? g_debug_spin_limit : kSpinLimit;
         for (int s = 0; s < kXStages; s++) {
             mbar_init(x_full(s), 1);
             mbar_init(x_empty(s), 1);
@@ -404,6 +405,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         // ---- TMA producer of this CTA's packed codes and ids ----
         int s = 0;
         uint32_t ph = 1;
+        const bool skip_first = g_debug_skip_first_code_stage != 0;   // test hook: see bd_debug_fault
         Tile t;
         for (int i = 0; next_tile(sc, cluster, i, t); i++) {
             const int w0 = t.w_pair * 256 + (int)rank * 128;
@@ -411,7 +413,7 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             const bool have_ids = my_row_tile < row_tiles_w;
             for (int kt = t.k_begin; kt < t.k_end; kt++) {
                 if (!mbar_wait(c_empty(s), ph, abort_flag)) break;
-                if (elect_one()) {
+                if (elect_one() && !(skip_first && i == 0 && kt == t.k_begin)) {
                     mbar_expect_tx(c_full(s), kCodeTile + (have_ids ? kIdAtomBytes : 0));
                     tma_load_2d(code_tile(s), &mapCodes, kt * (BK / 2), w0, c_full(s));
                     if (have_ids)
@@ -472,6 +474,13 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                     const bool x_ok = mbar_test_wait(x_full(s), ph_s), a_ok = mbar_test_wait(a_full(b), ph_b);
                     ready = x_ok && a_ok;
                 }
+                if (*abort_flag && elect_one()) {
+                    // this CTA is aborting: tell the peer before its epilogue warps are woken by the commit below,
+                    // so that they too skip their stores
+                    asm volatile("st.shared::cluster.u32 [%0], %1;\n\tfence.acq_rel.cluster;"
+                                 ::"r"(map_to_cta(smem_u32((const void *)abort_flag), 1)), "r"(1u) : "memory");
+                }
+                __syncwarp();
                 if (elect_one()) tcgen05_commit_pair(tmem_full_bar);
                 __syncwarp();
                 if (*abort_flag) break;
@@ -497,33 +506,43 @@ gemm_wtmem_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         int s = group % kCodeStages, b = group % kABufs;
         uint32_t s_par = 0, b_par = 1;
         static_assert(kDecodeGroups <= kCodeStages && kDecodeGroups <= kABufs, "one wrap per step at most");
+        // A warp whose wait ran out (or that saw the abort word) is `dead`: it stops waiting and working but keeps
+        // meeting its group at the named barrier of every remaining k-step.  The four warps wait on the same
+        // barriers, yet one may see the abort word where another still sees its barrier complete; a warp that left
+        // the loop would then leave the other at the named barrier for good.
+        bool dead = false;
         for (int g = group; g < total_k; g += kDecodeGroups) {
-            if (!mbar_wait(c_full(s), s_par, abort_flag)) break;
-            const uint8_t *codes = base_ptr + Smem::codes + s * kCodeTile + j * 64;
-            const uint32_t ids16 = *(const uint16_t *)(base_ptr + Smem::ids + s * kIdAtomBytes + (j % 32) * 8 + (j / 32) * 2);
             uint4 w[4];
+            uint32_t ids16 = 0;
+            if (!dead) dead = !mbar_wait(c_full(s), s_par, abort_flag);
+            if (!dead) {
+                const uint8_t *codes = base_ptr + Smem::codes + s * kCodeTile + j * 64;
+                ids16 = *(const uint16_t *)(base_ptr + Smem::ids + s * kIdAtomBytes + (j % 32) * 8 + (j / 32) * 2);
 #pragma unroll
-            for (int c = 0; c < 4; c++) w[c] = *(const uint4 *)(codes + 16 * (c ^ swz64));
-            // the codes are in registers: hand the stage back to its producer
-            __syncwarp();
-            if (lane == 0) mbar_arrive_local(c_empty(s));
-            if (!mbar_wait(a_empty(b), b_par, abort_flag)) break;
-            tcgen05_fence_after();                                // the MMAs that read this buffer have completed
-#pragma unroll
-            for (int c = 0; c < 4; c++) {
-                const uint32_t id = (ids16 >> (4 * c)) & 15u;
-                const uint32_t lo = luts[id], hi = luts[16 + id];
-                uint32_t o[8];
-                decode_word(w[c].x, lo, hi, o[0], o[1]);
-                decode_word(w[c].y, lo, hi, o[2], o[3]);
-                decode_word(w[c].z, lo, hi, o[4], o[5]);
-                decode_word(w[c].w, lo, hi, o[6], o[7]);
-                tcgen05_st_32x32b_x8(t_row + 32u * (uint32_t)b + 8u * (uint32_t)c, o);   // block c = columns 8c .. 8c + 7
+                for (int c = 0; c < 4; c++) w[c] = *(const uint4 *)(codes + 16 * (c ^ swz64));
+                // the codes are in registers: hand the stage back to its producer
+                __syncwarp();
+                if (lane == 0) mbar_arrive_local(c_empty(s));
+                dead = !mbar_wait(a_empty(b), b_par, abort_flag);
             }
-            tcgen05_wait_st();
-            tcgen05_fence_before();
+            if (!dead) {
+                tcgen05_fence_after();                            // the MMAs that read this buffer have completed
+#pragma unroll
+                for (int c = 0; c < 4; c++) {
+                    const uint32_t id = (ids16 >> (4 * c)) & 15u;
+                    const uint32_t lo = luts[id], hi = luts[16 + id];
+                    uint32_t o[8];
+                    decode_word(w[c].x, lo, hi, o[0], o[1]);
+                    decode_word(w[c].y, lo, hi, o[2], o[3]);
+                    decode_word(w[c].z, lo, hi, o[4], o[5]);
+                    decode_word(w[c].w, lo, hi, o[6], o[7]);
+                    tcgen05_st_32x32b_x8(t_row + 32u * (uint32_t)b + 8u * (uint32_t)c, o);   // block c = columns 8c .. 8c + 7
+                }
+                tcgen05_wait_st();
+                tcgen05_fence_before();
+            }
             asm volatile("bar.sync %0, 128;" ::"r"(1 + group) : "memory");   // the four warps of this group are done
-            if (group_leader) mbar_arrive_cluster(a_full_leader + 8u * b);
+            if (group_leader && !dead) mbar_arrive_cluster(a_full_leader + 8u * b);
             s += kDecodeGroups;
             if (s >= kCodeStages) { s -= kCodeStages; s_par ^= 1u; }
             b += kDecodeGroups;

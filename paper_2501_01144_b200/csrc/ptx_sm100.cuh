@@ -10,6 +10,10 @@ namespace bd {
 
 // Device status word, read and cleared by bd_poll_status (bits: kStatusNonfinite, kStatusTimeout).
 __device__ uint32_t g_status_word = 0;
+// Test hooks (bd_debug_fault): a lower poll limit for the bounded waits (0 = the built-in one) and "the code
+// producer of the tensor-core product leaves out its very first stage", which makes a wait run out on purpose.
+__device__ uint32_t g_debug_spin_limit = 0;
+__device__ uint32_t g_debug_skip_first_code_stage = 0;
 
 namespace tc {
 
@@ -49,6 +53,7 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // have completed" word: while it is zero the polls are not counted, because the wait then
 // includes the rest of the previous kernel, whose length is not this kernel's to bound (the
 // warp that waits for that kernel does so in hardware, without a limit, and sets the word).
+// abort_flag[2] is the poll limit of this launch (looked at every 1024 polls, like the abort word).
 // Returns false when the CTA is aborting (this wait or an earlier one ran out), so that a caller
 // in a hot loop need not read the flag again after every wait.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
@@ -59,6 +64,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if ((spin & 1023u) == 1023u) {
             if (*abort_flag) return false;
             if (!abort_flag[1]) spin = 0;
+            else if (spin >= abort_flag[2]) break;
         }
     }
     *abort_flag = 1;

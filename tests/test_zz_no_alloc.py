@@ -10,6 +10,8 @@ into the second, and that a problem beyond the array's size is refused.
 Collected last on purpose: a run that stops at the first failure has then already
 run every other test.
 """
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -33,6 +35,7 @@ def test_noalloc_matches_linear_on_two_calls_in_a_row():
     problems = [_problem(*c) for c in cases]
     expected = [bd.linear(x, wq, dtype=torch.float32) for x, wq in problems]
     outs = [torch.empty_like(e) for e in expected]              # outputs allocated before the calls
+    gc.collect()                                                # tensors of earlier tests must not be freed in between
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
     for (x, wq), out in zip(problems, outs):                    # back to back on one stream
@@ -58,6 +61,7 @@ def test_noalloc_decode_sized_calls_keep_their_partial_sums_in_the_builtin_array
     expected = [bd.linear(x, wq, dtype=dt) for (x, wq), dt in problems]
     outs = [torch.empty_like(e) for e in expected]
     big_out = torch.empty(384, 640, dtype=torch.float32, device="cuda")
+    gc.collect()                                                # tensors of earlier tests must not be freed in between
     torch.cuda.synchronize()
     free_before, _ = torch.cuda.mem_get_info()
     allocated_before = torch.cuda.memory_allocated()
