@@ -244,6 +244,30 @@ bd_status bd_kvcache_scores(const bd_kvcache *c, const bd_qtensor *Q, void *S, b
 bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int64_t ldp, void *Y, bd_dtype ydtype,
                         int64_t ldy, void *workspace, size_t workspace_bytes, void *stream);
 
+/* Full-path attention in one kernel (Sec. 4.1, scope "all": Q K^T and score x V are quantised
+ * like the linear layers; Sec. 3.3: softmax stays in high precision; appendix "Quantization
+ * Dimension": Q and K are cut into blocks along head_dim, the probabilities along the keys, V
+ * along the tokens).  Per head h:
+ *     S = dq(Q[h]) dq(K[h / group])^T * scale
+ *     P = softmax(S) row by row in fp32
+ *     O[h] = dq(quantise(P)) dq(V[h / group])^T     (P quantised with the online two-stage rule)
+ * Q: `heads` operands [Sq, d] (bd_quantize_act, BD_AXIS_CONTIG); K: heads / group operands
+ * [Sk, d]; V: heads / group operands [d, Sk] (bd_quantize_act of V [Sk, d] with BD_AXIS_STRIDED).
+ * Q, K, V are host arrays of descriptors.  d is 64 or 128; Sk a multiple of 32.  O is
+ * [heads][Sq][ldo] with stride_o elements between heads, BD_F32 or BD_BF16.  No mask.
+ * Neither S nor P goes to memory; the keys are walked twice (row maxima and sums first), because
+ * the blocks of P must be quantised from the final probabilities.  With `dump` (for checking;
+ * any member may be NULL) the kernel also writes S and P as fp32 [heads][Sq][Sk] and the
+ * canonical codes [heads][Sq][Sk/2], ids and scales [heads][Sq][Sk/32] of the quantised P.
+ * Accuracy: as the tensor-core product (fp32 accumulation of exact products). */
+typedef struct {
+    float *S, *P;
+    uint8_t *codes, *ids, *scales;
+} bd_attention_dump;
+bd_status bd_attention(const bd_qtensor *Q, const bd_qtensor *K, const bd_qtensor *V, int64_t heads, int64_t group,
+                       float scale, void *O, bd_dtype odtype, int64_t ldo, int64_t stride_o,
+                       const bd_attention_dump *dump, void *stream);
+
 /* bd_linear for callers that can neither allocate device memory nor hand in a
  * workspace (the paper has no counterpart; this is a convenience of the library).
  * Think of code that runs where cudaMalloc is off limits: inside a region whose

@@ -30,6 +30,11 @@ class _CQTensor(ctypes.Structure):
                 ("rows", ctypes.c_int64), ("K", ctypes.c_int64)]
 
 
+class _CAttentionDump(ctypes.Structure):
+    _fields_ = [("S", ctypes.c_void_p), ("P", ctypes.c_void_p), ("codes", ctypes.c_void_p), ("ids", ctypes.c_void_p),
+                ("scales", ctypes.c_void_p)]
+
+
 class _CKVCache(ctypes.Structure):
     _fields_ = [("k", _CQTensor), ("v", _CQTensor), ("v_recent", ctypes.c_void_p), ("dtype", ctypes.c_int),
                 ("capacity", ctypes.c_int64), ("head_dim", ctypes.c_int64), ("length", ctypes.c_int64)]
@@ -80,6 +85,7 @@ def load():
     lib.bd_kvcache_workspace_size.argtypes = [i64, i64, i64, szp]
     lib.bd_kvcache_scores.argtypes = [kp, qp, vp, ci, i64, vp, sz, vp]
     lib.bd_kvcache_pv.argtypes = [kp, vp, i64, i64, vp, ci, i64, vp, sz, vp]
+    lib.bd_attention.argtypes = [qp, qp, qp, i64, i64, ctypes.c_float, vp, ci, i64, i64, ctypes.POINTER(_CAttentionDump), vp]
     lib.bd_qtensor_sizes_bs.argtypes = [i64, i64, ci, szp, szp, szp]
     lib.bd_quantize_bs.argtypes = [vp, ci, i64, i64, i64, ci, ci, qp, vp]
     lib.bd_export_canonical_bs.argtypes = [qp, ci, vp, vp, vp, vp]
@@ -352,6 +358,32 @@ def linear_bs(X, Wq, block, out=None, dtype=torch.bfloat16, workspace=None, stre
     _check(load().bd_linear_bs(ptr, dt, M, K, ld, block, ctypes.byref(cw), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
                                out.stride(0), wptr, wbytes, _stream(stream)))
     return out
+
+
+def attention(Qs, Ks, Vs, group=1, scale=None, out=None, dtype=torch.bfloat16, dump=False, stream=None):
+    """Full-path attention in one kernel (Sec. 4.1 scope "all"; Sec. 3.3 softmax in high precision): Qs are `heads`
+    operands [Sq, d], Ks heads / group operands [Sk, d], Vs heads / group operands [d, Sk] (quantize_act with
+    AXIS_STRIDED).  Returns O [heads, Sq, d]; with dump=True also a dict of S, P (fp32 [heads, Sq, Sk]) and the
+    canonical codes, ids, scales of the quantised P, which the kernel then writes for checking."""
+    heads, sq, d, sk = len(Qs), Qs[0].rows, Qs[0].K, Ks[0].rows
+    dev = Qs[0].codes.device
+    if scale is None:
+        scale = d ** -0.5
+    if out is None:
+        out = torch.empty(heads, sq, d, dtype=dtype, device=dev)
+    cq = (_CQTensor * heads)(*[q.c_struct() for q in Qs])
+    ck = (_CQTensor * len(Ks))(*[k.c_struct() for k in Ks])
+    cv = (_CQTensor * len(Vs))(*[v.c_struct() for v in Vs])
+    extra, cd = None, None
+    if dump:
+        extra = {"S": torch.empty(heads, sq, sk, dtype=torch.float32, device=dev), "P": torch.empty(heads, sq, sk, dtype=torch.float32, device=dev),
+                 "codes": torch.empty(heads, sq, sk // 2, dtype=torch.uint8, device=dev),
+                 "ids": torch.empty(heads, sq, sk // 32, dtype=torch.uint8, device=dev),
+                 "scales": torch.empty(heads, sq, sk // 32, dtype=torch.uint8, device=dev)}
+        cd = ctypes.pointer(_CAttentionDump(*[extra[k].data_ptr() for k in ("S", "P", "codes", "ids", "scales")]))
+    _check(load().bd_attention(cq, ck, cv, heads, group, ctypes.c_float(scale), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
+                               out.stride(1), out.stride(0), cd, _stream(stream)))
+    return (out, extra) if dump else out
 
 
 class KVCache:

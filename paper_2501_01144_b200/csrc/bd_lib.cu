@@ -11,6 +11,7 @@
 #include "gemm_tc.cuh"
 #include "blocksize.cuh"
 #include "kvcache.cuh"
+#include "attention.cuh"
 #include "quantize.cuh"
 
 using namespace bd;
@@ -762,6 +763,63 @@ bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int
     }
     BD_KV_DISPATCH(c->dtype, launch_kv_finish, part, d, P, ldp, n_q, n_recent, c->v_recent, (int)d, q_rows, Y, ydtype, ldy, st);
     return launch_result();
+}
+
+// ---- fused full-path attention ----
+bd_status bd_attention(const bd_qtensor *Q, const bd_qtensor *K, const bd_qtensor *V, int64_t heads, int64_t group, float scale,
+                       void *O, bd_dtype odtype, int64_t ldo, int64_t stride_o, const bd_attention_dump *dump, void *stream) {
+    if (!Q || !K || !V || !O || heads <= 0 || group <= 0 || heads % group) return BD_ERR_INVALID_ARG;
+    if (odtype != BD_F32 && odtype != BD_BF16) return BD_ERR_INVALID_ARG;
+    const int64_t kv = heads / group, sq = Q[0].rows, hd = Q[0].K, sk = K[0].rows;
+    if (hd != 128 && hd != 64) return BD_ERR_UNSUPPORTED;
+    if (sk % kBlock || ldo < hd) return BD_ERR_SHAPE;
+    if (!aligned16(O) || (ldo * (odtype == BD_F32 ? 4 : 2)) % 16) return BD_ERR_ALIGN;
+    for (int64_t h = 0; h < heads; h++) {
+        bd_status s = check_qtensor(&Q[h]);
+        if (s) return s;
+        if (Q[h].rows != sq || Q[h].K != hd) return BD_ERR_SHAPE;
+    }
+    for (int64_t g = 0; g < kv; g++) {
+        bd_status s = check_qtensor(&K[g]);
+        if (s) return s;
+        s = check_qtensor(&V[g]);
+        if (s) return s;
+        if (K[g].rows != sk || K[g].K != hd || V[g].rows != hd || V[g].K != sk) return BD_ERR_SHAPE;
+    }
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        if (cudaFuncSetAttribute(attn::attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn::Layout<128>::total) != cudaSuccess ||
+            cudaFuncSetAttribute(attn::attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn::Layout<64>::total) != cudaSuccess)
+            return launch_result(0);
+        configured[dev] = true;
+    }
+    // heads per launch: whole KV groups, as many as the argument block holds
+    const int64_t groups_per_launch = std::max<int64_t>(1, std::min<int64_t>(attn::kMaxKvHeads, attn::kMaxHeads / group));
+    if (group > attn::kMaxHeads) return BD_ERR_UNSUPPORTED;
+    int kernels = 0;
+    for (int64_t g0 = 0; g0 < kv; g0 += groups_per_launch) {
+        const int64_t ng = std::min(groups_per_launch, kv - g0), nh = ng * group, h0 = g0 * group;
+        attn::Params p = {};
+        for (int64_t h = 0; h < nh; h++) {
+            p.q_codes[h] = (const uint8_t *)Q[h0 + h].codes; p.q_ids[h] = (const uint8_t *)Q[h0 + h].ids; p.q_scales[h] = (const uint8_t *)Q[h0 + h].scales;
+        }
+        for (int64_t g = 0; g < ng; g++) {
+            p.k_codes[g] = (const uint8_t *)K[g0 + g].codes; p.k_ids[g] = (const uint8_t *)K[g0 + g].ids; p.k_scales[g] = (const uint8_t *)K[g0 + g].scales;
+            p.v_codes[g] = (const uint8_t *)V[g0 + g].codes; p.v_ids[g] = (const uint8_t *)V[g0 + g].ids; p.v_scales[g] = (const uint8_t *)V[g0 + g].scales;
+        }
+        p.sq = sq; p.sk = sk; p.head0 = (int)h0; p.group = (int)group; p.scale = scale;
+        p.O = O; p.ldo = ldo; p.stride_o = stride_o; p.out_bf16 = odtype == BD_BF16 ? 1 : 0;
+        if (dump) {
+            p.dump_S = dump->S; p.dump_P = dump->P; p.dump_codes = dump->codes; p.dump_ids = dump->ids; p.dump_scales = dump->scales;
+        }
+        dim3 grid((unsigned)((sq + attn::kQTile - 1) / attn::kQTile), (unsigned)nh);
+        if (hd == 128) attn::attention_kernel<128><<<grid, attn::kThreads, attn::Layout<128>::total, (cudaStream_t)stream>>>(p);
+        else attn::attention_kernel<64><<<grid, attn::kThreads, attn::Layout<64>::total, (cudaStream_t)stream>>>(p);
+        kernels++;
+    }
+    return launch_result(kernels);
 }
 
 bd_status bd_export_canonical(const bd_qtensor *q, uint8_t *codes, uint8_t *ids, uint8_t *scales, void *stream) {
