@@ -669,6 +669,13 @@ def run_gpu(args, rank, world, local_rank):
 
         pv_two_streams(2)
         pv2_us = pv_two_streams(8) / grp
+        # the fused kernel: scores, softmax, quantisation of the probabilities and P V without S or P in memory
+        Vall = [bd.quantize_act(dev_bf16(Vb[g]), axis=bd.AXIS_STRIDED) for g in range(kvh)]
+        Aq2 = [bd.quantize_act(dev_bf16(Qb[h])) for h in range(heads)]
+        Bk2 = [bd.quantize_act(dev_bf16(Kb[g])) for g in range(kvh)]
+        o_fused = torch.empty(heads, S, hd, dtype=torch.bfloat16, device=dev)
+        fused_us = time_us(lambda: bd.attention(Aq2, Bk2, Vall, group=grp, out=o_fused), 3)
+        del Vall, Aq2, Bk2
         qk_bytes, pv_bytes = heads * S * S * 2.0, S * S * 4.0
         attention = {"workload": "QK^T: 32 heads x [4096,128] x [4096,128]^T (head-dim outlier channels), bf16 scores; "
                                  "PV: fp32 Dirichlet(0.1) rows P [4096,4096] per head quantised online x V (token-axis "
@@ -680,7 +687,12 @@ def run_gpu(args, rank, world, local_rank):
                      "pv_us_per_head": pv_us, "pv_read_gbs": pv_bytes / pv_us / 1e3,
                      "pv_frac_of_hbm": pv_bytes / pv_us / 1e3 / peaks["hbm_gbs"],
                      "pv_two_streams_us_per_head": pv2_us, "pv_two_streams_read_gbs": pv_bytes / pv2_us / 1e3,
-                     "pv_two_streams_frac_of_hbm": pv_bytes / pv2_us / 1e3 / peaks["hbm_gbs"]}
+                     "pv_two_streams_frac_of_hbm": pv_bytes / pv2_us / 1e3 / peaks["hbm_gbs"],
+                     # fused: all 32 heads in one call; the materialised route beside it is QK^T + P V of all heads
+                     # and does not even include the softmax between them
+                     "fused_us_32_heads": fused_us, "materialised_products_us_32_heads": qk_us + pv_us * heads,
+                     "fused_tflops": 3 * 2.0 * heads * S * S * hd / fused_us / 1e6,
+                     "fused_note": "flops counted: Q K^T twice (two walks over the keys) + P V; warp-level bf16 MMA"}
         del P, Aq, Bk
         bd.poll_status()
 

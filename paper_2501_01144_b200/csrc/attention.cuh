@@ -14,7 +14,7 @@
 //
 // Arithmetic: warp-level bf16 tensor-core instructions with fp32 accumulators.  Every DialectFP4 value is
 // 0.5 * h * 2^e with h <= 15, which bf16 holds exactly, and every product of two of them is exact in fp32, so the
-// only rounding is the fp32 accumulation (as in the other product kernels).  A CTA of four warps owns 64 queries
+// only rounding is the fp32 accumulation (as in the other product kernels).  A CTA of eight warps owns 128 queries
 // of one head; keys come in tiles of 64: their codes are expanded to bf16 tiles in shared memory (K as [key][d],
 // V as [channel][key]) and the warps read their operand fragments from there.
 //
@@ -32,7 +32,7 @@
 namespace bd {
 namespace attn {
 
-constexpr int kQTile = 64, kKTile = 64, kWarps = 4, kThreads = 32 * kWarps;
+constexpr int kQTile = 128, kKTile = 64, kWarps = 8, kThreads = 32 * kWarps;
 
 template <int HD>
 struct Layout {
@@ -78,16 +78,32 @@ __device__ __forceinline__ void bytes_to_bf16(uint32_t bytes, __nv_bfloat162 m1,
     hi = *(uint32_t *)&x1;
 }
 
-// Expands block b of operand row r (a view's codes, id, scale) into 32 bf16 values at dst (64 bytes, 16-byte aligned).
-// Rows or blocks outside the operand give zeros.
-__device__ __forceinline__ void expand_block(const uint8_t *codes, const uint8_t *ids, const uint8_t *scales, int64_t rows, int64_t ldc,
-                                             int64_t nb, int64_t r, int64_t b, const SmemTables &tab, uint8_t *dst) {
+// A block of an operand as it comes from memory: its 16 bytes of codes, dialect id and scale byte.  Fetching and
+// expanding are separate steps so that a thread's loads of a tile are all issued before the first is used.
+struct RawBlock {
+    uint4 codes;
+    uint32_t id, scale;
+    bool valid;
+};
+__device__ __forceinline__ RawBlock fetch_block(const uint8_t *codes, const uint8_t *ids, const uint8_t *scales, int64_t rows, int64_t ldc,
+                                                int64_t nb, int64_t r, int64_t b) {
+    RawBlock raw;
+    raw.valid = r < rows && b < nb;
+    if (raw.valid) {
+        raw.codes = __ldg((const uint4 *)(codes + r * ldc + b * 16));
+        raw.id = (__ldg(ids + id_byte_offset(rows, r, b)) >> (4 * (b & 1))) & 15u;
+        raw.scale = __ldg(scales + scale_offset(rows, r, b));
+    }
+    return raw;
+}
+// Expands a block into 32 bf16 values at dst (64 bytes, 16-byte aligned); blocks outside the operand give zeros.
+__device__ __forceinline__ void expand_block(const RawBlock &raw, const SmemTables &tab, uint8_t *dst) {
     uint4 out[4];
-    if (r < rows && b < nb) {
-        const uint4 u = *(const uint4 *)(codes + r * ldc + b * 16);
+    if (raw.valid) {
+        const uint4 u = raw.codes;
         const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-        const uint32_t id = (ids[id_byte_offset(rows, r, b)] >> (4 * (b & 1))) & 15u;
-        const int e = (int)scales[scale_offset(rows, r, b)] - 127;
+        const uint32_t id = raw.id;
+        const int e = (int)raw.scale - 127;
         // 2^(e + 120) as two bf16 factors, each inside the normal range
         const int e1 = (e + 120) / 2, e2 = e + 120 - e1;
         const __nv_bfloat162 m1 = __float2bfloat162_rn(__uint_as_float((uint32_t)(e1 + 127) << 23));
@@ -114,7 +130,7 @@ __device__ __forceinline__ void expand_block(const uint8_t *codes, const uint8_t
 __device__ __forceinline__ int key_of(int j, int n) { return 8 * (n >> 1) + 2 * j + (n & 1); }
 
 template <int HD>
-__global__ void __launch_bounds__(kThreads) attention_kernel(const __grid_constant__ Params p) {
+__global__ void __launch_bounds__(kThreads, 2) attention_kernel(const __grid_constant__ Params p) {
     using L = Layout<HD>;
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ SmemTables tab;
@@ -133,18 +149,38 @@ __global__ void __launch_bounds__(kThreads) attention_kernel(const __grid_consta
     // ---- the CTA's 64 query rows as bf16 ----
     for (int task = threadIdx.x; task < kQTile * NB; task += kThreads) {
         const int r = task / NB, b = task % NB;
-        expand_block(qc, qi, qs, p.sq, HD / 2, NB, q0 + r, b, tab, smem + L::q + r * L::row_stride + b * 64);
+        expand_block(fetch_block(qc, qi, qs, p.sq, HD / 2, NB, q0 + r, b), tab, smem + L::q + r * L::row_stride + b * 64);
     }
-    auto load_k_tile = [&](int64_t key0) {
-        for (int task = threadIdx.x; task < kKTile * NB; task += kThreads) {
-            const int r = task / NB, b = task % NB;
-            expand_block(kc, ki, ks, p.sk, HD / 2, NB, key0 + r, b, tab, smem + L::k + r * L::row_stride + b * 64);
+    // A tile of 64 keys is kKTile * NB key blocks and HD * 2 value blocks: with 256 threads one of each per thread
+    // (head_dim 128; half as many key blocks for head_dim 64).
+    constexpr int kKTasks = (kKTile * NB + kThreads - 1) / kThreads, kVTasks = (HD * (kKTile / kBlock) + kThreads - 1) / kThreads;
+    RawBlock raw_k[kKTasks], raw_v[kVTasks];
+    auto fetch_k_tile = [&](int64_t key0) {
+#pragma unroll
+        for (int i = 0; i < kKTasks; i++) {
+            const int task = threadIdx.x + i * kThreads, r = task / NB, b = task % NB;
+            raw_k[i] = fetch_block(kc, ki, ks, task < kKTile * NB ? p.sk : 0, HD / 2, NB, key0 + r, b);
         }
     };
-    auto load_v_tile = [&](int64_t key0) {
-        for (int task = threadIdx.x; task < HD * (kKTile / kBlock); task += kThreads) {
-            const int ch = task % HD, b = task / HD;              // neighbouring lanes = neighbouring channels
-            expand_block(vc, vi, vs, HD, p.sk / 2, nbk, ch, key0 / kBlock + b, tab, smem + L::v + ch * L::v_stride + b * 64);
+    auto expand_k_tile = [&]() {
+#pragma unroll
+        for (int i = 0; i < kKTasks; i++) {
+            const int task = threadIdx.x + i * kThreads, r = task / NB, b = task % NB;
+            if (task < kKTile * NB) expand_block(raw_k[i], tab, smem + L::k + r * L::row_stride + b * 64);
+        }
+    };
+    auto fetch_v_tile = [&](int64_t key0) {
+#pragma unroll
+        for (int i = 0; i < kVTasks; i++) {
+            const int task = threadIdx.x + i * kThreads, ch = task % HD, b = task / HD;   // neighbouring lanes = neighbouring channels
+            raw_v[i] = fetch_block(vc, vi, vs, task < HD * (kKTile / kBlock) ? HD : 0, p.sk / 2, nbk, ch, key0 / kBlock + b);
+        }
+    };
+    auto expand_v_tile = [&]() {
+#pragma unroll
+        for (int i = 0; i < kVTasks; i++) {
+            const int task = threadIdx.x + i * kThreads, ch = task % HD, b = task / HD;
+            if (task < HD * (kKTile / kBlock)) expand_block(raw_v[i], tab, smem + L::v + ch * L::v_stride + b * 64);
         }
     };
     // ---- scores of this warp's 16 queries against the 32 keys of block kb of the tile in shared memory ----
@@ -170,8 +206,9 @@ __global__ void __launch_bounds__(kThreads) attention_kernel(const __grid_consta
     // ---- first walk over the keys: row maxima and sums ----
     float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.0f, l_hi = 0.0f;
     for (int64_t key0 = 0; key0 < p.sk; key0 += kKTile) {
-        __syncthreads();
-        load_k_tile(key0);
+        __syncthreads();                                          // the previous tile has been used
+        fetch_k_tile(key0);
+        expand_k_tile();
         __syncthreads();
 #pragma unroll
         for (int kb = 0; kb < kKTile / kBlock; kb++) {
@@ -216,8 +253,10 @@ __global__ void __launch_bounds__(kThreads) attention_kernel(const __grid_consta
     const int64_t dump_row_lo = ((int64_t)head * p.sq + row_lo), dump_row_hi = dump_row_lo + 8;
     for (int64_t key0 = 0; key0 < p.sk; key0 += kKTile) {
         __syncthreads();
-        load_k_tile(key0);
-        load_v_tile(key0);
+        fetch_k_tile(key0);                                       // (keeping the next tile's blocks in registers through the
+        fetch_v_tile(key0);                                       // products, to hide this latency, costs more in spills)
+        expand_k_tile();
+        expand_v_tile();
         __syncthreads();
 #pragma unroll
         for (int kb = 0; kb < kKTile / kBlock; kb++) {

@@ -136,3 +136,40 @@ def test_attention_products_both_operands_online():
         ok, ratio = gemm_tolerance_ok(O[rows], Yref, T)
         assert ok, f"PV head {h}: max err / bound = {ratio}"
     bd.poll_status()
+
+
+def test_attention_fused_path_at_the_benchmark_size():
+    """Config 5 through the fused kernel: 32 query heads, 8 KV heads, 4096 tokens, head_dim 128, no S or P in
+    memory.  Three heads are run again with the kernel's checking dumps and compared link by link with the oracle on
+    sampled rows; their results must equal the full call's bit for bit."""
+    from oracle import attention as oa
+    heads, kv, S, d = 32, 8, 4096, 128
+    group = heads // kv
+    Q, Kt, _, V = inputs.attention_case(heads, kv, S, d, seed=4, p_heads=0)
+    Qs = [bd.quantize_act(to_device(Q[h], torch.bfloat16)) for h in range(heads)]
+    Ks = [bd.quantize_act(to_device(Kt[g], torch.bfloat16)) for g in range(kv)]
+    Vs = [bd.quantize_act(to_device(V[g], torch.bfloat16), axis=bd.AXIS_STRIDED) for g in range(kv)]
+    scale = d ** -0.5
+    O = bd.attention(Qs, Ks, Vs, group=group, scale=scale, dtype=torch.float32)
+    rows = np.array([0, 63, 64, 1000, 2049, S - 1])
+    for h in (0, 13, 31):
+        Oh, dump = bd.attention([Qs[h]], [Ks[h // group]], [Vs[h // group]], group=1, scale=scale, dtype=torch.float32, dump=True)
+        assert torch.equal(Oh[0], O[h]), f"head {h}: the result depends on the launch it was part of"
+        qq = oracle_quantize(Q[h][rows], torch.bfloat16)
+        kq = oracle_quantize(Kt[h // group], torch.bfloat16)
+        vq = oracle_quantize(np.ascontiguousarray(V[h // group].T), torch.bfloat16)
+        S_ref, T = oa.scores(qq, kq, scale)
+        S_lib = dump["S"][0].cpu().numpy()[rows]
+        ok, ratio = gemm_tolerance_ok(S_lib, S_ref, T)
+        assert ok, f"head {h} scores: max err / bound = {ratio}"
+        P_lib = dump["P"][0].cpu().numpy()[rows]
+        P_ref = oa.softmax_rows(S_lib)
+        # the scores of this case reach the thousands (outlier channels), so the fp32 exponent carries their rounding
+        assert np.abs(P_lib - P_ref).max() <= 2e-3, f"head {h} probabilities"
+        pq_ref = oracle.quantize(P_lib)
+        for name, j in (("scales", 2), ("ids", 1), ("codes", 0)):
+            assert np.array_equal(dump[name][0].cpu().numpy()[rows], pq_ref[j]), f"head {h}: {name} of the quantised probabilities"
+        O_ref, To = oracle.gemm(oracle.dequantize(*pq_ref), oracle.dequantize(*vq))
+        ok, ratio = gemm_tolerance_ok(O[h].cpu().numpy()[rows], O_ref, To)
+        assert ok, f"head {h} result: max err / bound = {ratio}"
+    bd.poll_status()
