@@ -760,7 +760,9 @@ def run_case(args):
     """A few launches of one kernel family on a small, fixed case (for ncu captures).
     quantizer: bd_quantize_act on bf16 [8192, 4096] (168 MiB of buffers in rotation).
     quantizer_f32: bd_quantize_act on fp32 [4096, 4096] (three buffer sets in rotation).
-    linear_<layer>: bd_linear of one LLaMA3-8B layer at M = 2048 (layer in qo_proj, kv_proj, gate_up, down)."""
+    linear_<layer>: bd_linear of one LLaMA3-8B layer at M = 2048 (layer in qo_proj, kv_proj, gate_up, down).
+    decode: bd_linear of 16 tokens against K = 11008, N = 4096.  quantizer_strided: the token-axis quantizer on V [4096, 128].
+    requant_gate_up: bd_linear_requant of the gate/up layer.  attention: bd_attention on four heads of 4096 tokens."""
     import torch
 
     import paper_2501_01144_b200 as bd
@@ -824,6 +826,73 @@ def run_case(args):
         torch.cuda.synchronize()
         print(json.dumps({"case": args.case, "us_per_step": e0.elapsed_time(e1) / reps * 1e3}))
         return
+    if args.case == "decode":
+        # a decode-sized call of the LLaMA2 MLP sweep: 16 tokens against K = 11008, N = 4096; six weight copies in rotation
+        K, N, M = 11008, 4096, 16
+        wsrc = dev_bf16(inputs.weights_normal(N, K, seed=3))
+        wqs = [bd.quantize_weights(wsrc, bd.SELECT_TWO_STAGE) for _ in range(6)]
+        x = dev_bf16(inputs.act_post_silu(M, K, seed=3))
+        y = torch.empty(M, N, dtype=torch.bfloat16, device=dev)
+        ws = torch.empty(bd.linear_workspace_size(M, N, K), dtype=torch.uint8, device=dev)
+        for i in range(args.warmup):
+            bd.linear(x, wqs[i % 6], out=y, workspace=ws)
+        e0.record()
+        for i in range(reps):
+            bd.linear(x, wqs[i % 6], out=y, workspace=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        print(json.dumps({"case": args.case, "us_per_call": e0.elapsed_time(e1) / reps * 1e3}))
+        return
+    if args.case == "quantizer_strided":
+        # the value matrix of one KV head, blocks along the token axis: V [4096 tokens, 128] bf16 -> operand [128, 4096]
+        vs = [dev_bf16(inputs.to_bf16_bits(np.random.default_rng(s).standard_normal((4096, 128)).astype(np.float32))) for s in range(2)]
+        qs = [bd.QTensor(128, 4096, dev) for _ in range(2)]
+        for i in range(args.warmup):
+            bd.quantize_act(vs[i % 2], axis=bd.AXIS_STRIDED, out=qs[i % 2])
+        e0.record()
+        for i in range(reps):
+            bd.quantize_act(vs[i % 2], axis=bd.AXIS_STRIDED, out=qs[i % 2])
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        print(json.dumps({"case": args.case, "us_per_launch": us, "GB/s": 4096 * 128 * BYTES_PER_ELEM_QUANT / us / 1e3}))
+        return
+    if args.case == "requant_gate_up":
+        # the gate/up layer at M = 2048 with the requantising epilogue
+        K, N = 4096, 14336
+        x = dev_bf16(inputs.act_student_t(M_TOKENS, K, seed=2))
+        wq = bd.quantize_weights(dev_bf16(inputs.weights_normal(N, K, seed=2)), bd.SELECT_TWO_STAGE)
+        hq = bd.QTensor(M_TOKENS, N, dev)
+        ws = torch.empty(bd.linear_requant_workspace_size(M_TOKENS, N, K), dtype=torch.uint8, device=dev)
+        for _ in range(args.warmup):
+            bd.linear_requant(x, wq, out=hq, workspace=ws)
+        e0.record()
+        for _ in range(reps):
+            bd.linear_requant(x, wq, out=hq, workspace=ws)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        print(json.dumps({"case": args.case, "us_per_call": us, "TFLOP/s": 2.0 * M_TOKENS * N * K / us / 1e6}))
+        return
+    if args.case == "attention":
+        # the fused attention kernel on four query heads of one KV head, 4096 tokens, head_dim 128
+        rng = np.random.default_rng(0)
+        mk = lambda n: inputs.to_bf16_bits(rng.standard_normal((n, 4096, 128)).astype(np.float32))
+        Qb, Kb, Vb = mk(4), mk(1), mk(1)
+        Qs = [bd.quantize_act(dev_bf16(Qb[h])) for h in range(4)]
+        Ks = [bd.quantize_act(dev_bf16(Kb[0]))]
+        Vs = [bd.quantize_act(dev_bf16(Vb[0]), axis=bd.AXIS_STRIDED)]
+        o = torch.empty(4, 4096, 128, dtype=torch.bfloat16, device=dev)
+        for _ in range(args.warmup):
+            bd.attention(Qs, Ks, Vs, group=4, out=o)
+        e0.record()
+        for _ in range(reps):
+            bd.attention(Qs, Ks, Vs, group=4, out=o)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        print(json.dumps({"case": args.case, "us_per_call": us, "TFLOP/s": 3 * 2.0 * 4 * 4096 * 4096 * 128 / us / 1e6}))
+        return
     name = args.case[len("linear_"):]
     K, N = {n: (k, nn) for n, k, nn in LAYERS}[name]
     x = dev_bf16(inputs.act_student_t(M_TOKENS, K, seed=2))
@@ -861,7 +930,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--case", default=None,
-                    choices=["quantizer", "quantizer_f32", "step"] + ["linear_" + n for n, _, _ in LAYERS],
+                    choices=["quantizer", "quantizer_f32", "step", "decode", "quantizer_strided", "requant_gate_up", "attention"]
+                    + ["linear_" + n for n, _, _ in LAYERS],
                     help="run a few launches of one small case (for profiler captures) instead of the benchmark")
     args = ap.parse_args()
     _lib_override()
