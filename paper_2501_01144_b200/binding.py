@@ -12,7 +12,7 @@ _SRC = os.path.join(_HERE, "csrc", "bd_lib.cu")
 F32, BF16, F16 = 0, 1, 2
 SELECT_TWO_STAGE, SELECT_MSE = 0, 1
 AXIS_CONTIG, AXIS_STRIDED = 0, 1
-GEMM_AUTO, GEMM_SIMT, GEMM_TCGEN05 = 0, 1, 2
+GEMM_AUTO, GEMM_SIMT, GEMM_TCGEN05, GEMM_WARP = 0, 1, 2, 3
 
 _TORCH_DTYPE = {torch.float32: F32, torch.bfloat16: BF16, torch.float16: F16}
 

@@ -9,6 +9,7 @@
 #include "bd_common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_warp.cuh"
 #include "blocksize.cuh"
 #include "kvcache.cuh"
 #include "attention.cuh"
@@ -384,8 +385,70 @@ bd_status bd_linear_workspace_size(int64_t M, int64_t N, int64_t K, size_t *byte
     const size_t tc_bytes = tc_supported(M, N, K) ? align256(s) + tc_gemm_workspace(M, N, K) : 0;
     const size_t simt_bytes = align256(c) + align256(i) + align256(s);
     *bytes = tc_bytes > simt_bytes ? tc_bytes : simt_bytes;
+    if (wk::supported(M, N, K)) *bytes = std::max(*bytes, align256(wk::record_bytes(K, 2)));
     return BD_OK;
 }
+
+namespace {
+// The warp-level kernel (gemm_warp.cuh) serves up to 16 tokens; the library's own choice takes it for up to 8 (one
+// token group per MMA), where it measured faster than the tensor-core path with its three launches; with two token
+// groups the activation records no longer fit beside the kernel's shared memory in L1 and it measured slower.
+bool use_warp(int64_t M, int64_t N, int64_t K) {
+    if (g_gemm_impl == BD_GEMM_WARP) return true;
+    return g_gemm_impl == BD_GEMM_AUTO && wk::supported(M, N, K) && M <= wk::kTokTile && (int64_t)N * K >= (1 << 20);
+}
+unsigned sm_count() {
+    static int sms[kMaxDevices] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= kMaxDevices) return 148;
+    if (!sms[dev]) {
+        cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev);
+        if (sms[dev] <= 0) sms[dev] = 148;
+    }
+    return (unsigned)sms[dev];
+}
+// Warps per CTA = shares of K of a row tile: as many as keep about 32 warps on every SM with all CTAs resident
+// at once, at most one per unit of K.
+int warp_kernel_warps(int64_t N, int64_t K) {
+    const int64_t tiles = N / wk::kRows, units = K / wk::kUnitK;
+    const int64_t per_sm = (tiles + sm_count() - 1) / sm_count();
+    int64_t w = 32 / per_sm;
+    if (const char *e = getenv("BD_WARP_KERNEL_WARPS")) w = atoi(e);
+    return (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(w, units), wk::kMaxWarps));
+}
+bd_status launch_warp_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, const QView &W, void *Y,
+                             bd_dtype ydtype, int64_t ldy, void *workspace, cudaStream_t st) {
+    const int nt = M > wk::kTokTile ? 2 : 1, nb = (int)(K / kBlock);
+    uint8_t *rec16 = (uint8_t *)workspace;
+    float *recs = (float *)(rec16 + (size_t)nb * nt * wk::kRecBytes);
+    const unsigned qgrid = grid_for((int64_t)nb * wk::kTokTile * nt, 128);
+    switch (xdtype) {
+    case BD_F32: launch_serialized(wk::quantize_records_kernel<BD_F32>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
+    case BD_BF16: launch_serialized(wk::quantize_records_kernel<BD_BF16>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
+    default: launch_serialized(wk::quantize_records_kernel<BD_F16>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
+    }
+    bd_status s = launch_result(1);
+    if (s) return s;
+    wk::Params p{W.codes, W.ids, W.scales, W.ldc, row_tiles(W.rows), rec16, recs, Y, ldy, (int)M, (int)(K / wk::kUnitK), ydtype == BD_BF16};
+    const int warps = warp_kernel_warps(W.rows, K);
+    const size_t smem = (size_t)warps * (wk::kStages * wk::kStageBytes + nt * 512);
+    const unsigned grid = (unsigned)(W.rows / wk::kRows);
+    static bool smem_set[kMaxDevices] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < kMaxDevices && !smem_set[dev]) {
+        const int most = wk::kMaxWarps * (wk::kStages * wk::kStageBytes + 2 * 512);
+        if (cudaFuncSetAttribute(wk::gemm_warp_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(wk::gemm_warp_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
+            return cuda_result(cudaGetLastError());
+        smem_set[dev] = true;
+    }
+    if (nt == 1) launch_serialized(wk::gemm_warp_kernel<1>, grid, 32u * warps, smem, st, p);
+    else launch_serialized(wk::gemm_warp_kernel<2>, grid, 32u * warps, smem, st, p);
+    return launch_result(1);
+}
+}  // namespace
 
 bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, const bd_qtensor *Wq, void *Y,
                     bd_dtype ydtype, int64_t ldy, void *workspace, size_t workspace_bytes, void *stream) {
@@ -404,6 +467,10 @@ bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_
     char *p = (char *)workspace;
     cudaStream_t st = (cudaStream_t)stream;
     const int64_t N = Wq->rows;
+    if (use_warp(M, N, K)) {
+        if (!wk::supported(M, N, K)) return BD_ERR_UNSUPPORTED;
+        return launch_warp_linear(X, xdtype, M, K, ldx, view_of(Wq), Y, ydtype, ldy, workspace, st);
+    }
     if (use_tc(M, N, K)) {
         if (!tc_supported(M, N, K)) return BD_ERR_UNSUPPORTED;
         // tensor-core path: the quantizer writes the operand bytes and the scale atoms directly
@@ -895,7 +962,7 @@ bd_status bd_poll_status(void *stream) {
 }
 
 bd_status bd_set_gemm_impl(bd_gemm_impl impl) {
-    if (impl != BD_GEMM_AUTO && impl != BD_GEMM_SIMT && impl != BD_GEMM_TCGEN05) return BD_ERR_INVALID_ARG;
+    if (impl != BD_GEMM_AUTO && impl != BD_GEMM_SIMT && impl != BD_GEMM_TCGEN05 && impl != BD_GEMM_WARP) return BD_ERR_INVALID_ARG;
     g_gemm_impl = impl;
     return BD_OK;
 }
