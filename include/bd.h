@@ -77,10 +77,10 @@ typedef enum {
     BD_GEMM_AUTO = 0,   /* by shape                                                    */
     BD_GEMM_SIMT = 1,   /* CUDA-core kernel: exact integer in-block sums, any shape     */
     BD_GEMM_TCGEN05 = 2, /* tensor-core kernel (block-scaled E4M3 MMA, TMEM accumulators) */
-    BD_GEMM_WARP = 3    /* bd_linear of at most 16 tokens: warp-level E4M3 MMA straight from the packed
-                           weights, one launch after the quantizer, no partial sums in memory; needs
-                           rows % 16 == 0 and K % 128 == 0 (BD_ERR_UNSUPPORTED otherwise; calls other than
-                           bd_linear treat it like BD_GEMM_AUTO) */
+    BD_GEMM_WARP = 3    /* products with at most 16 rows on the activation side (bd_linear of at most 16
+                           tokens, bd_gemm with A->rows <= 16, the KV-cache calls): warp-level fp16 MMA
+                           straight from the packed B operand, one launch after the kernel that prepares
+                           A, no partial sums in memory; BD_ERR_UNSUPPORTED for more rows */
 } bd_gemm_impl;
 
 /* A quantised [rows, K] operand in the library's physical layout.  All three
@@ -135,15 +135,14 @@ bd_status bd_quantize_act(const void *X, bd_dtype dtype, int64_t M, int64_t K, i
  *                     the guaranteed bound for ANY input is (K / 32) * 2^-21 * S (an
  *                     operand with blocks 2^28 apart and opposite signs gets close to
  *                     it).  Callers who need 1e-6 * S on such inputs select BD_GEMM_SIMT.
- *   BD_GEMM_WARP      (bd_linear, at most 16 tokens) in-block sums are exact (fp16 tensor-core
+ *   BD_GEMM_WARP      (at most 16 rows of A) in-block sums are exact (fp16 tensor-core
  *                     products of 4-bit integers, fp32 sums of 32 of them); each block's sum is
  *                     multiplied by its two power-of-two scales one after the other and the blocks
  *                     are added in fp32, the warps' shares of K in a fixed order: |err| <=
  *                     (K / 32 + 16) * 2^-24 * S.  Blocks whose scale lies below 2^-100 or above
  *                     2^100 may be flushed or overflow in the intermediate product.
- *   BD_GEMM_AUTO      picks BD_GEMM_TCGEN05 except for tiny problems, and BD_GEMM_WARP for
- *                     bd_linear of at most 8 tokens where that kernel serves the shape; the
- *                     chosen implementation's bound applies. */
+ *   BD_GEMM_AUTO      picks BD_GEMM_TCGEN05 except for tiny problems, and BD_GEMM_WARP for at most
+ *                     8 rows of A; the chosen implementation's bound applies. */
 bd_status bd_gemm_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes);
 bd_status bd_gemm(const bd_qtensor *A, const bd_qtensor *B, void *Y, bd_dtype ydtype, int64_t ldy,
                   void *workspace, size_t workspace_bytes, void *stream);

@@ -22,6 +22,7 @@ namespace {
 int g_last_cuda_error = 0;
 uint64_t g_launches = 0;
 bd_gemm_impl g_gemm_impl = BD_GEMM_AUTO;
+constexpr int kMaxDevices = 64;
 Formatbook g_book = kBook;            // the table bd_get_formatbook reports (host copy of what the device uses)
 
 bd_status cuda_result(cudaError_t e) {
@@ -160,8 +161,91 @@ bd_status check_gemm(const bd_qtensor *A, const bd_qtensor *B, const void *Y, bd
     return BD_OK;
 }
 
+// The warp-level kernel (gemm_warp.cuh) serves up to 16 tokens; the library's own choice takes it for up to 8 (one
+// token group per MMA), where it measured faster than the tensor-core path with its three launches; with two token
+// groups the activation records no longer fit beside the kernel's shared memory in L1 and it measured slower.
+bool use_warp(int64_t M, int64_t N, int64_t K) {
+    if (g_gemm_impl == BD_GEMM_WARP) return true;
+    return g_gemm_impl == BD_GEMM_AUTO && wk::supported(M, N, K) && M <= wk::kTokTile && (int64_t)N * K >= (1 << 18);
+}
+unsigned sm_count() {
+    static int sms[kMaxDevices] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= kMaxDevices) return 148;
+    if (!sms[dev]) {
+        cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev);
+        if (sms[dev] <= 0) sms[dev] = 148;
+    }
+    return (unsigned)sms[dev];
+}
+// Warps per CTA = shares of K of a row tile: as many as keep about 32 warps on every SM with all CTAs resident
+// at once, at most one per unit of K.
+int warp_kernel_warps(int64_t N, int64_t K) {
+    const int64_t tiles = N / wk::kRows, units = K / wk::kUnitK;
+    const int64_t per_sm = (tiles + sm_count() - 1) / sm_count();
+    int64_t w = 32 / per_sm;
+    if (const char *e = getenv("BD_WARP_KERNEL_WARPS")) w = atoi(e);
+    return (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(w, units), wk::kMaxWarps));
+}
+// The product kernel over records at `workspace` (rec16, then the factors).
+bd_status launch_warp_main(int64_t M, int64_t K, const QView &W, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace, cudaStream_t st) {
+    const int nt = M > wk::kTokTile ? 2 : 1;
+    const uint8_t *rec16 = (const uint8_t *)workspace;
+    const float *recs = (const float *)(rec16 + (size_t)wk::padded_blocks(K) * nt * wk::kRecBytes);
+    wk::Params p{W.codes, W.ids, W.scales, W.ldc, row_tiles(W.rows), rec16, recs, Y, ldy, W.rows, (int)M,
+                 (int)((K + wk::kUnitK - 1) / wk::kUnitK), (int)(K / kBlock % wk::kUnitBlocks), ydtype == BD_BF16};
+    const int warps = warp_kernel_warps((W.rows + wk::kRows - 1) / wk::kRows * wk::kRows, (K + wk::kUnitK - 1) / wk::kUnitK * wk::kUnitK);
+    const size_t smem = (size_t)warps * (wk::kStages * wk::kStageBytes + nt * 512);
+    const unsigned grid = (unsigned)((W.rows + wk::kRows - 1) / wk::kRows);
+    static bool smem_set[kMaxDevices] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < kMaxDevices && !smem_set[dev]) {
+        const int most = wk::kMaxWarps * (wk::kStages * wk::kStageBytes + 2 * 512);
+        if (cudaFuncSetAttribute(wk::gemm_warp_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(wk::gemm_warp_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
+            return cuda_result(cudaGetLastError());
+        smem_set[dev] = true;
+    }
+    if (nt == 1) launch_serialized(wk::gemm_warp_kernel<1>, grid, 32u * warps, smem, st, p);
+    else launch_serialized(wk::gemm_warp_kernel<2>, grid, 32u * warps, smem, st, p);
+    return launch_result(1);
+}
+bd_status launch_warp_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, const QView &W, void *Y,
+                             bd_dtype ydtype, int64_t ldy, void *workspace, cudaStream_t st) {
+    const int nt = M > wk::kTokTile ? 2 : 1, nb = (int)(K / kBlock);
+    uint8_t *rec16 = (uint8_t *)workspace;
+    float *recs = (float *)(rec16 + (size_t)wk::padded_blocks(K) * nt * wk::kRecBytes);
+    const unsigned qgrid = grid_for(wk::padded_blocks(K) * wk::kTokTile * nt, 128);
+    switch (xdtype) {
+    case BD_F32: launch_serialized(wk::quantize_records_kernel<BD_F32>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
+    case BD_BF16: launch_serialized(wk::quantize_records_kernel<BD_BF16>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
+    default: launch_serialized(wk::quantize_records_kernel<BD_F16>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
+    }
+    bd_status s = launch_result(1);
+    if (s) return s;
+    return launch_warp_main(M, K, W, Y, ydtype, ldy, workspace, st);
+}
+// bd_gemm with a few rows of A: records from the quantised A, then the same product kernel.
+bd_status launch_warp_gemm(const QView &A, const QView &B, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace, cudaStream_t st) {
+    const int nt = A.rows > wk::kTokTile ? 2 : 1;
+    uint8_t *rec16 = (uint8_t *)workspace;
+    float *recs = (float *)(rec16 + (size_t)wk::padded_blocks(A.K) * nt * wk::kRecBytes);
+    launch_serialized(wk::records_from_qtensor_kernel, grid_for(wk::padded_blocks(A.K) * wk::kTokTile * nt, 128), 128, 0, st, A, nt, rec16, recs);
+    bd_status s = launch_result(1);
+    if (s) return s;
+    return launch_warp_main(A.rows, A.K, B, Y, ydtype, ldy, workspace, st);
+}
+
 bd_status gemm_dispatch(const QView &A, const QView &B, void *Y, bd_dtype ydt, int64_t ldy, void *ws, size_t ws_bytes,
                         cudaStream_t st) {
+    if (use_warp(A.rows, B.rows, A.K)) {
+        if (!wk::supported(A.rows, B.rows, A.K)) return BD_ERR_UNSUPPORTED;
+        if (!ws || ws_bytes < wk::record_bytes(A.K, 2)) return BD_ERR_WORKSPACE;
+        if ((uintptr_t)ws & 255u) return BD_ERR_ALIGN;
+        return launch_warp_gemm(A, B, Y, ydt, ldy, ws, st);
+    }
     if (use_tc(A.rows, B.rows, A.K)) {
         if (!tc_supported(A.rows, B.rows, A.K)) return BD_ERR_UNSUPPORTED;
         size_t need = tc_gemm_workspace(A.rows, B.rows, A.K);
@@ -193,7 +277,6 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 static __device__ __align__(256) uint8_t g_noalloc_scratch[BD_NOALLOC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 void *g_noalloc_ptr[kMaxDevices] = {};
 }  // namespace
 
@@ -296,6 +379,7 @@ bd_status bd_gemm_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes)
     if (!bytes || M <= 0 || N <= 0 || K <= 0) return BD_ERR_INVALID_ARG;
     if (K % kBlock) return BD_ERR_SHAPE;
     *bytes = tc_supported(M, N, K) ? tc_gemm_workspace(M, N, K) : 0;
+    if (wk::supported(M, N, K)) *bytes = std::max(*bytes, (size_t)((wk::record_bytes(K, 2) + 255) & ~(size_t)255));
     return BD_OK;
 }
 
@@ -388,67 +472,6 @@ bd_status bd_linear_workspace_size(int64_t M, int64_t N, int64_t K, size_t *byte
     if (wk::supported(M, N, K)) *bytes = std::max(*bytes, align256(wk::record_bytes(K, 2)));
     return BD_OK;
 }
-
-namespace {
-// The warp-level kernel (gemm_warp.cuh) serves up to 16 tokens; the library's own choice takes it for up to 8 (one
-// token group per MMA), where it measured faster than the tensor-core path with its three launches; with two token
-// groups the activation records no longer fit beside the kernel's shared memory in L1 and it measured slower.
-bool use_warp(int64_t M, int64_t N, int64_t K) {
-    if (g_gemm_impl == BD_GEMM_WARP) return true;
-    return g_gemm_impl == BD_GEMM_AUTO && wk::supported(M, N, K) && M <= wk::kTokTile && (int64_t)N * K >= (1 << 20);
-}
-unsigned sm_count() {
-    static int sms[kMaxDevices] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev < 0 || dev >= kMaxDevices) return 148;
-    if (!sms[dev]) {
-        cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev);
-        if (sms[dev] <= 0) sms[dev] = 148;
-    }
-    return (unsigned)sms[dev];
-}
-// Warps per CTA = shares of K of a row tile: as many as keep about 32 warps on every SM with all CTAs resident
-// at once, at most one per unit of K.
-int warp_kernel_warps(int64_t N, int64_t K) {
-    const int64_t tiles = N / wk::kRows, units = K / wk::kUnitK;
-    const int64_t per_sm = (tiles + sm_count() - 1) / sm_count();
-    int64_t w = 32 / per_sm;
-    if (const char *e = getenv("BD_WARP_KERNEL_WARPS")) w = atoi(e);
-    return (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(w, units), wk::kMaxWarps));
-}
-bd_status launch_warp_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, const QView &W, void *Y,
-                             bd_dtype ydtype, int64_t ldy, void *workspace, cudaStream_t st) {
-    const int nt = M > wk::kTokTile ? 2 : 1, nb = (int)(K / kBlock);
-    uint8_t *rec16 = (uint8_t *)workspace;
-    float *recs = (float *)(rec16 + (size_t)nb * nt * wk::kRecBytes);
-    const unsigned qgrid = grid_for((int64_t)nb * wk::kTokTile * nt, 128);
-    switch (xdtype) {
-    case BD_F32: launch_serialized(wk::quantize_records_kernel<BD_F32>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
-    case BD_BF16: launch_serialized(wk::quantize_records_kernel<BD_BF16>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
-    default: launch_serialized(wk::quantize_records_kernel<BD_F16>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
-    }
-    bd_status s = launch_result(1);
-    if (s) return s;
-    wk::Params p{W.codes, W.ids, W.scales, W.ldc, row_tiles(W.rows), rec16, recs, Y, ldy, (int)M, (int)(K / wk::kUnitK), ydtype == BD_BF16};
-    const int warps = warp_kernel_warps(W.rows, K);
-    const size_t smem = (size_t)warps * (wk::kStages * wk::kStageBytes + nt * 512);
-    const unsigned grid = (unsigned)(W.rows / wk::kRows);
-    static bool smem_set[kMaxDevices] = {};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < kMaxDevices && !smem_set[dev]) {
-        const int most = wk::kMaxWarps * (wk::kStages * wk::kStageBytes + 2 * 512);
-        if (cudaFuncSetAttribute(wk::gemm_warp_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
-            cudaFuncSetAttribute(wk::gemm_warp_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
-            return cuda_result(cudaGetLastError());
-        smem_set[dev] = true;
-    }
-    if (nt == 1) launch_serialized(wk::gemm_warp_kernel<1>, grid, 32u * warps, smem, st, p);
-    else launch_serialized(wk::gemm_warp_kernel<2>, grid, 32u * warps, smem, st, p);
-    return launch_result(1);
-}
-}  // namespace
 
 bd_status bd_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, const bd_qtensor *Wq, void *Y,
                     bd_dtype ydtype, int64_t ldy, void *workspace, size_t workspace_bytes, void *stream) {
@@ -821,11 +844,16 @@ bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int
         bd_qtensor pq{p, p + align256(cb), p + align256(cb) + align256(ib), q_rows, n_q};
         char *gws = p + align256(cb) + align256(ib) + align256(sb);
         part = (float *)(gws + align256(g2));
-        s = launch_contig<BD_SELECT_TWO_STAGE, true, false>(P, BD_F32, ldp, view_of(&pq), nullptr, st);
-        if (s) return s;
         QView vals = view_of(&c->v);
         vals.K = n_q;                                             // the first n_q tokens of every channel; the pitch stays
-        s = gemm_dispatch(view_of(&pq), vals, part, BD_F32, d, gws, g2, st);
+        if (use_warp(q_rows, d, n_q) && wk::supported(q_rows, d, n_q)) {
+            // a few query rows: the probabilities go straight into the warp-level kernel's records
+            s = launch_warp_linear(P, BD_F32, q_rows, n_q, ldp, vals, part, BD_F32, d, gws, st);
+        } else {
+            s = launch_contig<BD_SELECT_TWO_STAGE, true, false>(P, BD_F32, ldp, view_of(&pq), nullptr, st);
+            if (s) return s;
+            s = gemm_dispatch(view_of(&pq), vals, part, BD_F32, d, gws, g2, st);
+        }
         if (s) return s;
     }
     BD_KV_DISPATCH(c->dtype, launch_kv_finish, part, d, P, ldp, n_q, n_recent, c->v_recent, (int)d, q_rows, Y, ydtype, ldy, st);

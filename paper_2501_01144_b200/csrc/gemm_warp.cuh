@@ -43,11 +43,13 @@ constexpr int kStages = 4;
 constexpr int kRecBytes = kTokTile * kBlock * 2;       // fp16 values of a record (8 tokens x 32)
 constexpr int kMaxWarps = 16;
 
+// Records cover whole units: K is rounded up to 128 and the blocks past it hold zeros.
+__host__ __device__ inline int64_t padded_blocks(int64_t K) { return (K + kUnitK - 1) / kUnitK * kUnitBlocks; }
 __host__ __device__ inline size_t record_bytes(int64_t K, int nt) {
-    return (size_t)(K / kBlock) * nt * (kRecBytes + kTokTile * sizeof(float));
+    return (size_t)padded_blocks(K) * nt * (kRecBytes + kTokTile * sizeof(float));
 }
 inline bool supported(int64_t M, int64_t N, int64_t K) {
-    return M >= 1 && M <= kMaxTokens && N % kRows == 0 && K % kUnitK == 0 && K / kBlock < (1 << 20);
+    return M >= 1 && M <= kMaxTokens && N >= 1 && K >= kBlock && K % kBlock == 0 && K / kBlock < (1 << 20);
 }
 
 // ---- the activations: two-stage quantisation of up to 16 token rows into MMA-ordered records ----
@@ -63,12 +65,12 @@ __global__ void __launch_bounds__(128) quantize_records_kernel(const void *__res
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     const int slots = kTokTile * nt;
     const int b = t / slots, m = t % slots;
-    if (b >= nb) return;
+    if (b >= (int)padded_blocks((int64_t)nb * kBlock)) return;
     uint4 out[4];
 #pragma unroll
     for (int i = 0; i < 4; i++) out[i] = make_uint4(0, 0, 0, 0);
     float factor = 1.0f;
-    if (m < M) {
+    if (m < M && b < nb) {
         uint32_t bits[32], unused[8];
         Loader<DT>::contiguous((const char *)X + ((int64_t)m * ldx + (int64_t)b * 32) * Loader<DT>::kElemBytes, bits);
         BlockResult res;
@@ -91,6 +93,49 @@ __global__ void __launch_bounds__(128) quantize_records_kernel(const void *__res
                     const uint32_t mag = ((idx < 4 ? tlo : thi) >> (8 * (idx & 3))) & 0xffu;
                     const uint32_t f16 = (uint32_t)__half_as_ushort(__int2half_rn((int)mag)) | word_sign(res.words[w], e) << 15;
                     pair |= f16 << (16 * j);
+                }
+                v[i] = pair;
+            }
+            out[w] = make_uint4(v[0], v[1], v[2], v[3]);
+        }
+    }
+    const size_t slot = (size_t)(b * nt + m / kTokTile) * kTokTile + m % kTokTile;
+    uint4 *dst = (uint4 *)(rec16 + slot * (kBlock * 2));
+#pragma unroll
+    for (int i = 0; i < 4; i++) dst[i] = out[i];
+    recs[slot] = factor;
+}
+
+// The same records from an operand that is already quantised (bd_gemm with a few rows of A).
+__global__ void __launch_bounds__(128) records_from_qtensor_kernel(QView a, int nt, uint8_t *__restrict__ rec16, float *__restrict__ recs) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    const int slots = kTokTile * nt, nb = (int)(a.K / kBlock);
+    const int b = t / slots, m = t % slots;
+    if (b >= (int)padded_blocks(a.K)) return;
+    uint4 out[4];
+#pragma unroll
+    for (int i = 0; i < 4; i++) out[i] = make_uint4(0, 0, 0, 0);
+    float factor = 1.0f;
+    if (m < a.rows && b < nb) {
+        const uint4 u = *(const uint4 *)(a.codes + (int64_t)m * a.ldc + (int64_t)b * 16);
+        const uint32_t words[4] = {u.x, u.y, u.z, u.w};
+        const uint32_t id = (a.ids[id_byte_offset(a.rows, m, b)] >> (4 * (b & 1))) & 15u, scale = a.scales[scale_offset(a.rows, m, b)];
+        factor = __uint_as_float(min(scale + 22u, 254u) << 23);
+        const uint32_t tlo = c_tables.int_lo[id], thi = c_tables.int_hi[id];
+#pragma unroll
+        for (int w = 0; w < 4; w++) {
+            uint32_t v[4];
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+                uint32_t pair = 0;
+#pragma unroll
+                for (int j = 0; j < 2; j++) {
+                    const int e = 2 * i + j;
+                    const uint32_t idx = word_index(words[w], e);
+                    const uint32_t mag = ((idx < 4 ? tlo : thi) >> (8 * (idx & 3))) & 0xffu;
+                    pair |= ((uint32_t)__half_as_ushort(__int2half_rn((int)mag)) | word_sign(words[w], e) << 15) << (16 * j);
                 }
                 v[i] = pair;
             }
@@ -155,7 +200,8 @@ struct Params {
     const float *recs;
     void *Y;
     int64_t ldy;
-    int M, units, y_bf16;
+    int64_t N;                             // weight rows (the last CTA's tile may reach past them)
+    int M, units, tail_blocks, y_bf16;     // units = ceil(K / 128); tail_blocks = blocks of the last unit if it is short, else 0
 };
 
 // Shared memory of a CTA: per warp kStages stages of kStageBytes, then the warps' sums [warps][NT][4][32] floats.
@@ -182,13 +228,21 @@ __global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_
                           ((int64_t)warp * p.row_tiles + rt) * matom;
     const int64_t mstep = (int64_t)warps * p.row_tiles * matom;
     const uint32_t mdst = ring_s + (uint32_t)(kCodeBytes + (lane < 16 ? 0 : kRows * 4) + mrow * 4);
+    // rows past N and blocks past K are not read: their codes become zeros (index 0 = value 0), so whatever their
+    // scale and id entries hold adds nothing
+    const bool row_ok_lo = r0 + crow < p.N, row_ok_hi = r0 + crow + 8 < p.N;
+    int next_unit = warp;
     auto issue = [&](int stage) {
         const uint32_t so = (uint32_t)stage * kStageBytes;
-        cp_async16(cdst + so, csrc);
-        cp_async16(cdst + so + 8 * 64, csrc + row8);
+        const bool piece_ok = !(p.tail_blocks && next_unit == p.units - 1 && cpiece >= p.tail_blocks);
+        if (row_ok_lo && piece_ok) cp_async16(cdst + so, csrc);
+        else asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(cdst + so), "r"(0) : "memory");
+        if (row_ok_hi && piece_ok) cp_async16(cdst + so + 8 * 64, csrc + row8);
+        else asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(cdst + so + 8 * 64), "r"(0) : "memory");
         cp_async4(mdst + so, msrc);
         csrc += cstep;
         msrc += mstep;
+        next_unit += warps;
     };
     // this warp's units: warp, warp + warps, ...
     const int n_units = p.units > warp ? (p.units - warp + warps - 1) / warps : 0;
@@ -220,7 +274,12 @@ __global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_
             w_lo[b] = *(const uint32_t *)(s + off);
             w_hi[b] = *(const uint32_t *)(s + off + 8 * 64);
         }
-        const uint32_t sc_lo = *(const uint32_t *)(s + kCodeBytes + g * 4), sc_hi = *(const uint32_t *)(s + kCodeBytes + (g + 8) * 4);
+        uint32_t sc_lo = *(const uint32_t *)(s + kCodeBytes + g * 4), sc_hi = *(const uint32_t *)(s + kCodeBytes + (g + 8) * 4);
+        if (p.tail_blocks && warp + i * warps == p.units - 1) {     // scale bytes past K may hold anything: make them 2^-127
+            const uint32_t keep = (1u << (8 * p.tail_blocks)) - 1u;
+            sc_lo &= keep;
+            sc_hi &= keep;
+        }
         const uint32_t id_lo = *(const uint32_t *)(s + kCodeBytes + kRows * 4 + g * 4) >> id_shift;
         const uint32_t id_hi = *(const uint32_t *)(s + kCodeBytes + kRows * 4 + (g + 8) * 4) >> id_shift;
         __syncwarp();                                            // everyone has read the stage: refill it
@@ -263,7 +322,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_
     __syncthreads();
     for (int o = threadIdx.x; o < kRows * kTokTile * NT; o += blockDim.x) {
         const int row = o % kRows, tok = o / kRows;
-        if (tok >= p.M) continue;
+        if (tok >= p.M || r0 + row >= p.N) continue;
         // accumulator c of lane (row % 8) * 4 + (tok % 8) / 2 holds (row, token): c = (row / 8) * 2 + tok % 2
         const int n = tok / kTokTile, tk = tok % kTokTile, src = ((n * 4) + (row / 8) * 2 + (tk & 1)) * 32 + (row % 8) * 4 + tk / 2;
         float y = 0.0f;
