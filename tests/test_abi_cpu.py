@@ -94,16 +94,20 @@ def test_workspace_sizes_follow_the_documented_parts():
         return b.value
 
     atoms = lambda M, K: ((M + 127) // 128) * ((K // 32 + 3) // 4) * 512
+    # at most 16 rows on the activation side: never less than the warp-level kernel's records (K rounded up to 128,
+    # two groups of 8 rows, 32 fp16 values and one fp32 factor per row and block)
+    records = lambda K: ((K + 127) // 128 * 4) * 2 * (8 * 32 * 2 + 8 * 4)
     # the benchmark's layers: operand bytes + scale atoms, nothing else
     assert gemm_ws(2048, 14336, 4096) == 2048 * 4096
     assert linear_ws(2048, 14336, 4096) == atoms(2048, 4096) + 2048 * 4096
     # up to 128 tokens against at most 37 pairs of 128 weight rows (half of the clusters): room for four splits of
     # [tokens rounded to 16][weight rows rounded to 256] fp32 partial sums behind the operand bytes
-    assert gemm_ws(16, 4096, 11008) == 16 * 11008 + 4 * 16 * 4096 * 4
-    assert gemm_ws(5, 300, 2144) == 256 * ((5 * 2144 + 255) // 256) + 4 * 16 * 512 * 4
+    assert gemm_ws(16, 4096, 11008) == 16 * 11008 + 4 * 16 * 4096 * 4 > records(11008)
+    assert gemm_ws(5, 300, 2144) == 256 * ((5 * 2144 + 255) // 256) + 4 * 16 * 512 * 4 > records(2144)
     assert gemm_ws(128, 9472, 4096) == 128 * 4096 + 4 * 128 * 9472 * 4
     # more weight rows than that, or more tokens: no split, no scratch
-    assert gemm_ws(16, 11008, 4096) == 16 * 4096
+    assert gemm_ws(16, 11008, 4096) == records(4096) > 16 * 4096
+    assert gemm_ws(17, 11008, 4096) == 17 * 4096
     assert gemm_ws(128, 9473, 4096) == 128 * 4096
     assert gemm_ws(129, 4096, 11008) == 256 * ((129 * 11008 + 255) // 256)
 
