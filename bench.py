@@ -568,18 +568,34 @@ def run_gpu(args, rank, world, local_rank):
             caches.append(cch)
         q_rows = [bd.quantize_act(dev_bf16(inputs.to_bf16_bits(rng_kv.standard_normal((grp, hd)).astype(np.float32)))) for _ in range(kvh)]
         pitch = (n_tok + 3) // 4 * 4
-        probs = [torch.softmax(torch.randn(grp, pitch, device=dev), -1)[:, :n_tok] for _ in range(kvh)]
-        s_out = torch.empty(grp, n_tok, dtype=torch.float32, device=dev)
-        o_out = torch.empty(grp, hd, dtype=torch.bfloat16, device=dev)
+        probs = torch.softmax(torch.randn(kvh, grp, pitch, device=dev), -1)[:, :, :n_tok]
+        s_out = torch.empty(kvh, grp, n_tok, dtype=torch.float32, device=dev)
+        o_out = torch.empty(kvh, grp, hd, dtype=torch.bfloat16, device=dev)
 
-        def attend():
+        def attend_per_head():
             for g in range(kvh):
-                caches[g].scores(q_rows[g], out=s_out)
-                caches[g].pv(probs[g], out=o_out)
+                caches[g].scores(q_rows[g], out=s_out[g])
+                caches[g].pv(probs[g], out=o_out[g])
+
+        def attend():                                         # all KV heads of the layer per call
+            bd.kvcache_scores_batched(caches, q_rows, out=s_out)
+            bd.kvcache_pv_batched(caches, probs, out=o_out)
+
+        for _ in range(3):
+            attend_per_head()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(10):
+            attend_per_head()
+        e1.record()
+        torch.cuda.synchronize()
+        per_head_us = e0.elapsed_time(e1) / 10 * 1e3
 
         for _ in range(3):
             attend()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches0 = bd.launch_count()
+        attend()
+        attend_launches = bd.launch_count() - launches0
         e0.record()
         for _ in range(10):
             attend()
@@ -595,8 +611,9 @@ def run_gpu(args, rank, world, local_rank):
         torch.cuda.synchronize()
         append_us = e0.elapsed_time(e1) / 10 * 1e3
         cache_bytes = kvh * 2 * n_tok * hd * 0.546875
-        kv_cache = {"workload": "8 KV heads x 4113 tokens x head_dim 128, 4 query heads per KV head, one object per KV head",
-                    "scores_and_pv_us_per_step": attend_us, "append_one_token_us_per_step": append_us,
+        kv_cache = {"workload": "8 KV heads x 4113 tokens x head_dim 128, 4 query heads per KV head, one object per KV head, scores and P x V of all heads per call",
+                    "scores_and_pv_us_per_step": attend_us, "launches_per_step": attend_launches, "scores_and_pv_us_per_step_head_by_head": per_head_us,
+                    "append_one_token_us_per_step": append_us,
                     "cache_bytes_read_per_step": cache_bytes, "cache_read_gbs": cache_bytes / attend_us / 1e3,
                     "stored_bits_per_value": 4.375, "recent_tokens_in_high_precision": n_tok % 32}
         del caches, probs

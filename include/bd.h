@@ -254,6 +254,17 @@ bd_status bd_kvcache_scores(const bd_kvcache *c, const bd_qtensor *Q, void *S, b
                             void *workspace, size_t workspace_bytes, void *stream);
 bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int64_t ldp, void *Y, bd_dtype ydtype,
                         int64_t ldy, void *workspace, size_t workspace_bytes, void *stream);
+/* The same two calls for the n KV heads of a layer in one decode step (n >= 1): c[i] all of one capacity,
+ * head_dim, dtype and length; Q[i] [q, head_dim] with the same q; head i reads P + i * stride_p and writes
+ * S + i * stride_s / Y + i * stride_y (strides in elements).  With q <= 8 and n <= 64 (and the library's own
+ * choice of product kernel) the heads share two (scores) or three (P x V) launches; otherwise the calls
+ * above run head by head.  workspace: bd_kvcache_batched_workspace_size bytes, 256-byte aligned. */
+bd_status bd_kvcache_batched_workspace_size(int64_t n, int64_t capacity, int64_t head_dim, int64_t q_rows, size_t *bytes);
+bd_status bd_kvcache_scores_batched(const bd_kvcache *c, int64_t n, const bd_qtensor *Q, void *S, bd_dtype sdtype,
+                                    int64_t lds, int64_t stride_s, void *workspace, size_t workspace_bytes, void *stream);
+bd_status bd_kvcache_pv_batched(const bd_kvcache *c, int64_t n, const float *P, int64_t q_rows, int64_t ldp,
+                                int64_t stride_p, void *Y, bd_dtype ydtype, int64_t ldy, int64_t stride_y,
+                                void *workspace, size_t workspace_bytes, void *stream);
 
 /* Full-path attention in one kernel (Sec. 4.1, scope "all": Q K^T and score x V are quantised
  * like the linear layers; Sec. 3.3: softmax stays in high precision; appendix "Quantization

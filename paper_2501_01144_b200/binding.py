@@ -85,6 +85,9 @@ def load():
     lib.bd_kvcache_workspace_size.argtypes = [i64, i64, i64, szp]
     lib.bd_kvcache_scores.argtypes = [kp, qp, vp, ci, i64, vp, sz, vp]
     lib.bd_kvcache_pv.argtypes = [kp, vp, i64, i64, vp, ci, i64, vp, sz, vp]
+    lib.bd_kvcache_batched_workspace_size.argtypes = [i64, i64, i64, i64, szp]
+    lib.bd_kvcache_scores_batched.argtypes = [kp, i64, qp, vp, ci, i64, i64, vp, sz, vp]
+    lib.bd_kvcache_pv_batched.argtypes = [kp, i64, vp, i64, i64, i64, vp, ci, i64, i64, vp, sz, vp]
     lib.bd_attention.argtypes = [qp, qp, qp, i64, i64, ctypes.c_float, vp, ci, i64, i64, ctypes.POINTER(_CAttentionDump), vp]
     lib.bd_qtensor_sizes_bs.argtypes = [i64, i64, ci, szp, szp, szp]
     lib.bd_quantize_bs.argtypes = [vp, ci, i64, i64, i64, ci, ci, qp, vp]
@@ -438,6 +441,42 @@ class KVCache:
         _check(load().bd_kvcache_pv(ctypes.byref(self._c), ctypes.c_void_p(P.data_ptr()), P.shape[0], P.stride(0),
                                     ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype), out.stride(0), wptr, wbytes, _stream(stream)))
         return out
+
+
+def _kv_batch(caches, q_rows):
+    n, c0 = len(caches), caches[0]
+    arr = (_CKVCache * n)(*[c._c for c in caches])
+    b = ctypes.c_size_t()
+    _check(load().bd_kvcache_batched_workspace_size(n, c0.capacity, c0.head_dim, q_rows, ctypes.byref(b)))
+    if c0._ws is None or c0._ws.numel() < b.value:
+        c0._ws = torch.empty(max(b.value, 256), dtype=torch.uint8, device=c0.k.codes.device)
+    return arr, ctypes.c_void_p(c0._ws.data_ptr()), c0._ws.numel()
+
+
+def kvcache_scores_batched(caches, Qs, out=None, dtype=torch.float32, stream=None):
+    """S [n, q, length]: the scores of n KV heads (same length) in one call; Qs[i] is head i's quantised query operand."""
+    n, q, length = len(caches), Qs[0].rows, caches[0].length
+    if out is None:
+        out = torch.empty(n, q, length, dtype=dtype, device=caches[0].k.codes.device)
+    arr, wptr, wbytes = _kv_batch(caches, q)
+    cq = (_CQTensor * n)(*[x.c_struct() for x in Qs])
+    _check(load().bd_kvcache_scores_batched(arr, n, cq, ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype), out.stride(1), out.stride(0),
+                                            wptr, wbytes, _stream(stream)))
+    return out
+
+
+def kvcache_pv_batched(caches, P, out=None, dtype=torch.float32, stream=None):
+    """O [n, q, head_dim] = P[i] V[i] for fp32 probabilities P [n, q, length] of n KV heads (same length) in one call."""
+    n = len(caches)
+    if P.dtype != torch.float32 or P.dim() != 3 or P.stride(2) != 1 or P.shape[0] != n or P.shape[2] != caches[0].length:
+        raise ValueError("P must be fp32 [n, q, length] with a contiguous last axis")
+    if out is None:
+        out = torch.empty(n, P.shape[1], caches[0].head_dim, dtype=dtype, device=P.device)
+    arr, wptr, wbytes = _kv_batch(caches, P.shape[1])
+    _check(load().bd_kvcache_pv_batched(arr, n, ctypes.c_void_p(P.data_ptr()), P.shape[1], P.stride(1), P.stride(0),
+                                        ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype), out.stride(1), out.stride(0), wptr, wbytes,
+                                        _stream(stream)))
+    return out
 
 
 NOALLOC_SCRATCH_BYTES = 32 << 20

@@ -66,9 +66,9 @@ unsigned quant_bf16_grid_limit() {
 // Launch with programmatic stream serialisation: the blocks may be scheduled while the previous kernel of the
 // stream drains; such a kernel waits for that kernel's results before it touches global memory.
 template <typename... Params, typename... Args>
-void launch_serialized(void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args... args) {
+void launch_serialized(void (*kernel)(Params...), dim3 grid, unsigned block, size_t smem, cudaStream_t st, Args... args) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
+    cfg.gridDim = grid;
     cfg.blockDim = dim3(block);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -188,42 +188,58 @@ int warp_kernel_warps(int64_t N, int64_t K) {
     if (const char *e = getenv("BD_WARP_KERNEL_WARPS")) w = atoi(e);
     return (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(w, units), wk::kMaxWarps));
 }
-// The product kernel over records at `workspace` (rec16, then the factors).
-bd_status launch_warp_main(int64_t M, int64_t K, const QView &W, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace, cudaStream_t st) {
+// The product kernel over records at `workspace` (rec16, then the factors).  batch: n problems with the operands
+// of `batch`, records rec_stride bytes apart and results y_stride elements apart.
+bd_status launch_warp_main(int64_t M, int64_t K, const QView &W, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace, cudaStream_t st,
+                           const wk::OperandBatch *batch = nullptr, int n = 1, int64_t rec_stride = 0, int64_t y_stride = 0) {
     const int nt = M > wk::kTokTile ? 2 : 1;
     const uint8_t *rec16 = (const uint8_t *)workspace;
     const float *recs = (const float *)(rec16 + (size_t)wk::padded_blocks(K) * nt * wk::kRecBytes);
-    wk::Params p{W.codes, W.ids, W.scales, W.ldc, row_tiles(W.rows), rec16, recs, Y, ldy, W.rows, (int)M,
+    wk::Params p{W.codes, W.ids, W.scales, W.ldc, row_tiles(W.rows), rec16, recs, Y, ldy, W.rows, rec_stride, y_stride, (int)M,
                  (int)((K + wk::kUnitK - 1) / wk::kUnitK), (int)(K / kBlock % wk::kUnitBlocks), ydtype == BD_BF16};
-    const int warps = warp_kernel_warps((W.rows + wk::kRows - 1) / wk::kRows * wk::kRows, (K + wk::kUnitK - 1) / wk::kUnitK * wk::kUnitK);
+    const int64_t tiles = (W.rows + wk::kRows - 1) / wk::kRows;
+    const int warps = warp_kernel_warps(tiles * n * wk::kRows, (K + wk::kUnitK - 1) / wk::kUnitK * wk::kUnitK);
     const size_t smem = (size_t)warps * (wk::kStages * wk::kStageBytes + nt * 512);
-    const unsigned grid = (unsigned)((W.rows + wk::kRows - 1) / wk::kRows);
+    const dim3 grid((unsigned)tiles, (unsigned)n);
     static bool smem_set[kMaxDevices] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < kMaxDevices && !smem_set[dev]) {
         const int most = wk::kMaxWarps * (wk::kStages * wk::kStageBytes + 2 * 512);
-        if (cudaFuncSetAttribute(wk::gemm_warp_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
-            cudaFuncSetAttribute(wk::gemm_warp_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
+        if (cudaFuncSetAttribute(wk::gemm_warp_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(wk::gemm_warp_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(wk::gemm_warp_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
+            cudaFuncSetAttribute(wk::gemm_warp_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
             return cuda_result(cudaGetLastError());
         smem_set[dev] = true;
     }
-    if (nt == 1) launch_serialized(wk::gemm_warp_kernel<1>, grid, 32u * warps, smem, st, p);
-    else launch_serialized(wk::gemm_warp_kernel<2>, grid, 32u * warps, smem, st, p);
+    const wk::OperandBatch none{};
+    if (batch) {
+        if (nt == 1) launch_serialized(wk::gemm_warp_kernel<1, true>, grid, 32u * warps, smem, st, p, *batch);
+        else launch_serialized(wk::gemm_warp_kernel<2, true>, grid, 32u * warps, smem, st, p, *batch);
+    } else {
+        if (nt == 1) launch_serialized(wk::gemm_warp_kernel<1, false>, grid, 32u * warps, smem, st, p, none);
+        else launch_serialized(wk::gemm_warp_kernel<2, false>, grid, 32u * warps, smem, st, p, none);
+    }
+    return launch_result(1);
+}
+// X: n problems x_stride elements apart (n = 1: one).
+bd_status launch_warp_records(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, void *workspace, cudaStream_t st, int n = 1,
+                              int64_t x_stride = 0, int64_t rec_stride = 0) {
+    const int nt = M > wk::kTokTile ? 2 : 1, nb = (int)(K / kBlock);
+    uint8_t *rec16 = (uint8_t *)workspace;
+    float *recs = (float *)(rec16 + (size_t)wk::padded_blocks(K) * nt * wk::kRecBytes);
+    const dim3 qgrid(grid_for(wk::padded_blocks(K) * wk::kTokTile * nt, 128), (unsigned)n);
+    switch (xdtype) {
+    case BD_F32: launch_serialized(wk::quantize_records_kernel<BD_F32>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs, x_stride, rec_stride); break;
+    case BD_BF16: launch_serialized(wk::quantize_records_kernel<BD_BF16>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs, x_stride, rec_stride); break;
+    default: launch_serialized(wk::quantize_records_kernel<BD_F16>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs, x_stride, rec_stride); break;
+    }
     return launch_result(1);
 }
 bd_status launch_warp_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t K, int64_t ldx, const QView &W, void *Y,
                              bd_dtype ydtype, int64_t ldy, void *workspace, cudaStream_t st) {
-    const int nt = M > wk::kTokTile ? 2 : 1, nb = (int)(K / kBlock);
-    uint8_t *rec16 = (uint8_t *)workspace;
-    float *recs = (float *)(rec16 + (size_t)wk::padded_blocks(K) * nt * wk::kRecBytes);
-    const unsigned qgrid = grid_for(wk::padded_blocks(K) * wk::kTokTile * nt, 128);
-    switch (xdtype) {
-    case BD_F32: launch_serialized(wk::quantize_records_kernel<BD_F32>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
-    case BD_BF16: launch_serialized(wk::quantize_records_kernel<BD_BF16>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
-    default: launch_serialized(wk::quantize_records_kernel<BD_F16>, qgrid, 128, 0, st, X, ldx, (int)M, nb, nt, rec16, recs); break;
-    }
-    bd_status s = launch_result(1);
+    bd_status s = launch_warp_records(X, xdtype, M, K, ldx, workspace, st);
     if (s) return s;
     return launch_warp_main(M, K, W, Y, ydtype, ldy, workspace, st);
 }
@@ -232,7 +248,9 @@ bd_status launch_warp_gemm(const QView &A, const QView &B, void *Y, bd_dtype ydt
     const int nt = A.rows > wk::kTokTile ? 2 : 1;
     uint8_t *rec16 = (uint8_t *)workspace;
     float *recs = (float *)(rec16 + (size_t)wk::padded_blocks(A.K) * nt * wk::kRecBytes);
-    launch_serialized(wk::records_from_qtensor_kernel, grid_for(wk::padded_blocks(A.K) * wk::kTokTile * nt, 128), 128, 0, st, A, nt, rec16, recs);
+    const wk::OperandBatch none{};
+    launch_serialized(wk::records_from_qtensor_kernel<false>, dim3(grid_for(wk::padded_blocks(A.K) * wk::kTokTile * nt, 128)), 128, 0, st, A, nt, rec16,
+                      recs, none, (int64_t)0);
     bd_status s = launch_result(1);
     if (s) return s;
     return launch_warp_main(A.rows, A.K, B, Y, ydtype, ldy, workspace, st);
@@ -294,10 +312,21 @@ template <int DT>
 void launch_kv_finish(const float *part, int64_t ld_part, const float *P, int64_t ldp, int64_t n_q, int n_recent, const void *recent,
                       int d, int64_t q_rows, void *Y, bd_dtype ydt, int64_t ldy, cudaStream_t st) {
     const unsigned grid = grid_for(q_rows * d, 256);
+    const RecentBatch none{};
     if (ydt == BD_BF16)
-        kv_pv_finish_kernel<DT, __nv_bfloat16><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, recent, d, q_rows, (__nv_bfloat16 *)Y, ldy);
+        kv_pv_finish_kernel<DT, __nv_bfloat16, false><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, recent, d, q_rows, (__nv_bfloat16 *)Y, ldy, none, 0, 0, 0);
     else
-        kv_pv_finish_kernel<DT, float><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, recent, d, q_rows, (float *)Y, ldy);
+        kv_pv_finish_kernel<DT, float, false><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, recent, d, q_rows, (float *)Y, ldy, none, 0, 0, 0);
+}
+template <int DT>
+void launch_kv_finish_batched(const float *part, int64_t ld_part, const float *P, int64_t ldp, int64_t n_q, int n_recent, const RecentBatch &recent,
+                              int n, int64_t part_stride, int64_t p_stride, int64_t y_stride, int d, int64_t q_rows, void *Y, bd_dtype ydt,
+                              int64_t ldy, cudaStream_t st) {
+    const dim3 grid(grid_for(q_rows * d, 256), (unsigned)n);
+    if (ydt == BD_BF16)
+        kv_pv_finish_kernel<DT, __nv_bfloat16, true><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, nullptr, d, q_rows, (__nv_bfloat16 *)Y, ldy, recent, part_stride, p_stride, y_stride);
+    else
+        kv_pv_finish_kernel<DT, float, true><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, nullptr, d, q_rows, (float *)Y, ldy, recent, part_stride, p_stride, y_stride);
 }
 #define BD_KV_DISPATCH(dt, fn, ...)                          \
     switch (dt) {                                            \
@@ -857,6 +886,125 @@ bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int
         if (s) return s;
     }
     BD_KV_DISPATCH(c->dtype, launch_kv_finish, part, d, P, ldp, n_q, n_recent, c->v_recent, (int)d, q_rows, Y, ydtype, ldy, st);
+    return launch_result();
+}
+
+// ---- the same two calls for the KV heads of a layer at once ----
+namespace {
+bd_status check_kvcache_batch(const bd_kvcache *c, int64_t n) {
+    if (!c || n <= 0) return BD_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < n; i++) {
+        bd_status s = check_kvcache(&c[i]);
+        if (s) return s;
+        if (c[i].capacity != c[0].capacity || c[i].head_dim != c[0].head_dim || c[i].length != c[0].length || c[i].dtype != c[0].dtype)
+            return BD_ERR_SHAPE;
+    }
+    return BD_OK;
+}
+bool kv_batch_fused(int64_t n, int64_t q_rows, int64_t N, int64_t K) {
+    return n <= wk::kMaxBatch && g_gemm_impl != BD_GEMM_SIMT && g_gemm_impl != BD_GEMM_TCGEN05 && q_rows <= wk::kTokTile && wk::supported(q_rows, N, K);
+}
+}  // namespace
+
+bd_status bd_kvcache_batched_workspace_size(int64_t n, int64_t capacity, int64_t head_dim, int64_t q_rows, size_t *bytes) {
+    if (n <= 0) return BD_ERR_INVALID_ARG;
+    size_t one;
+    bd_status s = bd_kvcache_workspace_size(capacity, head_dim, q_rows, &one);
+    if (s) return s;
+    *bytes = (size_t)n * align256(one);
+    return BD_OK;
+}
+
+bd_status bd_kvcache_scores_batched(const bd_kvcache *c, int64_t n, const bd_qtensor *Q, void *S, bd_dtype sdtype, int64_t lds,
+                                    int64_t stride_s, void *workspace, size_t workspace_bytes, void *stream) {
+    bd_status s = check_kvcache_batch(c, n);
+    if (s) return s;
+    if (!Q || !S || (sdtype != BD_F32 && sdtype != BD_BF16)) return BD_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < n; i++) {
+        s = check_qtensor(&Q[i]);
+        if (s) return s;
+        if (Q[i].K != c[0].head_dim || Q[i].rows != Q[0].rows) return BD_ERR_SHAPE;
+    }
+    const int64_t len = c[0].length, q_rows = Q[0].rows, hd = c[0].head_dim;
+    if (len == 0 || lds < len || (n > 1 && stride_s < q_rows * lds)) return BD_ERR_SHAPE;
+    size_t one, need;
+    bd_kvcache_workspace_size(c[0].capacity, hd, q_rows, &one);
+    bd_kvcache_batched_workspace_size(n, c[0].capacity, hd, q_rows, &need);
+    if (!workspace || workspace_bytes < need) return BD_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 255u) return BD_ERR_ALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t esz = sdtype == BD_F32 ? 4 : 2;
+    if (!kv_batch_fused(n, q_rows, len, hd)) {
+        for (int64_t i = 0; i < n; i++) {
+            s = bd_kvcache_scores(&c[i], &Q[i], (char *)S + i * stride_s * esz, sdtype, lds, (char *)workspace + i * align256(one), one, stream);
+            if (s) return s;
+        }
+        return BD_OK;
+    }
+    // one launch for the queries' records, one for the products: grid.y = head
+    wk::OperandBatch qa{}, kb{};
+    for (int64_t i = 0; i < n; i++) {
+        qa.codes[i] = (const uint8_t *)Q[i].codes; qa.ids[i] = (const uint8_t *)Q[i].ids; qa.scales[i] = (const uint8_t *)Q[i].scales;
+        kb.codes[i] = (const uint8_t *)c[i].k.codes; kb.ids[i] = (const uint8_t *)c[i].k.ids; kb.scales[i] = (const uint8_t *)c[i].k.scales;
+    }
+    const int nt = 1;
+    const int64_t rec_stride = (int64_t)align256(wk::record_bytes(hd, nt));
+    uint8_t *rec16 = (uint8_t *)workspace;
+    float *recs = (float *)(rec16 + (size_t)wk::padded_blocks(hd) * nt * wk::kRecBytes);
+    launch_serialized(wk::records_from_qtensor_kernel<true>, dim3(grid_for(wk::padded_blocks(hd) * wk::kTokTile * nt, 128), (unsigned)n), 128, 0, st,
+                      view_of(&Q[0]), nt, rec16, recs, qa, rec_stride);
+    s = launch_result(1);
+    if (s) return s;
+    QView keys = view_of(&c[0].k);
+    keys.rows = len;
+    return launch_warp_main(q_rows, hd, keys, S, sdtype, lds, workspace, st, &kb, (int)n, rec_stride, stride_s);
+}
+
+bd_status bd_kvcache_pv_batched(const bd_kvcache *c, int64_t n, const float *P, int64_t q_rows, int64_t ldp, int64_t stride_p, void *Y,
+                                bd_dtype ydtype, int64_t ldy, int64_t stride_y, void *workspace, size_t workspace_bytes, void *stream) {
+    bd_status s = check_kvcache_batch(c, n);
+    if (s) return s;
+    if (!P || !Y || q_rows <= 0 || (ydtype != BD_F32 && ydtype != BD_BF16)) return BD_ERR_INVALID_ARG;
+    const int64_t len = c[0].length, d = c[0].head_dim;
+    if (len == 0 || ldp < len || ldy < d || (n > 1 && (stride_p < q_rows * ldp || stride_y < q_rows * ldy))) return BD_ERR_SHAPE;
+    if (len >= kBlock && (!aligned16(P) || (ldp * 4) % 16 || (stride_p * 4) % 16)) return BD_ERR_ALIGN;
+    size_t one, need;
+    bd_kvcache_workspace_size(c[0].capacity, d, q_rows, &one);
+    bd_kvcache_batched_workspace_size(n, c[0].capacity, d, q_rows, &need);
+    if (!workspace || workspace_bytes < need) return BD_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 255u) return BD_ERR_ALIGN;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t esz = ydtype == BD_F32 ? 4 : 2;
+    const int64_t n_q = len / kBlock * kBlock;
+    const int n_recent = (int)(len - n_q);
+    if (!kv_batch_fused(n, q_rows, d, n_q ? n_q : kBlock)) {
+        for (int64_t i = 0; i < n; i++) {
+            s = bd_kvcache_pv(&c[i], P + i * stride_p, q_rows, ldp, (char *)Y + i * stride_y * esz, ydtype, ldy, (char *)workspace + i * align256(one), one, stream);
+            if (s) return s;
+        }
+        return BD_OK;
+    }
+    // records of all heads' probabilities, the products over the stored chunks (fp32, in the workspace), then the
+    // recent tokens in high precision and the result: three launches, grid.y = head
+    float *part = nullptr;
+    const int64_t part_stride = q_rows * d;
+    if (n_q) {
+        const int64_t rec_stride = (int64_t)align256(wk::record_bytes(n_q, 1));
+        part = (float *)((char *)workspace + (size_t)n * rec_stride);
+        s = launch_warp_records(P, BD_F32, q_rows, n_q, ldp, workspace, st, (int)n, stride_p, rec_stride);
+        if (s) return s;
+        wk::OperandBatch vb{};
+        for (int64_t i = 0; i < n; i++) {
+            vb.codes[i] = (const uint8_t *)c[i].v.codes; vb.ids[i] = (const uint8_t *)c[i].v.ids; vb.scales[i] = (const uint8_t *)c[i].v.scales;
+        }
+        QView vals = view_of(&c[0].v);
+        vals.K = n_q;
+        s = launch_warp_main(q_rows, n_q, vals, part, BD_F32, d, workspace, st, &vb, (int)n, rec_stride, part_stride);
+        if (s) return s;
+    }
+    RecentBatch rb{};
+    for (int64_t i = 0; i < n; i++) rb.ptr[i] = c[i].v_recent;
+    BD_KV_DISPATCH(c[0].dtype, launch_kv_finish_batched, part, d, P, ldp, n_q, n_recent, rb, (int)n, part_stride, stride_p, stride_y, (int)d, q_rows, Y, ydtype, ldy, st);
     return launch_result();
 }
 

@@ -56,8 +56,10 @@ inline bool supported(int64_t M, int64_t N, int64_t K) {
 // rec16: [K/32][nt][8 tokens][32 fp16]; recs: [K/32][nt][8] factors 2^(scale - 127 + 22) (anything finite for
 // an all-zero block or a token past M, whose values are zeros).  Thread = (block b, token slot m of 8 * nt), m fastest.
 template <int DT>
+// blockIdx.y = problem of a batch: X advances by x_stride elements, the records by rec_stride bytes.
 __global__ void __launch_bounds__(128) quantize_records_kernel(const void *__restrict__ X, int64_t ldx, int M, int nb, int nt,
-                                                               uint8_t *__restrict__ rec16, float *__restrict__ recs) {
+                                                               uint8_t *__restrict__ rec16, float *__restrict__ recs, int64_t x_stride,
+                                                               int64_t rec_stride) {
     __shared__ SmemTables tab;
     load_tables(tab);
     asm volatile("griddepcontrol.wait;" ::: "memory");           // X may be the previous kernel's result; the records
@@ -66,6 +68,9 @@ __global__ void __launch_bounds__(128) quantize_records_kernel(const void *__res
     const int slots = kTokTile * nt;
     const int b = t / slots, m = t % slots;
     if (b >= (int)padded_blocks((int64_t)nb * kBlock)) return;
+    X = (const char *)X + (int64_t)blockIdx.y * x_stride * Loader<DT>::kElemBytes;
+    rec16 += (int64_t)blockIdx.y * rec_stride;
+    recs = (float *)((uint8_t *)recs + (int64_t)blockIdx.y * rec_stride);
     uint4 out[4];
 #pragma unroll
     for (int i = 0; i < 4; i++) out[i] = make_uint4(0, 0, 0, 0);
@@ -106,10 +111,24 @@ __global__ void __launch_bounds__(128) quantize_records_kernel(const void *__res
     recs[slot] = factor;
 }
 
-// The same records from an operand that is already quantised (bd_gemm with a few rows of A).
-__global__ void __launch_bounds__(128) records_from_qtensor_kernel(QView a, int nt, uint8_t *__restrict__ rec16, float *__restrict__ recs) {
+constexpr int kMaxBatch = 64;
+struct OperandBatch {                      // the operands of a batch that differ per problem (same shape and pitch)
+    const uint8_t *codes[kMaxBatch], *ids[kMaxBatch], *scales[kMaxBatch];
+};
+// The same records from an operand that is already quantised (bd_gemm with a few rows of A).  BATCH: blockIdx.y
+// picks the operand from `batch` and the records advance by rec_stride bytes.
+template <bool BATCH>
+__global__ void __launch_bounds__(128) records_from_qtensor_kernel(QView a, int nt, uint8_t *__restrict__ rec16, float *__restrict__ recs,
+                                                                   const __grid_constant__ OperandBatch batch, int64_t rec_stride) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (BATCH) {
+        a.codes = (uint8_t *)batch.codes[blockIdx.y];
+        a.ids = (uint8_t *)batch.ids[blockIdx.y];
+        a.scales = (uint8_t *)batch.scales[blockIdx.y];
+        rec16 += (int64_t)blockIdx.y * rec_stride;
+        recs = (float *)((uint8_t *)recs + (int64_t)blockIdx.y * rec_stride);
+    }
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     const int slots = kTokTile * nt, nb = (int)(a.K / kBlock);
     const int b = t / slots, m = t % slots;
@@ -201,12 +220,13 @@ struct Params {
     void *Y;
     int64_t ldy;
     int64_t N;                             // weight rows (the last CTA's tile may reach past them)
+    int64_t rec_stride, y_stride;          // batch (blockIdx.y): bytes between the problems' records, elements between results
     int M, units, tail_blocks, y_bf16;     // units = ceil(K / 128); tail_blocks = blocks of the last unit if it is short, else 0
 };
 
 // Shared memory of a CTA: per warp kStages stages of kStageBytes, then the warps' sums [warps][NT][4][32] floats.
-template <int NT>
-__global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_constant__ Params p) {
+template <int NT, bool BATCH>
+__global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_constant__ Params p, const __grid_constant__ OperandBatch batch) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ uint2 lut[16];
     const int warps = blockDim.x / 32, warp = threadIdx.x / 32, lane = threadIdx.x % 32, g = lane >> 2, t = lane & 3;
@@ -219,12 +239,14 @@ __global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_
     // ---- copies of one unit into a stage: two 16-byte pieces of codes per lane, a scale word or an id word ----
     // (source pointers walk from one of the warp's units to its next)
     const int crow = lane >> 2, cpiece = lane & 3;               // rows crow and crow + 8, piece = block inside the unit
-    const uint8_t *csrc = p.codes + (r0 + crow) * p.ldc + cpiece * 16 + (int64_t)warp * (kUnitK / 2);
+    const uint8_t *w_codes = BATCH ? batch.codes[blockIdx.y] : p.codes, *w_ids = BATCH ? batch.ids[blockIdx.y] : p.ids,
+                  *w_scales = BATCH ? batch.scales[blockIdx.y] : p.scales;
+    const uint8_t *csrc = w_codes + (r0 + crow) * p.ldc + cpiece * 16 + (int64_t)warp * (kUnitK / 2);
     const int64_t cstep = (int64_t)warps * (kUnitK / 2), row8 = 8 * p.ldc;
     const uint32_t cdst = ring_s + (uint32_t)(crow * 64 + ((cpiece ^ (crow >> 1)) & 3) * 16);
     const int mrow = lane & 15, mrr = rr0 + mrow;                // lanes 0..15: scale word of row mrow; 16..31: id word
     const int64_t matom = lane < 16 ? kScaleAtomBytes : kIdAtomBytes;
-    const uint8_t *msrc = (lane < 16 ? p.scales + (mrr % 32) * 16 + (mrr / 32) * 4 : p.ids + (mrr % 32) * 8 + (mrr / 64) * 4) +
+    const uint8_t *msrc = (lane < 16 ? w_scales + (mrr % 32) * 16 + (mrr / 32) * 4 : w_ids + (mrr % 32) * 8 + (mrr / 64) * 4) +
                           ((int64_t)warp * p.row_tiles + rt) * matom;
     const int64_t mstep = (int64_t)warps * p.row_tiles * matom;
     const uint32_t mdst = ring_s + (uint32_t)(kCodeBytes + (lane < 16 ? 0 : kRows * 4) + mrow * 4);
@@ -258,8 +280,9 @@ __global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_
 #pragma unroll
     for (int n = 0; n < NT; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.0f;
     const int id_shift = ((rr0 / 32) & 1) * 16;                  // which half of the id word holds this row group
-    const uint8_t *my_rec = p.rec16 + g * (kBlock * 2) + t * 16 + (size_t)warp * (kUnitBlocks * NT * kRecBytes);
-    const float *my_fac = p.recs + 2 * t + (size_t)warp * (kUnitBlocks * NT * kTokTile);
+    const int64_t rec_off = BATCH ? (int64_t)blockIdx.y * p.rec_stride : 0;
+    const uint8_t *my_rec = p.rec16 + rec_off + g * (kBlock * 2) + t * 16 + (size_t)warp * (kUnitBlocks * NT * kRecBytes);
+    const float *my_fac = (const float *)((const uint8_t *)p.recs + rec_off) + 2 * t + (size_t)warp * (kUnitBlocks * NT * kTokTile);
     const size_t rec_step = (size_t)warps * (kUnitBlocks * NT * kRecBytes), fac_step = (size_t)warps * (kUnitBlocks * NT * kTokTile);
 
     for (int i = 0; i < n_units; i++) {
@@ -327,8 +350,9 @@ __global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_
         const int n = tok / kTokTile, tk = tok % kTokTile, src = ((n * 4) + (row / 8) * 2 + (tk & 1)) * 32 + (row % 8) * 4 + tk / 2;
         float y = 0.0f;
         for (int w = 0; w < warps; w++) y += red[w * NT * 128 + src];
-        if (p.y_bf16) ((__nv_bfloat16 *)p.Y)[(int64_t)tok * p.ldy + r0 + row] = __float2bfloat16_rn(y);
-        else ((float *)p.Y)[(int64_t)tok * p.ldy + r0 + row] = y;
+        const int64_t at = (BATCH ? (int64_t)blockIdx.y * p.y_stride : 0) + (int64_t)tok * p.ldy + r0 + row;
+        if (p.y_bf16) ((__nv_bfloat16 *)p.Y)[at] = __float2bfloat16_rn(y);
+        else ((float *)p.Y)[at] = y;
     }
 }
 

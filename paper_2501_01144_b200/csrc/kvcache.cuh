@@ -97,11 +97,22 @@ __global__ void __launch_bounds__(256) kv_quantize_chunks_kernel(const void *__r
 
 // O[q, c] = (product over the stored chunks, fp32, or nothing) + sum over the recent tokens of P[q, n_q + k] * V_recent[k, c],
 // the latter in fp32 on the source values ("maintained in high precision").  Thread = one output.
-template <int DT, typename OutT>
+// blockIdx.y = head of a batch: `recent` then is an array of the heads' pointers, part / P / Y advance by their strides.
+struct RecentBatch {
+    const void *ptr[64];
+};
+template <int DT, typename OutT, bool BATCH>
 __global__ void kv_pv_finish_kernel(const float *__restrict__ part, int64_t ld_part, const float *__restrict__ P, int64_t ldp, int64_t n_q,
-                                    int n_recent, const void *__restrict__ recent, int d, int64_t q_rows, OutT *__restrict__ Y, int64_t ldy) {
+                                    int n_recent, const void *__restrict__ recent, int d, int64_t q_rows, OutT *__restrict__ Y, int64_t ldy,
+                                    const __grid_constant__ RecentBatch batch, int64_t part_stride, int64_t p_stride, int64_t y_stride) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= q_rows * d) return;
+    if (BATCH) {
+        recent = batch.ptr[blockIdx.y];
+        if (part) part += (int64_t)blockIdx.y * part_stride;
+        P += (int64_t)blockIdx.y * p_stride;
+        Y += (int64_t)blockIdx.y * y_stride;
+    }
     const int64_t q = t / d;
     const int c = (int)(t % d);
     float acc = 0.0f;

@@ -106,3 +106,63 @@ def test_decoding_token_by_token_never_changes_a_stored_chunk():
     with pytest.raises(bd.BdError):
         cache.append(to_device(k[:64], kind), to_device(v[:64], kind))       # beyond the capacity
     bd.poll_status()
+
+
+@pytest.mark.parametrize("n,q_rows,heads,d", [(19, 4, 3, 128), (77, 4, 8, 128), (1000, 8, 2, 64), (4127, 4, 8, 128), (300, 12, 3, 128)])
+@pytest.mark.parametrize("impl", [bd.GEMM_AUTO, bd.GEMM_SIMT])
+def test_batched_heads_match_the_oracle_head_by_head(n, q_rows, heads, d, impl):
+    # the KV heads of a layer in one call (one launch sequence for all heads with at most 8 query rows, head by head
+    # otherwise): every head against its own oracle cache, guard bands around results and workspace strides
+    cap, kind = 4160, torch.bfloat16
+    caches, refs, Qs, Qrefs = [], [], [], []
+    rng = np.random.default_rng(n + q_rows + heads)
+    for h in range(heads):
+        k, v = _rows(n, d, kind, seed=n + 7 * h)
+        c, r = bd.KVCache(cap, d, dtype=kind), OracleCache(d)
+        c.append(to_device(k, kind), to_device(v, kind))
+        r.append(k, v)
+        caches.append(c)
+        refs.append(r)
+        qb = inputs.to_bf16_bits(rng.standard_normal((q_rows, d)).astype(np.float32))
+        Qs.append(bd.quantize_act(to_device(qb, torch.bfloat16)))
+        Qrefs.append(oracle.quantize(qb, dtype=oracle.BF16))
+    bd.set_gemm_impl(impl)
+    try:
+        pitch = (n + 3) // 4 * 4
+        S_all = torch.full((heads, q_rows, pitch + 4), -7.0, device="cuda")
+        S = S_all[:, :, :n]
+        before = bd.launch_count()
+        bd.kvcache_scores_batched(caches, Qs, out=S)
+        if impl == bd.GEMM_AUTO and q_rows <= 8:
+            assert bd.launch_count() - before == 2
+        assert (S_all[:, :, n:] == -7.0).all(), "write past the scores' rows"
+        Sh = S.cpu().numpy()
+        P = np.zeros((heads, q_rows, n), np.float32)
+        for h in range(heads):
+            Sref, T = refs[h].scores(Qrefs[h])
+            ok, ratio = gemm_tolerance_ok(Sh[h], Sref, T)
+            assert ok, f"head {h} scores: max err / bound = {ratio}"
+            z = Sh[h].astype(np.float64) / np.sqrt(d)
+            e = np.exp(z - z.max(-1, keepdims=True))
+            P[h] = (e / e.sum(-1, keepdims=True)).astype(np.float32)
+        Pd = torch.zeros(heads, q_rows, pitch, device="cuda")[:, :, :n]
+        Pd.copy_(torch.from_numpy(P))
+        O_all = torch.full((heads, q_rows, d + 8), -7.0, device="cuda")
+        before = bd.launch_count()
+        bd.kvcache_pv_batched(caches, Pd, out=O_all[:, :, :d])
+        if impl == bd.GEMM_AUTO and q_rows <= 8:
+            assert bd.launch_count() - before == (3 if n >= 32 else 1)
+        assert (O_all[:, :, d:] == -7.0).all(), "write past the result's rows"
+        Oh = O_all[:, :, :d].cpu().numpy()
+        for h in range(heads):
+            Oref, To = refs[h].pv(P[h])
+            ok, ratio = gemm_tolerance_ok(Oh[h], Oref, To)
+            assert ok, f"head {h} P V: max err / bound = {ratio}"
+            # and the single-head call agrees (the shares of K may be cut differently, so not bit for bit)
+            ok, ratio = gemm_tolerance_ok(caches[h].pv(Pd[h]).cpu().numpy(), Oref, To)
+            assert ok, f"head {h} P V, single call: max err / bound = {ratio}"
+        O16 = bd.kvcache_pv_batched(caches, Pd, dtype=torch.bfloat16)
+        assert torch.equal(O16.cpu(), torch.from_numpy(Oh).to(torch.bfloat16))
+    finally:
+        bd.set_gemm_impl(bd.GEMM_AUTO)
+    bd.poll_status()
