@@ -843,9 +843,11 @@ def run_case(args):
         torch.cuda.synchronize()
         print(json.dumps({"case": args.case, "us_per_step": e0.elapsed_time(e1) / reps * 1e3}))
         return
-    if args.case == "decode":
-        # a decode-sized call of the LLaMA2 MLP sweep: 16 tokens against K = 11008, N = 4096; six weight copies in rotation
-        K, N, M = 11008, 4096, 16
+    if args.case in ("decode", "decode8"):
+        # a decode-sized call of the LLaMA2 MLP sweep, six weight copies in rotation.  decode: 16 tokens against
+        # K = 11008, N = 4096 (tensor-core path with a K split); decode8: 8 tokens against K = 4096, N = 11008 (the
+        # warp-level kernel)
+        K, N, M = (11008, 4096, 16) if args.case == "decode" else (4096, 11008, 8)
         wsrc = dev_bf16(inputs.weights_normal(N, K, seed=3))
         wqs = [bd.quantize_weights(wsrc, bd.SELECT_TWO_STAGE) for _ in range(6)]
         x = dev_bf16(inputs.act_post_silu(M, K, seed=3))
@@ -947,7 +949,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--case", default=None,
-                    choices=["quantizer", "quantizer_f32", "step", "decode", "quantizer_strided", "requant_gate_up", "attention"]
+                    choices=["quantizer", "quantizer_f32", "step", "decode", "decode8", "quantizer_strided", "requant_gate_up", "attention"]
                     + ["linear_" + n for n, _, _ in LAYERS],
                     help="run a few launches of one small case (for profiler captures) instead of the benchmark")
     args = ap.parse_args()
