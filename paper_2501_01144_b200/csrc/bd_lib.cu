@@ -201,26 +201,22 @@ bd_status launch_warp_main(int64_t M, int64_t K, const QView &W, void *Y, bd_dty
     const int warps = warp_kernel_warps(tiles * n * wk::kRows, (K + wk::kUnitK - 1) / wk::kUnitK * wk::kUnitK);
     const size_t smem = (size_t)warps * (wk::kStages * wk::kStageBytes + nt * 512);
     const dim3 grid((unsigned)tiles, (unsigned)n);
+    const bool ragged = W.rows % wk::kRows != 0 || K % wk::kUnitK != 0;
+    using Kernel = void (*)(const wk::Params, const wk::OperandBatch);
+    static const Kernel kernels[8] = {wk::gemm_warp_kernel<1, false, false>, wk::gemm_warp_kernel<1, false, true>, wk::gemm_warp_kernel<1, true, false>,
+                                      wk::gemm_warp_kernel<1, true, true>,   wk::gemm_warp_kernel<2, false, false>, wk::gemm_warp_kernel<2, false, true>,
+                                      wk::gemm_warp_kernel<2, true, false>,  wk::gemm_warp_kernel<2, true, true>};
     static bool smem_set[kMaxDevices] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < kMaxDevices && !smem_set[dev]) {
         const int most = wk::kMaxWarps * (wk::kStages * wk::kStageBytes + 2 * 512);
-        if (cudaFuncSetAttribute(wk::gemm_warp_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
-            cudaFuncSetAttribute(wk::gemm_warp_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
-            cudaFuncSetAttribute(wk::gemm_warp_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess ||
-            cudaFuncSetAttribute(wk::gemm_warp_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess)
-            return cuda_result(cudaGetLastError());
+        for (Kernel k : kernels)
+            if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess) return cuda_result(cudaGetLastError());
         smem_set[dev] = true;
     }
     const wk::OperandBatch none{};
-    if (batch) {
-        if (nt == 1) launch_serialized(wk::gemm_warp_kernel<1, true>, grid, 32u * warps, smem, st, p, *batch);
-        else launch_serialized(wk::gemm_warp_kernel<2, true>, grid, 32u * warps, smem, st, p, *batch);
-    } else {
-        if (nt == 1) launch_serialized(wk::gemm_warp_kernel<1, false>, grid, 32u * warps, smem, st, p, none);
-        else launch_serialized(wk::gemm_warp_kernel<2, false>, grid, 32u * warps, smem, st, p, none);
-    }
+    launch_serialized(kernels[(nt - 1) * 4 + (batch ? 2 : 0) + (ragged ? 1 : 0)], grid, 32u * warps, smem, st, p, batch ? *batch : none);
     return launch_result(1);
 }
 // X: n problems x_stride elements apart (n = 1: one).

@@ -225,7 +225,9 @@ struct Params {
 };
 
 // Shared memory of a CTA: per warp kStages stages of kStageBytes, then the warps' sums [warps][NT][4][32] floats.
-template <int NT, bool BATCH>
+// RAGGED: the rows do not fill the last tile of 16 or K does not fill the last unit of 128 (guards in the copy and
+// store paths that whole shapes do without).
+template <int NT, bool BATCH, bool RAGGED>
 __global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_constant__ Params p, const __grid_constant__ OperandBatch batch) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ uint2 lut[16];
@@ -252,11 +254,11 @@ __global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_
     const uint32_t mdst = ring_s + (uint32_t)(kCodeBytes + (lane < 16 ? 0 : kRows * 4) + mrow * 4);
     // rows past N and blocks past K are not read: their codes become zeros (index 0 = value 0), so whatever their
     // scale and id entries hold adds nothing
-    const bool row_ok_lo = r0 + crow < p.N, row_ok_hi = r0 + crow + 8 < p.N;
+    const bool row_ok_lo = !RAGGED || r0 + crow < p.N, row_ok_hi = !RAGGED || r0 + crow + 8 < p.N;
     int next_unit = warp;
     auto issue = [&](int stage) {
         const uint32_t so = (uint32_t)stage * kStageBytes;
-        const bool piece_ok = !(p.tail_blocks && next_unit == p.units - 1 && cpiece >= p.tail_blocks);
+        const bool piece_ok = !RAGGED || !(p.tail_blocks && next_unit == p.units - 1 && cpiece >= p.tail_blocks);
         if (row_ok_lo && piece_ok) cp_async16(cdst + so, csrc);
         else asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(cdst + so), "r"(0) : "memory");
         if (row_ok_hi && piece_ok) cp_async16(cdst + so + 8 * 64, csrc + row8);
@@ -264,7 +266,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_
         cp_async4(mdst + so, msrc);
         csrc += cstep;
         msrc += mstep;
-        next_unit += warps;
+        if (RAGGED) next_unit += warps;
     };
     // this warp's units: warp, warp + warps, ...
     const int n_units = p.units > warp ? (p.units - warp + warps - 1) / warps : 0;
@@ -298,7 +300,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_
             w_hi[b] = *(const uint32_t *)(s + off + 8 * 64);
         }
         uint32_t sc_lo = *(const uint32_t *)(s + kCodeBytes + g * 4), sc_hi = *(const uint32_t *)(s + kCodeBytes + (g + 8) * 4);
-        if (p.tail_blocks && warp + i * warps == p.units - 1) {     // scale bytes past K may hold anything: make them 2^-127
+        if (RAGGED && p.tail_blocks && warp + i * warps == p.units - 1) {     // scale bytes past K may hold anything: make them 2^-127
             const uint32_t keep = (1u << (8 * p.tail_blocks)) - 1u;
             sc_lo &= keep;
             sc_hi &= keep;
@@ -345,7 +347,7 @@ __global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_
     __syncthreads();
     for (int o = threadIdx.x; o < kRows * kTokTile * NT; o += blockDim.x) {
         const int row = o % kRows, tok = o / kRows;
-        if (tok >= p.M || r0 + row >= p.N) continue;
+        if (tok >= p.M || (RAGGED && r0 + row >= p.N)) continue;
         // accumulator c of lane (row % 8) * 4 + (tok % 8) / 2 holds (row, token): c = (row / 8) * 2 + tok % 2
         const int n = tok / kTokTile, tk = tok % kTokTile, src = ((n * 4) + (row / 8) * 2 + (tk & 1)) * 32 + (row % 8) * 4 + tk / 2;
         float y = 0.0f;
