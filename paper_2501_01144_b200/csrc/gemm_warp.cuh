@@ -39,7 +39,7 @@ constexpr int kTokTile = 8;                // tokens per MMA (its N)
 constexpr int kMaxTokens = 16;
 constexpr int kCodeBytes = kRows * kUnitK / 2;         // 1024
 constexpr int kStageBytes = kCodeBytes + kRows * 4 + kRows * 4;   // + scale words + id words = 1152
-constexpr int kStages = 4;
+constexpr int kStages = 2;
 constexpr int kRecBytes = kTokTile * kBlock * 2;       // fp16 values of a record (8 tokens x 32)
 constexpr int kMaxWarps = 16;
 
@@ -228,7 +228,7 @@ struct Params {
 // RAGGED: the rows do not fill the last tile of 16 or K does not fill the last unit of 128 (guards in the copy and
 // store paths that whole shapes do without).
 template <int NT, bool BATCH, bool RAGGED>
-__global__ void __launch_bounds__(32 * kMaxWarps) gemm_warp_kernel(const __grid_constant__ Params p, const __grid_constant__ OperandBatch batch) {
+__global__ void __launch_bounds__(32 * kMaxWarps, 2) gemm_warp_kernel(const __grid_constant__ Params p, const __grid_constant__ OperandBatch batch) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ uint2 lut[16];
     const int warps = blockDim.x / 32, warp = threadIdx.x / 32, lane = threadIdx.x % 32, g = lane >> 2, t = lane & 3;
