@@ -603,17 +603,24 @@ def run_gpu(args, rank, world, local_rank):
         torch.cuda.synchronize()
         attend_us = e0.elapsed_time(e1) / 10 * 1e3
         new_k = dev_bf16(inputs.to_bf16_bits(rng_kv.standard_normal((1, hd)).astype(np.float32)))
+        new_kv = new_k.expand(kvh, 1, hd).contiguous()
         e0.record()
-        for _ in range(10):                                   # ten more tokens per head (27 recent tokens at the end)
+        for _ in range(5):                                    # five tokens per head, one call per head
             for g in range(kvh):
                 caches[g].append(new_k, new_k)
         e1.record()
         torch.cuda.synchronize()
-        append_us = e0.elapsed_time(e1) / 10 * 1e3
+        append_per_head_us = e0.elapsed_time(e1) / 5 * 1e3
+        e0.record()
+        for _ in range(5):                                    # five more tokens, all heads per call (27 recent tokens at the end)
+            bd.kvcache_append_batched(caches, new_kv, new_kv)
+        e1.record()
+        torch.cuda.synchronize()
+        append_us = e0.elapsed_time(e1) / 5 * 1e3
         cache_bytes = kvh * 2 * n_tok * hd * 0.546875
         kv_cache = {"workload": "8 KV heads x 4113 tokens x head_dim 128, 4 query heads per KV head, one object per KV head, scores and P x V of all heads per call",
                     "scores_and_pv_us_per_step": attend_us, "launches_per_step": attend_launches, "scores_and_pv_us_per_step_head_by_head": per_head_us,
-                    "append_one_token_us_per_step": append_us,
+                    "append_one_token_us_per_step": append_us, "append_one_token_us_per_step_head_by_head": append_per_head_us,
                     "cache_bytes_read_per_step": cache_bytes, "cache_read_gbs": cache_bytes / attend_us / 1e3,
                     "stored_bits_per_value": 4.375, "recent_tokens_in_high_precision": n_tok % 32}
         del caches, probs

@@ -256,9 +256,12 @@ bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int
                         int64_t ldy, void *workspace, size_t workspace_bytes, void *stream);
 /* The same two calls for the n KV heads of a layer in one decode step (n >= 1): c[i] all of one capacity,
  * head_dim, dtype and length; Q[i] [q, head_dim] with the same q; head i reads P + i * stride_p and writes
- * S + i * stride_s / Y + i * stride_y (strides in elements).  With q <= 8 and n <= 64 (and the library's own
+ * S + i * stride_s / Y + i * stride_y, and takes its t new tokens from Knew + i * stride_k, Vnew + i * stride_v
+ * (strides in elements; every head's length advances by t).  With q <= 8 and n <= 64 (and the library's own
  * choice of product kernel) the heads share two (scores) or three (P x V) launches; otherwise the calls
  * above run head by head.  workspace: bd_kvcache_batched_workspace_size bytes, 256-byte aligned. */
+bd_status bd_kvcache_append_batched(bd_kvcache *c, int64_t n, const void *Knew, const void *Vnew, int64_t t, int64_t ldk,
+                                    int64_t ldv, int64_t stride_k, int64_t stride_v, void *stream);
 bd_status bd_kvcache_batched_workspace_size(int64_t n, int64_t capacity, int64_t head_dim, int64_t q_rows, size_t *bytes);
 bd_status bd_kvcache_scores_batched(const bd_kvcache *c, int64_t n, const bd_qtensor *Q, void *S, bd_dtype sdtype,
                                     int64_t lds, int64_t stride_s, void *workspace, size_t workspace_bytes, void *stream);

@@ -85,6 +85,7 @@ def load():
     lib.bd_kvcache_workspace_size.argtypes = [i64, i64, i64, szp]
     lib.bd_kvcache_scores.argtypes = [kp, qp, vp, ci, i64, vp, sz, vp]
     lib.bd_kvcache_pv.argtypes = [kp, vp, i64, i64, vp, ci, i64, vp, sz, vp]
+    lib.bd_kvcache_append_batched.argtypes = [kp, i64, vp, vp, i64, i64, i64, i64, i64, vp]
     lib.bd_kvcache_batched_workspace_size.argtypes = [i64, i64, i64, i64, szp]
     lib.bd_kvcache_scores_batched.argtypes = [kp, i64, qp, vp, ci, i64, i64, vp, sz, vp]
     lib.bd_kvcache_pv_batched.argtypes = [kp, i64, vp, i64, i64, i64, vp, ci, i64, i64, vp, sz, vp]
@@ -451,6 +452,20 @@ def _kv_batch(caches, q_rows):
     if c0._ws is None or c0._ws.numel() < b.value:
         c0._ws = torch.empty(max(b.value, 256), dtype=torch.uint8, device=c0.k.codes.device)
     return arr, ctypes.c_void_p(c0._ws.data_ptr()), c0._ws.numel()
+
+
+def kvcache_append_batched(caches, k_new, v_new, stream=None):
+    """t new tokens for n KV heads of the same length in one call: k_new, v_new [n, t, head_dim] of the caches' dtype."""
+    n, c0 = len(caches), caches[0]
+    if k_new.shape != v_new.shape or k_new.dim() != 3 or k_new.shape[0] != n or k_new.shape[2] != c0.head_dim or k_new.stride(2) != 1 or v_new.stride(2) != 1:
+        raise ValueError("key / value rows must be [n, t, head_dim] with a contiguous last axis")
+    if _TORCH_DTYPE[k_new.dtype] != c0._c.dtype or v_new.dtype != k_new.dtype:
+        raise ValueError("key / value rows must have the caches' dtype")
+    arr = (_CKVCache * n)(*[c._c for c in caches])
+    _check(load().bd_kvcache_append_batched(arr, n, ctypes.c_void_p(k_new.data_ptr()), ctypes.c_void_p(v_new.data_ptr()), k_new.shape[1],
+                                            k_new.stride(1), v_new.stride(1), k_new.stride(0), v_new.stride(0), _stream(stream)))
+    for c, done in zip(caches, arr):
+        c._c.length = done.length
 
 
 def kvcache_scores_batched(caches, Qs, out=None, dtype=torch.float32, stream=None):

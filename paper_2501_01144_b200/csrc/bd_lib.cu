@@ -296,13 +296,28 @@ void *g_noalloc_ptr[kMaxDevices] = {};
 
 // launchers of the KV-cache kernels per source type
 template <int DT>
-void launch_kv_keys(const void *Knew, int64_t ldk, int64_t t, const QView &k, int64_t row0, cudaStream_t st) {
-    kv_append_keys_kernel<DT><<<grid_for(t * kBlocksPerAtom, 256), 256, 0, st>>>(Knew, ldk, t, k, row0, (int)(k.K / kBlock));
+void launch_kv_keys(const void *Knew, int64_t ldk, int64_t t, const QView &k, int64_t row0, cudaStream_t st, const KvBatch *batch = nullptr,
+                    int n = 1, int64_t src_stride = 0) {
+    const dim3 grid(grid_for(t * kBlocksPerAtom, 256), (unsigned)n);
+    const KvBatch none{};
+    if (batch) kv_append_keys_kernel<DT, true><<<grid, 256, 0, st>>>(Knew, ldk, t, k, row0, (int)(k.K / kBlock), *batch, src_stride);
+    else kv_append_keys_kernel<DT, false><<<grid, 256, 0, st>>>(Knew, ldk, t, k, row0, (int)(k.K / kBlock), none, 0);
 }
 template <int DT>
-void launch_kv_chunks(const void *src, int64_t ld, int n_chunks, const QView &v, int chunk0, cudaStream_t st) {
+void launch_kv_chunks(const void *src, int64_t ld, int n_chunks, const QView &v, int chunk0, cudaStream_t st, const KvBatch *batch = nullptr,
+                      int n = 1, int64_t src_stride = 0) {
     const int pairs = (chunk0 + n_chunks + 1) / 2 - chunk0 / 2;
-    kv_quantize_chunks_kernel<DT><<<grid_for(v.rows * pairs, 256), 256, 0, st>>>(src, ld, n_chunks, v, chunk0);
+    const dim3 grid(grid_for(v.rows * pairs, 256), (unsigned)n);
+    const KvBatch none{};
+    if (batch) kv_quantize_chunks_kernel<DT, true><<<grid, 256, 0, st>>>(src, ld, n_chunks, v, chunk0, *batch, src_stride);
+    else kv_quantize_chunks_kernel<DT, false><<<grid, 256, 0, st>>>(src, ld, n_chunks, v, chunk0, none, 0);
+}
+void launch_kv_recent(const void *Vnew, int64_t ldv_bytes, int rows, int row_bytes, void *recent, int slot0, cudaStream_t st,
+                      const KvBatch *batch = nullptr, int n = 1, int64_t src_stride_bytes = 0) {
+    const dim3 grid(grid_for((int64_t)rows * row_bytes / 2, 256), (unsigned)n);
+    const KvBatch none{};
+    if (batch) kv_store_recent_kernel<true><<<grid, 256, 0, st>>>(Vnew, ldv_bytes, rows, row_bytes, (uint8_t *)recent, slot0, *batch, src_stride_bytes);
+    else kv_store_recent_kernel<false><<<grid, 256, 0, st>>>(Vnew, ldv_bytes, rows, row_bytes, (uint8_t *)recent, slot0, none, 0);
 }
 template <int DT>
 void launch_kv_finish(const float *part, int64_t ld_part, const float *P, int64_t ldp, int64_t n_q, int n_recent, const void *recent,
@@ -775,30 +790,37 @@ bd_status bd_kvcache_reset(bd_kvcache *c, void *stream) {
     return BD_OK;
 }
 
-bd_status bd_kvcache_append(bd_kvcache *c, const void *Knew, const void *Vnew, int64_t t, int64_t ldk, int64_t ldv, void *stream) {
-    bd_status s = check_kvcache(c);
-    if (s) return s;
-    if (!Knew || !Vnew || t <= 0) return BD_ERR_INVALID_ARG;
+namespace {
+// t new tokens for n heads (n = 1: `c` alone, no batch): the same launches, grid.y = head.
+bd_status kv_append(bd_kvcache *c, int64_t n, const void *Knew, const void *Vnew, int64_t t, int64_t ldk, int64_t ldv, int64_t stride_k,
+                    int64_t stride_v, cudaStream_t st) {
     const int64_t d = c->head_dim;
     const int esz = elem_bytes(c->dtype);
-    if (ldk < d || ldv < d || c->length + t > c->capacity) return BD_ERR_SHAPE;
-    if (!aligned16(Knew) || !aligned16(Vnew) || (ldk * esz) % 16 || (ldv * esz) % 16) return BD_ERR_ALIGN;
-    cudaStream_t st = (cudaStream_t)stream;
+    KvBatch kb{}, vb{};
+    const KvBatch *pk = nullptr, *pv = nullptr;
+    if (n > 1) {
+        for (int64_t i = 0; i < n; i++) {
+            kb.codes[i] = (uint8_t *)c[i].k.codes; kb.ids[i] = (uint8_t *)c[i].k.ids; kb.scales[i] = (uint8_t *)c[i].k.scales;
+            vb.codes[i] = (uint8_t *)c[i].v.codes; vb.ids[i] = (uint8_t *)c[i].v.ids; vb.scales[i] = (uint8_t *)c[i].v.scales;
+            kb.recent[i] = vb.recent[i] = c[i].v_recent;
+        }
+        pk = &kb;
+        pv = &vb;
+    }
     const QView kq = view_of(&c->k), vq = view_of(&c->v);
     int kernels = 0;
     // keys: one quantisation per new token, appended as rows
-    BD_KV_DISPATCH(c->dtype, launch_kv_keys, Knew, ldk, t, kq, c->length, st);
+    BD_KV_DISPATCH(c->dtype, launch_kv_keys, Knew, ldk, t, kq, c->length, st, pk, (int)n, stride_k);
     kernels++;
     // values: complete the waiting chunk, then whole chunks straight from the source, then the new remainder
     int64_t done = 0, len = c->length;
     const int waiting = (int)(len % kBlock);
     if (waiting) {
         const int fill = (int)std::min<int64_t>(kBlock - waiting, t);
-        kv_store_recent_kernel<<<grid_for((int64_t)fill * d * esz / 2, 256), 256, 0, st>>>(Vnew, ldv * esz, fill, (int)(d * esz),
-                                                                                         (uint8_t *)c->v_recent, waiting);
+        launch_kv_recent(Vnew, ldv * esz, fill, (int)(d * esz), c->v_recent, waiting, st, pv, (int)n, stride_v * esz);
         kernels++;
         if (waiting + fill == kBlock) {
-            BD_KV_DISPATCH(c->dtype, launch_kv_chunks, c->v_recent, d, 1, vq, (int)(len / kBlock), st);
+            BD_KV_DISPATCH(c->dtype, launch_kv_chunks, n > 1 ? nullptr : c->v_recent, d, 1, vq, (int)(len / kBlock), st, pv, (int)n, (int64_t)0);
             kernels++;
         }
         done = fill;
@@ -806,18 +828,34 @@ bd_status bd_kvcache_append(bd_kvcache *c, const void *Knew, const void *Vnew, i
     }
     const int64_t whole = (t - done) / kBlock;
     if (whole) {
-        BD_KV_DISPATCH(c->dtype, launch_kv_chunks, (const char *)Vnew + done * ldv * esz, ldv, (int)whole, vq, (int)(len / kBlock), st);
+        BD_KV_DISPATCH(c->dtype, launch_kv_chunks, (const char *)Vnew + done * ldv * esz, ldv, (int)whole, vq, (int)(len / kBlock), st, pv, (int)n, stride_v);
         kernels++;
         done += whole * kBlock;
     }
     if (done < t) {
         const int rest = (int)(t - done);
-        kv_store_recent_kernel<<<grid_for((int64_t)rest * d * esz / 2, 256), 256, 0, st>>>((const char *)Vnew + done * ldv * esz, ldv * esz, rest,
-                                                                                         (int)(d * esz), (uint8_t *)c->v_recent, 0);
+        launch_kv_recent((const char *)Vnew + done * ldv * esz, ldv * esz, rest, (int)(d * esz), c->v_recent, 0, st, pv, (int)n, stride_v * esz);
         kernels++;
     }
-    c->length += t;
+    for (int64_t i = 0; i < n; i++) c[i].length += t;
     return launch_result(kernels);
+}
+bd_status check_append(const bd_kvcache *c, const void *Knew, const void *Vnew, int64_t t, int64_t ldk, int64_t ldv) {
+    if (!Knew || !Vnew || t <= 0) return BD_ERR_INVALID_ARG;
+    const int64_t d = c->head_dim;
+    const int esz = elem_bytes(c->dtype);
+    if (ldk < d || ldv < d || c->length + t > c->capacity) return BD_ERR_SHAPE;
+    if (!aligned16(Knew) || !aligned16(Vnew) || (ldk * esz) % 16 || (ldv * esz) % 16) return BD_ERR_ALIGN;
+    return BD_OK;
+}
+}  // namespace
+
+bd_status bd_kvcache_append(bd_kvcache *c, const void *Knew, const void *Vnew, int64_t t, int64_t ldk, int64_t ldv, void *stream) {
+    bd_status s = check_kvcache(c);
+    if (s) return s;
+    s = check_append(c, Knew, Vnew, t, ldk, ldv);
+    if (s) return s;
+    return kv_append(c, 1, Knew, Vnew, t, ldk, ldv, 0, 0, (cudaStream_t)stream);
 }
 
 bd_status bd_kvcache_workspace_size(int64_t capacity, int64_t head_dim, int64_t q_rows, size_t *bytes) {
@@ -901,6 +939,24 @@ bool kv_batch_fused(int64_t n, int64_t q_rows, int64_t N, int64_t K) {
     return n <= wk::kMaxBatch && g_gemm_impl != BD_GEMM_SIMT && g_gemm_impl != BD_GEMM_TCGEN05 && q_rows <= wk::kTokTile && wk::supported(q_rows, N, K);
 }
 }  // namespace
+
+bd_status bd_kvcache_append_batched(bd_kvcache *c, int64_t n, const void *Knew, const void *Vnew, int64_t t, int64_t ldk, int64_t ldv,
+                                    int64_t stride_k, int64_t stride_v, void *stream) {
+    bd_status s = check_kvcache_batch(c, n);
+    if (s) return s;
+    s = check_append(c, Knew, Vnew, t, ldk, ldv);
+    if (s) return s;
+    const int esz = elem_bytes(c->dtype);
+    if (n > 1 && ((stride_k * esz) % 16 || (stride_v * esz) % 16)) return BD_ERR_ALIGN;
+    if (n > kKvMaxBatch) {                                        // more heads than a launch takes: head by head
+        for (int64_t i = 0; i < n; i++) {
+            s = kv_append(&c[i], 1, (const char *)Knew + i * stride_k * esz, (const char *)Vnew + i * stride_v * esz, t, ldk, ldv, 0, 0, (cudaStream_t)stream);
+            if (s) return s;
+        }
+        return BD_OK;
+    }
+    return kv_append(c, n, Knew, Vnew, t, ldk, ldv, stride_k, stride_v, (cudaStream_t)stream);
+}
 
 bd_status bd_kvcache_batched_workspace_size(int64_t n, int64_t capacity, int64_t head_dim, int64_t q_rows, size_t *bytes) {
     if (n <= 0) return BD_ERR_INVALID_ARG;

@@ -17,12 +17,30 @@
 
 namespace bd {
 
+// The KV heads of a layer in one launch: blockIdx.y picks the head's operand and its high-precision rows; the sources
+// advance by a stride per head.  (kernels launched with BATCH = false ignore it.)
+constexpr int kKvMaxBatch = 64;
+struct KvBatch {
+    uint8_t *codes[kKvMaxBatch], *ids[kKvMaxBatch], *scales[kKvMaxBatch];
+    void *recent[kKvMaxBatch];
+};
+template <bool BATCH>
+__device__ __forceinline__ void kv_pick(QView &q, const KvBatch &batch) {
+    if (BATCH) {
+        q.codes = batch.codes[blockIdx.y];
+        q.ids = batch.ids[blockIdx.y];
+        q.scales = batch.scales[blockIdx.y];
+    }
+}
+
 // New key rows: thread = (new row i, block b of 4); the four lanes of a row merge scale bytes and id nibbles.
-template <int DT>
+template <int DT, bool BATCH>
 __global__ void __launch_bounds__(256) kv_append_keys_kernel(const void *__restrict__ Knew, int64_t ldk, int64_t t_new, QView k,
-                                                             int64_t row0, int nb) {
+                                                             int64_t row0, int nb, const __grid_constant__ KvBatch batch, int64_t src_stride) {
     __shared__ SmemTables tab;
     load_tables(tab);
+    kv_pick<BATCH>(k, batch);
+    if (BATCH) Knew = (const char *)Knew + (int64_t)blockIdx.y * src_stride * Loader<DT>::kElemBytes;
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t i = t / kBlocksPerAtom;
     const int b = (int)(t % kBlocksPerAtom);
@@ -51,8 +69,13 @@ __global__ void __launch_bounds__(256) kv_append_keys_kernel(const void *__restr
 }
 
 // Value rows that do not complete a chunk: copied as they are into the high-precision slots.
+template <bool BATCH>
 __global__ void kv_store_recent_kernel(const void *__restrict__ Vnew, int64_t ldv_bytes, int rows, int row_bytes, uint8_t *__restrict__ recent,
-                                       int slot0) {
+                                       int slot0, const __grid_constant__ KvBatch batch, int64_t src_stride_bytes) {
+    if (BATCH) {
+        recent = (uint8_t *)batch.recent[blockIdx.y];
+        Vnew = (const char *)Vnew + (int64_t)blockIdx.y * src_stride_bytes;
+    }
     const int t = blockIdx.x * blockDim.x + threadIdx.x;          // one 2-byte unit each
     const int units = row_bytes / 2;
     if (t >= rows * units) return;
@@ -63,10 +86,14 @@ __global__ void kv_store_recent_kernel(const void *__restrict__ Vnew, int64_t ld
 // Whole chunks of 32 value rows -> one block per channel.  Thread = (channel c, pair of chunks p): the chunks 2p and
 // 2p + 1 of a channel share an id byte, so one thread writes both nibbles; a nibble of an earlier call is kept.
 // src: [32 * n_chunks, ld] elements, the rows of chunks chunk0 .. chunk0 + n_chunks - 1.
-template <int DT>
-__global__ void __launch_bounds__(256) kv_quantize_chunks_kernel(const void *__restrict__ src, int64_t ld, int n_chunks, QView v, int chunk0) {
+// BATCH: src is nullptr for "the head's own high-precision rows", else the new rows, src_stride elements per head.
+template <int DT, bool BATCH>
+__global__ void __launch_bounds__(256) kv_quantize_chunks_kernel(const void *__restrict__ src, int64_t ld, int n_chunks, QView v, int chunk0,
+                                                                 const __grid_constant__ KvBatch batch, int64_t src_stride) {
     __shared__ SmemTables tab;
     load_tables(tab);
+    kv_pick<BATCH>(v, batch);
+    if (BATCH) src = src ? (const void *)((const char *)src + (int64_t)blockIdx.y * src_stride * Loader<DT>::kElemBytes) : batch.recent[blockIdx.y];
     const int d = (int)v.rows;
     const int pair0 = chunk0 / 2, n_pairs = (chunk0 + n_chunks + 1) / 2 - pair0;
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;

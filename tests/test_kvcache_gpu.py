@@ -166,3 +166,26 @@ def test_batched_heads_match_the_oracle_head_by_head(n, q_rows, heads, d, impl):
     finally:
         bd.set_gemm_impl(bd.GEMM_AUTO)
     bd.poll_status()
+
+
+@pytest.mark.parametrize("kind", [torch.bfloat16, torch.float32])
+def test_batched_appends_leave_every_head_in_the_oracle_state(kind):
+    # the heads of a layer take their new tokens in one call (pieces that cross chunk borders in every way); each
+    # head's stored keys, value chunks and high-precision rows against its own oracle cache after every piece
+    heads, d, total, cap = 5, 128, 203, 256
+    rows = [_rows(total, d, kind, seed=31 + h) for h in range(heads)]
+    caches = [bd.KVCache(cap, d, dtype=kind) for _ in range(heads)]
+    refs = [OracleCache(d, dtype=ORACLE_DTYPE[kind]) for _ in range(heads)]
+    pos = 0
+    for t in (1, 30, 1, 1, 64, 3, 40, 31, 32):
+        k_new = torch.stack([to_device(rows[h][0][pos:pos + t], kind) for h in range(heads)])
+        v_new = torch.stack([to_device(rows[h][1][pos:pos + t], kind) for h in range(heads)])
+        before = bd.launch_count()
+        bd.kvcache_append_batched(caches, k_new, v_new)
+        assert bd.launch_count() - before <= 5, "the heads share their launches"
+        for h in range(heads):
+            refs[h].append(rows[h][0][pos:pos + t], rows[h][1][pos:pos + t])
+            _check_state(caches[h], refs[h], kind)
+        pos += t
+    assert pos == total
+    bd.poll_status()
