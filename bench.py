@@ -433,7 +433,10 @@ def run_gpu(args, rank, world, local_rank):
                 ws = torch.empty(bd.linear_workspace_size(M, N, K), dtype=torch.uint8, device=dev)
                 for i in range(n_wsets):
                     bd.linear(x, wqs[i], out=y, workspace=ws)
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                l0 = bd.launch_count()
+                bd.linear(x, wqs[0], out=y, workspace=ws)
+                launches_per_call = bd.launch_count() - l0          # 2: quantizer + product (warp-level kernel for up to 8
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)   # tokens); 3: + the K split's sum
                 n_rep = 24 if M <= 1024 else 6
                 torch.cuda._sleep(2_000_000)                  # GPU head start: the events see kernel time, not launch rate
                 a.record()
@@ -453,7 +456,7 @@ def run_gpu(args, rank, world, local_rank):
                 bound_tf = min(2.0 * peaks["bf16_tflops"], flops / nbytes * peaks["hbm_gbs"] / 1e3)
                 sweep.append({"K": K, "N": N, "M": M, "us": us, "host_us_per_call": host_us, "tflops": flops / us / 1e6,
                               "gbs": nbytes / us / 1e3, "floor_us": flops / bound_tf / 1e6,
-                              "frac_of_roofline": flops / us / 1e6 / bound_tf})
+                              "frac_of_roofline": flops / us / 1e6 / bound_tf, "launches_per_call": launches_per_call})
             del wqs
         bd.poll_status()
 
