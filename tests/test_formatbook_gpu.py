@@ -48,6 +48,14 @@ def test_alternative_formatbook_end_to_end():
             bd.set_gemm_impl(impl)
             ok, ratio = gemm_tolerance_ok(bd.gemm(qx, qw).cpu().numpy(), Yref, T)
             assert ok, f"impl {impl}: max err / bound = {ratio}"
+        # the warp-level kernel reads the table of half-unit integers: a few rows of A through both of its front ends
+        bd.set_gemm_impl(bd.GEMM_WARP)
+        qx11 = bd.quantize_act(x[:11])
+        Yref11, T11 = oracle.gemm(oracle.dequantize(*oracle_quantize(xb[:11], torch.bfloat16)), oracle.dequantize(*ref_w))
+        ok, ratio = gemm_tolerance_ok(bd.gemm(qx11, qw).cpu().numpy(), Yref11, T11)
+        assert ok, f"warp-level kernel, bd_gemm: max err / bound = {ratio}"
+        ok, ratio = gemm_tolerance_ok(bd.linear(x[:11], qw, dtype=torch.float32).cpu().numpy(), Yref11, T11)
+        assert ok, f"warp-level kernel, bd_linear: max err / bound = {ratio}"
         bd.set_gemm_impl(bd.GEMM_AUTO)
         Y = bd.linear(x, bd.quantize_weights(w, bd.SELECT_TWO_STAGE), dtype=torch.float32).cpu().numpy()
         ref_w2 = oracle_quantize(wb, torch.bfloat16)
@@ -116,6 +124,9 @@ def test_random_formatbooks(seed):
             bd.set_gemm_impl(impl)
             ok, ratio = gemm_tolerance_ok(bd.linear(x, Wq, dtype=torch.float32).cpu().numpy(), Yref, T)
             assert ok, f"impl {impl}: max err / bound = {ratio}"
+        bd.set_gemm_impl(bd.GEMM_WARP)
+        ok, ratio = gemm_tolerance_ok(bd.linear(x[:7], Wq, dtype=torch.float32).cpu().numpy(), Yref[:7], T[:7])
+        assert ok, f"warp-level kernel: max err / bound = {ratio}"
     finally:
         bd.set_gemm_impl(bd.GEMM_AUTO)
         bd.set_formatbook(None)
