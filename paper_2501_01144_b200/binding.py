@@ -233,8 +233,11 @@ def _ydtype(dtype):
 
 
 def _ws(workspace, need, device):
-    if workspace is None and need:
-        workspace = torch.empty(need, dtype=torch.uint8, device=device)
+    """`need` may be a callable: the size query is skipped when the caller brings a workspace."""
+    if workspace is None:
+        need = need() if callable(need) else need
+        if need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=device)
     ptr = ctypes.c_void_p(workspace.data_ptr() if workspace is not None else 0)
     return workspace, ptr, (workspace.numel() if workspace is not None else 0)
 
@@ -243,7 +246,7 @@ def gemm(A, B, out=None, dtype=torch.float32, workspace=None, stream=None):
     """Y [M, N] = dq(A) dq(B)^T (Sec. 3.3, Fig. 6)."""
     if out is None:
         out = torch.empty(A.rows, B.rows, dtype=dtype, device=A.codes.device)
-    workspace, wptr, wbytes = _ws(workspace, gemm_workspace_size(A.rows, B.rows, A.K), A.codes.device)
+    workspace, wptr, wbytes = _ws(workspace, lambda: gemm_workspace_size(A.rows, B.rows, A.K), A.codes.device)
     ca, cb = A.c_struct(), B.c_struct()
     _check(load().bd_gemm(ctypes.byref(ca), ctypes.byref(cb), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
                           out.stride(0), wptr, wbytes, _stream(stream)))
@@ -276,7 +279,7 @@ def linear(X, Wq, out=None, dtype=torch.bfloat16, workspace=None, stream=None):
     M, K = X.shape
     if out is None:
         out = torch.empty(M, Wq.rows, dtype=dtype, device=X.device)
-    workspace, wptr, wbytes = _ws(workspace, linear_workspace_size(M, Wq.rows, K), X.device)
+    workspace, wptr, wbytes = _ws(workspace, lambda: linear_workspace_size(M, Wq.rows, K), X.device)
     cw = Wq.c_struct()
     _check(load().bd_linear(ptr, dt, M, K, ld, ctypes.byref(cw), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
                             out.stride(0), wptr, wbytes, _stream(stream)))
