@@ -605,6 +605,18 @@ def run_gpu(args, rank, world, local_rank):
         e1.record()
         torch.cuda.synchronize()
         attend_us = e0.elapsed_time(e1) / 10 * 1e3
+        o32 = torch.empty(kvh, grp, hd, dtype=torch.bfloat16, device=dev)
+        for _ in range(3):
+            bd.kvcache_attention(caches, q_rows, 1.0 / np.sqrt(hd), out=o32)
+        launches0 = bd.launch_count()
+        bd.kvcache_attention(caches, q_rows, 1.0 / np.sqrt(hd), out=o32)
+        step_launches = bd.launch_count() - launches0
+        e0.record()
+        for _ in range(10):                                   # scores, fp32 softmax and P x V of all heads in one call
+            bd.kvcache_attention(caches, q_rows, 1.0 / np.sqrt(hd), out=o32)
+        e1.record()
+        torch.cuda.synchronize()
+        step_us = e0.elapsed_time(e1) / 10 * 1e3
         new_k = dev_bf16(inputs.to_bf16_bits(rng_kv.standard_normal((1, hd)).astype(np.float32)))
         new_kv = new_k.expand(kvh, 1, hd).contiguous()
         e0.record()
@@ -622,6 +634,7 @@ def run_gpu(args, rank, world, local_rank):
         append_us = e0.elapsed_time(e1) / 5 * 1e3
         cache_bytes = kvh * 2 * n_tok * hd * 0.546875
         kv_cache = {"workload": "8 KV heads x 4113 tokens x head_dim 128, 4 query heads per KV head, one object per KV head, scores and P x V of all heads per call",
+                    "attention_us_per_step": step_us, "attention_launches_per_step": step_launches,
                     "scores_and_pv_us_per_step": attend_us, "launches_per_step": attend_launches, "scores_and_pv_us_per_step_head_by_head": per_head_us,
                     "append_one_token_us_per_step": append_us, "append_one_token_us_per_step_head_by_head": append_per_head_us,
                     "cache_bytes_read_per_step": cache_bytes, "cache_read_gbs": cache_bytes / attend_us / 1e3,

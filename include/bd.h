@@ -268,6 +268,16 @@ bd_status bd_kvcache_scores_batched(const bd_kvcache *c, int64_t n, const bd_qte
 bd_status bd_kvcache_pv_batched(const bd_kvcache *c, int64_t n, const float *P, int64_t q_rows, int64_t ldp,
                                 int64_t stride_p, void *Y, bd_dtype ydtype, int64_t ldy, int64_t stride_y,
                                 void *workspace, size_t workspace_bytes, void *stream);
+/* Attention of one decode step over the cached heads (Sec. 4.1 scope "all", Sec. 3.3): per head i
+ *     S = dq(Q[i]) dq(K_i)^T,  P = softmax(scale * S) row by row in fp32,  O_i = P V_i as in bd_kvcache_pv.
+ * O + i * stride_o is [q, head_dim] with row pitch ldo.  P_out, when not NULL, receives the fp32 probabilities
+ * (head i at P_out + i * stride_p_out, pitch ldp_out >= length; 16-byte aligned pointer and pitches) and is the
+ * buffer the second product reads; with NULL they stay in the workspace.  The calls it is made of are the batched
+ * ones above plus one softmax kernel.  workspace: bd_kvcache_attention_workspace_size bytes, 256-byte aligned. */
+bd_status bd_kvcache_attention_workspace_size(int64_t n, int64_t capacity, int64_t head_dim, int64_t q_rows, size_t *bytes);
+bd_status bd_kvcache_attention(const bd_kvcache *c, int64_t n, const bd_qtensor *Q, float scale, void *O, bd_dtype odtype,
+                               int64_t ldo, int64_t stride_o, float *P_out, int64_t ldp_out, int64_t stride_p_out,
+                               void *workspace, size_t workspace_bytes, void *stream);
 
 /* Full-path attention in one kernel (Sec. 4.1, scope "all": Q K^T and score x V are quantised
  * like the linear layers; Sec. 3.3: softmax stays in high precision; appendix "Quantization

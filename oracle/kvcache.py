@@ -69,6 +69,15 @@ class KVCache:
         """S = dq(Q) dq(K)^T for a quantised query operand [q, head_dim]; returns (S, T)."""
         return gemm(dequantize(*q_canonical), dequantize(*self.keys()))
 
+    def attention(self, q_canonical, scale):
+        """One decode step (Sec. 4.1 scope "all", Sec. 3.3): S = dq(Q) dq(K)^T, P = softmax(scale * S) in fp64 stored as
+        fp32, O = P V as in pv().  Returns (O, T, P32)."""
+        S, _ = self.scores(q_canonical)
+        z = np.exp(scale * S - (scale * S).max(axis=-1, keepdims=True))
+        P32 = (z / z.sum(axis=-1, keepdims=True)).astype(np.float32)
+        O, T = self.pv(P32)
+        return O, T, P32
+
     def pv(self, P):
         """O = P V with P [q, length] fp32: the part over full chunks is quantised along the keys (two-stage rule)
         and multiplied with the 4-bit values; the part over the recent tokens stays in high precision (fp64 here).

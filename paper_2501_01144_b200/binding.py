@@ -87,6 +87,8 @@ def load():
     lib.bd_kvcache_pv.argtypes = [kp, vp, i64, i64, vp, ci, i64, vp, sz, vp]
     lib.bd_kvcache_append_batched.argtypes = [kp, i64, vp, vp, i64, i64, i64, i64, i64, vp]
     lib.bd_kvcache_batched_workspace_size.argtypes = [i64, i64, i64, i64, szp]
+    lib.bd_kvcache_attention_workspace_size.argtypes = [i64, i64, i64, i64, szp]
+    lib.bd_kvcache_attention.argtypes = [kp, i64, qp, ctypes.c_float, vp, ci, i64, i64, vp, i64, i64, vp, sz, vp]
     lib.bd_kvcache_scores_batched.argtypes = [kp, i64, qp, vp, ci, i64, i64, vp, sz, vp]
     lib.bd_kvcache_pv_batched.argtypes = [kp, i64, vp, i64, i64, i64, vp, ci, i64, i64, vp, sz, vp]
     lib.bd_attention.argtypes = [qp, qp, qp, i64, i64, ctypes.c_float, vp, ci, i64, i64, ctypes.POINTER(_CAttentionDump), vp]
@@ -494,6 +496,24 @@ def kvcache_pv_batched(caches, P, out=None, dtype=torch.float32, stream=None):
     _check(load().bd_kvcache_pv_batched(arr, n, ctypes.c_void_p(P.data_ptr()), P.shape[1], P.stride(1), P.stride(0),
                                         ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype), out.stride(1), out.stride(0), wptr, wbytes,
                                         _stream(stream)))
+    return out
+
+
+def kvcache_attention(caches, Qs, scale, out=None, dtype=torch.float32, probs=None, stream=None):
+    """O [n, q, head_dim] of one decode step over n cached heads: scores, fp32 softmax of scale * S, P V.  `probs`
+    (fp32 [n, q, pitch >= length], pitch a multiple of 4) receives the probabilities when given."""
+    n, c0, q = len(caches), caches[0], Qs[0].rows
+    if out is None:
+        out = torch.empty(n, q, c0.head_dim, dtype=dtype, device=c0.k.codes.device)
+    arr = (_CKVCache * n)(*[c._c for c in caches])
+    b = ctypes.c_size_t()
+    _check(load().bd_kvcache_attention_workspace_size(n, c0.capacity, c0.head_dim, q, ctypes.byref(b)))
+    if c0._ws is None or c0._ws.numel() < b.value:
+        c0._ws = torch.empty(max(b.value, 256), dtype=torch.uint8, device=c0.k.codes.device)
+    cq = (_CQTensor * n)(*[x.c_struct() for x in Qs])
+    pp, ldp, sp = (ctypes.c_void_p(probs.data_ptr()), probs.stride(1), probs.stride(0)) if probs is not None else (None, 0, 0)
+    _check(load().bd_kvcache_attention(arr, n, cq, ctypes.c_float(scale), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype), out.stride(1),
+                                       out.stride(0), pp, ldp, sp, ctypes.c_void_p(c0._ws.data_ptr()), c0._ws.numel(), _stream(stream)))
     return out
 
 

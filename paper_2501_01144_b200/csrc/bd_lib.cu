@@ -1060,6 +1060,49 @@ bd_status bd_kvcache_pv_batched(const bd_kvcache *c, int64_t n, const float *P, 
     return launch_result();
 }
 
+// ---- a decode step's attention over the cached heads: scores, softmax in high precision, P x V ----
+bd_status bd_kvcache_attention_workspace_size(int64_t n, int64_t capacity, int64_t head_dim, int64_t q_rows, size_t *bytes) {
+    size_t kv;
+    bd_status s = bd_kvcache_batched_workspace_size(n, capacity, head_dim, q_rows, &kv);
+    if (s) return s;
+    *bytes = align256(kv) + align256((size_t)n * (size_t)q_rows * (size_t)capacity * sizeof(float));   // + the scores / probabilities
+    return BD_OK;
+}
+
+bd_status bd_kvcache_attention(const bd_kvcache *c, int64_t n, const bd_qtensor *Q, float scale, void *O, bd_dtype odtype, int64_t ldo,
+                               int64_t stride_o, float *P_out, int64_t ldp_out, int64_t stride_p_out, void *workspace,
+                               size_t workspace_bytes, void *stream) {
+    bd_status s = check_kvcache_batch(c, n);
+    if (s) return s;
+    if (!Q || !O) return BD_ERR_INVALID_ARG;
+    const int64_t q_rows = Q[0].rows, len = c[0].length, cap = c[0].capacity, d = c[0].head_dim;
+    if (q_rows <= 0 || len == 0) return BD_ERR_SHAPE;
+    size_t need, kv;
+    bd_kvcache_attention_workspace_size(n, cap, d, q_rows, &need);
+    bd_kvcache_batched_workspace_size(n, cap, d, q_rows, &kv);
+    if (!workspace || workspace_bytes < need) return BD_ERR_WORKSPACE;
+    if ((uintptr_t)workspace & 255u) return BD_ERR_ALIGN;
+    // the probabilities live in the caller's buffer when one is given (then it is also an output), else in the workspace
+    float *P = P_out ? P_out : (float *)((char *)workspace + align256(kv));
+    const int64_t ldp = P_out ? ldp_out : cap, stride_p = P_out ? stride_p_out : q_rows * cap;
+    if (P_out && (ldp < len || (n > 1 && stride_p < q_rows * ldp))) return BD_ERR_SHAPE;
+    if (P_out && (!aligned16(P_out) || (ldp * 4) % 16 || (stride_p * 4) % 16)) return BD_ERR_ALIGN;
+    s = bd_kvcache_scores_batched(c, n, Q, P, BD_F32, ldp, stride_p, workspace, kv, stream);
+    if (s) return s;
+    if (stride_p == q_rows * ldp) {
+        kv_softmax_rows_kernel<<<(unsigned)(n * q_rows), 256, 0, (cudaStream_t)stream>>>(P, ldp, len, scale);
+        s = launch_result(1);
+        if (s) return s;
+    } else {
+        for (int64_t i = 0; i < n; i++) {
+            kv_softmax_rows_kernel<<<(unsigned)q_rows, 256, 0, (cudaStream_t)stream>>>(P + i * stride_p, ldp, len, scale);
+            s = launch_result(1);
+            if (s) return s;
+        }
+    }
+    return bd_kvcache_pv_batched(c, n, P, q_rows, ldp, stride_p, O, odtype, ldo, stride_o, workspace, kv, stream);
+}
+
 // ---- fused full-path attention ----
 bd_status bd_attention(const bd_qtensor *Q, const bd_qtensor *K, const bd_qtensor *V, int64_t heads, int64_t group, float scale,
                        void *O, bd_dtype odtype, int64_t ldo, int64_t stride_o, const bd_attention_dump *dump, void *stream) {

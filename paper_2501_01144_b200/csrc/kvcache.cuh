@@ -150,4 +150,36 @@ __global__ void kv_pv_finish_kernel(const float *__restrict__ part, int64_t ld_p
     else ((float *)Y)[q * ldy + c] = y;
 }
 
+// Softmax between the two products of a decode step, in high precision (Sec. 3.3): row r of S [rows, length]
+// (fp32, pitch ld) becomes exp(scale * (s - max)) / sum in place, through exp2 of the scores in units of log2 e as
+// in the prefill kernel.  One CTA per row; three sweeps over the row (maximum, sum, store), which for the few
+// rows of a decode step sit in L1/L2.  Columns from `length` to the pitch are left alone.
+__global__ void __launch_bounds__(256) kv_softmax_rows_kernel(float *__restrict__ S, int64_t ld, int64_t length, float scale) {
+    __shared__ float red[8];
+    float *row = S + (int64_t)blockIdx.x * ld;
+    const float sl2 = scale * 1.4426950408889634f;
+    const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    auto block_reduce = [&](float v, bool take_max) {
+#pragma unroll
+        for (int d = 16; d; d >>= 1) {
+            const float o = __shfl_xor_sync(0xffffffffu, v, d);
+            v = take_max ? fmaxf(v, o) : v + o;
+        }
+        __syncthreads();                                          // the previous reduction's readers are done
+        if (lane == 0) red[warp] = v;
+        __syncthreads();
+        float r = red[0];
+        for (int w = 1; w < 8; w++) r = take_max ? fmaxf(r, red[w]) : r + red[w];     // fixed order
+        return r;
+    };
+    float m = -INFINITY;
+    for (int64_t k = threadIdx.x; k < length; k += blockDim.x) m = fmaxf(m, row[k] * sl2);
+    m = block_reduce(m, true);
+    float l = 0.0f;
+    for (int64_t k = threadIdx.x; k < length; k += blockDim.x) l += exp2f(row[k] * sl2 - m);
+    l = block_reduce(l, false);
+    const float inv = 1.0f / l;
+    for (int64_t k = threadIdx.x; k < length; k += blockDim.x) row[k] = exp2f(row[k] * sl2 - m) * inv;
+}
+
 }  // namespace bd

@@ -189,3 +189,45 @@ def test_batched_appends_leave_every_head_in_the_oracle_state(kind):
         pos += t
     assert pos == total
     bd.poll_status()
+
+
+@pytest.mark.parametrize("n,q_rows,heads,d", [(19, 4, 2, 128), (77, 1, 4, 64), (1000, 8, 3, 128), (4127, 4, 8, 128), (640, 12, 2, 128)])
+def test_decode_step_attention_link_by_link(n, q_rows, heads, d):
+    # scores -> fp32 softmax -> P V in one call.  The probabilities come back through the optional output: they are
+    # held against the oracle's fp64 softmax of its own scores, and the result against the oracle's P V of the
+    # LIBRARY's probabilities (a probability that differs in its last bit may round to another code, which is a
+    # different, equally valid, input to the second product); the call without the output buffer gives the same result
+    cap, kind, scale = 4160, torch.bfloat16, 1.0 / np.sqrt(d)
+    caches, refs, Qs, Qrefs = [], [], [], []
+    rng = np.random.default_rng(n + q_rows)
+    for h in range(heads):
+        k, v = _rows(n, d, kind, seed=n + 11 * h)
+        c, r = bd.KVCache(cap, d, dtype=kind), OracleCache(d)
+        c.append(to_device(k, kind), to_device(v, kind))
+        r.append(k, v)
+        caches.append(c)
+        refs.append(r)
+        qb = inputs.to_bf16_bits(rng.standard_normal((q_rows, d)).astype(np.float32))
+        Qs.append(bd.quantize_act(to_device(qb, torch.bfloat16)))
+        Qrefs.append(oracle.quantize(qb, dtype=oracle.BF16))
+    pitch = (n + 3) // 4 * 4
+    probs_all = torch.full((heads, q_rows, pitch + 4), -7.0, device="cuda")
+    probs = probs_all[:, :, :pitch]
+    O = bd.kvcache_attention(caches, Qs, scale, probs=probs).cpu().numpy()
+    assert (probs_all[:, :, pitch:] == -7.0).all()
+    P = probs[:, :, :n].cpu().numpy()
+    for h in range(heads):
+        _, _, Pref = refs[h].attention(Qrefs[h], scale)
+        assert np.abs(P[h].astype(np.float64) - Pref.astype(np.float64)).max() <= 2e-6, f"head {h}: probabilities"
+        assert np.abs(P[h].astype(np.float64).sum(-1) - 1.0).max() <= 1e-5
+        Oref, To = refs[h].pv(P[h])
+        ok, ratio = gemm_tolerance_ok(O[h], Oref, To)
+        assert ok, f"head {h}: P V of the library's probabilities: max err / bound = {ratio}"
+    O2 = bd.kvcache_attention(caches, Qs, scale).cpu().numpy()
+    for h in range(heads):
+        Oref, To = refs[h].pv(P[h])
+        ok, ratio = gemm_tolerance_ok(O2[h], Oref, To)
+        assert ok, f"head {h}: without the probabilities' buffer: max err / bound = {ratio}"
+    O16 = bd.kvcache_attention(caches, Qs, scale, dtype=torch.bfloat16)
+    assert torch.equal(O16.cpu(), torch.from_numpy(O2).to(torch.bfloat16))
+    bd.poll_status()

@@ -82,3 +82,31 @@ def test_fewer_tokens_than_a_block_is_the_exact_product():
     O, _ = c.pv(P)
     assert np.allclose(O, P.astype(np.float64) @ inputs.bf16_bits_to_f32(v).astype(np.float64), rtol=1e-14, atol=0)
     assert len(c.chunks) == 0
+
+
+def test_attention_special_cases():
+    # one cached token: its probability is 1 and it is still in high precision, so the result is that value row itself
+    d = 64
+    rng = np.random.default_rng(3)
+    k, v = rng.standard_normal((40, d)).astype(np.float32), rng.standard_normal((40, d)).astype(np.float32)
+    q = oracle.quantize(rng.standard_normal((3, d)).astype(np.float32))
+    c = KVCache(d, dtype=oracle.F32)
+    c.append(k[:1], v[:1])
+    O, _, P = c.attention(q, 0.3)
+    assert np.array_equal(P, np.ones((3, 1), np.float32)) and np.array_equal(O, np.repeat(v[:1].astype(np.float64), 3, 0))
+    # a query that is a large multiple of one key: the softmax is one-hot up to rounding, the result is that token's
+    # stored value (a full chunk, so the dequantised 4-bit row) and the rows of P are distributions
+    c = KVCache(d, dtype=oracle.F32)
+    c.append(k[:32], v[:32])
+    j = 7
+    q = oracle.quantize((64.0 * k[j:j + 1]).astype(np.float32))
+    O, _, P = c.attention(q, 1.0)
+    assert P.argmax() == j and P[0, j] > 1.0 - 1e-6 and abs(P.sum() - 1.0) < 1e-6
+    vq = oracle.dequantize(*c.values_quantised())                 # [d, 32]
+    assert np.allclose(O[0], vq[:, j], rtol=0, atol=1e-5 * np.abs(vq).max())
+    # scale 0: uniform probabilities over 40 tokens = the plain pv of a constant row
+    c.append(k[32:], v[32:])
+    O, _, P = c.attention(q, 0.0)
+    assert np.array_equal(P, np.full((1, 40), np.float32(1.0 / 40)))
+    O2, _ = c.pv(np.full((1, 40), 1.0 / 40, np.float32))
+    assert np.array_equal(O, O2)
