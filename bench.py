@@ -617,6 +617,21 @@ def run_gpu(args, rank, world, local_rank):
         e1.record()
         torch.cuda.synchronize()
         step_us = e0.elapsed_time(e1) / 10 * 1e3
+        # the same call replayed from a CUDA graph: the six launches without the host's share
+        gstream = torch.cuda.Stream(device=dev)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(gstream):
+            with torch.cuda.graph(graph, stream=gstream):
+                bd.kvcache_attention(caches, q_rows, 1.0 / np.sqrt(hd), out=o32)
+        for _ in range(3):
+            graph.replay()
+        e0.record()
+        for _ in range(20):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        step_graph_us = e0.elapsed_time(e1) / 20 * 1e3
+        del graph
         new_k = dev_bf16(inputs.to_bf16_bits(rng_kv.standard_normal((1, hd)).astype(np.float32)))
         new_kv = new_k.expand(kvh, 1, hd).contiguous()
         e0.record()
@@ -634,7 +649,7 @@ def run_gpu(args, rank, world, local_rank):
         append_us = e0.elapsed_time(e1) / 5 * 1e3
         cache_bytes = kvh * 2 * n_tok * hd * 0.546875
         kv_cache = {"workload": "8 KV heads x 4113 tokens x head_dim 128, 4 query heads per KV head, one object per KV head, scores and P x V of all heads per call",
-                    "attention_us_per_step": step_us, "attention_launches_per_step": step_launches,
+                    "attention_us_per_step": step_us, "attention_launches_per_step": step_launches, "attention_us_per_step_graph_replay": step_graph_us,
                     "scores_and_pv_us_per_step": attend_us, "launches_per_step": attend_launches, "scores_and_pv_us_per_step_head_by_head": per_head_us,
                     "append_one_token_us_per_step": append_us, "append_one_token_us_per_step_head_by_head": append_per_head_us,
                     "cache_bytes_read_per_step": cache_bytes, "cache_read_gbs": cache_bytes / attend_us / 1e3,
