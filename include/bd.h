@@ -294,14 +294,18 @@ bd_status bd_kvcache_attention(const bd_kvcache *c, int64_t n, const bd_qtensor 
  * the blocks of P must be quantised from the final probabilities.  With `dump` (for checking;
  * any member may be NULL) the kernel also writes S and P as fp32 [heads][Sq][Sk] and the
  * canonical codes [heads][Sq][Sk/2], ids and scales [heads][Sq][Sk/32] of the quantised P.
+ * With a workspace (bd_attention_workspace_size bytes, 256-byte aligned; NULL: none) the K and V operands of
+ * the launch's KV heads are first expanded to bf16 there, once, and the kernel copies its key tiles from that
+ * instead of expanding the codes again for every tile of 128 queries; the results are the same bit for bit.
  * Accuracy: as the tensor-core product (fp32 accumulation of exact products). */
 typedef struct {
     float *S, *P;
     uint8_t *codes, *ids, *scales;
 } bd_attention_dump;
+bd_status bd_attention_workspace_size(int64_t heads, int64_t group, int64_t sk, int64_t head_dim, size_t *bytes);
 bd_status bd_attention(const bd_qtensor *Q, const bd_qtensor *K, const bd_qtensor *V, int64_t heads, int64_t group,
                        float scale, void *O, bd_dtype odtype, int64_t ldo, int64_t stride_o,
-                       const bd_attention_dump *dump, void *stream);
+                       const bd_attention_dump *dump, void *workspace, size_t workspace_bytes, void *stream);
 
 /* bd_linear for callers that can neither allocate device memory nor hand in a
  * workspace (the paper has no counterpart; this is a convenience of the library).

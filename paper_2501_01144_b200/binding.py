@@ -91,7 +91,8 @@ def load():
     lib.bd_kvcache_attention.argtypes = [kp, i64, qp, ctypes.c_float, vp, ci, i64, i64, vp, i64, i64, vp, sz, vp]
     lib.bd_kvcache_scores_batched.argtypes = [kp, i64, qp, vp, ci, i64, i64, vp, sz, vp]
     lib.bd_kvcache_pv_batched.argtypes = [kp, i64, vp, i64, i64, i64, vp, ci, i64, i64, vp, sz, vp]
-    lib.bd_attention.argtypes = [qp, qp, qp, i64, i64, ctypes.c_float, vp, ci, i64, i64, ctypes.POINTER(_CAttentionDump), vp]
+    lib.bd_attention_workspace_size.argtypes = [i64, i64, i64, i64, szp]
+    lib.bd_attention.argtypes = [qp, qp, qp, i64, i64, ctypes.c_float, vp, ci, i64, i64, ctypes.POINTER(_CAttentionDump), vp, sz, vp]
     lib.bd_qtensor_sizes_bs.argtypes = [i64, i64, ci, szp, szp, szp]
     lib.bd_quantize_bs.argtypes = [vp, ci, i64, i64, i64, ci, ci, qp, vp]
     lib.bd_export_canonical_bs.argtypes = [qp, ci, vp, vp, vp, vp]
@@ -369,11 +370,18 @@ def linear_bs(X, Wq, block, out=None, dtype=torch.bfloat16, workspace=None, stre
     return out
 
 
-def attention(Qs, Ks, Vs, group=1, scale=None, out=None, dtype=torch.bfloat16, dump=False, stream=None):
+def attention_workspace_size(heads, group, sk, head_dim):
+    b = ctypes.c_size_t()
+    _check(load().bd_attention_workspace_size(heads, group, sk, head_dim, ctypes.byref(b)))
+    return b.value
+
+
+def attention(Qs, Ks, Vs, group=1, scale=None, out=None, dtype=torch.bfloat16, dump=False, workspace=True, stream=None):
     """Full-path attention in one kernel (Sec. 4.1 scope "all"; Sec. 3.3 softmax in high precision): Qs are `heads`
     operands [Sq, d], Ks heads / group operands [Sk, d], Vs heads / group operands [d, Sk] (quantize_act with
     AXIS_STRIDED).  Returns O [heads, Sq, d]; with dump=True also a dict of S, P (fp32 [heads, Sq, Sk]) and the
-    canonical codes, ids, scales of the quantised P, which the kernel then writes for checking."""
+    canonical codes, ids, scales of the quantised P, which the kernel then writes for checking.  workspace: True = allocate
+    the scratch in which K and V are expanded to bf16 once (faster), False / None = none, or a uint8 CUDA tensor."""
     heads, sq, d, sk = len(Qs), Qs[0].rows, Qs[0].K, Ks[0].rows
     dev = Qs[0].codes.device
     if scale is None:
@@ -390,8 +398,13 @@ def attention(Qs, Ks, Vs, group=1, scale=None, out=None, dtype=torch.bfloat16, d
                  "ids": torch.empty(heads, sq, sk // 32, dtype=torch.uint8, device=dev),
                  "scales": torch.empty(heads, sq, sk // 32, dtype=torch.uint8, device=dev)}
         cd = ctypes.pointer(_CAttentionDump(*[extra[k].data_ptr() for k in ("S", "P", "codes", "ids", "scales")]))
+    if workspace is True:
+        b = ctypes.c_size_t()
+        _check(load().bd_attention_workspace_size(heads, group, sk, d, ctypes.byref(b)))
+        workspace = torch.empty(b.value, dtype=torch.uint8, device=dev)
+    wptr, wbytes = (ctypes.c_void_p(workspace.data_ptr()), workspace.numel()) if isinstance(workspace, torch.Tensor) else (None, 0)
     _check(load().bd_attention(cq, ck, cv, heads, group, ctypes.c_float(scale), ctypes.c_void_p(out.data_ptr()), _ydtype(out.dtype),
-                               out.stride(1), out.stride(0), cd, _stream(stream)))
+                               out.stride(1), out.stride(0), cd, wptr, wbytes, _stream(stream)))
     return (out, extra) if dump else out
 
 

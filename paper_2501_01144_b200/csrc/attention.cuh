@@ -57,6 +57,8 @@ struct Params {
     void *O;                   // [heads][sq][ldo]
     int64_t ldo, stride_o;
     int out_bf16;
+    const uint8_t *k_exp, *v_exp;   // PRE: the KV heads' operands already expanded to bf16 (K [sk][d], V [d][sk]), exp_stride
+    int64_t exp_stride;             // bytes from one KV head of this launch to the next
     float *dump_S, *dump_P;    // optional [heads][sq][sk] fp32 (nullptr: not written)
     uint8_t *dump_codes, *dump_ids, *dump_scales;   // optional canonical form of quantise(P): [heads][sq][sk/2], [..][sk/32]
 };
@@ -125,11 +127,31 @@ __device__ __forceinline__ void expand_block(const RawBlock &raw, const SmemTabl
     for (int i = 0; i < 4; i++) *(uint4 *)(dst + 16 * i) = out[i];
 }
 
+// The K and V operands of a launch's KV heads expanded once to bf16 (exact: 0.5 h 2^e), for the kernel instantiation
+// that copies its key tiles instead of expanding them again for every tile of 128 queries (32 tiles x 4 heads of a
+// group share each KV head at the benchmark's shapes).  blockIdx.y = KV head, blockIdx.z = 0: K, 1: V.
+template <int HD>
+__global__ void __launch_bounds__(256) expand_kv_kernel(const __grid_constant__ Params p, uint8_t *__restrict__ k_exp, uint8_t *__restrict__ v_exp) {
+    __shared__ SmemTables tab;
+    load_tables(tab);
+    const int kvh = blockIdx.y;
+    const bool is_v = blockIdx.z != 0;
+    const int64_t rows = is_v ? HD : p.sk, nb = is_v ? p.sk / kBlock : HD / kBlock;
+    const int64_t task = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (task >= rows * nb) return;
+    const int64_t r = task / nb, b = task % nb;
+    const uint8_t *codes = is_v ? p.v_codes[kvh] : p.k_codes[kvh], *ids = is_v ? p.v_ids[kvh] : p.k_ids[kvh],
+                  *scales = is_v ? p.v_scales[kvh] : p.k_scales[kvh];
+    uint8_t *dst = (is_v ? v_exp : k_exp) + (int64_t)kvh * p.exp_stride + (r * nb + b) * 64;
+    expand_block(fetch_block(codes, ids, scales, rows, nb * 16, nb, r, b), tab, dst);
+}
+
 // Key of accumulator column n (0..7) of score tile j (0..3) inside a block of 32 keys: chosen so that lane t of a quad,
 // which owns columns 2 t and 2 t + 1 of every tile, ends up with the keys 8 t .. 8 t + 7 in order.
 __device__ __forceinline__ int key_of(int j, int n) { return 8 * (n >> 1) + 2 * j + (n & 1); }
 
-template <int HD>
+// PRE: the key and value tiles are copied from the bf16 operands expand_kv_kernel wrote, instead of expanded from codes.
+template <int HD, bool PRE>
 __global__ void __launch_bounds__(kThreads, 2) attention_kernel(const __grid_constant__ Params p) {
     using L = Layout<HD>;
     extern __shared__ __align__(128) uint8_t smem[];
@@ -155,6 +177,27 @@ __global__ void __launch_bounds__(kThreads, 2) attention_kernel(const __grid_con
     // (head_dim 128; half as many key blocks for head_dim 64).
     constexpr int kKTasks = (kKTile * NB + kThreads - 1) / kThreads, kVTasks = (HD * (kKTile / kBlock) + kThreads - 1) / kThreads;
     RawBlock raw_k[kKTasks], raw_v[kVTasks];
+    const uint8_t *k_exp = PRE ? p.k_exp + (int64_t)kvh * p.exp_stride : nullptr, *v_exp = PRE ? p.v_exp + (int64_t)kvh * p.exp_stride : nullptr;
+    const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(smem);
+    auto copy16 = [&](uint32_t dst, const uint8_t *src, bool ok) {
+        if (ok) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+        else asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
+    };
+    // PRE: 64 keys x HD bf16 = 16-byte pieces, HD / 8 per key; keys past sk become zeros
+    auto copy_k_tile = [&](int64_t key0) {
+        for (int c = threadIdx.x; c < kKTile * (HD / 8); c += kThreads) {
+            const int r = c / (HD / 8), piece = c % (HD / 8);
+            copy16(smem_s + L::k + r * L::row_stride + piece * 16, k_exp + ((key0 + r) * HD + piece * 8) * 2, key0 + r < p.sk);
+        }
+    };
+    // PRE: HD channels x 64 keys bf16 = 8 pieces per channel
+    auto copy_v_tile = [&](int64_t key0) {
+        for (int c = threadIdx.x; c < HD * (kKTile / 8); c += kThreads) {
+            const int ch = c / (kKTile / 8), piece = c % (kKTile / 8);
+            copy16(smem_s + L::v + ch * L::v_stride + piece * 16, v_exp + ((int64_t)ch * p.sk + key0 + piece * 8) * 2, key0 + piece * 8 < p.sk);
+        }
+    };
+    auto copies_done = [&]() { asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory"); };
     auto fetch_k_tile = [&](int64_t key0) {
 #pragma unroll
         for (int i = 0; i < kKTasks; i++) {
@@ -207,8 +250,13 @@ __global__ void __launch_bounds__(kThreads, 2) attention_kernel(const __grid_con
     float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.0f, l_hi = 0.0f;
     for (int64_t key0 = 0; key0 < p.sk; key0 += kKTile) {
         __syncthreads();                                          // the previous tile has been used
-        fetch_k_tile(key0);
-        expand_k_tile();
+        if (PRE) {
+            copy_k_tile(key0);
+            copies_done();
+        } else {
+            fetch_k_tile(key0);
+            expand_k_tile();
+        }
         __syncthreads();
 #pragma unroll
         for (int kb = 0; kb < kKTile / kBlock; kb++) {
@@ -253,10 +301,16 @@ __global__ void __launch_bounds__(kThreads, 2) attention_kernel(const __grid_con
     const int64_t dump_row_lo = ((int64_t)head * p.sq + row_lo), dump_row_hi = dump_row_lo + 8;
     for (int64_t key0 = 0; key0 < p.sk; key0 += kKTile) {
         __syncthreads();
-        fetch_k_tile(key0);                                       // (keeping the next tile's blocks in registers through the
-        fetch_v_tile(key0);                                       // products, to hide this latency, costs more in spills)
-        expand_k_tile();
-        expand_v_tile();
+        if (PRE) {
+            copy_k_tile(key0);
+            copy_v_tile(key0);
+            copies_done();
+        } else {
+            fetch_k_tile(key0);                                   // (keeping the next tile's blocks in registers through the
+            fetch_v_tile(key0);                                   // products, to hide this latency, costs more in spills)
+            expand_k_tile();
+            expand_v_tile();
+        }
         __syncthreads();
 #pragma unroll
         for (int kb = 0; kb < kKTile / kBlock; kb++) {

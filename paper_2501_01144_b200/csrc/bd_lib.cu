@@ -1104,8 +1104,17 @@ bd_status bd_kvcache_attention(const bd_kvcache *c, int64_t n, const bd_qtensor 
 }
 
 // ---- fused full-path attention ----
+bd_status bd_attention_workspace_size(int64_t heads, int64_t group, int64_t sk, int64_t head_dim, size_t *bytes) {
+    if (!bytes || heads <= 0 || group <= 0 || heads % group || sk <= 0 || head_dim <= 0) return BD_ERR_INVALID_ARG;
+    // K and V of the KV heads of one launch as bf16
+    const int64_t per_launch = std::min<int64_t>(heads / group, std::max<int64_t>(1, std::min<int64_t>(attn::kMaxKvHeads, attn::kMaxHeads / group)));
+    *bytes = (size_t)2 * (size_t)per_launch * align256((size_t)sk * head_dim * 2);
+    return BD_OK;
+}
+
 bd_status bd_attention(const bd_qtensor *Q, const bd_qtensor *K, const bd_qtensor *V, int64_t heads, int64_t group, float scale,
-                       void *O, bd_dtype odtype, int64_t ldo, int64_t stride_o, const bd_attention_dump *dump, void *stream) {
+                       void *O, bd_dtype odtype, int64_t ldo, int64_t stride_o, const bd_attention_dump *dump, void *workspace,
+                       size_t workspace_bytes, void *stream) {
     if (!Q || !K || !V || !O || heads <= 0 || group <= 0 || heads % group) return BD_ERR_INVALID_ARG;
     if (odtype != BD_F32 && odtype != BD_BF16) return BD_ERR_INVALID_ARG;
     const int64_t kv = heads / group, sq = Q[0].rows, hd = Q[0].K, sk = K[0].rows;
@@ -1128,14 +1137,27 @@ bd_status bd_attention(const bd_qtensor *Q, const bd_qtensor *K, const bd_qtenso
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(attn::attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn::Layout<128>::total) != cudaSuccess ||
-            cudaFuncSetAttribute(attn::attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn::Layout<64>::total) != cudaSuccess)
+        if (cudaFuncSetAttribute(attn::attention_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn::Layout<128>::total) != cudaSuccess ||
+            cudaFuncSetAttribute(attn::attention_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn::Layout<64>::total) != cudaSuccess ||
+            cudaFuncSetAttribute(attn::attention_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn::Layout<128>::total) != cudaSuccess ||
+            cudaFuncSetAttribute(attn::attention_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn::Layout<64>::total) != cudaSuccess)
             return launch_result(0);
         configured[dev] = true;
     }
     // heads per launch: whole KV groups, as many as the argument block holds
     const int64_t groups_per_launch = std::max<int64_t>(1, std::min<int64_t>(attn::kMaxKvHeads, attn::kMaxHeads / group));
     if (group > attn::kMaxHeads) return BD_ERR_UNSUPPORTED;
+    // with a workspace the KV heads' operands are expanded to bf16 once per launch and the kernel copies its key tiles
+    bool pre = false;
+    const size_t exp_bytes = align256((size_t)sk * hd * 2);
+    if (workspace) {
+        size_t need;
+        bd_attention_workspace_size(heads, group, sk, hd, &need);
+        if (workspace_bytes < need) return BD_ERR_WORKSPACE;
+        if ((uintptr_t)workspace & 255u) return BD_ERR_ALIGN;
+        pre = true;
+    }
+    uint8_t *k_exp = (uint8_t *)workspace, *v_exp = k_exp + (size_t)std::min(groups_per_launch, kv) * exp_bytes;
     int kernels = 0;
     for (int64_t g0 = 0; g0 < kv; g0 += groups_per_launch) {
         const int64_t ng = std::min(groups_per_launch, kv - g0), nh = ng * group, h0 = g0 * group;
@@ -1153,8 +1175,19 @@ bd_status bd_attention(const bd_qtensor *Q, const bd_qtensor *K, const bd_qtenso
             p.dump_S = dump->S; p.dump_P = dump->P; p.dump_codes = dump->codes; p.dump_ids = dump->ids; p.dump_scales = dump->scales;
         }
         dim3 grid((unsigned)((sq + attn::kQTile - 1) / attn::kQTile), (unsigned)nh);
-        if (hd == 128) attn::attention_kernel<128><<<grid, attn::kThreads, attn::Layout<128>::total, (cudaStream_t)stream>>>(p);
-        else attn::attention_kernel<64><<<grid, attn::kThreads, attn::Layout<64>::total, (cudaStream_t)stream>>>(p);
+        cudaStream_t st = (cudaStream_t)stream;
+        if (pre) {
+            p.k_exp = k_exp; p.v_exp = v_exp; p.exp_stride = (int64_t)exp_bytes;
+            const dim3 egrid(grid_for(sk * (hd / kBlock), 256), (unsigned)ng, 2);
+            if (hd == 128) attn::expand_kv_kernel<128><<<egrid, 256, 0, st>>>(p, k_exp, v_exp);
+            else attn::expand_kv_kernel<64><<<egrid, 256, 0, st>>>(p, k_exp, v_exp);
+            kernels++;
+            if (hd == 128) attn::attention_kernel<128, true><<<grid, attn::kThreads, attn::Layout<128>::total, st>>>(p);
+            else attn::attention_kernel<64, true><<<grid, attn::kThreads, attn::Layout<64>::total, st>>>(p);
+        } else {
+            if (hd == 128) attn::attention_kernel<128, false><<<grid, attn::kThreads, attn::Layout<128>::total, st>>>(p);
+            else attn::attention_kernel<64, false><<<grid, attn::kThreads, attn::Layout<64>::total, st>>>(p);
+        }
         kernels++;
     }
     return launch_result(kernels);

@@ -65,6 +65,14 @@ def test_fused_attention_link_by_link(heads, kv, sq, sk, d):
     # without the dump and with bf16 output: the same result, rounded
     O16 = bd.attention(Qs, Ks, Vs, group=heads // kv, scale=scale, dtype=torch.bfloat16)
     assert torch.equal(O16, O.to(torch.bfloat16))
+    # without the scratch for the expanded K and V the kernel expands its key tiles itself: the same bits
+    O_plain, dump_plain = bd.attention(Qs, Ks, Vs, group=heads // kv, scale=scale, dtype=torch.float32, dump=True, workspace=None)
+    assert torch.equal(O_plain, O) and all(torch.equal(dump_plain[k], dump[k]) for k in dump)
+    # a caller's scratch with guard bands
+    need = bd.attention_workspace_size(heads, heads // kv, sk, d)
+    raw = torch.full((need + 8192,), 0xA5, dtype=torch.uint8, device="cuda")
+    O_ws = bd.attention(Qs, Ks, Vs, group=heads // kv, scale=scale, dtype=torch.float32, workspace=raw[4096:4096 + need])
+    assert torch.equal(O_ws, O) and bool((raw[:4096] == 0xA5).all()) and bool((raw[4096 + need:] == 0xA5).all())
     bd.poll_status()
 
 
