@@ -344,34 +344,52 @@ __global__ void __launch_bounds__(kThreads, 2) attention_kernel(const __grid_con
                 amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
                 amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
                 const uint32_t eadj = max(amax >> 23, 2u);
-                const Scaler sc(eadj);
-                const uint32_t m5 = sc.q5(amax);
+                // The quantizer's packed arithmetic on this lane's eight elements (one code word of the block): the
+                // number of merged thresholds of the dialect pair above each 5-bit code, as nibbles; range counts by
+                // byte-permute lookup, summed over the quad; indices by nibble-parallel arithmetic (finish_two_stage).
+                float pv8[8];
+                uint32_t eadj_eff = eadj;
+                float amax_f = __uint_as_float(amax);
+#pragma unroll
+                for (int i = 0; i < 8; i++) pv8[i] = pr[h][i];
+                if (eadj < 4u) {                                  // block at the exponent clamp: 2^(131 - eadj) is no fp32
+#pragma unroll
+                    for (int i = 0; i < 8; i++) pv8[i] *= 18446744073709551616.0f;
+                    amax_f *= 18446744073709551616.0f;
+                    eadj_eff = eadj + 64u;
+                }
+                const float q_scale = __uint_as_float((258u - eadj_eff) << 23);      // 2^(2 - e), e = eadj - 129
+                const uint32_t m5 = __float_as_uint(__fmaf_rz(amax_f, q_scale, 8388608.0f)) & 63u;
                 const uint32_t pair = min(7u, 15u - min(15u, (m5 + 1u) >> 1));
-                const uint32_t even_mask = tab.even_mask[pair], odd_mask = tab.odd_mask[pair];
-                uint32_t q5[8], cnt = 0;                          // even count in the low half, odd count in the high half
+                const uint32_t above = tab.merged_above[pair];
+                uint32_t v = 0;
 #pragma unroll
                 for (int i = 0; i < 8; i++) {
-                    q5[i] = sc.q5(__float_as_uint(pr[h][i]));
-                    cnt += ((even_mask >> q5[i]) & 1u) + (((odd_mask >> q5[i]) & 1u) << 16);
+                    const uint32_t tq = __float_as_uint(__fmaf_rz(pv8[i], q_scale, 8388608.0f));
+                    v = (uint32_t)__popc(__funnelshift_r(above, 0u, tq)) * (1u << (4 * i)) + v;
                 }
+                const uint32_t acc = prmt_b32(0x10010100u, 0x00000010u, v) + prmt_b32(0x10010100u, 0x00000010u, v >> 16);
+                uint32_t cnt = byte_sum(acc & 0x0f0f0f0fu) | byte_sum((acc >> 4) & 0x0f0f0f0fu) << 16;   // even | odd << 16
                 cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
                 cnt += __shfl_xor_sync(0xffffffffu, cnt, 2);
-                const uint32_t id = 2u * pair + ((cnt >> 16) > (cnt & 0xffffu) ? 1u : 0u);    // equal counts: the even member
-                const uint32_t rmask = tab.round_mask[id];
-                const uint64_t lut = (uint64_t)int_lut[2 * id + 1] << 32 | int_lut[2 * id];
-                // value = 0.5 * h * 2^e with e = eadj - 129, exact in bf16
+                const uint32_t odd = (cnt >> 16) > (cnt & 0xffffu) ? 1u : 0u;                  // equal counts: the even member
+                const uint32_t id = 2u * pair + odd;
+                const uint32_t first_step = odd ? 0x11111111u : 0x22222222u, odd_mask = 0u - odd;
+                const uint32_t u = 0xaaaaaaaau - v;
+                const uint32_t b3 = (u >> 3) & 0x11111111u, b1 = (u >> 1) & 0x11111111u, b0 = u & 0x11111111u;
+                const uint32_t f = ((u + first_step) >> 3) & 0x11111111u;
+                const uint32_t top = b3 & (b1 | (b0 & ~odd_mask));
+                const uint32_t codes = u - f - b3 - top;           // index of element i in nibble i (probabilities carry no sign)
+                // values 0.5 h 2^e = h * unit as bf16: the half-unit integers through the dialect's byte table, each
+                // byte under the high byte 0x43 is the bf16 number 128 + h, and (128 + h) * unit - 128 * unit is exact
+                const uint32_t h_lo = prmt_b32(int_lut[2 * id], int_lut[2 * id + 1], codes), h_hi = prmt_b32(int_lut[2 * id], int_lut[2 * id + 1], codes >> 16);
                 const float unit = __uint_as_float((uint32_t)max((int)eadj - 130 + 127, 0) << 23);
-                uint32_t codes = 0;
-                float val[8];
-#pragma unroll
-                for (int i = 0; i < 8; i++) {
-                    const uint32_t idx = __popc(rmask & ((2u << q5[i]) - 1u));
-                    codes |= idx << (4 * i);
-                    val[i] = (float)((lut >> (8 * idx)) & 0xff) * unit;
-                }
+                const __nv_bfloat162 unit2 = __float2bfloat162_rn(unit), off2 = __float2bfloat162_rn(-128.0f * unit);
+                const uint32_t raw4[4] = {prmt_b32(h_lo, 0x43434343u, 0x4140u), prmt_b32(h_lo, 0x43434343u, 0x4342u),
+                                          prmt_b32(h_hi, 0x43434343u, 0x4140u), prmt_b32(h_hi, 0x43434343u, 0x4342u)};
 #pragma unroll
                 for (int i = 0; i < 4; i++) {
-                    const __nv_bfloat162 pk = __floats2bfloat162_rn(val[2 * i], val[2 * i + 1]);
+                    const __nv_bfloat162 pk = __hfma2(*(const __nv_bfloat162 *)&raw4[i], unit2, off2);
                     a_frag[h][i] = *(const uint32_t *)&pk;
                 }
                 const int64_t drow = h ? dump_row_hi : dump_row_lo;
