@@ -211,3 +211,34 @@ def test_graph_replay_and_back_to_back_calls():
         ok, ratio = gemm_tolerance_ok(y.cpu().numpy(), Yref, T)
         assert ok, ratio
     bd.poll_status()
+
+
+def _fuzz_cases():
+    rng = np.random.default_rng(77)
+    return [(int(rng.integers(1, 17)), int(rng.integers(1, 700)), 32 * int(rng.integers(1, 81)), [torch.bfloat16, torch.float32, torch.float16][i % 3])
+            for i in range(24)]
+
+
+@pytest.mark.parametrize("M,N,K,kind", _fuzz_cases())
+def test_random_shapes_against_the_exact_cuda_core_kernel(M, N, K, kind):
+    # every element against the library's CUDA-core product (exact integer block sums, fp64 across blocks), which
+    # shares nothing with this kernel after the weights' codes; guard bands as above
+    rng = np.random.default_rng(M + 31 * N + K)
+    x = (rng.standard_t(3, (M, K)) * np.exp2(rng.integers(-6, 7, (M, 1)))).astype(np.float32)
+    w = (rng.standard_normal((N, K)) * np.exp2(rng.integers(-8, 3, (N, 1)))).astype(np.float32)
+    host, _ = _host(x, kind)
+    xd = to_device(host, kind)
+    Wq = bd.quantize_weights(to_device(inputs.to_bf16_bits(w), torch.bfloat16), bd.SELECT_TWO_STAGE)
+    bd.set_gemm_impl(bd.GEMM_SIMT)
+    Yexact = bd.linear(xd, Wq, dtype=torch.float32)
+    bound = 2e-6 * (bd.dequantize(bd.quantize_act(xd)).abs() @ bd.dequantize(Wq).abs().T) + 2.0 ** -120
+    bd.set_gemm_impl(bd.GEMM_WARP)
+    ws_bytes = bd.linear_workspace_size(M, N, K)
+    raw_ws, ws = _guarded(ws_bytes)
+    raw_y, ybytes = _guarded(M * N * 4)
+    y = ybytes.view(torch.float32).view(M, N)
+    bd.linear(xd, Wq, out=y, workspace=ws)
+    torch.cuda.synchronize()
+    assert _intact(raw_y, M * N * 4) and _intact(raw_ws, ws_bytes), "write outside a buffer"
+    assert bool(((y - Yexact).abs() <= bound).all()), f"{M}x{N}x{K}: max err / bound = {float(((y - Yexact).abs() / bound).max())}"
+    bd.poll_status()
