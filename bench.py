@@ -460,6 +460,54 @@ def run_gpu(args, rank, world, local_rank):
             del wqs
         bd.poll_status()
 
+    # ---- one token through the four linear layers of a LLaMA3-8B block (the benchmark's shapes at M = 1): called one by
+    # one, and the same four calls replayed from a CUDA graph.  Weights of two blocks in rotation (152 MB > L2). ----
+    decode_block = None
+    if rank == 0:
+        blocks = []
+        for seed in (21, 22):
+            blocks.append([bd.quantize_weights(dev_bf16(inputs.weights_normal(N, K, seed=seed + 10 * i)), bd.SELECT_TWO_STAGE)
+                           for i, (_, K, N) in enumerate(LAYERS)])
+        xs1 = [dev_bf16(inputs.act_post_silu(1, K, seed=5)) for _, K, _ in LAYERS]
+        ys1 = [torch.empty(1, N, dtype=torch.bfloat16, device=dev) for _, _, N in LAYERS]
+        wss = [torch.empty(bd.linear_workspace_size(1, N, K), dtype=torch.uint8, device=dev) for _, K, N in LAYERS]
+
+        def one_token(b):
+            for i in range(len(LAYERS)):
+                bd.linear(xs1[i], blocks[b][i], out=ys1[i], workspace=wss[i])
+
+        for i in range(4):
+            one_token(i % 2)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(4_000_000)
+        e0.record()
+        for i in range(20):
+            one_token(i % 2)
+        e1.record()
+        torch.cuda.synchronize()
+        eager_us = e0.elapsed_time(e1) / 20 * 1e3
+        gs = torch.cuda.Stream(device=dev)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(gs):
+            with torch.cuda.graph(graph, stream=gs):
+                one_token(0)
+                one_token(1)
+        for _ in range(3):
+            graph.replay()
+        e0.record()
+        for _ in range(10):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        graph_us = e0.elapsed_time(e1) / 20 * 1e3
+        del graph
+        wbytes = sum(N * K for _, K, N in LAYERS) * 0.546875
+        decode_block = {"workload": "llama3-8b linear layers (q/o, k/v, gate/up, down) at M = 1, one after the other",
+                        "us_per_token": eager_us, "us_per_token_graph_replay": graph_us, "weight_bytes": wbytes,
+                        "floor_us": wbytes / peaks["hbm_gbs"] / 1e3, "frac_of_roofline": wbytes / peaks["hbm_gbs"] / 1e3 / graph_us}
+        del blocks
+        bd.poll_status()
+
     # ---- two chained layers (gate/up then down, M = 2048) with and without the requantising epilogue (Sec. 3.3,
     # last paragraph).  Without: the first layer writes bf16, the second layer's quantizer reads it back.  With: the
     # first product's epilogue writes the DialectFP4 operand and the second product takes it (its operand bytes are
@@ -795,6 +843,7 @@ def run_gpu(args, rank, world, local_rank):
         "cpu_baseline": cpu,
         "per_layer_gflop": {l["name"]: l["flops"] / 1e9 for l in layers},
         "llama2_mlp_m_sweep": sweep,
+        "decode_block": decode_block,
         "chained_layers": chained,
         "block_sizes": block_sizes,
         "kv_cache": kv_cache,
