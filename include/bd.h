@@ -142,7 +142,8 @@ bd_status bd_quantize_act(const void *X, bd_dtype dtype, int64_t M, int64_t K, i
  *                     (K / 32 + 16) * 2^-24 * S.  Blocks whose scale lies below 2^-100 or above
  *                     2^100 may be flushed or overflow in the intermediate product.
  *   BD_GEMM_AUTO      picks BD_GEMM_TCGEN05 except for tiny problems, and BD_GEMM_WARP for at most
- *                     8 rows of A; the chosen implementation's bound applies. */
+ *                     8 rows of A (at most 16 against up to 2^25 elements of B); the chosen
+ *                     implementation's bound applies. */
 bd_status bd_gemm_workspace_size(int64_t M, int64_t N, int64_t K, size_t *bytes);
 bd_status bd_gemm(const bd_qtensor *A, const bd_qtensor *B, void *Y, bd_dtype ydtype, int64_t ldy,
                   void *workspace, size_t workspace_bytes, void *stream);
@@ -257,7 +258,7 @@ bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int
 /* The same two calls for the n KV heads of a layer in one decode step (n >= 1): c[i] all of one capacity,
  * head_dim, dtype and length; Q[i] [q, head_dim] with the same q; head i reads P + i * stride_p and writes
  * S + i * stride_s / Y + i * stride_y, and takes its t new tokens from Knew + i * stride_k, Vnew + i * stride_v
- * (strides in elements; every head's length advances by t).  With q <= 8 and n <= 64 (and the library's own
+ * (strides in elements; every head's length advances by t).  With q <= 16 and n <= 64 (and the library's own
  * choice of product kernel) the heads share two (scores) or three (P x V) launches; otherwise the calls
  * above run head by head.  workspace: bd_kvcache_batched_workspace_size bytes, 256-byte aligned. */
 bd_status bd_kvcache_append_batched(bd_kvcache *c, int64_t n, const void *Knew, const void *Vnew, int64_t t, int64_t ldk,

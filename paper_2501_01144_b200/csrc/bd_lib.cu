@@ -161,12 +161,15 @@ bd_status check_gemm(const bd_qtensor *A, const bd_qtensor *B, const void *Y, bd
     return BD_OK;
 }
 
-// The warp-level kernel (gemm_warp.cuh) serves up to 16 tokens; the library's own choice takes it for up to 8 (one
-// token group per MMA), where it measured faster than the tensor-core path with its three launches; with two token
-// groups the activation records no longer fit beside the kernel's shared memory in L1 and it measured slower.
+// The warp-level kernel (gemm_warp.cuh) serves up to 16 activation rows.  The library's own choice takes it for up to 8
+// (one token group per MMA), where it measured faster than the tensor-core path with its three launches at every
+// size, and for 9 to 16 rows against at most 2^25 weights, where a call is mostly fixed cost and this kernel has
+// less of it (9.5 against 12.8 us at 4096 x 4096); against more weights the two token groups make it the slower one
+// (22 against 17 us at 4096 x 14336).
 bool use_warp(int64_t M, int64_t N, int64_t K) {
     if (g_gemm_impl == BD_GEMM_WARP) return true;
-    return g_gemm_impl == BD_GEMM_AUTO && wk::supported(M, N, K) && M <= wk::kTokTile && (int64_t)N * K >= (1 << 18);
+    if (g_gemm_impl != BD_GEMM_AUTO || !wk::supported(M, N, K) || (int64_t)N * K < (1 << 18)) return false;
+    return M <= wk::kTokTile || (int64_t)N * K <= (1 << 25);
 }
 unsigned sm_count() {
     static int sms[kMaxDevices] = {};
@@ -936,7 +939,7 @@ bd_status check_kvcache_batch(const bd_kvcache *c, int64_t n) {
     return BD_OK;
 }
 bool kv_batch_fused(int64_t n, int64_t q_rows, int64_t N, int64_t K) {
-    return n <= wk::kMaxBatch && g_gemm_impl != BD_GEMM_SIMT && g_gemm_impl != BD_GEMM_TCGEN05 && q_rows <= wk::kTokTile && wk::supported(q_rows, N, K);
+    return n <= wk::kMaxBatch && g_gemm_impl != BD_GEMM_SIMT && g_gemm_impl != BD_GEMM_TCGEN05 && wk::supported(q_rows, N, K);
 }
 }  // namespace
 
@@ -999,7 +1002,7 @@ bd_status bd_kvcache_scores_batched(const bd_kvcache *c, int64_t n, const bd_qte
         qa.codes[i] = (const uint8_t *)Q[i].codes; qa.ids[i] = (const uint8_t *)Q[i].ids; qa.scales[i] = (const uint8_t *)Q[i].scales;
         kb.codes[i] = (const uint8_t *)c[i].k.codes; kb.ids[i] = (const uint8_t *)c[i].k.ids; kb.scales[i] = (const uint8_t *)c[i].k.scales;
     }
-    const int nt = 1;
+    const int nt = q_rows > wk::kTokTile ? 2 : 1;
     const int64_t rec_stride = (int64_t)align256(wk::record_bytes(hd, nt));
     uint8_t *rec16 = (uint8_t *)workspace;
     float *recs = (float *)(rec16 + (size_t)wk::padded_blocks(hd) * nt * wk::kRecBytes);
@@ -1041,7 +1044,7 @@ bd_status bd_kvcache_pv_batched(const bd_kvcache *c, int64_t n, const float *P, 
     float *part = nullptr;
     const int64_t part_stride = q_rows * d;
     if (n_q) {
-        const int64_t rec_stride = (int64_t)align256(wk::record_bytes(n_q, 1));
+        const int64_t rec_stride = (int64_t)align256(wk::record_bytes(n_q, q_rows > wk::kTokTile ? 2 : 1));
         part = (float *)((char *)workspace + (size_t)n * rec_stride);
         s = launch_warp_records(P, BD_F32, q_rows, n_q, ldp, workspace, st, (int)n, stride_p, rec_stride);
         if (s) return s;
