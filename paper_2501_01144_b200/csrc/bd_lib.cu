@@ -188,7 +188,6 @@ int warp_kernel_warps(int64_t N, int64_t K) {
     const int64_t tiles = N / wk::kRows, units = K / wk::kUnitK;
     const int64_t per_sm = (tiles + sm_count() - 1) / sm_count();
     int64_t w = 32 / per_sm;
-    if (const char *e = getenv("BD_WARP_KERNEL_WARPS")) w = atoi(e);
     return (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(w, units), wk::kMaxWarps));
 }
 // The product kernel over records at `workspace` (rec16, then the factors).  batch: n problems with the operands
