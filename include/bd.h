@@ -259,7 +259,7 @@ bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int
  * head_dim, dtype and length; Q[i] [q, head_dim] with the same q; head i reads P + i * stride_p and writes
  * S + i * stride_s / Y + i * stride_y, and takes its t new tokens from Knew + i * stride_k, Vnew + i * stride_v
  * (strides in elements; every head's length advances by t).  With q <= 16 and n <= 64 (and the library's own
- * choice of product kernel) the heads share two (scores) or three (P x V) launches; otherwise the calls
+ * choice of product kernel) the heads share one (scores) or two (P x V) launches; otherwise the calls
  * above run head by head.  workspace: bd_kvcache_batched_workspace_size bytes, 256-byte aligned. */
 bd_status bd_kvcache_append_batched(bd_kvcache *c, int64_t n, const void *Knew, const void *Vnew, int64_t t, int64_t ldk,
                                     int64_t ldv, int64_t stride_k, int64_t stride_v, void *stream);
@@ -273,8 +273,9 @@ bd_status bd_kvcache_pv_batched(const bd_kvcache *c, int64_t n, const float *P, 
  *     S = dq(Q[i]) dq(K_i)^T,  P = softmax(scale * S) row by row in fp32,  O_i = P V_i as in bd_kvcache_pv.
  * O + i * stride_o is [q, head_dim] with row pitch ldo.  P_out, when not NULL, receives the fp32 probabilities
  * (head i at P_out + i * stride_p_out, pitch ldp_out >= length; 16-byte aligned pointer and pitches) and is the
- * buffer the second product reads; with NULL they stay in the workspace.  The calls it is made of are the batched
- * ones above plus one softmax kernel.  workspace: bd_kvcache_attention_workspace_size bytes, 256-byte aligned. */
+ * buffer the second product reads; with NULL they stay in the workspace.  Three launches where the batched calls
+ * above share theirs (scores; softmax, which also prepares the second product's operand; P x V), else those calls
+ * and a softmax kernel.  workspace: bd_kvcache_attention_workspace_size bytes, 256-byte aligned. */
 bd_status bd_kvcache_attention_workspace_size(int64_t n, int64_t capacity, int64_t head_dim, int64_t q_rows, size_t *bytes);
 bd_status bd_kvcache_attention(const bd_kvcache *c, int64_t n, const bd_qtensor *Q, float scale, void *O, bd_dtype odtype,
                                int64_t ldo, int64_t stride_o, float *P_out, int64_t ldp_out, int64_t stride_p_out,

@@ -241,6 +241,33 @@ bd_status launch_warp_linear(const void *X, bd_dtype xdtype, int64_t M, int64_t 
     if (s) return s;
     return launch_warp_main(M, K, W, Y, ydtype, ldy, workspace, st);
 }
+// The two products of a decode step's attention over n heads (gemm_warp.cuh, MODE 1 and 2): W is the view of head 0's
+// cached operand (shape, pitch), `ops` the heads' operand pointers, x the mode's extras.
+bd_status launch_warp_attn(int mode, int64_t M, int64_t K, const QView &W, void *Y, bd_dtype ydtype, int64_t ldy, int64_t y_stride,
+                           const void *records, int64_t rec_stride, const wk::OperandBatch &ops, const wk::Extra &x, int n, cudaStream_t st) {
+    const int nt = M > wk::kTokTile ? 2 : 1;
+    const uint8_t *rec16 = (const uint8_t *)records;
+    const float *recs = (const float *)(rec16 + (size_t)wk::padded_blocks(K) * nt * wk::kRecBytes);
+    wk::Params p{W.codes, W.ids, W.scales, W.ldc, row_tiles(W.rows), rec16, recs, Y, ldy, W.rows, rec_stride, y_stride, (int)M,
+                 (int)((K + wk::kUnitK - 1) / wk::kUnitK), (int)(K / kBlock % wk::kUnitBlocks), ydtype == BD_BF16};
+    const int64_t tiles = (W.rows + wk::kRows - 1) / wk::kRows;
+    const int warps = warp_kernel_warps(tiles * n * wk::kRows, (K + wk::kUnitK - 1) / wk::kUnitK * wk::kUnitK);
+    const size_t smem = (size_t)warps * (wk::kStages * wk::kStageBytes + nt * 512);
+    using Kernel = void (*)(const wk::Params, const wk::OperandBatch, const wk::Extra);
+    static const Kernel kernels[4] = {wk::gemm_warp_attn_kernel<1, 1>, wk::gemm_warp_attn_kernel<2, 1>, wk::gemm_warp_attn_kernel<1, 2>,
+                                      wk::gemm_warp_attn_kernel<2, 2>};
+    static bool smem_set[kMaxDevices] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < kMaxDevices && !smem_set[dev]) {
+        const int most = wk::kMaxWarps * (wk::kStages * wk::kStageBytes + 2 * 512);
+        for (Kernel k : kernels)
+            if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, most) != cudaSuccess) return cuda_result(cudaGetLastError());
+        smem_set[dev] = true;
+    }
+    launch_serialized(kernels[(mode - 1) * 2 + (nt - 1)], dim3((unsigned)tiles, (unsigned)n), 32u * warps, smem, st, p, ops, x);
+    return launch_result(1);
+}
 // bd_gemm with a few rows of A: records from the quantised A, then the same product kernel.
 bd_status launch_warp_gemm(const QView &A, const QView &B, void *Y, bd_dtype ydtype, int64_t ldy, void *workspace, cudaStream_t st) {
     const int nt = A.rows > wk::kTokTile ? 2 : 1;
@@ -330,16 +357,6 @@ void launch_kv_finish(const float *part, int64_t ld_part, const float *P, int64_
         kv_pv_finish_kernel<DT, __nv_bfloat16, false><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, recent, d, q_rows, (__nv_bfloat16 *)Y, ldy, none, 0, 0, 0);
     else
         kv_pv_finish_kernel<DT, float, false><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, recent, d, q_rows, (float *)Y, ldy, none, 0, 0, 0);
-}
-template <int DT>
-void launch_kv_finish_batched(const float *part, int64_t ld_part, const float *P, int64_t ldp, int64_t n_q, int n_recent, const RecentBatch &recent,
-                              int n, int64_t part_stride, int64_t p_stride, int64_t y_stride, int d, int64_t q_rows, void *Y, bd_dtype ydt,
-                              int64_t ldy, cudaStream_t st) {
-    const dim3 grid(grid_for(q_rows * d, 256), (unsigned)n);
-    if (ydt == BD_BF16)
-        kv_pv_finish_kernel<DT, __nv_bfloat16, true><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, nullptr, d, q_rows, (__nv_bfloat16 *)Y, ldy, recent, part_stride, p_stride, y_stride);
-    else
-        kv_pv_finish_kernel<DT, float, true><<<grid, 256, 0, st>>>(part, ld_part, P, ldp, n_q, n_recent, nullptr, d, q_rows, (float *)Y, ldy, recent, part_stride, p_stride, y_stride);
 }
 #define BD_KV_DISPATCH(dt, fn, ...)                          \
     switch (dt) {                                            \
@@ -937,6 +954,21 @@ bd_status check_kvcache_batch(const bd_kvcache *c, int64_t n) {
     }
     return BD_OK;
 }
+// P x V of n heads with the probabilities' records at `records` (rec_stride bytes per head): the product over the stored
+// chunks and, in its epilogue, the recent tokens in high precision.
+bd_status kv_pv_product(const bd_kvcache *c, int64_t n, const float *P, int64_t q_rows, int64_t ldp, int64_t stride_p, int64_t n_q, int n_recent,
+                        const void *records, int64_t rec_stride, void *Y, bd_dtype ydtype, int64_t ldy, int64_t stride_y, cudaStream_t st) {
+    wk::OperandBatch vb{};
+    wk::Extra x{};
+    for (int64_t i = 0; i < n; i++) {
+        vb.codes[i] = (const uint8_t *)c[i].v.codes; vb.ids[i] = (const uint8_t *)c[i].v.ids; vb.scales[i] = (const uint8_t *)c[i].v.scales;
+        x.recent[i] = c[i].v_recent;
+    }
+    x.P = P; x.ldp = ldp; x.p_stride = stride_p; x.n_q = (int)n_q; x.n_recent = n_recent; x.recent_dt = (int)c[0].dtype;
+    QView vals = view_of(&c[0].v);
+    vals.K = n_q;
+    return launch_warp_attn(2, q_rows, n_q, vals, Y, ydtype, ldy, stride_y, records, rec_stride, vb, x, (int)n, st);
+}
 bool kv_batch_fused(int64_t n, int64_t q_rows, int64_t N, int64_t K) {
     return n <= wk::kMaxBatch && g_gemm_impl != BD_GEMM_SIMT && g_gemm_impl != BD_GEMM_TCGEN05 && wk::supported(q_rows, N, K);
 }
@@ -995,23 +1027,17 @@ bd_status bd_kvcache_scores_batched(const bd_kvcache *c, int64_t n, const bd_qte
         }
         return BD_OK;
     }
-    // one launch for the queries' records, one for the products: grid.y = head
-    wk::OperandBatch qa{}, kb{};
+    // one launch, grid.y = head: the product kernel builds its B fragments from the queries' codes
+    wk::OperandBatch kb{};
+    wk::Extra x{};
     for (int64_t i = 0; i < n; i++) {
-        qa.codes[i] = (const uint8_t *)Q[i].codes; qa.ids[i] = (const uint8_t *)Q[i].ids; qa.scales[i] = (const uint8_t *)Q[i].scales;
+        x.a_codes[i] = (const uint8_t *)Q[i].codes; x.a_ids[i] = (const uint8_t *)Q[i].ids; x.a_scales[i] = (const uint8_t *)Q[i].scales;
         kb.codes[i] = (const uint8_t *)c[i].k.codes; kb.ids[i] = (const uint8_t *)c[i].k.ids; kb.scales[i] = (const uint8_t *)c[i].k.scales;
     }
-    const int nt = q_rows > wk::kTokTile ? 2 : 1;
-    const int64_t rec_stride = (int64_t)align256(wk::record_bytes(hd, nt));
-    uint8_t *rec16 = (uint8_t *)workspace;
-    float *recs = (float *)(rec16 + (size_t)wk::padded_blocks(hd) * nt * wk::kRecBytes);
-    launch_serialized(wk::records_from_qtensor_kernel<true>, dim3(grid_for(wk::padded_blocks(hd) * wk::kTokTile * nt, 128), (unsigned)n), 128, 0, st,
-                      view_of(&Q[0]), nt, rec16, recs, qa, rec_stride);
-    s = launch_result(1);
-    if (s) return s;
+    x.a_ldc = hd / 2;
     QView keys = view_of(&c[0].k);
     keys.rows = len;
-    return launch_warp_main(q_rows, hd, keys, S, sdtype, lds, workspace, st, &kb, (int)n, rec_stride, stride_s);
+    return launch_warp_attn(1, q_rows, hd, keys, S, sdtype, lds, stride_s, workspace, 0, kb, x, (int)n, st);
 }
 
 bd_status bd_kvcache_pv_batched(const bd_kvcache *c, int64_t n, const float *P, int64_t q_rows, int64_t ldp, int64_t stride_p, void *Y,
@@ -1038,28 +1064,14 @@ bd_status bd_kvcache_pv_batched(const bd_kvcache *c, int64_t n, const float *P, 
         }
         return BD_OK;
     }
-    // records of all heads' probabilities, the products over the stored chunks (fp32, in the workspace), then the
-    // recent tokens in high precision and the result: three launches, grid.y = head
-    float *part = nullptr;
-    const int64_t part_stride = q_rows * d;
+    // records of all heads' probabilities over the stored chunks, then one product kernel whose epilogue adds the
+    // recent tokens in high precision and writes the result: two launches, grid.y = head
+    const int64_t rec_stride = n_q ? (int64_t)align256(wk::record_bytes(n_q, q_rows > wk::kTokTile ? 2 : 1)) : 0;
     if (n_q) {
-        const int64_t rec_stride = (int64_t)align256(wk::record_bytes(n_q, q_rows > wk::kTokTile ? 2 : 1));
-        part = (float *)((char *)workspace + (size_t)n * rec_stride);
         s = launch_warp_records(P, BD_F32, q_rows, n_q, ldp, workspace, st, (int)n, stride_p, rec_stride);
         if (s) return s;
-        wk::OperandBatch vb{};
-        for (int64_t i = 0; i < n; i++) {
-            vb.codes[i] = (const uint8_t *)c[i].v.codes; vb.ids[i] = (const uint8_t *)c[i].v.ids; vb.scales[i] = (const uint8_t *)c[i].v.scales;
-        }
-        QView vals = view_of(&c[0].v);
-        vals.K = n_q;
-        s = launch_warp_main(q_rows, n_q, vals, part, BD_F32, d, workspace, st, &vb, (int)n, rec_stride, part_stride);
-        if (s) return s;
     }
-    RecentBatch rb{};
-    for (int64_t i = 0; i < n; i++) rb.ptr[i] = c[i].v_recent;
-    BD_KV_DISPATCH(c[0].dtype, launch_kv_finish_batched, part, d, P, ldp, n_q, n_recent, rb, (int)n, part_stride, stride_p, stride_y, (int)d, q_rows, Y, ydtype, ldy, st);
-    return launch_result();
+    return kv_pv_product(c, n, P, q_rows, ldp, stride_p, n_q, n_recent, workspace, rec_stride, Y, ydtype, ldy, stride_y, st);
 }
 
 // ---- a decode step's attention over the cached heads: scores, softmax in high precision, P x V ----
@@ -1091,13 +1103,28 @@ bd_status bd_kvcache_attention(const bd_kvcache *c, int64_t n, const bd_qtensor 
     if (P_out && (!aligned16(P_out) || (ldp * 4) % 16 || (stride_p * 4) % 16)) return BD_ERR_ALIGN;
     s = bd_kvcache_scores_batched(c, n, Q, P, BD_F32, ldp, stride_p, workspace, kv, stream);
     if (s) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t n_q = len / kBlock * kBlock;
+    if (kv_batch_fused(n, q_rows, d, n_q ? n_q : kBlock)) {
+        // the softmax kernel also quantises its rows into the second product's records; that product's epilogue adds
+        // the recent tokens: three launches for the step
+        const int nt = q_rows > wk::kTokTile ? 2 : 1;
+        const int64_t rec_stride = (int64_t)align256(wk::record_bytes(n_q ? n_q : kBlock, nt));
+        uint8_t *rec16 = (uint8_t *)workspace;
+        float *recs = (float *)(rec16 + (size_t)wk::padded_blocks(n_q) * nt * wk::kRecBytes);
+        launch_serialized(kv_softmax_records_kernel, dim3((unsigned)(wk::kTokTile * nt), (unsigned)n), 256, 0, st, P, ldp, stride_p, len, scale,
+                          (int)q_rows, nt, (int)n_q, (int)wk::padded_blocks(n_q), rec16, recs, rec_stride);
+        s = launch_result(1);
+        if (s) return s;
+        return kv_pv_product(c, n, P, q_rows, ldp, stride_p, n_q, (int)(len - n_q), workspace, rec_stride, O, odtype, ldo, stride_o, st);
+    }
     if (stride_p == q_rows * ldp) {
-        kv_softmax_rows_kernel<<<(unsigned)(n * q_rows), 256, 0, (cudaStream_t)stream>>>(P, ldp, len, scale);
+        kv_softmax_rows_kernel<<<(unsigned)(n * q_rows), 256, 0, st>>>(P, ldp, len, scale);
         s = launch_result(1);
         if (s) return s;
     } else {
         for (int64_t i = 0; i < n; i++) {
-            kv_softmax_rows_kernel<<<(unsigned)q_rows, 256, 0, (cudaStream_t)stream>>>(P + i * stride_p, ldp, len, scale);
+            kv_softmax_rows_kernel<<<(unsigned)q_rows, 256, 0, st>>>(P + i * stride_p, ldp, len, scale);
             s = launch_result(1);
             if (s) return s;
         }

@@ -224,11 +224,24 @@ struct Params {
     int M, units, tail_blocks, y_bf16;     // units = ceil(K / 128); tail_blocks = blocks of the last unit if it is short, else 0
 };
 
+// What the decode-step attention adds to a batched launch (blockIdx.y = KV head).
+//   MODE 1 (scores): no records; the B fragments come straight from the quantised queries' codes (a few rows, K = head_dim).
+//   MODE 2 (P x V): after the product over the stored chunks the epilogue adds the recent tokens in high precision,
+//                   sum_k P[q, n_q + k] * V_recent[k, c] in fp32 on the source values (kv_pv_finish_kernel's arithmetic).
+struct Extra {
+    const uint8_t *a_codes[kMaxBatch], *a_ids[kMaxBatch], *a_scales[kMaxBatch];   // MODE 1: the heads' query operands [M, K]
+    int64_t a_ldc;
+    const void *recent[kMaxBatch];         // MODE 2: the heads' high-precision value rows [32, N]
+    const float *P;                        // MODE 2: probabilities, head y at P + y * p_stride, row pitch ldp
+    int64_t ldp, p_stride;
+    int n_q, n_recent, recent_dt;
+};
+
 // Shared memory of a CTA: per warp kStages stages of kStageBytes, then the warps' sums [warps][NT][4][32] floats.
 // RAGGED: the rows do not fill the last tile of 16 or K does not fill the last unit of 128 (guards in the copy and
 // store paths that whole shapes do without).
-template <int NT, bool BATCH, bool RAGGED>
-__global__ void __launch_bounds__(32 * kMaxWarps, 2) gemm_warp_kernel(const __grid_constant__ Params p, const __grid_constant__ OperandBatch batch) {
+template <int NT, bool BATCH, bool RAGGED, int MODE>
+__device__ __forceinline__ void gemm_warp_body(const Params &p, const OperandBatch &batch, const Extra &x) {
     extern __shared__ __align__(16) uint8_t smem[];
     __shared__ uint2 lut[16];
     const int warps = blockDim.x / 32, warp = threadIdx.x / 32, lane = threadIdx.x % 32, g = lane >> 2, t = lane & 3;
@@ -270,14 +283,27 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) gemm_warp_kernel(const __gr
     };
     // this warp's units: warp, warp + warps, ...
     const int n_units = p.units > warp ? (p.units - warp + warps - 1) / warps : 0;
+    // The first copies go out before the wait when a record kernel sits in front: it lets this kernel start only after
+    // everything before it has completed (it waits before it lets its dependents go), so the B operand is final.
+    // MODE 1 has no such kernel in front and its B operand is the key cache, which the kernel just before may have
+    // appended to: there the copies wait too (the scores are one unit of K per warp, so nothing is lost).
+    if (MODE != 1) {
 #pragma unroll
-    for (int s = 0; s < kStages; s++) {
-        if (s < n_units) issue(s);
-        asm volatile("cp.async.commit_group;" ::: "memory");
+        for (int s = 0; s < kStages; s++) {
+            if (s < n_units) issue(s);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
     }
     __syncthreads();                                             // the byte tables
-    asm volatile("griddepcontrol.wait;" ::: "memory");           // the records
+    asm volatile("griddepcontrol.wait;" ::: "memory");           // the records (MODE 1: the queries and the keys)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (MODE == 1) {
+#pragma unroll
+        for (int s = 0; s < kStages; s++) {
+            if (s < n_units) issue(s);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+    }
     float acc[NT][4];
 #pragma unroll
     for (int n = 0; n < NT; n++) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.0f;
@@ -321,8 +347,29 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) gemm_warp_kernel(const __gr
             const float f_hi = __uint_as_float((b < 3 ? sc_hi << (23 - 8 * b) : sc_hi >> 1) & 0x7f800000u);
 #pragma unroll
             for (int n = 0; n < NT; n++) {
-                const uint4 bb = *(const uint4 *)(my_rec + (b * NT + n) * kRecBytes);
-                const float2 fa = *(const float2 *)(my_fac + (b * NT + n) * kTokTile);
+                uint4 bb;
+                float2 fa;
+                if (MODE == 1) {
+                    // lane group g is query row 8 n + g: its code word t of this block, expanded like the weights';
+                    // the columns of this lane's sums are rows 8 n + 2 t, + 1: their block scales, with 2^46 for the
+                    // two subnormal encodings and the half-units (clamped as the records' factors are)
+                    const int blk = (warp + i * warps) * kUnitBlocks + b, row = n * kTokTile + g;
+                    const bool blk_ok = !(p.tail_blocks && warp + i * warps == p.units - 1 && b >= p.tail_blocks);
+                    uint32_t f[4] = {0, 0, 0, 0};
+                    if (row < p.M && blk_ok) {
+                        const uint32_t wq = *(const uint32_t *)(x.a_codes[blockIdx.y] + row * x.a_ldc + blk * 16 + t * 4);
+                        const uint32_t idq = (x.a_ids[blockIdx.y][(blk / 4) * kIdAtomBytes + row * 8 + (blk % 4) / 2] >> (4 * (blk & 1))) & 15u;
+                        word_to_f16(wq, lut[idq].x, lut[idq].y, f);
+                    }
+                    bb = make_uint4(f[0], f[1], f[2], f[3]);
+                    const int c0 = n * kTokTile + 2 * t;
+                    const uint8_t *sq = x.a_scales[blockIdx.y] + (blk / 4) * kScaleAtomBytes + (blk % 4);
+                    fa.x = c0 < p.M && blk_ok ? __uint_as_float(min((uint32_t)sq[c0 * 16] + 46u, 254u) << 23) : 0.0f;
+                    fa.y = c0 + 1 < p.M && blk_ok ? __uint_as_float(min((uint32_t)sq[(c0 + 1) * 16] + 46u, 254u) << 23) : 0.0f;
+                } else {
+                    bb = *(const uint4 *)(my_rec + (b * NT + n) * kRecBytes);
+                    fa = *(const float2 *)(my_fac + (b * NT + n) * kTokTile);
+                }
                 const float zero[4] = {0.0f, 0.0f, 0.0f, 0.0f};
                 float d0[4], d[4];
                 mma_f16(d0, a_lo[0], a_hi[0], a_lo[1], a_hi[1], bb.x, bb.y, zero);
@@ -352,10 +399,33 @@ __global__ void __launch_bounds__(32 * kMaxWarps, 2) gemm_warp_kernel(const __gr
         const int n = tok / kTokTile, tk = tok % kTokTile, src = ((n * 4) + (row / 8) * 2 + (tk & 1)) * 32 + (row % 8) * 4 + tk / 2;
         float y = 0.0f;
         for (int w = 0; w < warps; w++) y += red[w * NT * 128 + src];
+        if (MODE == 2) {                                          // the recent tokens, in fp32 on the source values
+            const float *prow = x.P + (int64_t)blockIdx.y * x.p_stride + (int64_t)tok * x.ldp + x.n_q;
+            const char *rec = (const char *)x.recent[blockIdx.y];
+            float add = 0.0f;
+            for (int k = 0; k < x.n_recent; k++) {
+                const int64_t e = (int64_t)k * p.N + r0 + row;
+                const uint32_t bits = x.recent_dt == BD_F32 ? Loader<BD_F32>::one(rec + e * 4)
+                                    : x.recent_dt == BD_BF16 ? Loader<BD_BF16>::one(rec + e * 2) : Loader<BD_F16>::one(rec + e * 2);
+                add = fmaf(prow[k], __uint_as_float(bits), add);
+            }
+            y += add;
+        }
         const int64_t at = (BATCH ? (int64_t)blockIdx.y * p.y_stride : 0) + (int64_t)tok * p.ldy + r0 + row;
         if (p.y_bf16) ((__nv_bfloat16 *)p.Y)[at] = __float2bfloat16_rn(y);
         else ((float *)p.Y)[at] = y;
     }
+}
+
+template <int NT, bool BATCH, bool RAGGED>
+__global__ void __launch_bounds__(32 * kMaxWarps, 2) gemm_warp_kernel(const __grid_constant__ Params p, const __grid_constant__ OperandBatch batch) {
+    gemm_warp_body<NT, BATCH, RAGGED, 0>(p, batch, Extra{});
+}
+// The decode-step attention's two products (always batched, guards for ragged shapes on).
+template <int NT, int MODE>
+__global__ void __launch_bounds__(32 * kMaxWarps, 2) gemm_warp_attn_kernel(const __grid_constant__ Params p, const __grid_constant__ OperandBatch batch,
+                                                                           const __grid_constant__ Extra x) {
+    gemm_warp_body<NT, true, true, MODE>(p, batch, x);
 }
 
 }  // namespace wk

@@ -12,6 +12,8 @@
 // pitch of the full capacity).  With head_dim <= 128 the key operand has one scale atom along K and the value
 // operand one row tile, so the atom order of both does not depend on the capacity.
 #pragma once
+#include <cuda_fp16.h>
+
 #include "bd_common.cuh"
 #include "quantize.cuh"
 
@@ -180,6 +182,95 @@ __global__ void __launch_bounds__(256) kv_softmax_rows_kernel(float *__restrict_
     l = block_reduce(l, false);
     const float inv = 1.0f / l;
     for (int64_t k = threadIdx.x; k < length; k += blockDim.x) row[k] = exp2f(row[k] * sl2 - m) * inv;
+}
+
+// The same softmax followed by the two-stage quantisation of the row's probabilities over the stored chunks (the first
+// n_q columns) into the warp-level product kernel's records (gemm_warp.cuh: [block][group of 8 rows][row][32 fp16] and
+// a factor per row and block; blocks from n_q / 32 up to `padded_blocks` are zeros).  Grid: (8 * nt row slots, heads);
+// row slots past q_rows only write zero records.  The probabilities are stored (fp32) first and the blocks are
+// quantised from what was stored, so the codes are those of the two-kernel route bit for bit.
+__global__ void __launch_bounds__(256) kv_softmax_records_kernel(float *__restrict__ S, int64_t ld, int64_t s_stride, int64_t length, float scale,
+                                                                 int q_rows, int nt, int n_q, int padded_blocks, uint8_t *__restrict__ rec16,
+                                                                 float *__restrict__ recs, int64_t rec_stride) {
+    __shared__ float red[8];
+    __shared__ SmemTables tab;
+    load_tables(tab);
+    asm volatile("griddepcontrol.wait;" ::: "memory");           // the scores
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int m = blockIdx.x;                                     // row slot
+    rec16 += (int64_t)blockIdx.y * rec_stride;
+    recs = (float *)((uint8_t *)recs + (int64_t)blockIdx.y * rec_stride);
+    const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    float *row = S + (int64_t)blockIdx.y * s_stride + (int64_t)m * ld;
+    if (m < q_rows) {
+        const float sl2 = scale * 1.4426950408889634f;
+        auto block_reduce = [&](float v, bool take_max) {
+#pragma unroll
+            for (int d = 16; d; d >>= 1) {
+                const float o = __shfl_xor_sync(0xffffffffu, v, d);
+                v = take_max ? fmaxf(v, o) : v + o;
+            }
+            __syncthreads();
+            if (lane == 0) red[warp] = v;
+            __syncthreads();
+            float r = red[0];
+            for (int w = 1; w < 8; w++) r = take_max ? fmaxf(r, red[w]) : r + red[w];
+            return r;
+        };
+        float mx = -INFINITY;
+        for (int64_t k = threadIdx.x; k < length; k += blockDim.x) mx = fmaxf(mx, row[k] * sl2);
+        mx = block_reduce(mx, true);
+        float l = 0.0f;
+        for (int64_t k = threadIdx.x; k < length; k += blockDim.x) l += exp2f(row[k] * sl2 - mx);
+        l = block_reduce(l, false);
+        const float inv = 1.0f / l;
+        for (int64_t k = threadIdx.x; k < length; k += blockDim.x) row[k] = exp2f(row[k] * sl2 - mx) * inv;
+        __syncthreads();                                          // the blocks below read what other threads stored
+    }
+    const int nb = n_q / kBlock;
+    for (int b = threadIdx.x; b < padded_blocks; b += blockDim.x) {
+        uint4 out[4];
+#pragma unroll
+        for (int i = 0; i < 4; i++) out[i] = make_uint4(0, 0, 0, 0);
+        float factor = 1.0f;
+        if (m < q_rows && b < nb) {
+            uint32_t bits[32], unused[8];
+            const uint4 *src = (const uint4 *)(row + (int64_t)b * 32);   // plain loads: this kernel wrote the row
+#pragma unroll
+            for (int i = 0; i < 8; i++) {
+                const uint4 u = src[i];
+                bits[4 * i] = u.x; bits[4 * i + 1] = u.y; bits[4 * i + 2] = u.z; bits[4 * i + 3] = u.w;
+            }
+            BlockResult res;
+            bool nonfinite;
+            quantize_two_stage_f32<false>(bits, tab, res, unused, nonfinite);
+            if (nonfinite) atomicOr(&g_status_word, kStatusNonfinite);
+            factor = __uint_as_float(min(res.scale + 22u, 254u) << 23);
+            const uint32_t tlo = c_tables.int_lo[res.id], thi = c_tables.int_hi[res.id];
+#pragma unroll
+            for (int w = 0; w < 4; w++) {
+                uint32_t v[4];
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    uint32_t pair = 0;
+#pragma unroll
+                    for (int j = 0; j < 2; j++) {
+                        const int e = 2 * i + j;
+                        const uint32_t idx = word_index(res.words[w], e);
+                        const uint32_t mag = ((idx < 4 ? tlo : thi) >> (8 * (idx & 3))) & 0xffu;
+                        pair |= ((uint32_t)__half_as_ushort(__int2half_rn((int)mag)) | word_sign(res.words[w], e) << 15) << (16 * j);
+                    }
+                    v[i] = pair;
+                }
+                out[w] = make_uint4(v[0], v[1], v[2], v[3]);
+            }
+        }
+        const size_t slot = (size_t)(b * nt + m / 8) * 8 + m % 8;
+        uint4 *dst = (uint4 *)(rec16 + slot * (kBlock * 2));
+#pragma unroll
+        for (int i = 0; i < 4; i++) dst[i] = out[i];
+        recs[slot] = factor;
+    }
 }
 
 }  // namespace bd
