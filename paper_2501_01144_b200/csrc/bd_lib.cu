@@ -889,6 +889,10 @@ bd_status bd_kvcache_workspace_size(int64_t capacity, int64_t head_dim, int64_t 
     return BD_OK;
 }
 
+namespace {
+bool kv_batch_fused(int64_t n, int64_t q_rows, int64_t N, int64_t K);   // (with the batched calls below)
+}
+
 bd_status bd_kvcache_scores(const bd_kvcache *c, const bd_qtensor *Q, void *S, bd_dtype sdtype, int64_t lds, void *workspace,
                             size_t workspace_bytes, void *stream) {
     bd_status s = check_kvcache(c);
@@ -897,6 +901,8 @@ bd_status bd_kvcache_scores(const bd_kvcache *c, const bd_qtensor *Q, void *S, b
     if (s) return s;
     if (Q->K != c->head_dim || c->length == 0 || lds < c->length) return BD_ERR_SHAPE;
     if (!S || (sdtype != BD_F32 && sdtype != BD_BF16)) return BD_ERR_INVALID_ARG;
+    if (kv_batch_fused(1, Q->rows, c->length, c->head_dim))       // a few query rows: the batched route with one head
+        return bd_kvcache_scores_batched(c, 1, Q, S, sdtype, lds, Q->rows * lds, workspace, workspace_bytes, stream);
     QView keys = view_of(&c->k);
     keys.rows = c->length;                                        // the rows stored so far (one scale atom along K: the
     return gemm_dispatch(view_of(Q), keys, S, sdtype, lds, workspace, workspace_bytes, (cudaStream_t)stream);   // atom order ignores the row count)
@@ -909,6 +915,8 @@ bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int
     if (!P || !Y || q_rows <= 0 || (ydtype != BD_F32 && ydtype != BD_BF16)) return BD_ERR_INVALID_ARG;
     if (c->length == 0 || ldp < c->length || ldy < c->head_dim) return BD_ERR_SHAPE;
     if (c->length >= kBlock && (!aligned16(P) || (ldp * 4) % 16)) return BD_ERR_ALIGN;   // the quantizer reads P in 16-byte pieces
+    if (kv_batch_fused(1, q_rows, c->head_dim, c->length >= kBlock ? c->length / kBlock * kBlock : kBlock))
+        return bd_kvcache_pv_batched(c, 1, P, q_rows, ldp, q_rows * ldp, Y, ydtype, ldy, q_rows * ldy, workspace, workspace_bytes, stream);
     size_t need;
     bd_kvcache_workspace_size(c->capacity, c->head_dim, q_rows, &need);
     if (!workspace || workspace_bytes < need) return BD_ERR_WORKSPACE;
