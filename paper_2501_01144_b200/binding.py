@@ -127,8 +127,9 @@ def _check(status):
 
 
 def _stream(stream=None):
-    s = torch.cuda.current_stream() if stream is None else stream
-    return ctypes.c_void_p(s.cuda_stream)
+    if stream is None:
+        return ctypes.c_void_p(torch._C._cuda_getCurrentRawStream(torch.cuda.current_device()))
+    return ctypes.c_void_p(stream.cuda_stream)
 
 
 def version():
@@ -184,8 +185,15 @@ class QTensor:
         self.ids = torch.empty(i.value, dtype=torch.uint8, device=device)
         self.scales = torch.empty(s.value, dtype=torch.uint8, device=device)
 
+    def __setattr__(self, name, value):
+        object.__setattr__(self, name, value)
+        object.__setattr__(self, "_c", None)                      # a buffer or a shape changed: the descriptor is rebuilt
+
     def c_struct(self):
-        return _CQTensor(self.codes.data_ptr(), self.ids.data_ptr(), self.scales.data_ptr(), self.rows, self.K)
+        """The C descriptor (kept until a member changes: a decode step passes dozens of these per call)."""
+        if self._c is None:
+            object.__setattr__(self, "_c", _CQTensor(self.codes.data_ptr(), self.ids.data_ptr(), self.scales.data_ptr(), self.rows, self.K))
+        return self._c
 
     def nbytes(self):
         return self.codes.numel() + self.ids.numel() + self.scales.numel()
