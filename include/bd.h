@@ -157,7 +157,9 @@ bd_status bd_gemm(const bd_qtensor *A, const bd_qtensor *B, void *Y, bd_dtype yd
  * With a workspace of bd_gemm_batched_workspace_size bytes, results of a group that
  * are contiguous in Y (stride_y == M * ldy) and M a multiple of 128, the b_group
  * products of a group run as one stacked launch; otherwise (any workspace of at
- * least bd_gemm_workspace_size bytes) one launch per product. */
+ * least bd_gemm_workspace_size bytes) one launch per product.  With at most 16 rows
+ * per A operand (where BD_GEMM_WARP serves the call) all products share launches of
+ * up to 64, whatever the strides; no workspace is touched then. */
 bd_status bd_gemm_batched_workspace_size(int64_t M, int64_t N, int64_t K, int64_t b_group, size_t *bytes);
 bd_status bd_gemm_batched(const bd_qtensor *A, const bd_qtensor *B, int64_t batch, int64_t b_group,
                           void *Y, bd_dtype ydtype, int64_t ldy, int64_t stride_y, void *workspace,

@@ -480,6 +480,24 @@ bd_status bd_gemm_batched(const bd_qtensor *A, const bd_qtensor *B, int64_t batc
     bd_gemm_batched_workspace_size(M, N, K, b_group, &stacked_need);
     // Grouped products share their B operand: when the group's results are contiguous in Y and the operands are
     // whole row tiles, the group's A operands are decoded into one stacked matrix and the group is one launch.
+    // A few rows of A per product (decode-shaped attention without the cache object): the warp-level kernel takes the
+    // whole batch through grid.y, 64 products per launch, and expands the A operands' code words itself.
+    if (use_warp(M, N, K) && wk::supported(M, N, K)) {
+        for (int64_t i0 = 0; i0 < batch; i0 += wk::kMaxBatch) {
+            const int count = (int)std::min<int64_t>(wk::kMaxBatch, batch - i0);
+            wk::OperandBatch ops{};
+            wk::Extra x{};
+            for (int h = 0; h < count; h++) {
+                const bd_qtensor &a = A[i0 + h], &b = B[(i0 + h) / b_group];
+                x.a_codes[h] = (const uint8_t *)a.codes; x.a_ids[h] = (const uint8_t *)a.ids; x.a_scales[h] = (const uint8_t *)a.scales;
+                ops.codes[h] = (const uint8_t *)b.codes; ops.ids[h] = (const uint8_t *)b.ids; ops.scales[h] = (const uint8_t *)b.scales;
+            }
+            x.a_ldc = K / 2;
+            bd_status s = launch_warp_attn(1, M, K, view_of(&B[0]), (uint8_t *)Y + i0 * stride_y * ysz, ydtype, ldy, stride_y, nullptr, 0, ops, x, count, st);
+            if (s) return s;
+        }
+        return BD_OK;
+    }
     const bool stack = b_group > 1 && M % kRowTile == 0 && stride_y == M * ldy && use_tc(M * b_group, N, K) &&
                        tc_supported(M * b_group, N, K) && workspace && workspace_bytes >= stacked_need &&
                        !((uintptr_t)workspace & 255u);

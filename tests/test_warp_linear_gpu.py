@@ -242,3 +242,32 @@ def test_random_shapes_against_the_exact_cuda_core_kernel(M, N, K, kind):
     assert _intact(raw_y, M * N * 4) and _intact(raw_ws, ws_bytes), "write outside a buffer"
     assert bool(((y - Yexact).abs() <= bound).all()), f"{M}x{N}x{K}: max err / bound = {float(((y - Yexact).abs() / bound).max())}"
     bd.poll_status()
+
+
+@pytest.mark.parametrize("heads,group,M,N,K", [(8, 4, 4, 4113, 128), (6, 1, 1, 130, 160), (70, 2, 9, 48, 64), (4, 2, 16, 257, 1056)])
+@pytest.mark.parametrize("ydt", [torch.float32, torch.bfloat16])
+def test_batched_products_with_a_few_rows_share_a_launch(heads, group, M, N, K, ydt):
+    # bd_gemm_batched with at most 16 rows of A per product: all products (64 per launch) through grid.y of the
+    # warp-level kernel, which expands the A operands' code words itself; every head against the oracle
+    rng = np.random.default_rng(heads + 31 * M + 977 * N + K)
+    a = inputs.to_bf16_bits((rng.standard_t(4, (heads, M, K)) * np.exp2(rng.integers(-3, 4, (heads, M, 1)))).astype(np.float32))
+    b = inputs.to_bf16_bits(rng.standard_normal((heads // group, N, K)).astype(np.float32))
+    As = [bd.quantize_act(to_device(a[h], torch.bfloat16)) for h in range(heads)]
+    Bs = [bd.quantize_act(to_device(b[g], torch.bfloat16)) for g in range(heads // group)]
+    esz = 4 if ydt == torch.float32 else 2
+    raw_y, ybytes = _guarded(heads * M * N * esz)
+    out = ybytes.view(ydt).view(heads, M, N)
+    ws_bytes = bd.gemm_batched_workspace_size(M, N, K, group)
+    raw_ws, ws = _guarded(max(ws_bytes, 256))
+    bd.set_gemm_impl(bd.GEMM_WARP)                                # (the library's own choice leaves tiny products to the CUDA-core kernel)
+    before = bd.launch_count()
+    bd.gemm_batched(As, Bs, b_group=group, out=out, workspace=ws)
+    torch.cuda.synchronize()
+    assert bd.launch_count() - before == (heads + 63) // 64
+    assert _intact(raw_y, heads * M * N * esz) and _intact(raw_ws, max(ws_bytes, 256)), "write outside a buffer"
+    for h in range(heads):
+        Yref, T = oracle.gemm(oracle.dequantize(*oracle.quantize(a[h], dtype=oracle.BF16)), oracle.dequantize(*oracle.quantize(b[h // group], dtype=oracle.BF16)))
+        err = np.abs(out[h].float().cpu().numpy().astype(np.float64) - Yref)
+        bound = 1e-6 * T + (2.0 ** -8 * np.abs(Yref) if ydt == torch.bfloat16 else 0.0) + 2.0 ** -120
+        assert (err <= bound).all(), f"head {h}: max err / bound = {float((err / bound).max())}"
+    bd.poll_status()
