@@ -949,6 +949,27 @@ def run_case(args):
         torch.cuda.synchronize()
         print(json.dumps({"case": args.case, "us_per_call": e0.elapsed_time(e1) / reps * 1e3}))
         return
+    if args.case == "kv_attention":
+        # the attention of one decode step over 8 cached KV heads x 4113 tokens x 128, 4 query rows per head
+        rng = np.random.default_rng(6)
+        kvh, grp, hd, n_tok, cap = 8, 4, 128, 4113, 4224
+        caches = []
+        for g in range(kvh):
+            c = bd.KVCache(cap, hd, device=dev)
+            c.append(dev_bf16(inputs.to_bf16_bits(rng.standard_normal((n_tok, hd)).astype(np.float32))),
+                     dev_bf16(inputs.to_bf16_bits(rng.standard_normal((n_tok, hd)).astype(np.float32))))
+            caches.append(c)
+        qs = [bd.quantize_act(dev_bf16(inputs.to_bf16_bits(rng.standard_normal((grp, hd)).astype(np.float32)))) for _ in range(kvh)]
+        o = torch.empty(kvh, grp, hd, dtype=torch.bfloat16, device=dev)
+        for _ in range(args.warmup):
+            bd.kvcache_attention(caches, qs, hd ** -0.5, out=o)
+        e0.record()
+        for _ in range(reps):
+            bd.kvcache_attention(caches, qs, hd ** -0.5, out=o)
+        e1.record()
+        torch.cuda.synchronize()
+        print(json.dumps({"case": args.case, "us_per_call": e0.elapsed_time(e1) / reps * 1e3}))
+        return
     if args.case == "quantizer_strided":
         # the value matrix of one KV head, blocks along the token axis: V [4096 tokens, 128] bf16 -> operand [128, 4096]
         vs = [dev_bf16(inputs.to_bf16_bits(np.random.default_rng(s).standard_normal((4096, 128)).astype(np.float32))) for s in range(2)]
@@ -1036,7 +1057,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--case", default=None,
-                    choices=["quantizer", "quantizer_f32", "step", "decode", "decode8", "quantizer_strided", "requant_gate_up", "attention"]
+                    choices=["quantizer", "quantizer_f32", "step", "decode", "decode8", "kv_attention", "quantizer_strided", "requant_gate_up", "attention"]
                     + ["linear_" + n for n, _, _ in LAYERS],
                     help="run a few launches of one small case (for profiler captures) instead of the benchmark")
     args = ap.parse_args()
