@@ -233,3 +233,44 @@ def test_decode_step_attention_link_by_link(n, q_rows, heads, d):
     O16 = bd.kvcache_attention(caches, Qs, scale, dtype=torch.bfloat16)
     assert torch.equal(O16.cpu(), torch.from_numpy(O2).to(torch.bfloat16))
     bd.poll_status()
+
+
+def test_decode_loop_appends_and_attends_back_to_back():
+    # token by token: the new token of every head is appended and the step's attention follows at once on the same
+    # stream, with nothing in between (the scores kernel's copies of the key cache must wait for the append kernels);
+    # every step's result against the oracle caches, which take the same tokens
+    heads, d, kind, start, steps = 3, 128, torch.bfloat16, 50, 40
+    scale = 1.0 / np.sqrt(d)
+    rows = [_rows(start + steps, d, kind, seed=71 + h) for h in range(heads)]
+    caches = [bd.KVCache(128, d, dtype=kind) for _ in range(heads)]
+    refs = [OracleCache(d) for _ in range(heads)]
+    for h in range(heads):
+        caches[h].append(to_device(rows[h][0][:start], kind), to_device(rows[h][1][:start], kind))
+        refs[h].append(rows[h][0][:start], rows[h][1][:start])
+    rng = np.random.default_rng(3)
+    qb = [inputs.to_bf16_bits(rng.standard_normal((steps, 2, d)).astype(np.float32)) for _ in range(heads)]
+    k_all = torch.stack([to_device(rows[h][0][start:], kind) for h in range(heads)])      # [heads, steps, d]
+    v_all = torch.stack([to_device(rows[h][1][start:], kind) for h in range(heads)])
+    Qs_all = [[bd.quantize_act(to_device(qb[h][t], torch.bfloat16)) for h in range(heads)] for t in range(steps)]
+    outs, probs = [], []
+    torch.cuda.synchronize()
+    for t in range(steps):                                        # no synchronisation inside the loop
+        bd.kvcache_append_batched(caches, k_all[:, t:t + 1], v_all[:, t:t + 1])
+        n = start + t + 1
+        p = torch.zeros(heads, 2, (n + 3) // 4 * 4, device="cuda")
+        outs.append(bd.kvcache_attention(caches, Qs_all[t], scale, probs=p))
+        probs.append(p)
+    torch.cuda.synchronize()
+    for t in range(steps):
+        n = start + t + 1
+        for h in range(heads):
+            refs[h].append(rows[h][0][n - 1:n], rows[h][1][n - 1:n])
+            P = probs[t][h, :, :n].cpu().numpy()
+            _, _, Pref = refs[h].attention(oracle.quantize(qb[h][t], dtype=oracle.BF16), scale)
+            assert np.abs(P.astype(np.float64) - Pref.astype(np.float64)).max() <= 2e-6, f"step {t} head {h}: probabilities"
+            Oref, To = refs[h].pv(P)
+            ok, ratio = gemm_tolerance_ok(outs[t][h].cpu().numpy(), Oref, To)
+            assert ok, f"step {t} head {h}: max err / bound = {ratio}"
+    for h in range(heads):
+        _check_state(caches[h], refs[h], kind)
+    bd.poll_status()
