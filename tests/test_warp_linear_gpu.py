@@ -271,3 +271,30 @@ def test_batched_products_with_a_few_rows_share_a_launch(heads, group, M, N, K, 
         bound = 1e-6 * T + (2.0 ** -8 * np.abs(Yref) if ydt == torch.bfloat16 else 0.0) + 2.0 ** -120
         assert (err <= bound).all(), f"head {h}: max err / bound = {float((err / bound).max())}"
     bd.poll_status()
+
+
+def test_weights_quantised_right_before_the_call():
+    # the weights are rewritten by bd_quantize_weights and used by the next call on the stream with nothing in between,
+    # twelve times over the same buffers: the product kernel's early copies of the weights must not overtake the kernel
+    # that writes them (the record kernel in front waits for it before it lets the product kernel start)
+    rng = np.random.default_rng(21)
+    M, N, K, reps = 4, 512, 1024, 12
+    xb = inputs.to_bf16_bits(rng.standard_t(4, (M, K)).astype(np.float32))
+    xd = to_device(xb, torch.bfloat16)
+    ws_host = [inputs.to_bf16_bits((rng.standard_normal((N, K)) * np.exp2(rng.integers(-6, 1, (N, 1)))).astype(np.float32)) for _ in range(reps)]
+    ws_dev = [to_device(w, torch.bfloat16) for w in ws_host]
+    Wq = bd.QTensor(N, K)
+    ws = torch.empty(bd.linear_workspace_size(M, N, K), dtype=torch.uint8, device="cuda")
+    ys = [torch.empty(M, N, dtype=torch.float32, device="cuda") for _ in range(reps)]
+    bd.set_gemm_impl(bd.GEMM_WARP)
+    torch.cuda.synchronize()
+    for i in range(reps):
+        bd.quantize_weights(ws_dev[i], bd.SELECT_TWO_STAGE, out=Wq)
+        bd.linear(xd, Wq, out=ys[i], workspace=ws)
+    torch.cuda.synchronize()
+    xq = oracle.dequantize(*oracle.quantize(xb, dtype=oracle.BF16))
+    for i in range(reps):
+        Yref, T = oracle.gemm(xq, oracle.dequantize(*oracle.quantize(ws_host[i], dtype=oracle.BF16)))
+        ok, ratio = gemm_tolerance_ok(ys[i].cpu().numpy(), Yref, T)
+        assert ok, f"call {i}: max err / bound = {ratio}"
+    bd.poll_status()
