@@ -262,7 +262,9 @@ bd_status bd_kvcache_pv(const bd_kvcache *c, const float *P, int64_t q_rows, int
  * S + i * stride_s / Y + i * stride_y, and takes its t new tokens from Knew + i * stride_k, Vnew + i * stride_v
  * (strides in elements; every head's length advances by t).  With q <= 16 and n <= 64 (and the library's own
  * choice of product kernel) the heads share one (scores) or two (P x V) launches; otherwise the calls
- * above run head by head.  workspace: bd_kvcache_batched_workspace_size bytes, 256-byte aligned. */
+ * above run head by head.  BD_ERR_SHAPE when the heads differ in capacity, head_dim, dtype or length, or the strides
+ * are shorter than a head's rows; otherwise the errors of the one-head calls.  workspace:
+ * bd_kvcache_batched_workspace_size bytes, 256-byte aligned. */
 bd_status bd_kvcache_append_batched(bd_kvcache *c, int64_t n, const void *Knew, const void *Vnew, int64_t t, int64_t ldk,
                                     int64_t ldv, int64_t stride_k, int64_t stride_v, void *stream);
 bd_status bd_kvcache_batched_workspace_size(int64_t n, int64_t capacity, int64_t head_dim, int64_t q_rows, size_t *bytes);
